@@ -1,0 +1,147 @@
+"""Ozaki Scheme II in Python big integers and exact fractions -- tiny inputs only.
+
+TEST INFRASTRUCTURE ONLY.  A second, independent statement of the method used to
+pin the C oracle: nothing here calls the C library, and every quantity is exact
+(`int`, `fractions.Fraction`), so there is no rounding anywhere except the single
+final conversion that the method itself prescribes (Sec. 2, step (iv)).
+
+Follows Sec. 2 Eq. 1-5, Algorithm 2 with Lemma 1, and Algorithm 3.
+"""
+from __future__ import annotations
+
+import math
+from fractions import Fraction
+
+SETS = {
+    "S": [1089, 1024, 961, 841, 625, 529, 511, 509, 503, 499, 491, 487],
+    "E": [1089, 1024, 961, 841, 625, 529, 251, 247, 241, 239, 233, 229, 227],
+}
+
+
+def product(ms):
+    out = 1
+    for m in ms:
+        out *= m
+    return out
+
+
+def floor_log2(x: Fraction) -> int:
+    """floor(log2 x) for an exact positive rational."""
+    e = x.numerator.bit_length() - x.denominator.bit_length()
+    if Fraction(2) ** e > x:
+        e -= 1
+    while Fraction(2) ** (e + 1) <= x:
+        e += 1
+    return e
+
+
+def budget_maxexp(ms, k):
+    T = ((product(ms) - 1) // 2 // k).bit_length() - 1
+    return T - T // 2, T // 2
+
+
+def cs_bound(ms, k):
+    bnd = math.isqrt((product(ms) - 1) // 2)
+    g = 0
+    while 4 * g * g < k:
+        g += 1
+    return bnd - g
+
+
+def shift_of_line(line, ms, rule, tbits, k):
+    """line: list of floats (finite).  Returns sigma (Eq. 1)."""
+    nz = [abs(Fraction(x)) for x in line if x != 0]
+    if not nz:
+        return 0
+    E = max(floor_log2(x) for x in nz)
+    if rule == "MAXEXP":
+        return tbits - 1 - E
+    S = sum(math.ceil(x * Fraction(2) ** (9 - E)) ** 2 for x in nz)
+    G2 = cs_bound(ms, k) ** 2
+    p = 0
+    while 4 ** (p + 1) * S <= G2:
+        p += 1
+    return p + 9 - E
+
+
+def quantise(x: float, sigma: int, quant: str) -> int:
+    v = Fraction(x) * Fraction(2) ** sigma
+    if quant == "TZ":
+        return int(v)  # int() truncates toward zero
+    return round(v)  # Fraction.__round__ rounds half to even
+
+
+def centred(x: int, m: int) -> int:
+    d = x % m
+    return d - m if 2 * d >= m else d
+
+
+def e4m3_integers():
+    """All integers exactly representable in E4M3 (the set of Lemma 1)."""
+    vals = set()
+    for e in range(16):
+        for f in range(8):
+            if e == 15 and f == 7:
+                continue
+            v = Fraction(f, 8) * Fraction(2) ** -6 if e == 0 else (1 + Fraction(f, 8)) * Fraction(2) ** (e - 7)
+            if v.denominator == 1:
+                vals.add(int(v))
+                vals.add(-int(v))
+    return vals
+
+
+_E = e4m3_integers()
+
+
+def split(d: int, m: int):
+    s = math.isqrt(m)
+    if s * s == m:
+        lo = s // 2
+        d0 = (d + lo) % s - lo
+        return [d0, (d - d0) // s]
+    d0 = (d + 8) % 16 - 8
+    d1 = (d - d0) // 16
+    if d0 + d1 not in _E:
+        sg = (d0 > 0) - (d0 < 0)
+        d0, d1 = d0 - 16 * sg, d1 + sg
+    return [d0, d1, d0 + d1]
+
+
+def garner(res, ms) -> int:
+    v = []
+    for j, m in enumerate(ms):
+        if j == 0:
+            v.append(res[0] % m)
+            continue
+        partial, weight = 0, 1
+        for l in range(j):
+            partial += v[l] * weight
+            weight *= ms[l]
+        w = pow(weight, -1, m)
+        v.append(((res[j] - partial) * w) % m)
+    x = 0
+    for j in reversed(range(len(ms))):
+        x = x * ms[j] + v[j]
+    M = product(ms)
+    return x - M if 2 * x >= M else x
+
+
+def int_to_float_rn(x: int) -> float:
+    return float(Fraction(x))  # exact rational -> nearest double, ties to even
+
+
+def dgemm(A, B, set_name="S", quant="RN", rule="CS"):
+    """A: m x k nested lists, B: k x n nested lists -> (C, sigma, tau, R, Cint)."""
+    ms = SETS[set_name]
+    m, k, n = len(A), len(B), len(B[0])
+    tA, tB = budget_maxexp(ms, k)
+    sig = [shift_of_line(A[i], ms, rule, tA, k) for i in range(m)]
+    tau = [shift_of_line([B[kk][j] for kk in range(k)], ms, rule, tB, k) for j in range(n)]
+    QA = [[quantise(A[i][kk], sig[i], quant) for kk in range(k)] for i in range(m)]
+    QB = [[quantise(B[kk][j], tau[j], quant) for kk in range(k)] for j in range(n)]
+    R = [[[sum(centred(QA[i][kk], mm) * centred(QB[j][kk], mm) for kk in range(k)) % mm
+           for i in range(m)] for j in range(n)] for mm in ms]
+    Cint = [[garner([R[q][j][i] for q in range(len(ms))], ms) for j in range(n)] for i in range(m)]
+    Cf = [[float(Fraction(int_to_float_rn(Cint[i][j])) * Fraction(2) ** -(sig[i] + tau[j]))
+           for j in range(n)] for i in range(m)]
+    return Cf, sig, tau, R, Cint

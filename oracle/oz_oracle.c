@@ -1,0 +1,666 @@
+/*
+ * Ozaki Scheme II FP64 GEMM emulation -- plain CPU oracle.
+ *
+ * TEST INFRASTRUCTURE ONLY.  This file is the slow, exact-integer statement of
+ * what the GPU library must compute.  It shares no code, header, table or
+ * constant generator with the CUDA path and is never called by it; only the
+ * tests, the smoke check and the benchmark's CPU-baseline leg load it.
+ *
+ * Every function follows the paper's steps in the paper's order:
+ *   Sec. 2 "The scheme in equations", Eq. 1-5  (scale, residues, products, Garner)
+ *   Sec. 2 "The FP8 variant", Eq. 6-7          (two-limb planes, 3 products / modulus)
+ *   Algorithm 2 (Deconstruct), Lemma 1, Eq. 8  (digit split, carry, stored planes)
+ *   Algorithm 3 (Reconstruct), Eq. 4-5         (mixed-radix digits, Horner, lift)
+ *   Sec. "Modulus/Encoding Codesign"           (sets S and E)
+ * No blocking, fusion or reordering beyond what those passages state.
+ *
+ * Parity status: every function here is pinned by tests/test_oracle_*.py against
+ * values the paper prints, closed forms, exhaustive identities or a Python
+ * big-integer restatement -- except the accuracy of the method against the true
+ * product on inputs with a very wide exponent spread, for which the paper prints
+ * no bound: "parity unpinned" for that one quantity (it is measured, not asserted).
+ *
+ * Storage conventions (column-major BLAS shapes, Sec. 2: C = AB, A m x k, B k x n):
+ *   side 0: X is m x k, "line" i is row i,    element (i,kk) at X[i + kk*ldx]
+ *   side 1: X is k x n, "line" j is column j, element (kk,j) at X[kk + j*ldx]
+ *   quantised integers  Q[line*k + kk]                 (int64)
+ *   centred residues    D[(mod*lines + line)*k + kk]   (int16)
+ *   stored planes       P[plane*plane_stride + line*row_pitch + kk] (uint8)
+ *   residue products    R[(mod*n + j)*m + i]           (uint16, canonical [0,m_i))
+ *   exact integers      CI[(j*m + i)*2 + {0,1}] = {low, high} 64-bit words of a
+ *                       two's-complement 128-bit value
+ */
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#include <math.h>
+
+typedef __int128 i128;
+typedef unsigned __int128 u128;
+
+enum { OZO_SET_S = 0, OZO_SET_E = 1 };
+enum { OZO_QUANT_RN = 0, OZO_QUANT_TZ = 1 };
+enum { OZO_SCALE_MAXEXP = 0, OZO_SCALE_CS = 1 };
+enum { OZO_SUB_FP8 = 0, OZO_SUB_INT8 = 1 };
+
+#define OZO_NONFINITE_SHIFT INT32_MIN
+
+/* ------------------------------------------------------------------ */
+/* Modulus sets (Sec. 2 Eq. 2 text for S; "Candidate E" paragraph)     */
+/* ------------------------------------------------------------------ */
+static const int SET_S[12] = {1089, 1024, 961, 841, 625, 529, 511, 509, 503, 499, 491, 487};
+static const int SET_E[13] = {1089, 1024, 961, 841, 625, 529, 251, 247, 241, 239, 233, 229, 227};
+
+int ozo_modset(int set, int *moduli)
+{
+    const int *src = (set == OZO_SET_S) ? SET_S : SET_E;
+    int r = (set == OZO_SET_S) ? 12 : 13;
+    if (set != OZO_SET_S && set != OZO_SET_E) return 0;
+    for (int i = 0; i < r; ++i) moduli[i] = src[i];
+    return r;
+}
+
+/* integer square root of a modulus if it is a perfect square, else 0 */
+int ozo_square_root(int m)
+{
+    for (int s = 1; s * s <= m; ++s)
+        if (s * s == m) return s;
+    return 0;
+}
+
+/* stored planes per modulus: 2 for a square, 3 otherwise (Sec. 2, FP8 variant) */
+int ozo_planes_of(int m) { return ozo_square_root(m) ? 2 : 3; }
+
+int ozo_pstore(int set)
+{
+    int mod[16], r = ozo_modset(set, mod), p = 0;
+    for (int i = 0; i < r; ++i) p += ozo_planes_of(mod[i]);
+    return p;
+}
+
+static u128 modset_product(int set)
+{
+    int mod[16], r = ozo_modset(set, mod);
+    u128 M = 1;
+    for (int i = 0; i < r; ++i) M *= (u128)mod[i];
+    return M;
+}
+
+void ozo_M(int set, uint64_t out[2])
+{
+    u128 M = modset_product(set);
+    out[0] = (uint64_t)M;
+    out[1] = (uint64_t)(M >> 64);
+}
+
+/* ------------------------------------------------------------------ */
+/* Range budget (Eq. 2: |c'| <= k 2^(2t) = mu,  M > 2 mu)              */
+/* ------------------------------------------------------------------ */
+static int bitlen128(u128 v)
+{
+    int n = 0;
+    while (v) { ++n; v >>= 1; }
+    return n;
+}
+
+/* MAXEXP rule: T = floor(log2(floor((M-1)/2)/k)), t_A = T - floor(T/2), t_B = floor(T/2).
+ * With |a'| <= 2^t_A and |b'| <= 2^t_B:  |c'| <= k 2^T <= (M-1)/2.            */
+int ozo_budget_maxexp(int set, int64_t k, int *tA, int *tB)
+{
+    if (k <= 0) { *tA = *tB = 0; return 0; }
+    u128 half = (modset_product(set) - 1) / 2;
+    u128 v = half / (u128)k;
+    int T = bitlen128(v) - 1;
+    *tB = T / 2;
+    *tA = T - *tB;
+    return T;
+}
+
+static u128 isqrt128(u128 v)
+{
+    u128 r = 0;
+    for (int b = 63; b >= 0; --b) {
+        u128 c = r | ((u128)1 << b);
+        if (c * c <= v) r = c;
+    }
+    return r;
+}
+
+/* CS rule bound: G = floor(sqrt((M-1)/2)) - ceil(sqrt(k)/2).
+ * ||a'||_2 <= 2^p sqrt(S) + sqrt(k)/2 (round-to-nearest adds at most 1/2 per entry),
+ * and |c'_ij| <= ||a'_i|| ||b'_j|| (Cauchy-Schwarz) <= floor(sqrt((M-1)/2))^2.      */
+uint64_t ozo_cs_bound(int set, int64_t k)
+{
+    u128 half = (modset_product(set) - 1) / 2;
+    uint64_t bnd = (uint64_t)isqrt128(half);
+    uint64_t g = 0;
+    while ((u128)4 * g * g < (u128)k) ++g; /* smallest g with 2g >= sqrt(k) */
+    return bnd - g;
+}
+
+/* ------------------------------------------------------------------ */
+/* IEEE-754 double decoding: |x| = sig * 2^(ex-52)                      */
+/* ------------------------------------------------------------------ */
+typedef struct { int neg; int kind; /* 0 zero, 1 finite nonzero, 2 inf/nan */
+                 uint64_t sig; int ex; int e; /* e = floor(log2|x|) */ } fp_parts;
+
+static fp_parts decode(double x)
+{
+    fp_parts p;
+    uint64_t bits;
+    memcpy(&bits, &x, 8);
+    p.neg = (int)(bits >> 63);
+    int be = (int)((bits >> 52) & 0x7FF);
+    uint64_t frac = bits & 0xFFFFFFFFFFFFFull;
+    p.sig = 0; p.ex = 0; p.e = 0;
+    if (be == 0x7FF) { p.kind = 2; return p; }
+    if (be == 0 && frac == 0) { p.kind = 0; return p; }
+    p.kind = 1;
+    if (be == 0) { p.sig = frac; p.ex = -1022; }
+    else { p.sig = frac | (1ull << 52); p.ex = be - 1023; }
+    int top = 63;
+    while (!((p.sig >> top) & 1)) --top;
+    p.e = p.ex - 52 + top;
+    return p;
+}
+
+static const double *elem(const double *X, int64_t ldx, int side, int64_t line, int64_t kk)
+{
+    return side == 0 ? &X[line + kk * ldx] : &X[kk + line * ldx];
+}
+
+/* ------------------------------------------------------------------ */
+/* Step (i) of Sec. 2: per-row / per-column exponents sigma, tau        */
+/* ------------------------------------------------------------------ */
+/* MAXEXP: sigma = t - 1 - max_k floor(log2|x|), so |x 2^sigma| < 2^t.
+ * CS:     abar = ceil(|x| 2^(9-E)) in [0,2^10], S = sum abar^2 (exact integer),
+ *         p = largest integer with 4^p S <= G^2,  sigma = p + 9 - E.
+ * A line of zeros gets shift 0; a line holding Inf/NaN gets the sentinel.    */
+void ozo_shifts(int side, int64_t lines, int64_t k, const double *X, int64_t ldx,
+                int set, int rule, int tbits, int32_t *shift)
+{
+    uint64_t G = ozo_cs_bound(set, k > 0 ? k : 1);
+    u128 G2 = (u128)G * G;
+#pragma omp parallel for schedule(static)
+    for (int64_t l = 0; l < lines; ++l) {
+        int any = 0, bad = 0, E = 0;
+        for (int64_t kk = 0; kk < k; ++kk) {
+            fp_parts p = decode(*elem(X, ldx, side, l, kk));
+            if (p.kind == 2) bad = 1;
+            if (p.kind == 1) { if (!any || p.e > E) E = p.e; any = 1; }
+        }
+        if (bad) { shift[l] = OZO_NONFINITE_SHIFT; continue; }
+        if (!any) { shift[l] = 0; continue; }
+        if (rule == OZO_SCALE_MAXEXP) { shift[l] = tbits - 1 - E; continue; }
+        u128 S = 0;
+        for (int64_t kk = 0; kk < k; ++kk) {
+            fp_parts p = decode(*elem(X, ldx, side, l, kk));
+            if (p.kind != 1) continue;
+            /* |x| 2^(9-E) = sig 2^(ex-52+9-E) = sig / 2^sh, sh = 43 + E - ex >= 43-52... */
+            int sh = 43 + E - p.ex;
+            uint64_t abar;
+            if (sh >= 64) abar = 1;
+            else if (sh <= 0) abar = p.sig << (-sh);
+            else abar = (p.sig >> sh) + ((p.sig & ((1ull << sh) - 1)) ? 1 : 0);
+            S += (u128)abar * abar;
+        }
+        int pw = 0;
+        while (pw < 60 && S <= (G2 >> (2 * (pw + 1)))) ++pw;
+        shift[l] = pw + 9 - E;
+    }
+}
+
+/* ------------------------------------------------------------------ */
+/* Eq. 1: a' = quant(2^sigma a) -- RN (ties to even) or truncation      */
+/* ------------------------------------------------------------------ */
+static int64_t quantise_one(double x, int32_t sigma, int quant)
+{
+    fp_parts p = decode(x);
+    if (p.kind != 1) return 0;
+    /* |x| 2^sigma = sig 2^(ex-52+sigma) = sig / 2^sh */
+    int64_t sh = 52 - (int64_t)p.ex - (int64_t)sigma;
+    uint64_t q;
+    if (sh <= 0) {
+        q = p.sig << (-sh);
+    } else if (sh >= 64) {
+        q = 0; /* sig < 2^53 <= 2^(sh-1): below one half */
+    } else {
+        q = p.sig >> sh;
+        if (quant == OZO_QUANT_RN) {
+            uint64_t rem = p.sig & ((1ull << sh) - 1);
+            uint64_t half = 1ull << (sh - 1);
+            if (rem > half || (rem == half && (q & 1))) ++q;
+        }
+    }
+    return p.neg ? -(int64_t)q : (int64_t)q;
+}
+
+void ozo_quantise(int side, int64_t lines, int64_t k, const double *X, int64_t ldx,
+                  const int32_t *shift, int quant, int64_t *Q)
+{
+#pragma omp parallel for schedule(static)
+    for (int64_t l = 0; l < lines; ++l)
+        for (int64_t kk = 0; kk < k; ++kk)
+            Q[l * k + kk] = (shift[l] == OZO_NONFINITE_SHIFT)
+                                ? 0
+                                : quantise_one(*elem(X, ldx, side, l, kk), shift[l], quant);
+}
+
+/* ------------------------------------------------------------------ */
+/* Eq. 3 operands: centred residues in [-m/2, m/2), -m/2 included       */
+/* ------------------------------------------------------------------ */
+int ozo_centred_residue(int64_t x, int m)
+{
+    int64_t d = x % m;
+    if (d < 0) d += m;
+    if (2 * d >= m) d -= m;
+    return (int)d;
+}
+
+void ozo_residues(int64_t lines, int64_t k, const int64_t *Q, int set, int16_t *D)
+{
+    int mod[16], r = ozo_modset(set, mod);
+    for (int i = 0; i < r; ++i) {
+#pragma omp parallel for schedule(static)
+        for (int64_t e = 0; e < lines * k; ++e)
+            D[(int64_t)i * lines * k + e] = (int16_t)ozo_centred_residue(Q[e], mod[i]);
+    }
+}
+
+/* ------------------------------------------------------------------ */
+/* E4M3 (OCP FP8, 4 exponent bits bias 7, 3 mantissa bits, max 448)     */
+/* ------------------------------------------------------------------ */
+/* value of a byte code, by the format's definition; NaN codes return NAN */
+double ozo_e4m3_value(int code)
+{
+    int s = (code >> 7) & 1, e = (code >> 3) & 15, f = code & 7;
+    double v;
+    if (e == 15 && f == 7) return NAN;
+    if (e == 0) v = ldexp((double)f / 8.0, -6);
+    else v = ldexp(1.0 + (double)f / 8.0, e - 7);
+    return s ? -v : v;
+}
+
+/* the set E of Lemma 1: is the integer exactly representable? */
+int ozo_in_e4m3(int v)
+{
+    for (int c = 0; c < 256; ++c) {
+        double x = ozo_e4m3_value(c);
+        if (x == (double)v) return 1;
+    }
+    return 0;
+}
+
+/* byte code of an exactly representable integer (zero is +0, code 0x00); -1 if none */
+int ozo_e4m3_encode(int v)
+{
+    if (v == 0) return 0;
+    for (int c = 0; c < 256; ++c) {
+        double x = ozo_e4m3_value(c);
+        if (x == (double)v) return c;
+    }
+    return -1;
+}
+
+/* ------------------------------------------------------------------ */
+/* Algorithm 2 lines for the digit split; Lemma 1 carry                 */
+/* ------------------------------------------------------------------ */
+static int floor_mod(int a, int b) { int r = a % b; return r < 0 ? r + b : r; }
+
+/* d -> (d0, d1[, d0+d1]); returns the number of stored planes (2 or 3) */
+int ozo_split(int d, int m, int out[3])
+{
+    int s = ozo_square_root(m);
+    if (s) {
+        /* balanced base-s digits: odd s in [-(s-1)/2,(s-1)/2]; even s in [-s/2, s/2-1] */
+        int lo = s / 2; /* (s-1)/2 for odd s, s/2 for even s */
+        int d0 = floor_mod(d + lo, s) - lo;
+        int d1 = (d - d0) / s;
+        out[0] = d0; out[1] = d1; out[2] = 0;
+        return 2;
+    }
+    int d0 = floor_mod(d + 8, 16) - 8;
+    int d1 = (d - d0) / 16;
+    if (!ozo_in_e4m3(d0 + d1)) {
+        int sg = (d0 > 0) - (d0 < 0);
+        d0 -= 16 * sg;
+        d1 += sg;
+    }
+    out[0] = d0; out[1] = d1; out[2] = d0 + d1;
+    return 3;
+}
+
+/* stored planes, published modulus order, plane order d0, d1[, d0+d1];
+ * FP8 substrate: E4M3 byte; INT8 substrate: two's-complement byte.
+ * Bytes kk in [k, row_pitch) of every line are written as zero.          */
+int ozo_planes(int64_t lines, int64_t k, const int16_t *D, int set, int substrate,
+               uint8_t *P, int64_t plane_stride, int64_t row_pitch)
+{
+    int mod[16], r = ozo_modset(set, mod), plane = 0, bad = 0;
+    for (int i = 0; i < r; ++i) {
+        int np = ozo_planes_of(mod[i]);
+        for (int64_t l = 0; l < lines; ++l) {
+            for (int64_t kk = 0; kk < row_pitch; ++kk) {
+                int dg[3] = {0, 0, 0};
+                if (kk < k) ozo_split(D[((int64_t)i * lines + l) * k + kk], mod[i], dg);
+                for (int q = 0; q < np; ++q) {
+                    int byte;
+                    if (substrate == OZO_SUB_FP8) {
+                        byte = ozo_e4m3_encode(dg[q]);
+                        if (byte < 0) { bad = 1; byte = 0x7F; }
+                    } else {
+                        if (dg[q] < -128 || dg[q] > 127) bad = 1;
+                        byte = dg[q] & 0xFF;
+                    }
+                    P[(int64_t)(plane + q) * plane_stride + l * row_pitch + kk] = (uint8_t)byte;
+                }
+            }
+        }
+        plane += np;
+    }
+    return bad ? -1 : plane;
+}
+
+static int plane_digit(uint8_t byte, int substrate)
+{
+    if (substrate == OZO_SUB_FP8) return (int)ozo_e4m3_value(byte);
+    return (int)(int8_t)byte;
+}
+
+/* ------------------------------------------------------------------ */
+/* Eq. 3: C^(i) = A^(i) B^(i) mod m_i, int64 accumulation               */
+/* ------------------------------------------------------------------ */
+void ozo_products(int64_t m, int64_t n, int64_t k, const int16_t *DA, const int16_t *DB,
+                  int set, uint16_t *R)
+{
+    int mod[16], r = ozo_modset(set, mod);
+    for (int i = 0; i < r; ++i) {
+        const int16_t *a = DA + (int64_t)i * m * k;
+        const int16_t *b = DB + (int64_t)i * n * k;
+#pragma omp parallel for schedule(static)
+        for (int64_t j = 0; j < n; ++j)
+            for (int64_t ii = 0; ii < m; ++ii) {
+                int64_t acc = 0;
+                for (int64_t kk = 0; kk < k; ++kk)
+                    acc += (int64_t)a[ii * k + kk] * (int64_t)b[j * k + kk];
+                int64_t c = acc % mod[i];
+                if (c < 0) c += mod[i];
+                R[((int64_t)i * n + j) * m + ii] = (uint16_t)c;
+            }
+    }
+}
+
+/* The same residues through the stored planes (Sec. 2 FP8 variant; Eq. 8):
+ *   square    : (D0.E0) + s (D1.E0 + D0.E1)                 mod m
+ *   nonsquare : -15 (D0.E0) + 16 (D0+D1).(E0+E1) + 240 (D1.E1) mod m
+ * Writes R like ozo_products and returns the largest |accumulator| met
+ * (for the exact-accumulation limit 2^24 of the FP8 route).               */
+int64_t ozo_plane_products(int64_t m, int64_t n, int64_t k, const uint8_t *PA,
+                           int64_t strideA, int64_t pitchA, const uint8_t *PB, int64_t strideB,
+                           int64_t pitchB, int set, int substrate, uint16_t *R)
+{
+    int mod[16], r = ozo_modset(set, mod), plane = 0;
+    int64_t worst = 0;
+    for (int i = 0; i < r; ++i) {
+        int s = ozo_square_root(mod[i]);
+        int np = s ? 2 : 3;
+        int64_t worst_i = 0;
+#pragma omp parallel for schedule(static) reduction(max : worst_i)
+        for (int64_t j = 0; j < n; ++j)
+            for (int64_t ii = 0; ii < m; ++ii) {
+                int64_t acc[3] = {0, 0, 0};
+                for (int64_t kk = 0; kk < k; ++kk) {
+                    int a[3], b[3];
+                    for (int q = 0; q < np; ++q) {
+                        a[q] = plane_digit(PA[(plane + q) * strideA + ii * pitchA + kk], substrate);
+                        b[q] = plane_digit(PB[(plane + q) * strideB + j * pitchB + kk], substrate);
+                    }
+                    if (s) {
+                        acc[0] += (int64_t)a[0] * b[0];
+                        acc[1] += (int64_t)a[1] * b[0] + (int64_t)a[0] * b[1];
+                    } else {
+                        acc[0] += (int64_t)a[0] * b[0];
+                        acc[1] += (int64_t)a[2] * b[2];
+                        acc[2] += (int64_t)a[1] * b[1];
+                    }
+                }
+                for (int q = 0; q < 3; ++q) {
+                    int64_t v = acc[q] < 0 ? -acc[q] : acc[q];
+                    if (v > worst_i) worst_i = v;
+                }
+                int64_t t = s ? acc[0] + (int64_t)s * acc[1]
+                              : -15 * acc[0] + 16 * acc[1] + 240 * acc[2];
+                int64_t c = t % mod[i];
+                if (c < 0) c += mod[i];
+                R[((int64_t)i * n + j) * m + ii] = (uint16_t)c;
+            }
+        if (worst_i > worst) worst = worst_i;
+        plane += np;
+    }
+    return worst;
+}
+
+/* ------------------------------------------------------------------ */
+/* Eq. 4-5 / Algorithm 3: Garner mixed-radix digits, Horner, lift       */
+/* ------------------------------------------------------------------ */
+/* w_j = (m_1 ... m_{j-1})^{-1} mod m_j, found by trial (w_1 unused = 0) */
+void ozo_garner_constants(int set, int *w)
+{
+    int mod[16], r = ozo_modset(set, mod);
+    w[0] = 0;
+    for (int j = 1; j < r; ++j) {
+        int64_t prod = 1;
+        for (int l = 0; l < j; ++l) prod = (prod * mod[l]) % mod[j];
+        w[j] = 0;
+        for (int c = 1; c < mod[j]; ++c)
+            if ((prod * c) % mod[j] == 1) { w[j] = c; break; }
+    }
+}
+
+static i128 crt_one(const int *mod, const int *w, int r, const int *c, u128 M)
+{
+    int v[16];
+    v[0] = c[0] % mod[0];
+    for (int j = 1; j < r; ++j) {
+        /* (v_1 + v_2 m_1 + ... + v_{j} m_1...m_{j-1}) mod m_j, by Horner from the top */
+        int64_t acc = 0;
+        for (int l = j - 1; l >= 0; --l) acc = (acc * mod[l] + v[l]) % mod[j];
+        int64_t t = ((int64_t)c[j] - acc) % mod[j];
+        if (t < 0) t += mod[j];
+        v[j] = (int)((t * w[j]) % mod[j]);
+    }
+    u128 x = 0;
+    for (int j = r - 1; j >= 0; --j) x = x * (u128)mod[j] + (u128)v[j];
+    /* symmetric lift: representatives u >= M/2 map to u - M, so -M/2 is included */
+    if (2 * x >= M) return (i128)x - (i128)M;
+    return (i128)x;
+}
+
+void ozo_crt(int64_t m, int64_t n, const uint16_t *R, int set, int64_t *CI)
+{
+    int mod[16], w[16], r = ozo_modset(set, mod);
+    u128 M = modset_product(set);
+    ozo_garner_constants(set, w);
+#pragma omp parallel for schedule(static)
+    for (int64_t e = 0; e < m * n; ++e) {
+        int c[16];
+        for (int i = 0; i < r; ++i) c[i] = R[(int64_t)i * m * n + e];
+        i128 x = crt_one(mod, w, r, c, M);
+        CI[2 * e] = (int64_t)(uint64_t)(u128)x;
+        CI[2 * e + 1] = (int64_t)(x >> 64);
+    }
+}
+
+/* CRT of one residue vector (for round-trip pins) */
+void ozo_crt_single(int set, const int *c, int64_t out[2])
+{
+    int mod[16], w[16], r = ozo_modset(set, mod);
+    ozo_garner_constants(set, w);
+    i128 x = crt_one(mod, w, r, c, modset_product(set));
+    out[0] = (int64_t)(uint64_t)(u128)x;
+    out[1] = (int64_t)(x >> 64);
+}
+
+/* the plain definition of C' = A'B' in 128-bit integers */
+void ozo_direct(int64_t m, int64_t n, int64_t k, const int64_t *QA, const int64_t *QB,
+                int64_t *CI)
+{
+#pragma omp parallel for schedule(static)
+    for (int64_t j = 0; j < n; ++j)
+        for (int64_t i = 0; i < m; ++i) {
+            i128 acc = 0;
+            for (int64_t kk = 0; kk < k; ++kk) acc += (i128)QA[i * k + kk] * (i128)QB[j * k + kk];
+            CI[2 * (j * m + i)] = (int64_t)(uint64_t)(u128)acc;
+            CI[2 * (j * m + i) + 1] = (int64_t)(acc >> 64);
+        }
+}
+
+/* ------------------------------------------------------------------ */
+/* Final step of Sec. 2 (iv): unscale and round once to FP64            */
+/* ------------------------------------------------------------------ */
+/* nearest double to a 128-bit integer, ties to even, written out by hand */
+double ozo_i128_to_double(int64_t lo, int64_t hi)
+{
+    i128 x = ((i128)hi << 64) | (i128)(u128)(uint64_t)lo;
+    int neg = x < 0;
+    u128 a = neg ? (u128)0 - (u128)x : (u128)x;
+    int bl = bitlen128(a);
+    double v;
+    if (bl <= 53) {
+        v = (double)(uint64_t)a;
+    } else {
+        int sh = bl - 53;
+        u128 q = a >> sh;
+        u128 rem = a & (((u128)1 << sh) - 1);
+        u128 half = (u128)1 << (sh - 1);
+        if (rem > half || (rem == half && (q & 1))) ++q;
+        v = ldexp((double)(uint64_t)q, sh);
+    }
+    return neg ? -v : v;
+}
+
+/* P_ij = RN(c'_ij) 2^-(sigma_i+tau_j);  C = P  (beta=0)  or  C = RN(C_old + alpha P) */
+void ozo_output(int64_t m, int64_t n, const int64_t *CI, const int32_t *shiftA,
+                const int32_t *shiftB, double alpha, double beta, double *C, int64_t ldc)
+{
+#pragma omp parallel for schedule(static)
+    for (int64_t j = 0; j < n; ++j)
+        for (int64_t i = 0; i < m; ++i) {
+            double p;
+            if (shiftA[i] == OZO_NONFINITE_SHIFT || shiftB[j] == OZO_NONFINITE_SHIFT) {
+                p = NAN;
+            } else {
+                double v = ozo_i128_to_double(CI[2 * (j * m + i)], CI[2 * (j * m + i) + 1]);
+                p = ldexp(v, -(shiftA[i] + shiftB[j]));
+            }
+            double *c = &C[i + j * ldc];
+            if (beta == 0.0) *c = alpha * p;
+            else *c = beta * (*c) + alpha * p; /* alpha = +-1, beta = 1: one rounding */
+        }
+}
+
+/* ------------------------------------------------------------------ */
+/* Second reference: double-double GEMM (error-free products and sums)  */
+/* ------------------------------------------------------------------ */
+static void dd_add_prod(double *hi, double *lo, double a, double b)
+{
+    double p = a * b;
+    double pe = fma(a, b, -p);       /* exact product = p + pe */
+    double s = *hi + p;
+    double bb = s - *hi;
+    double se = (*hi - (s - bb)) + (p - bb); /* exact sum = s + se */
+    double l = *lo + (se + pe);
+    double h = s + l;
+    *lo = l - (h - s);
+    *hi = h;
+}
+
+void ozo_dd_gemm(int64_t m, int64_t n, int64_t k, const double *A, int64_t lda, const double *B,
+                 int64_t ldb, double *Chi, double *Clo, double *absAB)
+{
+#pragma omp parallel for schedule(static)
+    for (int64_t j = 0; j < n; ++j)
+        for (int64_t i = 0; i < m; ++i) {
+            double hi = 0.0, lo = 0.0, ahi = 0.0, alo = 0.0;
+            for (int64_t kk = 0; kk < k; ++kk) {
+                double a = A[i + kk * lda], b = B[kk + j * ldb];
+                dd_add_prod(&hi, &lo, a, b);
+                dd_add_prod(&ahi, &alo, fabs(a), fabs(b));
+            }
+            Chi[i + j * m] = hi;
+            Clo[i + j * m] = lo;
+            absAB[i + j * m] = ahi;
+        }
+}
+
+/* ------------------------------------------------------------------ */
+/* The whole method in one call (steps in the order of Sec. 2)          */
+/* ------------------------------------------------------------------ */
+/* Returns 0, or -1 on allocation failure / bad arguments.  Optional outputs may be NULL. */
+int ozo_dgemm(int64_t m, int64_t n, int64_t k, const double *A, int64_t lda, const double *B,
+              int64_t ldb, double *C, int64_t ldc, int set, int quant, int rule, double alpha,
+              double beta, int32_t *shiftA_out, int32_t *shiftB_out, uint16_t *R_out)
+{
+    int mod[16], r = ozo_modset(set, mod), tA = 0, tB = 0;
+    if (!r || m < 0 || n < 0 || k < 0) return -1;
+    if (m == 0 || n == 0) return 0;
+    ozo_budget_maxexp(set, k > 0 ? k : 1, &tA, &tB);
+    int64_t kk = k > 0 ? k : 1;
+    int32_t *sA = malloc(sizeof(int32_t) * m), *sB = malloc(sizeof(int32_t) * n);
+    int64_t *QA = malloc(sizeof(int64_t) * m * kk), *QB = malloc(sizeof(int64_t) * n * kk);
+    int16_t *DA = malloc(sizeof(int16_t) * r * m * kk), *DB = malloc(sizeof(int16_t) * r * n * kk);
+    uint16_t *R = malloc(sizeof(uint16_t) * r * m * n);
+    int64_t *CI = malloc(sizeof(int64_t) * 2 * m * n);
+    if (!sA || !sB || !QA || !QB || !DA || !DB || !R || !CI) return -1;
+    ozo_shifts(0, m, k, A, lda, set, rule, tA, sA);
+    ozo_shifts(1, n, k, B, ldb, set, rule, tB, sB);
+    ozo_quantise(0, m, k, A, lda, sA, quant, QA);
+    ozo_quantise(1, n, k, B, ldb, sB, quant, QB);
+    ozo_residues(m, k, QA, set, DA);
+    ozo_residues(n, k, QB, set, DB);
+    ozo_products(m, n, k, DA, DB, set, R);
+    ozo_crt(m, n, R, set, CI);
+    ozo_output(m, n, CI, sA, sB, alpha, beta, C, ldc);
+    if (shiftA_out) memcpy(shiftA_out, sA, sizeof(int32_t) * m);
+    if (shiftB_out) memcpy(shiftB_out, sB, sizeof(int32_t) * n);
+    if (R_out) memcpy(R_out, R, sizeof(uint16_t) * r * m * n);
+    free(sA); free(sB); free(QA); free(QB); free(DA); free(DB); free(R); free(CI);
+    return 0;
+}
+
+/* ------------------------------------------------------------------ */
+/* Byte-plane reduction identity ("O2" paragraph; dp4a worked example)  */
+/* ------------------------------------------------------------------ */
+/* x mod m from the eight bytes of the two's-complement pattern of x:
+ *   U = sum_j byte_j (2^(8j) mod m), split R = R0 + 256 R1, minus [x<0] (2^64 mod m).
+ * Outputs the two limb partial sums of the low `nbytes` bytes and returns the
+ * canonical residue in [0,m).                                               */
+int ozo_byteplane_residue(int64_t x, int m, int nbytes, int *u0, int *u1, int *maxconst,
+                          int *maxhigh)
+{
+    uint64_t pat = (uint64_t)x;
+    int64_t s0 = 0, s1 = 0;
+    int mc = 0, mh = 0;
+    int64_t pw = 1 % m;
+    for (int j = 0; j < nbytes; ++j) {
+        int c = (int)pw;
+        int b = (int)((pat >> (8 * j)) & 0xFF);
+        s0 += (int64_t)b * (c & 0xFF);
+        s1 += (int64_t)b * (c >> 8);
+        if (c > mc) mc = c;
+        if ((c >> 8) > mh) mh = c >> 8;
+        pw = (pw * 256) % m;
+    }
+    if (u0) *u0 = (int)s0;
+    if (u1) *u1 = (int)s1;
+    if (maxconst) *maxconst = mc;
+    if (maxhigh) *maxhigh = mh;
+    int64_t U = s0 + 256 * s1;
+    if (nbytes == 8 && x < 0) {
+        /* pw now equals 2^64 mod m */
+        U -= pw;
+    }
+    int64_t res = U % m;
+    if (res < 0) res += m;
+    return (int)res;
+}

@@ -1,0 +1,444 @@
+"""Pins for the CPU oracle: values the paper prints, closed forms, exhaustive
+identities and a Python big-integer restatement.  No GPU, no CUDA library."""
+import math
+import os
+import random
+from fractions import Fraction
+
+import numpy as np
+import pytest
+
+from oracle import oz_bigint as big
+from oracle import oz_oracle as ozo
+import synth_inputs as syn
+
+GOLD = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def read_golden(name):
+    out = {}
+    with open(os.path.join(GOLD, name)) as fh:
+        for line in fh:
+            line = line.split("#")[0].strip()
+            if "=" in line:
+                key, val = [t.strip() for t in line.split("=", 1)]
+                out[key] = val
+    return out
+
+
+PAPER = read_golden("paper_constants.txt")
+SETS = {"S": ozo.SET_S, "E": ozo.SET_E}
+
+
+# ----------------------------------------------------------------- P1: the sets
+def test_modulus_sets_match_paper():
+    S = [int(v) for v in PAPER["set_S"].split()]
+    assert ozo.modset(ozo.SET_S) == S
+    tail = [int(v) for v in PAPER["set_E_tail"].split()]
+    assert ozo.modset(ozo.SET_E) == S[:6] + tail
+
+
+@pytest.mark.parametrize("name", ["S", "E"])
+def test_set_counts_and_range(name):
+    ms = ozo.modset(SETS[name])
+    for i, a in enumerate(ms):
+        for b in ms[i + 1:]:
+            assert math.gcd(a, b) == 1
+    M = math.prod(ms)
+    assert ozo.M(SETS[name]) == M
+    assert round(math.log2(M), 1) == float(PAPER[f"log2M_{name}"])
+    squares = sum(1 for m in ms if math.isqrt(m) ** 2 == m)
+    assert squares == int(PAPER[f"squares_{name}"])
+    assert ozo.pstore(SETS[name]) == int(PAPER[f"pstore_{name}"])
+    assert 3 * len(ms) == int(PAPER[f"pmma_{name}"])
+    assert 3 * len(ms) + 1 == int(PAPER[f"alpha_{name}"])
+    assert sum(ozo.planes_of(m) for m in ms) == 2 * squares + 3 * (len(ms) - squares)
+
+
+# ----------------------------------------------------------------- range budget
+@pytest.mark.parametrize("name", ["S", "E"])
+@pytest.mark.parametrize("k", [1, 7, 256, 1024, 4096, 5003, 32768])
+def test_budget_is_inside_crt_range(name, k):
+    M = math.prod(ozo.modset(SETS[name]))
+    tA, tB = ozo.budget_maxexp(SETS[name], k)
+    assert tA - tB in (0, 1)
+    assert k * 2 ** (tA + tB) <= (M - 1) // 2          # Eq. 2 with |a'| <= 2^t
+    assert k * 2 ** (tA + tB + 1) > (M - 1) // 2       # and T is the largest such
+    assert (tA, tB) == big.budget_maxexp(ozo.modset(SETS[name]), k)
+    G = ozo.cs_bound(SETS[name], k)
+    assert G == big.cs_bound(ozo.modset(SETS[name]), k)
+    g = math.isqrt((M - 1) // 2) - G
+    assert 2 * g >= math.sqrt(k) and 2 * (g - 1) < math.sqrt(k)
+
+
+# ----------------------------------------------------------------- P2/P3: byte-plane reduction
+def test_dp4a_worked_example():
+    ex = read_golden("dp4a_worked_example.txt")
+    m = int(ex["m"])
+    x = int(ex["x"], 16)
+    consts = [pow(256, j, m) for j in range(4)]
+    assert consts == [int(v) for v in ex["constants"].split()]
+    assert [c & 255 for c in consts] == [int(v) for v in ex["constants_low_limb"].split()]
+    assert [c >> 8 for c in consts] == [int(v) for v in ex["constants_high_limb"].split()]
+    res, u0, u1, _, _ = ozo.byteplane_residue(x, m, 4)
+    assert [(x >> (8 * j)) & 255 for j in range(4)] == [int(v) for v in ex["planes"].split()]
+    assert (u0, u1) == (int(ex["partial_low"]), int(ex["partial_high"]))
+    assert u0 + 256 * u1 == int(ex["recombined"])
+    assert res == int(ex["residue"]) == x % m
+    a, b = [int(v) for v in ex["identical_high_limbs"].split()]
+    assert [pow(256, j, a) >> 8 for j in range(8)] == [pow(256, j, b) >> 8 for j in range(8)]
+
+
+def test_byteplane_identity_signed_equivalence():
+    rng = random.Random(3)
+    worst_c = 0
+    for m in ozo.modset(ozo.SET_S):
+        xs = list(range(-2**15, 2**15, 7)) + [-2**63, 2**63 - 1, -1, 0, 1, -m, m, -m // 2]
+        xs += [rng.randrange(-2**63, 2**63) for _ in range(300)]
+        xs += [rng.randrange(-2**b, 2**b) for b in range(8, 63, 6) for _ in range(20)]
+        for x in xs:
+            res, u0, u1, mc, mh = ozo.byteplane_residue(x, m, 8)
+            assert res == x % m
+            assert 0 <= u0 < int(PAPER["byte_dot_bound"]) and 0 <= u1 < int(PAPER["byte_dot_bound"])
+            assert mh <= 4
+            worst_c = max(worst_c, mc)
+            # the centred residue function agrees with the canonical one
+            d = ozo.centred_residue(x, m)
+            assert (d - x) % m == 0 and -m <= 2 * d < m
+    assert worst_c == int(PAPER["max_reduction_constant_S"])
+
+
+def test_centred_interval_endpoint_rule():
+    # "for even x the endpoint -x/2 is included and +x/2 excluded"
+    assert ozo.centred_residue(512, 1024) == -512
+    assert ozo.centred_residue(-512, 1024) == -512
+    assert ozo.centred_residue(511, 1024) == 511
+    assert ozo.centred_residue(544, 1089) == 544
+    assert ozo.centred_residue(545, 1089) == -544
+
+
+# ----------------------------------------------------------------- P4: Lemma 1, exhaustive
+def test_e4m3_set_definition():
+    # integers M*2^e with |M| <= 15 and magnitude at most 448
+    want = set()
+    for mant in range(-15, 16):
+        for e in range(0, 9):
+            v = mant * 2 ** e
+            if abs(v) <= 448:
+                want.add(v)
+    got = {v for v in range(-600, 601) if ozo.in_e4m3(v)}
+    assert got == want == {v for v in big.e4m3_integers() if abs(v) <= 600}
+    for v in sorted(want):
+        code = ozo.e4m3_encode(v)
+        assert 0 <= code < 256 and ozo.e4m3_value(code) == v
+    assert ozo.e4m3_encode(0) == 0
+    assert not any(ozo.in_e4m3(v) for v in (17, 19, 21, 23, -17, 449))
+    # a few codes fixed by the format itself: 1.0 = 0x38, 448 = 0x7E, -2 = 0xC0
+    assert ozo.e4m3_value(0x38) == 1.0 and ozo.e4m3_value(0x7E) == 448.0
+    assert ozo.e4m3_value(0xC0) == -2.0 and ozo.e4m3_value(0x01) == 2.0 ** -9
+
+
+@pytest.mark.parametrize("m", [487, 491, 499, 503, 509, 511])
+def test_lemma1_exhaustive(m):
+    lo, hi = -(m // 2), (m - 1) // 2
+    planes = {d: ozo.split(d, m) for d in range(lo, hi + 1)}
+    carries = 0
+    for d, (d0, d1, ds) in planes.items():
+        assert d == d0 + 16 * d1 and ds == d0 + d1
+        assert all(ozo.in_e4m3(v) for v in (d0, d1, ds))
+        assert abs(d0) <= int(PAPER["lemma1_d0_max"])
+        assert abs(d1) <= int(PAPER["lemma1_d1_max"])
+        assert abs(ds) <= int(PAPER["lemma1_sum_max"])
+        canon0 = (d + 8) % 16 - 8
+        if d0 != canon0:
+            carries += 1
+            assert abs(canon0 + (d - canon0) // 16) in [int(v) for v in PAPER["lemma1_failing_sums"].split()]
+        assert planes[d] == big.split(d, m)
+    if m == 511:
+        assert carries == int(PAPER["lemma1_carries_at_511"])
+    worst_prod = worst_merged = 0
+    for d, (d0, d1, ds) in planes.items():
+        for e, (e0, e1, es) in planes.items():
+            assert d * e == -15 * d0 * e0 + 16 * ds * es + 240 * d1 * e1          # Eq. 8
+            assert d * e == -15 * (d0 * e0 - 16 * d1 * e1) + 16 * ds * es          # merged form
+            worst_prod = max(worst_prod, abs(d0 * e0), abs(ds * es), abs(d1 * e1))
+            worst_merged = max(worst_merged, abs(d0 * e0 - 16 * d1 * e1))
+    assert worst_prod <= int(PAPER["lemma1_product_max"])
+    assert worst_merged <= int(PAPER["merged_term_max"])
+    if m == 511:
+        assert worst_prod == int(PAPER["lemma1_product_max"])
+    assert 2 ** 24 // int(PAPER["lemma1_product_max"]) == int(PAPER["lemma1_K_exact"])
+    assert 2 ** 24 // int(PAPER["merged_term_max"]) == int(PAPER["merged_K_exact"])
+
+
+def test_lemma1_is_sharp_at_513():
+    def rule(d):
+        d0 = (d + 8) % 16 - 8
+        d1 = (d - d0) // 16
+        if not ozo.in_e4m3(d0 + d1):
+            sg = (d0 > 0) - (d0 < 0)
+            d0, d1 = d0 - 16 * sg, d1 + sg
+        return d0, d1
+    for m, ok in ((513, True), (514, False)):
+        good = all(all(ozo.in_e4m3(v) for v in (*rule(d), sum(rule(d))))
+                   for d in range(-(m // 2), (m - 1) // 2 + 1))
+        assert good == ok
+
+
+def test_byte_moduli_never_carry():
+    lo_s, hi_s = [int(v) for v in PAPER["byte_modulus_sum_range"].split()]
+    for m in ozo.modset(ozo.SET_E)[6:]:
+        for d in range(-(m // 2), (m - 1) // 2 + 1):
+            d0, d1, ds = ozo.split(d, m)
+            assert d0 == (d + 8) % 16 - 8 and d == d0 + 16 * d1
+            assert abs(d0) <= 8 and abs(d1) <= int(PAPER["byte_modulus_digit_max"])
+            assert lo_s <= ds <= hi_s
+
+
+# ----------------------------------------------------------------- P5: squares
+@pytest.mark.parametrize("m", [1089, 1024, 961, 841, 625, 529])
+def test_square_split_exhaustive(m):
+    s = math.isqrt(m)
+    lo, hi = -(m // 2), (m - 1) // 2
+    digs = {d: ozo.split(d, m) for d in range(lo, hi + 1)}
+    worst = 0
+    for d, (d0, d1) in digs.items():
+        assert d == d0 + s * d1
+        assert ozo.in_e4m3(d0) and ozo.in_e4m3(d1)
+        worst = max(worst, abs(d0), abs(d1))
+        assert digs[d] == big.split(d, m)
+        if s % 2 == 0:
+            assert -s // 2 <= d0 <= s // 2 - 1
+    assert worst <= int(PAPER["square_digit_max"])
+    if m == 1089:
+        assert worst == int(PAPER["square_digit_max"])          # "exactly tight at s=33"
+    vals = list(digs.items())[:: max(1, len(digs) // 257)] + [(lo, digs[lo]), (hi, digs[hi])]
+    for d, (d0, d1) in vals:
+        for e, (e0, e1) in digs.items():
+            assert (d * e - (d0 * e0 + s * (d1 * e0 + d0 * e1))) % m == 0   # epilogue {1,s,s}
+
+
+# ----------------------------------------------------------------- P6: CRT round trip
+@pytest.mark.parametrize("name", ["S", "E"])
+def test_crt_round_trip(name):
+    ms = ozo.modset(SETS[name])
+    M = math.prod(ms)
+    w = ozo.garner_constants(SETS[name])
+    for j in range(1, len(ms)):
+        assert (w[j] * math.prod(ms[:j])) % ms[j] == 1 and 0 < w[j] < ms[j]
+    rng = random.Random(11)
+    xs = [0, 1, -1, -(M // 2), (M - 1) // 2, M // 2 - 1, -(M // 2) + 1, 12345678901234567890]
+    xs += [rng.randrange(-(M // 2), (M + 1) // 2) for _ in range(400)]
+    xs += [rng.randrange(-2**b, 2**b) for b in range(1, 110, 9)]
+    for x in xs:
+        res = [x % m for m in ms]
+        assert ozo.crt_single(SETS[name], res) == x
+        assert big.garner(res, ms) == x
+
+
+def test_int128_to_double_is_correctly_rounded():
+    rng = random.Random(5)
+    xs = [0, 1, -1, 2**53, 2**53 + 1, 2**53 + 2, 2**53 + 3, -(2**53 + 1), 2**54 + 2, 2**54 + 6,
+          2**100 + 2**47, 2**100 + 2**47 + 1, 2**100 + 3 * 2**47, -(2**110) - 2**57, 2**112 - 1]
+    xs += [rng.randrange(-2**b, 2**b) for b in range(40, 120) for _ in range(25)]
+    for x in xs:
+        assert ozo.i128_to_double(x) == float(x), x   # Python's int -> float is RN-even
+
+
+# ----------------------------------------------------------------- quantiser / shifts
+def test_quantiser_against_exact_rationals():
+    rng = np.random.default_rng(2)
+    xs = np.concatenate([rng.standard_normal(200) * 10.0 ** rng.integers(-30, 30, 200),
+                         [0.0, -0.0, 5e-324, -5e-324, 2.0**-1040, 1.5, 2.5, -2.5, 0.5, -0.5, 3.5]])
+    for sigma in (-80, -3, 0, 1, 40, 52, 1074):
+        for x in xs:
+            X = np.asfortranarray(np.array([[x]]))
+            sh = np.array([sigma], dtype=np.int32)
+            v = Fraction(float(x)) * Fraction(2) ** sigma
+            if abs(v) >= 2**62:
+                continue
+            assert int(ozo.quantise(0, X, sh, ozo.QUANT_RN)[0, 0]) == round(v)
+            assert int(ozo.quantise(0, X, sh, ozo.QUANT_TZ)[0, 0]) == int(v)
+    # ties go to even
+    X = np.asfortranarray(np.array([[0.5, 1.5, 2.5, -0.5, -1.5]]))
+    q = ozo.quantise(0, X, np.zeros(1, dtype=np.int32), ozo.QUANT_RN)
+    assert q.tolist() == [[0, 2, 2, 0, -2]]
+
+
+@pytest.mark.parametrize("rule", ["MAXEXP", "CS"])
+@pytest.mark.parametrize("name", ["S", "E"])
+def test_shifts_keep_product_in_range(rule, name):
+    rng = np.random.default_rng(9)
+    ms = ozo.modset(SETS[name])
+    M = math.prod(ms)
+    m, n, k = 9, 7, 33
+    A = np.asfortranarray((rng.random((m, k)) - 0.5) * np.exp(3 * rng.standard_normal((m, k))))
+    B = np.asfortranarray((rng.random((k, n)) - 0.5) * np.exp(3 * rng.standard_normal((k, n))))
+    A[3, :] = A[3, 0]            # parallel row/column: the Cauchy-Schwarz bound is tight
+    B[:, 2] = A[3, 0]
+    A[5, 1:] = 0.0               # a single nonzero
+    tA, tB = ozo.budget_maxexp(SETS[name], k)
+    r = ozo.SCALE_MAXEXP if rule == "MAXEXP" else ozo.SCALE_CS
+    sA = ozo.shifts(0, A, SETS[name], r, tA)
+    sB = ozo.shifts(1, B, SETS[name], r, tB)
+    for i in range(m):
+        assert sA[i] == big.shift_of_line(A[i, :].tolist(), ms, rule, tA, k)
+    for j in range(n):
+        assert sB[j] == big.shift_of_line(B[:, j].tolist(), ms, rule, tB, k)
+    for quant in (ozo.QUANT_RN, ozo.QUANT_TZ):
+        QA = ozo.quantise(0, A, sA, quant).astype(object)
+        QB = ozo.quantise(1, B, sB, quant).astype(object)
+        Cp = QA @ QB.T
+        assert max(abs(int(v)) for v in Cp.ravel()) <= (M - 1) // 2
+        if rule == "MAXEXP":
+            assert max(abs(int(v)) for v in QA.ravel()) <= 2**tA
+            assert max(abs(int(v)) for v in QB.ravel()) <= 2**tB
+            # the shift is the largest allowed: the top entry of a line uses bit t-1
+            assert all(max(abs(int(v)) for v in QA[i]) >= 2**(tA - 1) for i in range(m))
+
+
+# ----------------------------------------------------------------- P7: brute force / big ints
+@pytest.mark.parametrize("name,quant,rule", [("S", "RN", "CS"), ("S", "TZ", "MAXEXP"),
+                                             ("E", "RN", "MAXEXP"), ("E", "TZ", "CS")])
+def test_whole_method_against_big_integers(name, quant, rule):
+    rng = np.random.default_rng(21)
+    m, n, k = 5, 4, 19
+    A = np.asfortranarray((rng.random((m, k)) - 0.5) * np.exp(2 * rng.standard_normal((m, k))))
+    B = np.asfortranarray((rng.random((k, n)) - 0.5) * np.exp(2 * rng.standard_normal((k, n))))
+    A[2, 3] = 0.0
+    q = ozo.QUANT_RN if quant == "RN" else ozo.QUANT_TZ
+    r = ozo.SCALE_CS if rule == "CS" else ozo.SCALE_MAXEXP
+    Cm, sA, sB, R = ozo.dgemm(A, B, SETS[name], q, r, want_stages=True)
+    Cf, sig, tau, Rb, Cint = big.dgemm(A.tolist(), B.tolist(), name, quant, rule)
+    assert sA.tolist() == sig and sB.tolist() == tau
+    assert R.tolist() == Rb
+    assert Cm.tolist() == Cf
+    # the residue path equals the plain 128-bit product A'B' (CRT uniqueness)
+    QA = ozo.quantise(0, A, sA, q)
+    QB = ozo.quantise(1, B, sB, q)
+    assert (ozo.crt(R, SETS[name], as_int=True) == ozo.direct(QA, QB, as_int=True)).all()
+    assert ozo.direct(QA, QB, as_int=True).tolist() == Cint
+
+
+@pytest.mark.parametrize("name,sub", [("S", ozo.SUB_FP8), ("S", ozo.SUB_INT8), ("E", ozo.SUB_FP8)])
+def test_planes_reproduce_residue_products(name, sub):
+    rng = np.random.default_rng(4)
+    m, n, k = 6, 5, 37
+    ms = ozo.modset(SETS[name])
+    QA = rng.integers(-2**50, 2**50, size=(m, k))
+    QB = rng.integers(-2**50, 2**50, size=(n, k))
+    QA[0, :] = [(-1) ** i * (ms[i % len(ms)] // 2) for i in range(k)]   # endpoint residues
+    DA, DB = ozo.residues(QA, SETS[name]), ozo.residues(QB, SETS[name])
+    for i, mm in enumerate(ms):
+        assert ((DA[i].astype(np.int64) - QA) % mm == 0).all()
+        assert (2 * DA[i].astype(np.int64) >= -mm).all() and (2 * DA[i].astype(np.int64) < mm).all()
+    PA, PB = ozo.planes(DA, SETS[name], sub), ozo.planes(DB, SETS[name], sub)
+    assert PA.shape == (ozo.pstore(SETS[name]), m, 48) and (PA[:, :, k:] == 0).all()
+    R1 = ozo.products(DA, DB, SETS[name])
+    R2, worst = ozo.plane_products(PA, PB, k, SETS[name], sub)
+    assert (R1 == R2).all() and worst <= 2 * 256 * k
+    want = (QA.astype(object) @ QB.astype(object).T)
+    for i, mm in enumerate(ms):
+        assert (R1[i].T.astype(object) == want % mm).all()
+
+
+# ----------------------------------------------------------------- P10: reduces to an exact product
+def test_exact_on_small_integers():
+    A, B = syn.special_operands("small_integers", 12, 10, 64)
+    want = (A.astype(np.int64).astype(object) @ B.astype(np.int64).astype(object))
+    for name in ("S", "E"):
+        for quant in (ozo.QUANT_RN, ozo.QUANT_TZ):
+            for rule in (ozo.SCALE_MAXEXP, ozo.SCALE_CS):
+                Cm = ozo.dgemm(A, B, SETS[name], quant, rule)
+                assert (Cm == want.astype(np.float64)).all()
+    assert (A @ B == want.astype(np.float64)).all()       # and so does plain FP64 here
+
+
+# ----------------------------------------------------------------- P8: accuracy vs the true product
+def _dd_exact(A, B):
+    m, k = A.shape
+    n = B.shape[1]
+    out = np.empty((m, n), dtype=object)
+    for i in range(m):
+        for j in range(n):
+            out[i, j] = sum(Fraction(A[i, t]) * Fraction(B[t, j]) for t in range(k))
+    return out
+
+
+def test_double_double_reference_is_accurate():
+    rng = np.random.default_rng(8)
+    A = np.asfortranarray(rng.standard_normal((4, 50)) * np.exp(4 * rng.standard_normal((4, 50))))
+    B = np.asfortranarray(rng.standard_normal((50, 3)))
+    hi, lo, ab = ozo.dd_gemm(A, B)
+    ex = _dd_exact(A, B)
+    exab = _dd_exact(np.abs(A), np.abs(B))
+    for i in range(4):
+        for j in range(3):
+            err = abs(Fraction(hi[i, j]) + Fraction(lo[i, j]) - ex[i, j])
+            assert err <= Fraction(2) ** -100 * exab[i, j]
+            assert abs(Fraction(ab[i, j]) - exab[i, j]) <= Fraction(2) ** -50 * exab[i, j]
+
+
+@pytest.mark.parametrize("cfg_id,scale", [(1, 1.0), (2, 1.0), (3, 1.0), (4, 1.0)])
+def test_rn_error_bound_and_fp64_grade(cfg_id, scale):
+    """Derived a-priori bound for round-to-nearest (from Eq. 1):
+         |2^(s_i+t_j) (AB)_ij - c'_ij| <= 1/2 sum|a'| + 1/2 sum|b'| + k/4
+       and, with the CS rule, the result is within 2 u (|A||B|)_ij of the true product
+       on the well-scaled configurations."""
+    cfg = syn.CONFIGS[cfg_id]
+    m, n, k = 24, 20, min(cfg.k, 1024)
+    A, B = syn.operands(cfg, m, n, k)
+    s = SETS[cfg.sets[0]]
+    Cm, sA, sB, R = ozo.dgemm(A, B, s, ozo.QUANT_RN, ozo.SCALE_CS, want_stages=True)
+    QA = ozo.quantise(0, A, sA, ozo.QUANT_RN).astype(object)
+    QB = ozo.quantise(1, B, sB, ozo.QUANT_RN).astype(object)
+    Cp = ozo.crt(R, s, as_int=True)
+    ex = _dd_exact(A, B)
+    exab = _dd_exact(np.abs(A), np.abs(B))
+    hi, lo, ab = ozo.dd_gemm(A, B)
+    u = Fraction(2) ** -53
+    worst = Fraction(0)
+    for i in range(m):
+        for j in range(n):
+            scaled = ex[i, j] * Fraction(2) ** int(sA[i] + sB[j])
+            bound = Fraction(sum(abs(v) for v in QA[i]) + sum(abs(v) for v in QB[j]), 2) + Fraction(k, 4)
+            assert abs(scaled - int(Cp[i, j])) <= bound
+            err = abs(Fraction(Cm[i, j]) - ex[i, j])
+            worst = max(worst, err / (2 * u * exab[i, j]))
+            assert abs(Fraction(hi[i, j]) + Fraction(lo[i, j]) - ex[i, j]) <= u * u * 4 * exab[i, j]
+    assert worst <= 1
+
+
+# ----------------------------------------------------------------- edge inputs
+def test_zero_lines_subnormals_spikes_and_nonfinite():
+    for kind in ("zero_lines", "subnormal", "spike"):
+        A, B = syn.special_operands(kind, 8, 6, 24)
+        for rule in (ozo.SCALE_MAXEXP, ozo.SCALE_CS):
+            Cm, sA, sB, R = ozo.dgemm(A, B, ozo.SET_S, ozo.QUANT_RN, rule, want_stages=True)
+            Cf, sig, tau, Rb, _ = big.dgemm(A.tolist(), B.tolist(), "S", "RN",
+                                            "CS" if rule == ozo.SCALE_CS else "MAXEXP")
+            assert sA.tolist() == sig and sB.tolist() == tau and R.tolist() == Rb
+            assert Cm.tolist() == Cf
+            if kind == "zero_lines":
+                assert (Cm[4, :] == 0).all() and (Cm[:, 2] == 0).all() and sA[4] == 0 and sB[2] == 0
+    A, B = syn.special_operands("spike", 8, 6, 24)
+    A[2, 5] = np.inf
+    B[7, 1] = np.nan
+    Cm, sA, sB, _ = ozo.dgemm(A, B, want_stages=True)
+    assert sA[2] == ozo.NONFINITE_SHIFT and sB[1] == ozo.NONFINITE_SHIFT
+    assert np.isnan(Cm[2, :]).all() and np.isnan(Cm[:, 1]).all()
+    mask = np.ones_like(Cm, dtype=bool)
+    mask[2, :] = False
+    mask[:, 1] = False
+    assert np.isfinite(Cm[mask]).all()
+
+
+def test_update_form_and_empty_shapes():
+    cfg = syn.CONFIGS[3]
+    A, B, C0 = syn.operands(cfg, 16, 12, 32, want_c=True)
+    P = ozo.dgemm(A, B, ozo.SET_E)
+    Cm = ozo.dgemm(A, B, ozo.SET_E, alpha=-1.0, beta=1.0, C0=C0)
+    assert (Cm == C0 - P).all()
+    Z = ozo.dgemm(np.zeros((3, 0), order="F"), np.zeros((0, 2), order="F"))
+    assert Z.shape == (3, 2) and (Z == 0).all()
+    assert ozo.dgemm(np.zeros((0, 4), order="F"), np.zeros((4, 2), order="F")).shape == (0, 2)
