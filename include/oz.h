@@ -1,0 +1,153 @@
+/*
+ * oz.h -- C ABI of the B200 (sm_100a) Ozaki Scheme II emulated-FP64 GEMM library.
+ *
+ * The library computes C = A B for FP64 matrices through exact integer residue
+ * arithmetic on the FP8 / INT8 tensor cores (paper Sec. 2, "The scheme in
+ * equations", Eq. 1-5, and "The FP8 variant", Eq. 6-7):
+ *   1. deconstruction (Algorithm 2): per-row / per-column power-of-two scaling, quantisation
+ *      to integers, centred residues modulo each modulus of the set, two-limb digit
+ *      split with the carry of Lemma 1, stored as K-major 8-bit planes;
+ *   2. residue products (Algorithm 1, the loop over moduli): three exact plane GEMMs per modulus,
+ *      combined and reduced modulo m_i in the epilogue (Eq. 8 for non-squares,
+ *      weights {1,s,s} for squares m = s^2);
+ *   3. reconstruction (Algorithm 3, Eq. 4-5): CRT, lift to [-M/2, M/2), inverse scaling,
+ *      one rounding to FP64.
+ *
+ * General conventions
+ *   - Matrices are column-major, no transposes: A is m x k (lda >= m), B is k x n
+ *     (ldb >= k), C is m x n (ldc >= m).
+ *   - Every pointer is a DEVICE pointer owned by the caller unless a comment says
+ *     "host".  The library never allocates or frees device memory; scratch comes
+ *     from the workspace registered with oz_set_workspace().
+ *   - All work is enqueued on `stream` (a cudaStream_t passed as void*; NULL is the
+ *     default stream).  No call synchronises the host except oz_query_status().
+ *   - Host-detectable errors return at once with nothing enqueued.  Conditions
+ *     found on the device (non-finite input, a bounded wait that ran out) set a
+ *     sticky per-device status word that oz_query_status() returns and clears.
+ *     Kernels never trap and never spin without a limit.
+ *   - m, n or k equal to zero is OZ_OK (k = 0 gives C = 0, or C unchanged for beta = 1).
+ *   - Non-finite contract: an Inf or NaN anywhere in row i of A (column j of B)
+ *     makes every C(i,:) (C(:,j)) NaN and sets OZ_ERR_NONFINITE_INPUT.
+ *   - k is limited to OZ_K_MAX, the depth to which the FP32 accumulators of the FP8
+ *     route stay exact (Lemma 1 and the accumulation invariant of Algorithm 2).
+ */
+#ifndef OZ_H_
+#define OZ_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    OZ_OK = 0,
+    OZ_ERR_INVALID_ARG = 1,     /* null pointer, negative size, bad leading dimension, bad enum */
+    OZ_ERR_UNSUPPORTED = 2,     /* k > OZ_K_MAX, alpha/beta outside {+-1}/{0,1}                 */
+    OZ_ERR_WORKSPACE = 3,       /* no workspace registered, or it is too small                  */
+    OZ_ERR_CUDA = 4,            /* a CUDA runtime / driver call failed                          */
+    OZ_ERR_NONFINITE_INPUT = 5, /* device: Inf/NaN met in an operand                            */
+    OZ_ERR_RANGE = 6,           /* device: a quantised value left the representable range       */
+    OZ_ERR_TIMEOUT = 7          /* device: a bounded barrier wait ran out                       */
+} oz_status_t;
+
+/* Modulus sets: S = the published 12-modulus set (Sec. 2, step (ii));
+ * E = the hybrid set, six squares of S plus seven byte moduli ("Candidate E"). */
+typedef enum { OZ_SET_S = 0, OZ_SET_E = 1 } oz_modset_t;
+
+/* route bit field: one substrate, one quantiser, one scale rule (0 picks the default) */
+#define OZ_SUB_FP8      0x001u  /* planes are E4M3 bytes, FP32 accumulation (default)          */
+#define OZ_SUB_INT8     0x002u  /* same digits as two's-complement bytes, INT32 accumulation   */
+#define OZ_QUANT_RN     0x010u  /* round to nearest, ties to even (variant Ozaki-II-RN, default) */
+#define OZ_QUANT_TZ     0x020u  /* truncate toward zero (variant Ozaki-II-TZ)                  */
+#define OZ_SCALE_MAXEXP 0x100u  /* shift from the largest exponent of the line (Eq. 2 read literally) */
+#define OZ_SCALE_CS     0x200u  /* shift from the 2-norm of the line, Cauchy-Schwarz bound (default) */
+
+#define OZ_K_MAX 32768
+#define OZ_NONFINITE_SHIFT INT32_MIN  /* value of shift[] for a line that holds Inf/NaN */
+
+/* Number of moduli r and of stored planes p_store of a set (Table "tuples": 12/30, 13/33).
+ * Returns OZ_ERR_INVALID_ARG for an unknown set.  `moduli` (host, may be NULL) receives r ints. */
+oz_status_t oz_set_info(oz_modset_t set, int *r, int *p_store, int *moduli);
+
+/* Pitch in bytes of one plane row for inner dimension k: k rounded up to 16 (TMA stride rule). */
+int64_t oz_row_pitch(int64_t k);
+
+/* Bytes of scratch that oz_dgemm needs for this shape (planes of A and B, residues, shifts). */
+size_t oz_workspace_bytes(int64_t m, int64_t n, int64_t k, oz_modset_t set, uint32_t route);
+
+/* Register caller-owned device scratch (256-byte aligned) for oz_dgemm / oz_dgemm_ex on the
+ * current device.  The library keeps only the pointer; the caller frees it after the last call
+ * has finished.  Passing NULL unregisters. */
+oz_status_t oz_set_workspace(void *workspace, size_t bytes);
+
+/* C = A B  (Sec. 2: the whole method).  Needs a registered workspace of at least
+ * oz_workspace_bytes().  Kernels launched: scan, deconstruct (A and B), residue GEMM, reconstruct. */
+oz_status_t oz_dgemm(int64_t m, int64_t n, int64_t k, const double *A, int64_t lda,
+                     const double *B, int64_t ldb, double *C, int64_t ldc, oz_modset_t set,
+                     uint32_t route, void *stream);
+
+/* C = beta C + alpha A B with alpha in {+1,-1}, beta in {0,1} (the HPL trailing update
+ * C <- C - A B of Sec. "HPL" is alpha = -1, beta = 1).  With beta = 1 the result carries two
+ * roundings: the method's single rounding of the product, then the FP64 addition. */
+oz_status_t oz_dgemm_ex(int64_t m, int64_t n, int64_t k, double alpha, const double *A,
+                        int64_t lda, const double *B, int64_t ldb, double beta, double *C,
+                        int64_t ldc, oz_modset_t set, uint32_t route, void *stream);
+
+/* Same as oz_dgemm_ex but A, B, C are HOST pointers (pinned memory recommended).  The operands
+ * are copied to staging areas inside the registered workspace, which must hold
+ * oz_workspace_bytes() + 8 (m k + k n + m n) bytes, and C is copied back; the call returns after
+ * enqueueing (the host buffers must stay valid until the stream has drained). */
+oz_status_t oz_dgemm_host(int64_t m, int64_t n, int64_t k, double alpha, const double *A_host,
+                          int64_t lda, const double *B_host, int64_t ldb, double beta,
+                          double *C_host, int64_t ldc, oz_modset_t set, uint32_t route,
+                          void *stream);
+
+/* Deconstruction of one operand (Algorithm 2; scaling of Eq. 1).
+ *   side 0: X is m x k column-major, lines = m rows,    element (i,kk) at X[i + kk*ldx]
+ *   side 1: X is k x n column-major, lines = n columns, element (kk,j) at X[kk + j*ldx]
+ * Outputs: shift[lines] (int32; sigma_i or tau_j of Eq. 1, OZ_NONFINITE_SHIFT for a line with
+ * Inf/NaN) and p_store planes, plane p / line l / inner index kk at
+ *   planes[p*plane_stride + l*row_pitch + kk],
+ * in the set's modulus order, plane order d0, d1[, d0+d1] per modulus; bytes kk in [k,row_pitch)
+ * are written as zero.  row_pitch >= k and plane_stride >= lines*row_pitch, both multiples of 16;
+ * `planes` 16-byte aligned.  `scratch` is 16*lines + 256 bytes of device memory (256-byte aligned). */
+oz_status_t oz_deconstruct(int side, int64_t lines, int64_t k, const double *X, int64_t ldx,
+                           oz_modset_t set, uint32_t route, uint8_t *planes,
+                           int64_t plane_stride, int64_t row_pitch, int32_t *shift,
+                           void *scratch, void *stream);
+
+/* Residue products (Eq. 3 through the plane identities of Sec. 2 "FP8 variant" and Eq. 8):
+ * for every modulus i,  R_i = (A_i B_i) mod m_i  from the stored planes of A (lines = m) and
+ * B (lines = n), on the tensor cores.  Output R[i*mod_stride + j*ldr + row], uint16 in [0, m_i).
+ * ldr >= m, mod_stride >= n*ldr (in elements).  Planes as written by oz_deconstruct with the
+ * same set and substrate; plane bases 16-byte aligned, pitches and strides multiples of 16. */
+oz_status_t oz_residue_gemm(int64_t m, int64_t n, int64_t k, const uint8_t *PA,
+                            int64_t plane_strideA, int64_t row_pitchA, const uint8_t *PB,
+                            int64_t plane_strideB, int64_t row_pitchB, oz_modset_t set,
+                            uint32_t route, uint16_t *R, int64_t ldr, int64_t mod_stride,
+                            void *stream);
+
+/* Reconstruction (Algorithm 3; Eq. 4-5 and the final step of Sec. 2 (iv)): the integer
+ * c'_ij in [-M/2, M/2) congruent to the residues, times 2^-(shiftA[i]+shiftB[j]), rounded once;
+ * C = alpha P (beta = 0) or C = C + alpha P (beta = 1).  The CRT is evaluated exactly. */
+oz_status_t oz_reconstruct(int64_t m, int64_t n, const uint16_t *R, int64_t ldr,
+                           int64_t mod_stride, const int32_t *shiftA, const int32_t *shiftB,
+                           oz_modset_t set, double alpha, double beta, double *C, int64_t ldc,
+                           void *stream);
+
+/* Synchronises `stream`, then returns and clears the device status word of the current device
+ * (OZ_OK, OZ_ERR_NONFINITE_INPUT, OZ_ERR_RANGE, OZ_ERR_TIMEOUT or OZ_ERR_CUDA). */
+oz_status_t oz_query_status(void *stream);
+
+/* Number of kernels launched by the library on this process since load (for benchmarks). */
+uint64_t oz_launch_count(void);
+
+/* Human-readable name of a status code (host string, never NULL). */
+const char *oz_status_string(oz_status_t status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* OZ_H_ */

@@ -1,0 +1,443 @@
+// C-ABI entry points of liboz_b200.so: argument checks, per-device set-up, workspace carving
+// and the oz_dgemm driver (Algorithm 1 reduced to materialised planes and three stages).
+#include <atomic>
+#include <cmath>
+#include <mutex>
+
+#include "oz_internal.h"
+
+namespace oz {
+
+// ------------------------------------------------------------------------------------------
+// per-device objects: plane lookup tables and the sticky status word
+// ------------------------------------------------------------------------------------------
+__device__ uint32_t g_lut[2][2][kLutWords];
+__device__ unsigned int g_status[4];
+
+namespace {
+
+constexpr int kMaxDevices = 64;
+std::mutex g_mutex;
+bool g_ready[kMaxDevices] = {};
+const uint32_t *g_lut_addr[kMaxDevices] = {};
+unsigned int *g_status_addr[kMaxDevices] = {};
+void *g_workspace[kMaxDevices] = {};
+size_t g_workspace_bytes[kMaxDevices] = {};
+std::atomic<uint64_t> g_launches{0};
+
+// Is the integer v exactly representable in E4M3 (the set of Lemma 1)?  If so return its
+// byte code through *code.  OCP E4M3: bias 7, 3 mantissa bits, largest finite value 448.
+bool e4m3_code(int v, int *code)
+{
+    if (v == 0) { *code = 0; return true; }
+    int a = v < 0 ? -v : v;
+    if (a > 448) return false;
+    int e = 0;
+    while ((2 << e) <= a) ++e;              // e = floor(log2 a)
+    int scaled = a << 3;                     // a * 8
+    if (scaled % (1 << e) != 0) return false;
+    int mant = (scaled >> e) - 8;            // 0..7
+    *code = ((v < 0) ? 0x80 : 0) | ((e + 7) << 3) | mant;
+    return true;
+}
+
+int floor_mod(int a, int b) { int r = a % b; return r < 0 ? r + b : r; }
+
+// Packed plane bytes of the canonical residue u of modulus m (Algorithm 2, split lines):
+// byte 0 = d0, byte 1 = d1, byte 2 = d0+d1 (zero for a square modulus).
+uint32_t lut_entry(int u, int m, int substrate)
+{
+    int d = (2 * u >= m) ? u - m : u;        // centred, -m/2 included
+    int s = square_root(m);
+    int dig[3] = {0, 0, 0};
+    if (s) {
+        int half = s / 2;
+        dig[0] = floor_mod(d + half, s) - half;
+        dig[1] = (d - dig[0]) / s;
+    } else {
+        dig[0] = floor_mod(d + 8, 16) - 8;
+        dig[1] = (d - dig[0]) / 16;
+        int code;
+        if (!e4m3_code(dig[0] + dig[1], &code)) {        // Lemma 1: one predicated carry
+            int sg = (dig[0] > 0) - (dig[0] < 0);
+            dig[0] -= 16 * sg;
+            dig[1] += sg;
+        }
+        dig[2] = dig[0] + dig[1];
+    }
+    uint32_t word = 0;
+    for (int q = 0; q < 3; ++q) {
+        int byte = 0;
+        if (substrate == 0) e4m3_code(dig[q], &byte);
+        else byte = dig[q] & 0xFF;
+        word |= static_cast<uint32_t>(byte) << (8 * q);
+    }
+    return word;
+}
+
+unsigned __int128 set_product(int set)
+{
+    unsigned __int128 M = 1;
+    for (int i = 0; i < set_r(set); ++i) M *= static_cast<unsigned>(modulus(set, i));
+    return M;
+}
+
+uint64_t isqrt_u128(unsigned __int128 v)
+{
+    uint64_t r = static_cast<uint64_t>(sqrtl(static_cast<long double>(v)));
+    while (static_cast<unsigned __int128>(r) * r > v) --r;
+    while (static_cast<unsigned __int128>(r + 1) * (r + 1) <= v) ++r;
+    return r;
+}
+
+}  // namespace
+
+bool decode_route(uint32_t route, Route *out)
+{
+    uint32_t sub = route & 0x00Fu, q = route & 0x0F0u, sc = route & 0xF00u;
+    if (route & ~0xFFFu) return false;
+    if (sub == 0 || sub == OZ_SUB_FP8) out->substrate = 0;
+    else if (sub == OZ_SUB_INT8) out->substrate = 1;
+    else return false;
+    if (q == 0 || q == OZ_QUANT_RN) out->quant = 0;
+    else if (q == OZ_QUANT_TZ) out->quant = 1;
+    else return false;
+    if (sc == 0 || sc == OZ_SCALE_CS) out->rule = 1;
+    else if (sc == OZ_SCALE_MAXEXP) out->rule = 0;
+    else return false;
+    return true;
+}
+
+void budget_maxexp(int set, int64_t k, int *tA, int *tB)
+{
+    unsigned __int128 v = (set_product(set) - 1) / 2 / static_cast<unsigned __int128>(k > 0 ? k : 1);
+    int T = -1;
+    while (v) { ++T; v >>= 1; }
+    *tB = T / 2;
+    *tA = T - T / 2;
+}
+
+void cs_bound_squared(int set, int64_t k, uint64_t *lo, uint64_t *hi)
+{
+    uint64_t bnd = isqrt_u128((set_product(set) - 1) / 2);
+    uint64_t kk = static_cast<uint64_t>(k > 0 ? k : 1);
+    uint64_t s = isqrt_u128(kk);
+    uint64_t g = (s * s == kk) ? (s + 1) / 2 : s / 2 + 1;   // ceil(sqrt(k)/2)
+    unsigned __int128 G = bnd - g;
+    unsigned __int128 G2 = G * G;
+    *lo = static_cast<uint64_t>(G2);
+    *hi = static_cast<uint64_t>(G2 >> 64);
+}
+
+oz_status_t ensure_device_ready()
+{
+    int dev = 0;
+    OZ_CUDA_CHECK(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return OZ_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(g_mutex);
+    if (g_ready[dev]) return OZ_OK;
+    static uint32_t host_lut[2][2][kLutWords];
+    for (int set = 0; set < 2; ++set)
+        for (int sub = 0; sub < 2; ++sub) {
+            int off = 0;
+            for (int i = 0; i < set_r(set); ++i) {
+                int m = modulus(set, i);
+                for (int u = 0; u < m; ++u) host_lut[set][sub][off + u] = lut_entry(u, m, sub);
+                off += m;
+            }
+            for (; off < kLutWords; ++off) host_lut[set][sub][off] = 0;
+        }
+    OZ_CUDA_CHECK(cudaMemcpyToSymbol(g_lut, host_lut, sizeof(host_lut)));
+    unsigned int zero[4] = {0, 0, 0, 0};
+    OZ_CUDA_CHECK(cudaMemcpyToSymbol(g_status, zero, sizeof(zero)));
+    void *p = nullptr;
+    OZ_CUDA_CHECK(cudaGetSymbolAddress(&p, g_lut));
+    g_lut_addr[dev] = static_cast<const uint32_t *>(p);
+    OZ_CUDA_CHECK(cudaGetSymbolAddress(&p, g_status));
+    g_status_addr[dev] = static_cast<unsigned int *>(p);
+    oz_status_t st = upload_reconstruct_constants();
+    if (st != OZ_OK) return st;
+    g_ready[dev] = true;
+    return OZ_OK;
+}
+
+const uint32_t *device_lut(int set, int substrate)
+{
+    int dev = 0;
+    cudaGetDevice(&dev);
+    return g_lut_addr[dev] + (static_cast<size_t>(set) * 2 + substrate) * kLutWords;
+}
+
+unsigned int *device_status_word()
+{
+    int dev = 0;
+    cudaGetDevice(&dev);
+    return g_status_addr[dev];
+}
+
+void count_launch(int n) { g_launches.fetch_add(static_cast<uint64_t>(n)); }
+
+namespace {
+
+struct Carve {
+    size_t off = 0;
+    size_t take(size_t bytes)
+    {
+        size_t at = off;
+        off += static_cast<size_t>(round_up(static_cast<int64_t>(bytes), 256));
+        return at;
+    }
+};
+
+struct Layout {
+    size_t shiftA, shiftB, scrA, scrB, PA, PB, R, total;
+    int64_t pitch, strideA, strideB, ldr, mod_stride;
+};
+
+Layout make_layout(int64_t m, int64_t n, int64_t k, int set)
+{
+    Layout L{};
+    Carve c;
+    L.pitch = oz_row_pitch(k);
+    L.strideA = m * L.pitch;
+    L.strideB = n * L.pitch;
+    L.ldr = round_up(m, 8);
+    L.mod_stride = n * L.ldr;
+    L.shiftA = c.take(4 * static_cast<size_t>(m));
+    L.shiftB = c.take(4 * static_cast<size_t>(n));
+    L.scrA = c.take(16 * static_cast<size_t>(m) + 256);
+    L.scrB = c.take(16 * static_cast<size_t>(n) + 256);
+    L.PA = c.take(static_cast<size_t>(p_store(set)) * L.strideA);
+    L.PB = c.take(static_cast<size_t>(p_store(set)) * L.strideB);
+    L.R = c.take(2 * static_cast<size_t>(set_r(set)) * L.mod_stride);
+    L.total = c.off;
+    return L;
+}
+
+bool valid_set(int set) { return set == OZ_SET_S || set == OZ_SET_E; }
+
+oz_status_t dgemm_impl(int64_t m, int64_t n, int64_t k, double alpha, const double *A, int64_t lda,
+                       const double *B, int64_t ldb, double beta, double *C, int64_t ldc, int set,
+                       uint32_t route, cudaStream_t stream, char *ws, size_t ws_bytes)
+{
+    Route rt;
+    if (!valid_set(set) || !decode_route(route, &rt)) return OZ_ERR_INVALID_ARG;
+    if (m < 0 || n < 0 || k < 0) return OZ_ERR_INVALID_ARG;
+    if (!(alpha == 1.0 || alpha == -1.0) || !(beta == 0.0 || beta == 1.0)) return OZ_ERR_UNSUPPORTED;
+    if (k > OZ_K_MAX) return OZ_ERR_UNSUPPORTED;
+    if (m == 0 || n == 0) return OZ_OK;
+    if (!C || ldc < m) return OZ_ERR_INVALID_ARG;
+    if (k == 0) {
+        if (beta == 0.0)
+            OZ_CUDA_CHECK(cudaMemset2DAsync(C, sizeof(double) * ldc, 0, sizeof(double) * m, n, stream));
+        return OZ_OK;
+    }
+    if (!A || !B || lda < m || ldb < k) return OZ_ERR_INVALID_ARG;
+    Layout L = make_layout(m, n, k, set);
+    if (!ws || ws_bytes < L.total) return OZ_ERR_WORKSPACE;
+    oz_status_t st = ensure_device_ready();
+    if (st != OZ_OK) return st;
+
+    int32_t *shiftA = reinterpret_cast<int32_t *>(ws + L.shiftA);
+    int32_t *shiftB = reinterpret_cast<int32_t *>(ws + L.shiftB);
+    uint8_t *PA = reinterpret_cast<uint8_t *>(ws + L.PA);
+    uint8_t *PB = reinterpret_cast<uint8_t *>(ws + L.PB);
+    uint16_t *R = reinterpret_cast<uint16_t *>(ws + L.R);
+
+    st = launch_deconstruct(0, m, k, A, lda, set, rt, PA, L.strideA, L.pitch, shiftA, ws + L.scrA, stream);
+    if (st != OZ_OK) return st;
+    st = launch_deconstruct(1, n, k, B, ldb, set, rt, PB, L.strideB, L.pitch, shiftB, ws + L.scrB, stream);
+    if (st != OZ_OK) return st;
+    st = launch_residue_gemm(m, n, k, PA, L.strideA, L.pitch, PB, L.strideB, L.pitch, set, rt, R,
+                             L.ldr, L.mod_stride, stream);
+    if (st != OZ_OK) return st;
+    return launch_reconstruct(m, n, R, L.ldr, L.mod_stride, shiftA, shiftB, set, alpha, beta, C,
+                              ldc, stream);
+}
+
+}  // namespace
+}  // namespace oz
+
+using namespace oz;
+
+extern "C" {
+
+oz_status_t oz_set_info(oz_modset_t set, int *r, int *pstore, int *moduli)
+{
+    if (!valid_set(set)) return OZ_ERR_INVALID_ARG;
+    if (r) *r = set_r(set);
+    if (pstore) *pstore = p_store(set);
+    if (moduli)
+        for (int i = 0; i < set_r(set); ++i) moduli[i] = modulus(set, i);
+    return OZ_OK;
+}
+
+int64_t oz_row_pitch(int64_t k) { return round_up(k > 0 ? k : 1, 16); }
+
+size_t oz_workspace_bytes(int64_t m, int64_t n, int64_t k, oz_modset_t set, uint32_t route)
+{
+    Route rt;
+    if (!valid_set(set) || !decode_route(route, &rt) || m < 0 || n < 0 || k < 0) return 0;
+    return make_layout(m > 0 ? m : 1, n > 0 ? n : 1, k > 0 ? k : 1, set).total;
+}
+
+oz_status_t oz_set_workspace(void *workspace, size_t bytes)
+{
+    int dev = 0;
+    OZ_CUDA_CHECK(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return OZ_ERR_CUDA;
+    if (workspace && (reinterpret_cast<uintptr_t>(workspace) & 255u)) return OZ_ERR_INVALID_ARG;
+    std::lock_guard<std::mutex> lock(g_mutex);
+    g_workspace[dev] = workspace;
+    g_workspace_bytes[dev] = workspace ? bytes : 0;
+    return OZ_OK;
+}
+
+oz_status_t oz_dgemm_ex(int64_t m, int64_t n, int64_t k, double alpha, const double *A, int64_t lda,
+                        const double *B, int64_t ldb, double beta, double *C, int64_t ldc,
+                        oz_modset_t set, uint32_t route, void *stream)
+{
+    int dev = 0;
+    OZ_CUDA_CHECK(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return OZ_ERR_CUDA;
+    return dgemm_impl(m, n, k, alpha, A, lda, B, ldb, beta, C, ldc, set, route,
+                      static_cast<cudaStream_t>(stream), static_cast<char *>(g_workspace[dev]),
+                      g_workspace_bytes[dev]);
+}
+
+oz_status_t oz_dgemm(int64_t m, int64_t n, int64_t k, const double *A, int64_t lda, const double *B,
+                     int64_t ldb, double *C, int64_t ldc, oz_modset_t set, uint32_t route,
+                     void *stream)
+{
+    return oz_dgemm_ex(m, n, k, 1.0, A, lda, B, ldb, 0.0, C, ldc, set, route, stream);
+}
+
+oz_status_t oz_dgemm_host(int64_t m, int64_t n, int64_t k, double alpha, const double *A_host,
+                          int64_t lda, const double *B_host, int64_t ldb, double beta,
+                          double *C_host, int64_t ldc, oz_modset_t set, uint32_t route,
+                          void *stream)
+{
+    int dev = 0;
+    OZ_CUDA_CHECK(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return OZ_ERR_CUDA;
+    Route rt;
+    if (!valid_set(set) || !decode_route(route, &rt)) return OZ_ERR_INVALID_ARG;
+    if (m < 0 || n < 0 || k < 0) return OZ_ERR_INVALID_ARG;
+    if (m == 0 || n == 0) return OZ_OK;
+    if (!C_host || ldc < m || (k > 0 && (!A_host || !B_host || lda < m || ldb < k)))
+        return OZ_ERR_INVALID_ARG;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    char *ws = static_cast<char *>(g_workspace[dev]);
+    int64_t kk = k > 0 ? k : 1;
+    size_t core = make_layout(m, n, kk, set).total;
+    size_t bytesA = 8 * static_cast<size_t>(m) * kk, bytesB = 8 * static_cast<size_t>(kk) * n;
+    size_t bytesC = 8 * static_cast<size_t>(m) * n;
+    size_t offA = core, offB = offA + round_up(bytesA, 256), offC = offB + round_up(bytesB, 256);
+    if (!ws || g_workspace_bytes[dev] < offC + bytesC) return OZ_ERR_WORKSPACE;
+    double *dA = reinterpret_cast<double *>(ws + offA);
+    double *dB = reinterpret_cast<double *>(ws + offB);
+    double *dC = reinterpret_cast<double *>(ws + offC);
+    if (k > 0) {
+        OZ_CUDA_CHECK(cudaMemcpy2DAsync(dA, 8 * m, A_host, 8 * lda, 8 * m, k, cudaMemcpyHostToDevice, s));
+        OZ_CUDA_CHECK(cudaMemcpy2DAsync(dB, 8 * k, B_host, 8 * ldb, 8 * k, n, cudaMemcpyHostToDevice, s));
+    }
+    if (beta != 0.0)
+        OZ_CUDA_CHECK(cudaMemcpy2DAsync(dC, 8 * m, C_host, 8 * ldc, 8 * m, n, cudaMemcpyHostToDevice, s));
+    oz_status_t st = dgemm_impl(m, n, k, alpha, dA, m, dB, kk, beta, dC, m, set, route, s, ws, core);
+    if (st != OZ_OK) return st;
+    OZ_CUDA_CHECK(cudaMemcpy2DAsync(C_host, 8 * ldc, dC, 8 * m, 8 * m, n, cudaMemcpyDeviceToHost, s));
+    return OZ_OK;
+}
+
+oz_status_t oz_deconstruct(int side, int64_t lines, int64_t k, const double *X, int64_t ldx,
+                           oz_modset_t set, uint32_t route, uint8_t *planes, int64_t plane_stride,
+                           int64_t row_pitch, int32_t *shift, void *scratch, void *stream)
+{
+    Route rt;
+    if (!valid_set(set) || !decode_route(route, &rt) || (side != 0 && side != 1))
+        return OZ_ERR_INVALID_ARG;
+    if (lines < 0 || k < 0) return OZ_ERR_INVALID_ARG;
+    if (k > OZ_K_MAX) return OZ_ERR_UNSUPPORTED;
+    if (lines == 0) return OZ_OK;
+    if (!planes || !shift || !scratch || (k > 0 && !X)) return OZ_ERR_INVALID_ARG;
+    if (row_pitch < k || row_pitch < 16 || (row_pitch & 15) || (plane_stride & 15) ||
+        plane_stride < lines * row_pitch || (reinterpret_cast<uintptr_t>(planes) & 15u) ||
+        (reinterpret_cast<uintptr_t>(scratch) & 255u))
+        return OZ_ERR_INVALID_ARG;
+    if (k > 0 && ldx < (side == 0 ? lines : k)) return OZ_ERR_INVALID_ARG;
+    oz_status_t st = ensure_device_ready();
+    if (st != OZ_OK) return st;
+    return launch_deconstruct(side, lines, k, X, ldx, set, rt, planes, plane_stride, row_pitch, shift,
+                              scratch, static_cast<cudaStream_t>(stream));
+}
+
+oz_status_t oz_residue_gemm(int64_t m, int64_t n, int64_t k, const uint8_t *PA, int64_t strideA,
+                            int64_t pitchA, const uint8_t *PB, int64_t strideB, int64_t pitchB,
+                            oz_modset_t set, uint32_t route, uint16_t *R, int64_t ldr,
+                            int64_t mod_stride, void *stream)
+{
+    Route rt;
+    if (!valid_set(set) || !decode_route(route, &rt)) return OZ_ERR_INVALID_ARG;
+    if (m < 0 || n < 0 || k < 0) return OZ_ERR_INVALID_ARG;
+    if (k > OZ_K_MAX) return OZ_ERR_UNSUPPORTED;
+    if (m == 0 || n == 0) return OZ_OK;
+    if (!PA || !PB || !R || ldr < m || mod_stride < n * ldr) return OZ_ERR_INVALID_ARG;
+    if ((pitchA & 15) || (pitchB & 15) || (strideA & 15) || (strideB & 15) || pitchA < k ||
+        pitchB < k || pitchA < 16 || pitchB < 16 || strideA < m * pitchA || strideB < n * pitchB ||
+        (reinterpret_cast<uintptr_t>(PA) & 15u) || (reinterpret_cast<uintptr_t>(PB) & 15u))
+        return OZ_ERR_INVALID_ARG;
+    oz_status_t st = ensure_device_ready();
+    if (st != OZ_OK) return st;
+    return launch_residue_gemm(m, n, k, PA, strideA, pitchA, PB, strideB, pitchB, set, rt, R, ldr,
+                               mod_stride, static_cast<cudaStream_t>(stream));
+}
+
+oz_status_t oz_reconstruct(int64_t m, int64_t n, const uint16_t *R, int64_t ldr, int64_t mod_stride,
+                           const int32_t *shiftA, const int32_t *shiftB, oz_modset_t set,
+                           double alpha, double beta, double *C, int64_t ldc, void *stream)
+{
+    if (!valid_set(set) || m < 0 || n < 0) return OZ_ERR_INVALID_ARG;
+    if (!(alpha == 1.0 || alpha == -1.0) || !(beta == 0.0 || beta == 1.0)) return OZ_ERR_UNSUPPORTED;
+    if (m == 0 || n == 0) return OZ_OK;
+    if (!R || !shiftA || !shiftB || !C || ldr < m || mod_stride < n * ldr || ldc < m)
+        return OZ_ERR_INVALID_ARG;
+    oz_status_t st = ensure_device_ready();
+    if (st != OZ_OK) return st;
+    return launch_reconstruct(m, n, R, ldr, mod_stride, shiftA, shiftB, set, alpha, beta, C, ldc,
+                              static_cast<cudaStream_t>(stream));
+}
+
+oz_status_t oz_query_status(void *stream)
+{
+    oz_status_t st = ensure_device_ready();
+    if (st != OZ_OK) return st;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    unsigned int word[4] = {0, 0, 0, 0}, zero[4] = {0, 0, 0, 0};
+    OZ_CUDA_CHECK(cudaStreamSynchronize(s));
+    OZ_CUDA_CHECK(cudaMemcpyFromSymbol(word, g_status, sizeof(word)));
+    OZ_CUDA_CHECK(cudaMemcpyToSymbol(g_status, zero, sizeof(zero)));
+    if (cudaGetLastError() != cudaSuccess) return OZ_ERR_CUDA;
+    if (word[0] & (1u << OZ_ERR_TIMEOUT)) return OZ_ERR_TIMEOUT;
+    if (word[0] & (1u << OZ_ERR_RANGE)) return OZ_ERR_RANGE;
+    if (word[0] & (1u << OZ_ERR_NONFINITE_INPUT)) return OZ_ERR_NONFINITE_INPUT;
+    return OZ_OK;
+}
+
+uint64_t oz_launch_count(void) { return g_launches.load(); }
+
+const char *oz_status_string(oz_status_t status)
+{
+    switch (status) {
+        case OZ_OK: return "ok";
+        case OZ_ERR_INVALID_ARG: return "invalid argument";
+        case OZ_ERR_UNSUPPORTED: return "unsupported (k above OZ_K_MAX, or alpha/beta not in {+-1}/{0,1})";
+        case OZ_ERR_WORKSPACE: return "workspace missing or too small";
+        case OZ_ERR_CUDA: return "CUDA call failed";
+        case OZ_ERR_NONFINITE_INPUT: return "Inf/NaN in an operand";
+        case OZ_ERR_RANGE: return "quantised value out of range";
+        case OZ_ERR_TIMEOUT: return "bounded device wait ran out";
+    }
+    return "unknown status";
+}
+
+}  // extern "C"

@@ -1,0 +1,401 @@
+// Deconstruction (Algorithm 2; scaling of Eq. 1): FP64 operand -> per-line shifts and K-major
+// 8-bit residue planes.
+//
+// Kernels, in launch order for one operand:
+//   scan_init      clears the per-line scratch (largest exponent, non-finite flag, sum of squares)
+//   scan_maxexp    largest floor(log2|x|) of every line, Inf/NaN detection
+//   scan_sumsq     CS rule only: exact integer sum of ceil(|x| 2^(9-E))^2 per line
+//   scan_finalize  shift[line] (sigma_i or tau_j of Eq. 1)
+//   convert        quantise, reduce modulo every modulus, look the plane bytes up, store
+//
+// The scan is split over the inner dimension with integer atomics (max / or / add), so its
+// result does not depend on the order of the partial results: the shifts are bit-reproducible.
+//
+// Residue of a 64-bit two's-complement integer a' modulo m (the paper's byte-plane identity of
+// paragraph "O2", applied to 16-bit limbs so that every partial sum stays below 2^32):
+//   a' mod m = (l0 + l1 (2^16 mod m) + l2 (2^32 mod m) + l3 (2^48 mod m) + [a'<0] ((-2^64) mod m)) mod m
+// followed by one Barrett step with floor(2^32/m).  The digit split, the Lemma 1 carry and the
+// E4M3 / INT8 encoding are folded into a per-modulus table indexed by the canonical residue
+// (built on the host at set-up), held in shared memory.
+#include <utility>
+
+#include "oz_internal.h"
+
+namespace oz {
+namespace {
+
+constexpr int kConvThreads = 256;
+constexpr int kChunk = 128;            // inner-dimension bytes handled per warp step (4 per lane)
+constexpr int kTileLines = 32;         // side 0: lines per shared-memory transposition tile
+constexpr int kTilePitch = kChunk + 1; // doubles per tile row (+1: conflict-free column writes)
+
+struct ScanScratch {
+    unsigned long long *sumsq;  // [lines]
+    int *emax;                  // [lines]
+    int *nonfinite;             // [lines]
+};
+
+__host__ __device__ inline ScanScratch carve_scratch(void *scratch, int64_t lines)
+{
+    ScanScratch s;
+    char *base = static_cast<char *>(scratch);
+    s.sumsq = reinterpret_cast<unsigned long long *>(base);
+    s.emax = reinterpret_cast<int *>(base + 8 * lines);
+    s.nonfinite = reinterpret_cast<int *>(base + 12 * lines);
+    return s;
+}
+
+__device__ __forceinline__ const double *element(const double *X, int64_t ldx, int side,
+                                                 int64_t line, int64_t kk)
+{
+    return side == 0 ? X + line + kk * ldx : X + kk + line * ldx;
+}
+
+// classification of a double: returns 0 zero, 1 finite non-zero (e = floor(log2|x|)), 2 Inf/NaN
+__device__ __forceinline__ int classify(double x, int *e)
+{
+    unsigned long long bits = static_cast<unsigned long long>(__double_as_longlong(x));
+    int be = static_cast<int>((bits >> 52) & 0x7FF);
+    unsigned long long frac = bits & 0xFFFFFFFFFFFFFull;
+    if (be == 0x7FF) return 2;
+    if (be == 0) {
+        if (frac == 0) return 0;
+        *e = -1011 - __clzll(static_cast<long long>(frac));   // subnormal: normalise the fraction
+        return 1;
+    }
+    *e = be - 1023;
+    return 1;
+}
+
+__global__ void scan_init_kernel(ScanScratch s, int64_t lines)
+{
+    int64_t i = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x;
+    if (i < lines) {
+        s.sumsq[i] = 0ull;
+        s.emax[i] = INT32_MIN;
+        s.nonfinite[i] = 0;
+    }
+}
+
+// One pass over the operand.  PASS 0: largest exponent + non-finite flag.  PASS 1: sum of squares.
+// side 0: thread = line, loop over a k-range (loads coalesced across lines).
+// side 1: warp = line, lanes stride over a k-range (loads coalesced along k), shuffle reduction.
+template <int SIDE, int PASS>
+__global__ void __launch_bounds__(256)
+scan_kernel(const double *__restrict__ X, int64_t ldx, int64_t lines, int64_t k, int64_t kspan,
+            ScanScratch s)
+{
+    int64_t k0 = static_cast<int64_t>(blockIdx.y) * kspan;
+    int64_t k1 = k0 + kspan < k ? k0 + kspan : k;
+    int lane = threadIdx.x & 31;
+    int64_t line;
+    int64_t kstart, kstep;
+    if (SIDE == 0) {
+        line = blockIdx.x * 256ll + threadIdx.x;
+        kstart = k0;
+        kstep = 1;
+    } else {
+        line = blockIdx.x * 8ll + (threadIdx.x >> 5);
+        kstart = k0 + lane;
+        kstep = 32;
+    }
+    bool live = line < lines;
+    int emax = INT32_MIN, bad = 0;
+    unsigned long long acc = 0;
+    int E = 0;
+    if (PASS == 1 && live) E = s.emax[line];
+    if (live && !(PASS == 1 && E == INT32_MIN)) {
+        for (int64_t kk = kstart; kk < k1; kk += kstep) {
+            double x = *element(X, ldx, SIDE, line, kk);
+            if (PASS == 0) {
+                int e;
+                int c = classify(x, &e);
+                if (c == 2) bad = 1;
+                if (c == 1 && e > emax) emax = e;
+            } else {
+                unsigned long long bits = static_cast<unsigned long long>(__double_as_longlong(x));
+                int be = static_cast<int>((bits >> 52) & 0x7FF);
+                unsigned long long frac = bits & 0xFFFFFFFFFFFFFull;
+                if (be == 0x7FF || (be == 0 && frac == 0)) continue;
+                unsigned long long sig = be ? (frac | (1ull << 52)) : frac;
+                int ex = be ? be - 1023 : -1022;
+                int sh = 43 + E - ex;                 // |x| 2^(9-E) = sig / 2^sh
+                unsigned long long abar;
+                if (sh >= 64) abar = 1;
+                else if (sh <= 0) abar = sig << (-sh);
+                else abar = (sig >> sh) + ((sig & ((1ull << sh) - 1)) ? 1ull : 0ull);
+                acc += abar * abar;
+            }
+        }
+    }
+    if (SIDE == 1) {
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            if (PASS == 0) {
+                int other = __shfl_xor_sync(0xFFFFFFFFu, emax, o);
+                emax = other > emax ? other : emax;
+                bad |= __shfl_xor_sync(0xFFFFFFFFu, bad, o);
+            } else {
+                acc += __shfl_xor_sync(0xFFFFFFFFu, acc, o);
+            }
+        }
+        if (lane != 0) live = false;
+    }
+    if (!live) return;
+    if (PASS == 0) {
+        if (emax != INT32_MIN) atomicMax(&s.emax[line], emax);
+        if (bad) atomicOr(&s.nonfinite[line], 1);
+    } else if (acc) {
+        atomicAdd(&s.sumsq[line], acc);
+    }
+}
+
+// shift[line]: MAXEXP  t - 1 - E;  CS  p + 9 - E with p the largest integer such that
+// 4^p * S <= G^2  (G^2 passed as two 64-bit words).
+__global__ void scan_finalize_kernel(ScanScratch s, int64_t lines, int rule, int tbits,
+                                     unsigned long long g2lo, unsigned long long g2hi,
+                                     int32_t *shift, unsigned int *status)
+{
+    int64_t i = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x;
+    if (i >= lines) return;
+    if (s.nonfinite[i]) {
+        shift[i] = OZ_NONFINITE_SHIFT;
+        atomicOr(status, 1u << OZ_ERR_NONFINITE_INPUT);
+        return;
+    }
+    int E = s.emax[i];
+    if (E == INT32_MIN) { shift[i] = 0; return; }
+    if (rule == 0) { shift[i] = tbits - 1 - E; return; }
+    unsigned __int128 G2 = (static_cast<unsigned __int128>(g2hi) << 64) | g2lo;
+    unsigned __int128 q = G2 / static_cast<unsigned __int128>(s.sumsq[i]);   // >= 4^p  <=>  4^p S <= G^2
+    unsigned long long qhi = static_cast<unsigned long long>(q >> 64);
+    unsigned long long qlo = static_cast<unsigned long long>(q);
+    int top = qhi ? 127 - __clzll(static_cast<long long>(qhi)) : 63 - __clzll(static_cast<long long>(qlo));
+    shift[i] = (top >> 1) + 9 - E;
+}
+
+// Eq. 1 for one element: a' = quant(x 2^sigma) as a 64-bit integer.
+__device__ __forceinline__ long long quantise(double x, int sigma, bool tz)
+{
+    unsigned long long bits = static_cast<unsigned long long>(__double_as_longlong(x));
+    int be = static_cast<int>((bits >> 52) & 0x7FF);
+    unsigned long long frac = bits & 0xFFFFFFFFFFFFFull;
+    unsigned long long sig = be ? (frac | (1ull << 52)) : frac;
+    int ex = be ? be - 1023 : -1022;
+    int sh = 52 - ex - sigma;                       // |x| 2^sigma = sig / 2^sh
+    unsigned long long q;
+    if (sh <= 0) {
+        q = sig << (sh < -63 ? 63 : -sh);
+    } else {
+        if (sh > 63) sh = 63;                       // sig < 2^53: anything past 54 rounds to zero
+        if (tz) q = sig >> sh;
+        else q = (sig + ((1ull << (sh - 1)) - 1ull) + ((sig >> sh) & 1ull)) >> sh;  // ties to even
+    }
+    return (bits >> 63) ? -static_cast<long long>(q) : static_cast<long long>(q);
+}
+
+// One modulus (compile-time index I of set SET) for four consecutive inner-dimension elements:
+// residues, table look-up, byte transposition, 2 or 3 four-byte plane stores.
+template <int SET, int I>
+__device__ __forceinline__ void convert_modulus(const uint32_t (&l0)[4], const uint32_t (&l1)[4],
+                                                const uint32_t (&l2)[4], const uint32_t (&l3)[4],
+                                                const uint32_t (&neg)[4],
+                                                const uint32_t *__restrict__ lut, uint8_t *out,
+                                                int64_t plane_stride)
+{
+    constexpr uint32_t m = modulus(SET, I);
+    constexpr uint32_t c1 = pow2_mod(16, m), c2 = pow2_mod(32, m), c3 = pow2_mod(48, m);
+    constexpr uint32_t corr = (m - pow2_mod(64, m)) % m;     // (-2^64) mod m
+    constexpr uint32_t magic = barrett_magic(m);
+    constexpr int off = lut_offset(SET, I);
+    constexpr int plane = first_plane(SET, I);
+    static_assert(65535ull * (1ull + c1 + c2 + c3) + corr < 0x100000000ull, "limb sum fits 32 bits");
+    uint32_t w[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+        uint32_t v = l0[e] + l1[e] * c1 + l2[e] * c2 + l3[e] * c3 + neg[e] * corr;
+        uint32_t q = __umulhi(v, magic);
+        uint32_t r = v - q * m;                  // in [0, 2m)
+        r = min(r, r - m);                       // unsigned: picks r - m when r >= m
+        w[e] = lut[off + r];
+    }
+    uint32_t t01 = __byte_perm(w[0], w[1], 0x5140);
+    uint32_t t23 = __byte_perm(w[2], w[3], 0x5140);
+    *reinterpret_cast<uint32_t *>(out + plane * plane_stride) = __byte_perm(t01, t23, 0x5410);
+    *reinterpret_cast<uint32_t *>(out + (plane + 1) * plane_stride) = __byte_perm(t01, t23, 0x7632);
+    if (planes_of(m) == 3) {
+        uint32_t u01 = __byte_perm(w[0], w[1], 0x0062);
+        uint32_t u23 = __byte_perm(w[2], w[3], 0x0062);
+        *reinterpret_cast<uint32_t *>(out + (plane + 2) * plane_stride) = __byte_perm(u01, u23, 0x5410);
+    }
+}
+
+template <int SET, int... I>
+__device__ __forceinline__ void convert_all_moduli(std::integer_sequence<int, I...>,
+                                                   const uint32_t (&l0)[4], const uint32_t (&l1)[4],
+                                                   const uint32_t (&l2)[4], const uint32_t (&l3)[4],
+                                                   const uint32_t (&neg)[4],
+                                                   const uint32_t *__restrict__ lut, uint8_t *out,
+                                                   int64_t plane_stride)
+{
+    (convert_modulus<SET, I>(l0, l1, l2, l3, neg, lut, out, plane_stride), ...);
+}
+
+// Four consecutive inner-dimension elements of one line -> 4 bytes of every stored plane.
+template <int SET>
+__device__ __forceinline__ void convert4(const double (&x)[4], int sigma, bool tz,
+                                         const uint32_t *__restrict__ lut, uint8_t *out,
+                                         int64_t plane_stride)
+{
+    uint32_t l0[4], l1[4], l2[4], l3[4], neg[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+        long long a = quantise(x[e], sigma, tz);
+        unsigned long long p = static_cast<unsigned long long>(a);
+        uint32_t lo = static_cast<uint32_t>(p), hi = static_cast<uint32_t>(p >> 32);
+        l0[e] = lo & 0xFFFFu;
+        l1[e] = lo >> 16;
+        l2[e] = hi & 0xFFFFu;
+        l3[e] = hi >> 16;
+        neg[e] = hi >> 31;
+    }
+    convert_all_moduli<SET>(std::make_integer_sequence<int, set_r(SET)>{}, l0, l1, l2, l3, neg, lut,
+                            out, plane_stride);
+}
+
+template <int SET, int SIDE>
+__global__ void __launch_bounds__(kConvThreads)
+convert_kernel(const double *__restrict__ X, int64_t ldx, int64_t lines, int64_t k,
+               const int32_t *__restrict__ shift, const uint32_t *__restrict__ lut_global,
+               uint8_t *__restrict__ planes, int64_t plane_stride, int64_t row_pitch, int tz)
+{
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    uint32_t *lut = reinterpret_cast<uint32_t *>(smem_raw);
+    for (int i = threadIdx.x; i < kLutWords; i += kConvThreads) lut[i] = lut_global[i];
+    __syncthreads();
+
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int64_t nchunks = (row_pitch + kChunk - 1) / kChunk;
+
+    if (SIDE == 1) {
+        const int64_t items = lines * nchunks;
+        for (int64_t item = blockIdx.x * 8ll + warp; item < items; item += gridDim.x * 8ll) {
+            int64_t line = item / nchunks;
+            int64_t kb = (item - line * nchunks) * kChunk + lane * 4;
+            if (kb >= row_pitch) continue;
+            int sigma = shift[line];
+            bool dead = sigma == OZ_NONFINITE_SHIFT;
+            double x[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e)
+                x[e] = (!dead && kb + e < k) ? X[kb + e + line * ldx] : 0.0;
+            convert4<SET>(x, dead ? 0 : sigma, tz != 0, lut, planes + line * row_pitch + kb, plane_stride);
+        }
+    } else {
+        double *tile = reinterpret_cast<double *>(smem_raw + kLutWords * 4);
+        const int64_t ltiles = (lines + kTileLines - 1) / kTileLines;
+        const int64_t items = ltiles * nchunks;
+        for (int64_t item = blockIdx.x; item < items; item += gridDim.x) {
+            int64_t lt = item % ltiles;           // neighbouring blocks read neighbouring rows
+            int64_t kc = item / ltiles;
+            int64_t line_l = lt * kTileLines + lane;
+            for (int kk = warp; kk < kChunk; kk += kConvThreads / 32) {
+                int64_t kg = kc * kChunk + kk;
+                tile[lane * kTilePitch + kk] =
+                    (line_l < lines && kg < k) ? X[line_l + kg * ldx] : 0.0;
+            }
+            __syncthreads();
+            int64_t kb = kc * kChunk + lane * 4;
+#pragma unroll 1
+            for (int li = warp * 4; li < warp * 4 + 4; ++li) {
+                int64_t line = lt * kTileLines + li;
+                if (line >= lines || kb >= row_pitch) continue;
+                int sigma = shift[line];
+                bool dead = sigma == OZ_NONFINITE_SHIFT;
+                double x[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) x[e] = dead ? 0.0 : tile[li * kTilePitch + lane * 4 + e];
+                convert4<SET>(x, dead ? 0 : sigma, tz != 0, lut, planes + line * row_pitch + kb, plane_stride);
+            }
+            __syncthreads();
+        }
+    }
+}
+
+template <int SET, int SIDE>
+oz_status_t launch_convert(const double *X, int64_t ldx, int64_t lines, int64_t k,
+                           const int32_t *shift, const uint32_t *lut, uint8_t *planes,
+                           int64_t plane_stride, int64_t row_pitch, int tz, cudaStream_t stream)
+{
+    size_t smem = kLutWords * 4 + (SIDE == 0 ? sizeof(double) * kTileLines * kTilePitch : 0);
+    OZ_CUDA_CHECK(cudaFuncSetAttribute(convert_kernel<SET, SIDE>,
+                                       cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       static_cast<int>(smem)));
+    int64_t nchunks = (row_pitch + kChunk - 1) / kChunk;
+    int64_t need = SIDE == 1 ? (lines * nchunks + 7) / 8
+                             : ((lines + kTileLines - 1) / kTileLines) * nchunks;
+    int sms = 148;
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, 0);
+    int64_t cap = static_cast<int64_t>(sms) * (SIDE == 1 ? 6 : 3);
+    int grid = static_cast<int>(need < cap ? need : cap);
+    convert_kernel<SET, SIDE><<<grid, kConvThreads, smem, stream>>>(
+        X, ldx, lines, k, shift, lut, planes, plane_stride, row_pitch, tz);
+    count_launch();
+    OZ_CUDA_CHECK(cudaGetLastError());
+    return OZ_OK;
+}
+
+}  // namespace
+
+oz_status_t launch_deconstruct(int side, int64_t lines, int64_t k, const double *X, int64_t ldx,
+                               int set, const Route &rt, uint8_t *planes, int64_t plane_stride,
+                               int64_t row_pitch, int32_t *shift, void *scratch,
+                               cudaStream_t stream)
+{
+    ScanScratch s = carve_scratch(scratch, lines);
+    unsigned int *status = device_status_word();
+    int blocks1d = static_cast<int>((lines + 255) / 256);
+    scan_init_kernel<<<blocks1d, 256, 0, stream>>>(s, lines);
+    count_launch();
+
+    // split the inner dimension so that the scan fills the machine even for few lines
+    int64_t line_blocks = side == 0 ? (lines + 255) / 256 : (lines + 7) / 8;
+    int64_t want_split = (148 * 8 + line_blocks - 1) / line_blocks;
+    int64_t max_split = (k + 63) / 64;
+    int64_t split = want_split < max_split ? want_split : max_split;
+    if (split < 1) split = 1;
+    if (split > 65535) split = 65535;
+    int64_t kspan = (k + split - 1) / split;
+    split = k > 0 ? (k + kspan - 1) / kspan : 0;
+
+    int tA = 0, tB = 0;
+    budget_maxexp(set, k, &tA, &tB);
+    uint64_t g2lo = 0, g2hi = 0;
+    cs_bound_squared(set, k, &g2lo, &g2hi);
+
+    if (k > 0) {
+        dim3 grid(static_cast<unsigned>(line_blocks), static_cast<unsigned>(split));
+        if (side == 0) scan_kernel<0, 0><<<grid, 256, 0, stream>>>(X, ldx, lines, k, kspan, s);
+        else scan_kernel<1, 0><<<grid, 256, 0, stream>>>(X, ldx, lines, k, kspan, s);
+        count_launch();
+        if (rt.rule == 1) {
+            if (side == 0) scan_kernel<0, 1><<<grid, 256, 0, stream>>>(X, ldx, lines, k, kspan, s);
+            else scan_kernel<1, 1><<<grid, 256, 0, stream>>>(X, ldx, lines, k, kspan, s);
+            count_launch();
+        }
+    }
+    scan_finalize_kernel<<<blocks1d, 256, 0, stream>>>(s, lines, rt.rule, side == 0 ? tA : tB, g2lo,
+                                                       g2hi, shift, status);
+    count_launch();
+    OZ_CUDA_CHECK(cudaGetLastError());
+
+    const uint32_t *lut = device_lut(set, rt.substrate);
+    if (set == 0) {
+        return side == 0 ? launch_convert<0, 0>(X, ldx, lines, k, shift, lut, planes, plane_stride, row_pitch, rt.quant, stream)
+                         : launch_convert<0, 1>(X, ldx, lines, k, shift, lut, planes, plane_stride, row_pitch, rt.quant, stream);
+    }
+    return side == 0 ? launch_convert<1, 0>(X, ldx, lines, k, shift, lut, planes, plane_stride, row_pitch, rt.quant, stream)
+                     : launch_convert<1, 1>(X, ldx, lines, k, shift, lut, planes, plane_stride, row_pitch, rt.quant, stream);
+}
+
+}  // namespace oz

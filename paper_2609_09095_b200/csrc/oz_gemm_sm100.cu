@@ -1,0 +1,540 @@
+// Residue GEMMs on the 5th-generation tensor cores (Algorithm 1, the loop over moduli; Sec. 2
+// "FP8 variant"; Eq. 8), with the per-modulus combination and `mod m_i` fused into the epilogue.
+//
+// For every modulus the product of two centred residues is rebuilt from exact plane products:
+//   square m = s^2 (planes d0,d1):        d e = d0 e0 + s (d1 e0 + d0 e1)              (mod m)
+//   non-square (planes d0,d1,dS=d0+d1):   d e = -15 d0 e0 + 16 dS eS + 240 d1 e1       (Eq. 8)
+// so one (modulus, output tile) work item is a short list of "accumulator jobs", each a K-loop
+// of tcgen05.mma instructions into one TMEM accumulator:
+//   square:      job 0 = D0.E0 (weight 1);  job 1 = [D1|D0].[E0|E1] (two K-loops, weight s)
+//   non-square:  job 0 = D0.E0 (-15);  job 1 = DS.ES (16);  job 2 = D1.E1 (240)
+// Three MMA K-loops per modulus either way (p_mma = 3r).
+//
+// Kernel structure (one persistent CTA per SM, 320 threads):
+//   warp 0      TMA producer: 128-byte-swizzled K-major tiles of A (128 rows) and B (256 rows)
+//               into a 4-stage shared-memory ring, no multicast
+//   warp 1      MMA issuer: one lane issues tcgen05.mma (M=128, N=256, K=32, cta_group::1);
+//               accumulators live in TMEM, two slots of 256 columns used alternately per job
+//   warps 2..9  epilogue: tcgen05.ld the finished slot, reduce each accumulator modulo m_i in
+//               FP32 (all values are integers below 2^24, every step exact), fold it with the
+//               job's weight into a per-thread running combination held in registers, release
+//               the slot; after the last job reduce once more and store 16-bit residues
+// so the epilogue of one job overlaps the K-loop of the next, and TMEM never needs the three
+// accumulators of a non-square modulus at once.
+//
+// Exactness: the FP8 route relies on integer-valued partial sums below 2^24 being accumulated
+// without rounding (accumulation invariant of Algorithm 2, Lemma 1); the INT8 route accumulates in
+// INT32.  Both are converted to FP32 exactly because k <= OZ_K_MAX keeps |acc| < 2^24.
+//
+// Every barrier wait is bounded: on expiry the CTA records OZ_ERR_TIMEOUT in the device status
+// word, every role leaves its loops, in-flight copies are given a bounded time to land, TMEM is
+// freed and the kernel returns.
+#include <cuda.h>
+
+#include "oz_internal.h"
+
+namespace oz {
+namespace {
+
+constexpr int BLOCK_M = 128;
+constexpr int BLOCK_N = 256;
+constexpr int BLOCK_K = 128;                       // bytes = elements (8-bit operands)
+constexpr int UMMA_K = 32;                         // 8-bit operands: 32 elements per instruction
+constexpr int STAGES = 4;
+constexpr int A_BYTES = BLOCK_M * BLOCK_K;         // 16 KiB
+constexpr int B_BYTES = BLOCK_N * BLOCK_K;         // 32 KiB
+constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+constexpr int TMEM_COLS = 512;                     // two accumulator slots of BLOCK_N columns
+constexpr int NUM_THREADS = 320;
+constexpr int EPI_WARPS = 8;
+constexpr int COLS_PER_WARP = BLOCK_N / 2;         // two warps share a TMEM lane quarter
+constexpr size_t SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+
+struct ModInfo {
+    float m, inv_m;
+    float w[3];           // weight of each job
+    int njobs;            // 2 (square) or 3
+    int plane0;           // first stored plane of this modulus
+};
+
+struct GemmParams {
+    int64_t m, n, k;
+    int tiles_m, tiles_n, nk;       // nk = K chunks of BLOCK_K
+    int r;
+    int64_t total_items;
+    uint16_t *R;
+    int64_t ldr, mod_stride;
+    unsigned int *status;
+    ModInfo mod[kMaxR];
+};
+
+// ---------------------------------------------------------------- PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void *p)
+{
+    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes)
+                 : "memory");
+}
+
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+
+__device__ __forceinline__ unsigned long long global_timer_ns()
+{
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
+
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s per wait
+
+// Bounded wait.  Returns false when the wait ran out or another role already gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag,
+                                          unsigned int *status)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    unsigned long long start = global_timer_ns();
+    for (;;) {
+#pragma unroll 1
+        for (int it = 0; it < 256; ++it)
+            if (mbar_try_wait(bar, parity)) return true;
+        if (*abort_flag) return false;
+        if (global_timer_ns() - start > kWaitLimitNs) {
+            *abort_flag = 1;
+            atomicOr(status, 1u << OZ_ERR_TIMEOUT);
+            return false;
+        }
+    }
+}
+
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map, uint32_t bar,
+                                            int c0, int c1, int c2)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes "
+        "[%0], [%1, {%3, %4, %5}], [%2];"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
+        : "memory");
+}
+
+__device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t cols)
+{
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem),
+                 "r"(cols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols)
+{
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols)
+                 : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+template <int SUB>
+__device__ __forceinline__ void umma(uint32_t d_tmem, uint64_t da, uint64_t db, uint32_t idesc,
+                                     uint32_t accumulate)
+{
+    if (SUB == 0) {
+        asm volatile(
+            "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+            "tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], %1, %2, %3, p;\n\t}"
+            ::"r"(d_tmem), "l"(da), "l"(db), "r"(idesc), "r"(accumulate)
+            : "memory");
+    } else {
+        asm volatile(
+            "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+            "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
+            ::"r"(d_tmem), "l"(da), "l"(db), "r"(idesc), "r"(accumulate)
+            : "memory");
+    }
+}
+
+// mbarrier arrives once every MMA issued so far by this thread has completed
+__device__ __forceinline__ void umma_commit(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar)
+                 : "memory");
+}
+
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]),
+          "=r"(v[7]), "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]),
+          "=r"(v[14]), "=r"(v[15]), "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]),
+          "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]),
+          "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+        : "r"(taddr)
+        : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+// shared-memory matrix descriptor: K-major operand, 128-byte swizzle, 8-row groups 1024 B apart
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr)
+{
+    uint64_t d = 0;
+    d |= static_cast<uint64_t>((addr >> 4) & 0x3FFFu);   // start address / 16
+    d |= static_cast<uint64_t>(1) << 16;                 // leading byte offset (unused here) / 16
+    d |= static_cast<uint64_t>(1024 >> 4) << 32;         // stride byte offset / 16
+    d |= static_cast<uint64_t>(1) << 46;                 // descriptor version of sm_100
+    d |= static_cast<uint64_t>(2) << 61;                 // 128-byte swizzle
+    return d;
+}
+
+// instruction descriptor: D format, A/B formats, K-major both, N/8 at bit 17, M/16 at bit 24
+template <int SUB>
+__host__ __device__ constexpr uint32_t instr_desc()
+{
+    uint32_t cfmt = SUB == 0 ? 1u /*f32*/ : 2u /*s32*/;
+    uint32_t abfmt = SUB == 0 ? 0u /*e4m3*/ : 1u /*s8*/;
+    return (cfmt << 4) | (abfmt << 7) | (abfmt << 10) | (static_cast<uint32_t>(BLOCK_N >> 3) << 17) |
+           (static_cast<uint32_t>(BLOCK_M >> 4) << 24);
+}
+
+// work item -> (modulus, tile_m, tile_n): modulus-major so that one modulus' planes stay in L2;
+// inside a modulus, bands of 16 tile rows are swept column by column.
+struct Item { int mod, tm, tn; };
+
+__device__ __forceinline__ Item decode_item(int64_t item, const GemmParams &p)
+{
+    constexpr int BAND = 16;
+    int64_t per_mod = static_cast<int64_t>(p.tiles_m) * p.tiles_n;
+    Item it;
+    it.mod = static_cast<int>(item / per_mod);
+    int64_t t = item - it.mod * per_mod;
+    int64_t band_size = static_cast<int64_t>(BAND) * p.tiles_n;
+    int band = static_cast<int>(t / band_size);
+    int64_t in_band = t - band * band_size;
+    int rows = p.tiles_m - band * BAND < BAND ? p.tiles_m - band * BAND : BAND;
+    it.tn = static_cast<int>(in_band / rows);
+    it.tm = band * BAND + static_cast<int>(in_band - static_cast<int64_t>(it.tn) * rows);
+    return it;
+}
+
+// plane pair (A plane, B plane) of K-loop `pair` of job `job`
+__device__ __forceinline__ void job_planes(const ModInfo &mi, int job, int pair, int *pa, int *pb)
+{
+    if (mi.njobs == 3) {
+        // non-square: stored order d0, d1, dS; jobs d0e0, dSeS, d1e1
+        int sel = job == 0 ? 0 : (job == 1 ? 2 : 1);
+        *pa = mi.plane0 + sel;
+        *pb = mi.plane0 + sel;
+    } else if (job == 0) {
+        *pa = mi.plane0;
+        *pb = mi.plane0;
+    } else {
+        *pa = mi.plane0 + (pair == 0 ? 1 : 0);
+        *pb = mi.plane0 + (pair == 0 ? 0 : 1);
+    }
+}
+
+__device__ __forceinline__ int job_pairs(const ModInfo &mi, int job) { return (mi.njobs == 2 && job == 1) ? 2 : 1; }
+
+template <int SUB>
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+residue_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB,
+                    const __grid_constant__ GemmParams p)
+{
+    extern __shared__ unsigned char smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t tiles = (raw + 1023u) & ~1023u;                     // 1024-byte aligned ring
+    const uint32_t bars = tiles + STAGES * STAGE_BYTES;
+    const uint32_t full_bar = bars;                                   // STAGES x 8 bytes
+    const uint32_t empty_bar = bars + 8 * STAGES;
+    const uint32_t tfull_bar = bars + 16 * STAGES;                    // 2 x 8
+    const uint32_t tempty_bar = tfull_bar + 16;                       // 2 x 8
+    const uint32_t tmem_slot = tempty_bar + 16;                       // 4 bytes: TMEM base address
+    unsigned char *gen = smem_raw + (tiles - raw) + STAGES * STAGE_BYTES;
+    volatile uint32_t *tmem_base_ptr = reinterpret_cast<volatile uint32_t *>(gen + 16 * STAGES + 32);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(gen + 16 * STAGES + 40);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(full_bar + 8 * s, 1);
+            mbar_init(empty_bar + 8 * s, 1);
+        }
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(tfull_bar + 8 * s, 1);
+            mbar_init(tempty_bar + 8 * s, EPI_WARPS);
+        }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) tmem_alloc(tmem_slot, TMEM_COLS);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_base_ptr;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            int stage = 0;
+            uint32_t phase = 0;
+            bool ok = true;
+            for (int64_t item = blockIdx.x; ok && item < p.total_items; item += gridDim.x) {
+                Item it = decode_item(item, p);
+                const ModInfo &mi = p.mod[it.mod];
+                for (int job = 0; ok && job < mi.njobs; ++job) {
+                    int npairs = job_pairs(mi, job);
+                    for (int pair = 0; ok && pair < npairs; ++pair) {
+                        int pa, pb;
+                        job_planes(mi, job, pair, &pa, &pb);
+                        for (int kc = 0; kc < p.nk; ++kc) {
+                            ok = mbar_wait(empty_bar + 8 * stage, phase ^ 1u, abort_flag, p.status);
+                            if (!ok) break;
+                            uint32_t fb = full_bar + 8 * stage;
+                            mbar_expect_tx(fb, STAGE_BYTES);
+                            uint32_t sa = tiles + stage * STAGE_BYTES;
+                            tma_load_3d(sa, &mapA, fb, kc * BLOCK_K, it.tm * BLOCK_M, pa);
+                            tma_load_3d(sa + A_BYTES, &mapB, fb, kc * BLOCK_K, it.tn * BLOCK_N, pb);
+                            if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                        }
+                    }
+                }
+            }
+            if (!ok) {
+                // give copies already in flight a bounded time to land before the CTA exits
+                unsigned long long t0 = global_timer_ns();
+                while (global_timer_ns() - t0 < 2000000ull) { }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            constexpr uint32_t idesc = instr_desc<SUB>();
+            int stage = 0;
+            uint32_t phase = 0;
+            int slot = 0;
+            uint32_t slot_phase = 0;   // bit s = phase of slot s
+            bool ok = true;
+            for (int64_t item = blockIdx.x; ok && item < p.total_items; item += gridDim.x) {
+                Item it = decode_item(item, p);
+                const ModInfo &mi = p.mod[it.mod];
+                for (int job = 0; ok && job < mi.njobs; ++job) {
+                    ok = mbar_wait(tempty_bar + 8 * slot, ((slot_phase >> slot) & 1u) ^ 1u, abort_flag, p.status);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(slot * BLOCK_N);
+                    uint32_t accumulate = 0;
+                    int steps = job_pairs(mi, job) * p.nk;
+                    for (int st = 0; st < steps; ++st) {
+                        ok = mbar_wait(full_bar + 8 * stage, phase, abort_flag, p.status);
+                        if (!ok) break;
+                        tc_fence_after();
+                        uint32_t sa = tiles + stage * STAGE_BYTES;
+                        uint64_t da = smem_desc(sa), db = smem_desc(sa + A_BYTES);
+#pragma unroll
+                        for (int ks = 0; ks < BLOCK_K / UMMA_K; ++ks) {
+                            // advancing K inside the 128-byte swizzle atom: +32 bytes = +2 in the address field
+                            umma<SUB>(d_tmem, da + static_cast<uint64_t>(ks * (UMMA_K >> 4)),
+                                      db + static_cast<uint64_t>(ks * (UMMA_K >> 4)), idesc, accumulate);
+                            accumulate = 1;
+                        }
+                        umma_commit(empty_bar + 8 * stage);     // frees the stage when these MMAs finish
+                        if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                    }
+                    if (!ok) break;
+                    umma_commit(tfull_bar + 8 * slot);           // accumulator complete
+                    slot_phase ^= 1u << slot;
+                    slot ^= 1;
+                }
+            }
+            if (!ok) {
+                unsigned long long t0 = global_timer_ns();
+                while (global_timer_ns() - t0 < 2000000ull) { }
+            }
+        }
+    } else {
+        // ------------------------------------------------------------ epilogue
+        const int q = warp & 3;                       // TMEM lane quarter this warp may read
+        const int half = (warp - 2) >> 2;             // which half of the tile's columns
+        int slot = 0;
+        uint32_t slot_phase = 0;   // bit s = phase of slot s
+        bool ok = true;
+        for (int64_t item = blockIdx.x; ok && item < p.total_items; item += gridDim.x) {
+            Item it = decode_item(item, p);
+            const ModInfo &mi = p.mod[it.mod];
+            const float mm = mi.m, inv_m = mi.inv_m;
+            float comb[COLS_PER_WARP];
+#pragma unroll
+            for (int c = 0; c < COLS_PER_WARP; ++c) comb[c] = 0.0f;
+            for (int job = 0; ok && job < mi.njobs; ++job) {
+                ok = mbar_wait(tfull_bar + 8 * slot, (slot_phase >> slot) & 1u, abort_flag, p.status);
+                if (!ok) break;
+                tc_fence_after();
+                const float wj = mi.w[job];
+                const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) +
+                                       static_cast<uint32_t>(slot * BLOCK_N + half * COLS_PER_WARP);
+#pragma unroll
+                for (int c0 = 0; c0 < COLS_PER_WARP; c0 += 32) {
+                    uint32_t v[32];
+                    tmem_ld32(taddr + c0, v);
+#pragma unroll
+                    for (int e = 0; e < 32; ++e) {
+                        float acc = SUB == 0 ? __uint_as_float(v[e])
+                                             : __int2float_rn(static_cast<int>(v[e]));
+                        float quot = fmaf(acc, inv_m, 12582912.0f) - 12582912.0f;   // rint(acc/m)
+                        float res = fmaf(-quot, mm, acc);                            // exact, |res| <= ~m/2
+                        comb[c0 + e] = fmaf(res, wj, comb[c0 + e]);                  // exact, < 2^24
+                    }
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(tempty_bar + 8 * slot);
+                slot_phase ^= 1u << slot;
+                slot ^= 1;
+            }
+            if (!ok) break;
+            const int64_t row = static_cast<int64_t>(it.tm) * BLOCK_M + q * 32 + lane;
+            const int64_t col0 = static_cast<int64_t>(it.tn) * BLOCK_N + half * COLS_PER_WARP;
+            if (row < p.m) {
+                uint16_t *dst = p.R + it.mod * p.mod_stride + col0 * p.ldr + row;
+#pragma unroll
+                for (int c = 0; c < COLS_PER_WARP; ++c) {
+                    if (col0 + c < p.n) {
+                        float t = comb[c];
+                        float quot = fmaf(t, inv_m, 12582912.0f) - 12582912.0f;
+                        float res = fmaf(-quot, mm, t);
+                        res = res < 0.0f ? res + mm : res;                           // canonical [0, m)
+                        uint32_t bits = __float_as_uint(res + 8388608.0f);           // integer in the low mantissa bits
+                        dst[c * p.ldr] = static_cast<uint16_t>(bits & 0xFFFFu);
+                    }
+                }
+            }
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, TMEM_COLS);
+    }
+}
+
+// ---------------------------------------------------------------- host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *,
+                                  const cuuint64_t *, const cuuint64_t *, const cuuint32_t *,
+                                  const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn()
+{
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void *sym = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(sym);
+    }
+    return fn;
+}
+
+// 3-D map over planes[plane][line][kbyte]; box = 128 bytes x box_lines lines x 1 plane,
+// 128-byte swizzle, out-of-range elements read as zero.
+bool make_plane_map(CUtensorMap *map, const uint8_t *base, int64_t lines, int64_t pitch,
+                    int64_t plane_stride, int planes, int box_lines)
+{
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    cuuint64_t dims[3] = {static_cast<cuuint64_t>(pitch), static_cast<cuuint64_t>(lines),
+                          static_cast<cuuint64_t>(planes)};
+    cuuint64_t strides[2] = {static_cast<cuuint64_t>(pitch), static_cast<cuuint64_t>(plane_stride)};
+    cuuint32_t box[3] = {static_cast<cuuint32_t>(BLOCK_K), static_cast<cuuint32_t>(box_lines), 1};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult rc = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<uint8_t *>(base), dims, strides,
+                     box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                     CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return rc == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+oz_status_t launch_residue_gemm(int64_t m, int64_t n, int64_t k, const uint8_t *PA, int64_t strideA,
+                                int64_t pitchA, const uint8_t *PB, int64_t strideB, int64_t pitchB,
+                                int set, const Route &rt, uint16_t *R, int64_t ldr,
+                                int64_t mod_stride, cudaStream_t stream)
+{
+    GemmParams p{};
+    p.m = m; p.n = n; p.k = k;
+    p.tiles_m = static_cast<int>((m + BLOCK_M - 1) / BLOCK_M);
+    p.tiles_n = static_cast<int>((n + BLOCK_N - 1) / BLOCK_N);
+    p.nk = static_cast<int>((k + BLOCK_K - 1) / BLOCK_K);
+    p.r = set_r(set);
+    p.total_items = static_cast<int64_t>(p.r) * p.tiles_m * p.tiles_n;
+    p.R = R; p.ldr = ldr; p.mod_stride = mod_stride;
+    p.status = device_status_word();
+    for (int i = 0; i < p.r; ++i) {
+        int mi = modulus(set, i), s = square_root(mi);
+        p.mod[i].m = static_cast<float>(mi);
+        p.mod[i].inv_m = 1.0f / static_cast<float>(mi);
+        p.mod[i].plane0 = first_plane(set, i);
+        if (s) {
+            p.mod[i].njobs = 2;
+            p.mod[i].w[0] = 1.0f; p.mod[i].w[1] = static_cast<float>(s); p.mod[i].w[2] = 0.0f;
+        } else {
+            p.mod[i].njobs = 3;
+            p.mod[i].w[0] = -15.0f; p.mod[i].w[1] = 16.0f; p.mod[i].w[2] = 240.0f;
+        }
+    }
+    if (k == 0) p.nk = 1;   // one all-zero chunk (the planes' padding) gives residues 0
+
+    CUtensorMap mapA, mapB;
+    if (!make_plane_map(&mapA, PA, m, pitchA, strideA, p_store(set), BLOCK_M) ||
+        !make_plane_map(&mapB, PB, n, pitchB, strideB, p_store(set), BLOCK_N))
+        return OZ_ERR_CUDA;
+
+    int dev = 0, sms = 148;
+    OZ_CUDA_CHECK(cudaGetDevice(&dev));
+    OZ_CUDA_CHECK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    int grid = static_cast<int>(p.total_items < sms ? p.total_items : sms);
+    if (rt.substrate == 0) {
+        OZ_CUDA_CHECK(cudaFuncSetAttribute(residue_gemm_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                           static_cast<int>(SMEM_BYTES)));
+        residue_gemm_kernel<0><<<grid, NUM_THREADS, SMEM_BYTES, stream>>>(mapA, mapB, p);
+    } else {
+        OZ_CUDA_CHECK(cudaFuncSetAttribute(residue_gemm_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                           static_cast<int>(SMEM_BYTES)));
+        residue_gemm_kernel<1><<<grid, NUM_THREADS, SMEM_BYTES, stream>>>(mapA, mapB, p);
+    }
+    count_launch();
+    OZ_CUDA_CHECK(cudaGetLastError());
+    return OZ_OK;
+}
+
+}  // namespace oz

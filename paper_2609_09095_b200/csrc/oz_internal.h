@@ -1,0 +1,116 @@
+// Internal declarations shared by the translation units of liboz_b200.so.
+// Nothing here is part of the public ABI (see include/oz.h).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "oz.h"
+
+namespace oz {
+
+constexpr int kMaxR = 13;          // moduli in the largest supported set (E)
+constexpr int kMaxPlanes = 33;     // stored planes of set E
+constexpr int kLutWords = 8208;    // >= sum of the moduli of either set (S: 8197, E: 6838)
+
+// ---- modulus sets (Sec. 2 step (ii) for S; "Candidate E" paragraph for E) ----------------
+__host__ __device__ constexpr int set_r(int set) { return set == 0 ? 12 : 13; }
+
+__host__ __device__ constexpr int modulus(int set, int i)
+{
+    constexpr int S[13] = {1089, 1024, 961, 841, 625, 529, 511, 509, 503, 499, 491, 487, 1};
+    constexpr int E[13] = {1089, 1024, 961, 841, 625, 529, 251, 247, 241, 239, 233, 229, 227};
+    return set == 0 ? S[i] : E[i];
+}
+
+// square root of a square modulus, 0 otherwise
+__host__ __device__ constexpr int square_root(int m)
+{
+    for (int s = 2; s * s <= m; ++s)
+        if (s * s == m) return s;
+    return 0;
+}
+
+__host__ __device__ constexpr int planes_of(int m) { return square_root(m) ? 2 : 3; }
+
+__host__ __device__ constexpr int first_plane(int set, int i)
+{
+    int p = 0;
+    for (int j = 0; j < i; ++j) p += planes_of(modulus(set, j));
+    return p;
+}
+
+__host__ __device__ constexpr int p_store(int set) { return first_plane(set, set_r(set)); }
+
+__host__ __device__ constexpr int lut_offset(int set, int i)
+{
+    int o = 0;
+    for (int j = 0; j < i; ++j) o += modulus(set, j);
+    return o;
+}
+
+// 2^e mod m
+__host__ __device__ constexpr uint32_t pow2_mod(int e, uint32_t m)
+{
+    uint32_t v = 1 % m;
+    for (int j = 0; j < e; ++j) v = (v * 2u) % m;
+    return v;
+}
+
+// floor(2^32 / m)
+__host__ __device__ constexpr uint32_t barrett_magic(uint32_t m)
+{
+    return static_cast<uint32_t>(0x100000000ull / m);
+}
+
+inline int64_t round_up(int64_t v, int64_t a) { return (v + a - 1) / a * a; }
+
+// ---- route decoding ----------------------------------------------------------------------
+struct Route {
+    int substrate;  // 0 fp8, 1 int8
+    int quant;      // 0 rn, 1 tz
+    int rule;       // 0 maxexp, 1 cs
+};
+bool decode_route(uint32_t route, Route *out);
+
+// ---- per-device state --------------------------------------------------------------------
+// Builds the lookup tables and constant blocks on the current device the first time it is used.
+oz_status_t ensure_device_ready();
+
+// device addresses of the per-device objects (valid after ensure_device_ready())
+const uint32_t *device_lut(int set, int substrate);  // kLutWords packed plane bytes
+unsigned int *device_status_word();
+
+void count_launch(int n = 1);
+
+// quantisation budgets (host)
+void budget_maxexp(int set, int64_t k, int *tA, int *tB);
+void cs_bound_squared(int set, int64_t k, uint64_t *lo, uint64_t *hi);  // G^2 as 128 bits
+
+// ---- stage launchers (host side of each .cu) ---------------------------------------------
+oz_status_t launch_deconstruct(int side, int64_t lines, int64_t k, const double *X, int64_t ldx,
+                               int set, const Route &rt, uint8_t *planes, int64_t plane_stride,
+                               int64_t row_pitch, int32_t *shift, void *scratch,
+                               cudaStream_t stream);
+
+oz_status_t launch_residue_gemm(int64_t m, int64_t n, int64_t k, const uint8_t *PA,
+                                int64_t strideA, int64_t pitchA, const uint8_t *PB,
+                                int64_t strideB, int64_t pitchB, int set, const Route &rt,
+                                uint16_t *R, int64_t ldr, int64_t mod_stride,
+                                cudaStream_t stream);
+
+oz_status_t launch_reconstruct(int64_t m, int64_t n, const uint16_t *R, int64_t ldr,
+                               int64_t mod_stride, const int32_t *shiftA, const int32_t *shiftB,
+                               int set, double alpha, double beta, double *C, int64_t ldc,
+                               cudaStream_t stream);
+
+// uploads the reconstruction constants of both sets to the current device
+oz_status_t upload_reconstruct_constants();
+
+#define OZ_CUDA_CHECK(expr)                                  \
+    do {                                                     \
+        cudaError_t e__ = (expr);                            \
+        if (e__ != cudaSuccess) return OZ_ERR_CUDA;          \
+    } while (0)
+
+}  // namespace oz

@@ -1,0 +1,227 @@
+// Reconstruction (Algorithm 3; Eq. 4-5 and the last step of Sec. 2 (iv)): residues -> the integer
+// c' in [-M/2, M/2), unscaled by 2^-(sigma_i + tau_j) and rounded once to FP64.
+//
+// The paper's SIMT branch walks Garner's mixed-radix digits (r(r-1)/2 multiply-reduce steps).
+// CRT fixes c' uniquely, so any exact evaluation gives the same integer; this kernel uses the
+// weighted form
+//     c' = sum_i t_i (M/m_i)  -  kappa M,     t_i = (c_i (M/m_i)^-1) mod m_i  (balanced),
+// with every M/m_i and M cut into three 38-bit chunks.  |t_i| <= (m_i+1)/2 < 2^10, so each of
+// the three chunk sums is an integer below 2^52 and is formed EXACTLY by FP64 fused
+// multiply-adds (the FP64 pipe is otherwise idle in this kernel).  kappa = round(S/M) comes from
+// a floating estimate and is then made exact by a 128-bit range test, so the result is the
+// unique representative in [-M/2, M/2) in every case.  The final conversion of the 128-bit
+// integer to FP64 is a single round-to-nearest-even done in integer arithmetic.
+#include <utility>
+
+#include "oz_internal.h"
+
+namespace oz {
+namespace {
+
+struct ReconConst {
+    float m[kMaxR];
+    float inv_m[kMaxR];
+    float q[kMaxR];            // (M/m_i)^-1 mod m_i
+    double W[kMaxR][3];        // M/m_i = W0 + W1 2^38 + W2 2^76
+    double Mc[3];              // M     = M0 + M1 2^38 + M2 2^76
+    double inv_M;              // 1/M (rounded)
+    unsigned long long M_lo, M_hi;
+};
+
+__constant__ ReconConst c_recon[2];
+
+constexpr double kTwo38 = 274877906944.0;             // 2^38
+constexpr double kTwoM38 = 1.0 / 274877906944.0;      // 2^-38
+constexpr double kTwo76 = kTwo38 * kTwo38;            // 2^76
+constexpr double kRint = 6755399441055744.0;          // 1.5 * 2^52: (x + kRint) - kRint = rint(x)
+
+// nearest double (ties to even) of a 128-bit integer times 2^scale
+__device__ __forceinline__ double i128_to_double(__int128 v, int scale)
+{
+    bool neg = v < 0;
+    unsigned __int128 a = neg ? static_cast<unsigned __int128>(0) - static_cast<unsigned __int128>(v)
+                              : static_cast<unsigned __int128>(v);
+    unsigned long long hi = static_cast<unsigned long long>(a >> 64);
+    unsigned long long lo = static_cast<unsigned long long>(a);
+    double d;
+    if (hi == 0) {
+        d = __ull2double_rn(lo);
+    } else {
+        int lz = __clzll(static_cast<long long>(hi));
+        unsigned long long top = lz ? ((hi << lz) | (lo >> (64 - lz))) : hi;
+        unsigned long long rest = lz ? (lo << lz) : lo;
+        top |= (rest != 0ull) ? 1ull : 0ull;     // sticky bit, far below the rounding position
+        d = __ull2double_rn(top);
+        scale += 64 - lz;
+    }
+    d = scalbn(d, scale);
+    return neg ? -d : d;
+}
+
+template <int SET, int I>
+__device__ __forceinline__ void crt_term(uint32_t c, double &S0, double &S1, double &S2)
+{
+    const ReconConst &K = c_recon[SET];
+    float cf = __uint_as_float(0x4B000000u | c) - 8388608.0f;          // exact: c < 2^16
+    float x = cf * K.q[I];                                              // < 2^21, exact
+    float quot = fmaf(x, K.inv_m[I], 12582912.0f) - 12582912.0f;        // rint(x / m) up to +-1
+    float t = fmaf(-quot, K.m[I], x);                                   // exact, |t| <= (m+1)/2
+    double td = static_cast<double>(t);
+    S0 = fma(td, K.W[I][0], S0);
+    S1 = fma(td, K.W[I][1], S1);
+    S2 = fma(td, K.W[I][2], S2);
+}
+
+template <int SET, int... I>
+__device__ __forceinline__ void crt_sum(std::integer_sequence<int, I...>, const uint32_t (&c)[kMaxR],
+                                        double &S0, double &S1, double &S2)
+{
+    (crt_term<SET, I>(c[I], S0, S1, S2), ...);
+}
+
+template <int SET>
+__device__ __forceinline__ double reconstruct_one(const uint32_t (&c)[kMaxR], int shift_sum)
+{
+    const ReconConst &K = c_recon[SET];
+    double S0 = 0.0, S1 = 0.0, S2 = 0.0;
+    crt_sum<SET>(std::make_integer_sequence<int, set_r(SET)>{}, c, S0, S1, S2);
+    double val = fma(S2, kTwo76, fma(S1, kTwo38, S0));
+    double kappa = (val * K.inv_M + kRint) - kRint;
+    double T0 = fma(-kappa, K.Mc[0], S0);
+    double T1 = fma(-kappa, K.Mc[1], S1);
+    double T2 = fma(-kappa, K.Mc[2], S2);
+    // carry-normalise so that the three chunks do not overlap
+    double c0 = (T0 * kTwoM38 + kRint) - kRint;
+    T0 = fma(-c0, kTwo38, T0);
+    T1 += c0;
+    double c1 = (T1 * kTwoM38 + kRint) - kRint;
+    T1 = fma(-c1, kTwo38, T1);
+    T2 += c1;
+    const __int128 one = 1;
+    __int128 v = static_cast<__int128>(__double2ll_rn(T2)) * (one << 76);
+    v += static_cast<__int128>(__double2ll_rn(T1)) * (one << 38);
+    v += static_cast<__int128>(__double2ll_rn(T0));
+    // exact lift to [-M/2, M/2)  (M is even for both sets)
+    const __int128 M = static_cast<__int128>((static_cast<unsigned __int128>(K.M_hi) << 64) | K.M_lo);
+    const __int128 Mh = M >> 1;
+    if (v >= Mh) v -= M;
+    else if (v < -Mh) v += M;
+    return i128_to_double(v, -shift_sum);
+}
+
+template <int SET>
+__global__ void __launch_bounds__(256)
+reconstruct_kernel(const uint16_t *__restrict__ R, int64_t ldr, int64_t mod_stride, int64_t m,
+                   int64_t n, const int32_t *__restrict__ shiftA, const int32_t *__restrict__ shiftB,
+                   double alpha, double beta, double *__restrict__ C, int64_t ldc, int vecR, int vecC)
+{
+    const int64_t pairs = (m + 1) >> 1;
+    int64_t idx = blockIdx.x * 256ll + threadIdx.x;
+    if (idx >= pairs * n) return;
+    int64_t j = idx / pairs;
+    int64_t row = (idx - j * pairs) * 2;
+    bool two = row + 1 < m;
+    constexpr int r = set_r(SET);
+
+    uint32_t c0[kMaxR], c1[kMaxR];
+    const uint16_t *base = R + j * ldr + row;
+#pragma unroll
+    for (int i = 0; i < r; ++i) {
+        if (vecR) {
+            uint32_t w = *reinterpret_cast<const uint32_t *>(base + i * mod_stride);
+            c0[i] = w & 0xFFFFu;
+            c1[i] = w >> 16;
+        } else {
+            c0[i] = base[i * mod_stride];
+            c1[i] = two ? base[i * mod_stride + 1] : 0u;
+        }
+    }
+    int sb = shiftB[j];
+    int sa0 = shiftA[row], sa1 = two ? shiftA[row + 1] : 0;
+    const double nan = __longlong_as_double(0x7FF8000000000000ll);
+    double p0 = (sb == OZ_NONFINITE_SHIFT || sa0 == OZ_NONFINITE_SHIFT) ? nan
+                                                                         : reconstruct_one<SET>(c0, sa0 + sb);
+    double p1 = 0.0;
+    if (two)
+        p1 = (sb == OZ_NONFINITE_SHIFT || sa1 == OZ_NONFINITE_SHIFT) ? nan
+                                                                      : reconstruct_one<SET>(c1, sa1 + sb);
+    p0 *= alpha;
+    p1 *= alpha;
+    double *out = C + row + j * ldc;
+    if (vecC && two) {
+        double2 o;
+        if (beta != 0.0) {
+            double2 old = *reinterpret_cast<const double2 *>(out);
+            o.x = old.x + p0;
+            o.y = old.y + p1;
+        } else {
+            o.x = p0;
+            o.y = p1;
+        }
+        *reinterpret_cast<double2 *>(out) = o;
+    } else {
+        out[0] = beta != 0.0 ? out[0] + p0 : p0;
+        if (two) out[1] = beta != 0.0 ? out[1] + p1 : p1;
+    }
+}
+
+}  // namespace
+
+oz_status_t upload_reconstruct_constants()
+{
+    static ReconConst host[2];
+    for (int set = 0; set < 2; ++set) {
+        unsigned __int128 M = 1;
+        for (int i = 0; i < set_r(set); ++i) M *= static_cast<unsigned>(modulus(set, i));
+        const unsigned __int128 mask = (static_cast<unsigned __int128>(1) << 38) - 1;
+        ReconConst &K = host[set];
+        for (int i = 0; i < kMaxR; ++i) {
+            K.m[i] = 1.0f; K.inv_m[i] = 1.0f; K.q[i] = 0.0f;
+            K.W[i][0] = K.W[i][1] = K.W[i][2] = 0.0;
+        }
+        for (int i = 0; i < set_r(set); ++i) {
+            unsigned mi = static_cast<unsigned>(modulus(set, i));
+            unsigned __int128 W = M / mi;
+            unsigned wm = static_cast<unsigned>(W % mi), inv = 0;
+            for (unsigned c = 1; c < mi; ++c)
+                if ((static_cast<unsigned long long>(wm) * c) % mi == 1) { inv = c; break; }
+            K.m[i] = static_cast<float>(mi);
+            K.inv_m[i] = 1.0f / static_cast<float>(mi);
+            K.q[i] = static_cast<float>(inv);
+            K.W[i][0] = static_cast<double>(static_cast<unsigned long long>(W & mask));
+            K.W[i][1] = static_cast<double>(static_cast<unsigned long long>((W >> 38) & mask));
+            K.W[i][2] = static_cast<double>(static_cast<unsigned long long>(W >> 76));
+        }
+        K.Mc[0] = static_cast<double>(static_cast<unsigned long long>(M & mask));
+        K.Mc[1] = static_cast<double>(static_cast<unsigned long long>((M >> 38) & mask));
+        K.Mc[2] = static_cast<double>(static_cast<unsigned long long>(M >> 76));
+        K.inv_M = 1.0 / static_cast<double>(M);
+        K.M_lo = static_cast<unsigned long long>(M);
+        K.M_hi = static_cast<unsigned long long>(M >> 64);
+    }
+    OZ_CUDA_CHECK(cudaMemcpyToSymbol(c_recon, host, sizeof(host)));
+    return OZ_OK;
+}
+
+oz_status_t launch_reconstruct(int64_t m, int64_t n, const uint16_t *R, int64_t ldr,
+                               int64_t mod_stride, const int32_t *shiftA, const int32_t *shiftB,
+                               int set, double alpha, double beta, double *C, int64_t ldc,
+                               cudaStream_t stream)
+{
+    int vecR = ((ldr & 1) == 0 && (mod_stride & 1) == 0 && (reinterpret_cast<uintptr_t>(R) & 3u) == 0) ? 1 : 0;
+    int vecC = ((ldc & 1) == 0 && (reinterpret_cast<uintptr_t>(C) & 15u) == 0) ? 1 : 0;
+    int64_t total = ((m + 1) >> 1) * n;
+    int64_t blocks = (total + 255) / 256;
+    if (blocks > 0x7FFFFFFFll) return OZ_ERR_UNSUPPORTED;
+    if (set == 0)
+        reconstruct_kernel<0><<<static_cast<unsigned>(blocks), 256, 0, stream>>>(
+            R, ldr, mod_stride, m, n, shiftA, shiftB, alpha, beta, C, ldc, vecR, vecC);
+    else
+        reconstruct_kernel<1><<<static_cast<unsigned>(blocks), 256, 0, stream>>>(
+            R, ldr, mod_stride, m, n, shiftA, shiftB, alpha, beta, C, ldc, vecR, vecC);
+    count_launch();
+    OZ_CUDA_CHECK(cudaGetLastError());
+    return OZ_OK;
+}
+
+}  // namespace oz

@@ -1,0 +1,99 @@
+"""Glue for the GPU parity tests: moves seeded host arrays to the device, calls the C-ABI
+through the Python binding, brings results back as numpy arrays.  No arithmetic of the method."""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+import paper_2609_09095_b200 as oz
+
+SETS = {"S": oz.OZ_SET_S, "E": oz.OZ_SET_E}
+
+
+def route(sub="fp8", quant="RN", rule="CS") -> int:
+    r = oz.OZ_SUB_FP8 if sub == "fp8" else oz.OZ_SUB_INT8
+    r |= oz.OZ_QUANT_RN if quant == "RN" else oz.OZ_QUANT_TZ
+    r |= oz.OZ_SCALE_CS if rule == "CS" else oz.OZ_SCALE_MAXEXP
+    return r
+
+
+def to_dev(X: np.ndarray) -> torch.Tensor:
+    """Column-major numpy matrix -> device tensor with the same memory image."""
+    assert X.flags.f_contiguous
+    return torch.from_numpy(np.ascontiguousarray(X.T)).cuda()
+
+
+def from_dev(t: torch.Tensor) -> np.ndarray:
+    return t.cpu().numpy().T
+
+
+def sync_status() -> int:
+    return oz.oz_query_status()
+
+
+def deconstruct(side: int, X: np.ndarray, set_name: str, rt: int):
+    lines = X.shape[0] if side == 0 else X.shape[1]
+    k = X.shape[1] if side == 0 else X.shape[0]
+    ldx = max(X.shape[0], 1)
+    r, p, _ = oz.oz_set_info(SETS[set_name])
+    pitch = oz.oz_row_pitch(k)
+    dX = to_dev(X) if X.size else torch.zeros(1, dtype=torch.float64, device="cuda")
+    planes = torch.full((p, lines, pitch), 0xAA, dtype=torch.uint8, device="cuda")
+    shift = torch.full((lines,), 12345, dtype=torch.int32, device="cuda")
+    scratch = torch.zeros(16 * lines + 256, dtype=torch.uint8, device="cuda")
+    oz.check(oz.oz_deconstruct(side, lines, k, dX, ldx, SETS[set_name], rt, planes, lines * pitch,
+                               pitch, shift, scratch), "oz_deconstruct")
+    st = sync_status()
+    return planes.cpu().numpy(), shift.cpu().numpy(), st
+
+
+def residue_gemm(PA: np.ndarray, PB: np.ndarray, k: int, set_name: str, rt: int, ldr=None):
+    p, m, pa = PA.shape
+    _, n, pb = PB.shape
+    r, _, _ = oz.oz_set_info(SETS[set_name])
+    ldr = m if ldr is None else ldr
+    dA, dB = torch.from_numpy(PA).cuda(), torch.from_numpy(PB).cuda()
+    R = torch.full((r, n, ldr), 0xFFFF, dtype=torch.uint16, device="cuda")
+    oz.check(oz.oz_residue_gemm(m, n, k, dA, m * pa, pa, dB, n * pb, pb, SETS[set_name], rt, R, ldr,
+                                n * ldr), "oz_residue_gemm")
+    st = sync_status()
+    return R.cpu().numpy()[:, :, :m], st
+
+
+def reconstruct(R: np.ndarray, sA: np.ndarray, sB: np.ndarray, set_name: str, alpha=1.0, beta=0.0,
+                C0: np.ndarray | None = None):
+    r, n, m = R.shape
+    dR = torch.from_numpy(np.ascontiguousarray(R)).cuda()
+    dC = to_dev(np.asfortranarray(C0)) if C0 is not None else torch.zeros((n, m), dtype=torch.float64, device="cuda")
+    oz.check(oz.oz_reconstruct(m, n, dR, m, n * m, torch.from_numpy(sA).cuda(), torch.from_numpy(sB).cuda(),
+                               SETS[set_name], alpha, beta, dC, m), "oz_reconstruct")
+    st = sync_status()
+    return from_dev(dC), st
+
+
+_ws = None
+
+
+def ensure_workspace(nbytes: int):
+    global _ws
+    if _ws is None or _ws.numel() < nbytes:
+        oz.oz_set_workspace(None)
+        _ws = None
+        torch.cuda.empty_cache()
+        _ws = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+    oz.check(oz.oz_set_workspace(_ws, _ws.numel()), "oz_set_workspace")
+    return _ws
+
+
+def dgemm(A: np.ndarray, B: np.ndarray, set_name: str, rt: int, alpha=1.0, beta=0.0,
+          C0: np.ndarray | None = None, keep_device=False):
+    m, k = A.shape
+    n = B.shape[1]
+    ensure_workspace(oz.oz_workspace_bytes(m, n, k, SETS[set_name], rt))
+    dA = to_dev(A) if A.size else torch.zeros(1, dtype=torch.float64, device="cuda")
+    dB = to_dev(B) if B.size else torch.zeros(1, dtype=torch.float64, device="cuda")
+    dC = to_dev(np.asfortranarray(C0)) if C0 is not None else torch.full((n, m), 7.0, dtype=torch.float64, device="cuda")
+    oz.check(oz.oz_dgemm_ex(m, n, k, alpha, dA, max(m, 1), dB, max(k, 1), beta, dC, max(m, 1),
+                            SETS[set_name], rt), "oz_dgemm_ex")
+    st = sync_status()
+    return (dC if keep_device else from_dev(dC)), st

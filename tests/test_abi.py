@@ -1,0 +1,40 @@
+"""The C-ABI library loads without a GPU and exports every symbol that include/oz.h declares."""
+import ctypes
+import os
+import re
+
+import paper_2609_09095_b200 as oz
+from paper_2609_09095_b200 import build as ozbuild
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def declared_functions():
+    text = open(os.path.join(ROOT, "include", "oz.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(oz_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_library_builds_and_exports_the_header():
+    ozbuild.build_library()
+    lib = ctypes.CDLL(oz.LIB_PATH)
+    names = declared_functions()
+    assert len(names) >= 12
+    for name in names:
+        assert hasattr(lib, name), name
+    assert sorted(names) == sorted(oz.EXPORTS)
+
+
+def test_host_only_queries():
+    r, p, mods = oz.oz_set_info(oz.OZ_SET_S)
+    assert (r, p) == (12, 30) and mods[0] == 1089 and mods[-1] == 487
+    r, p, mods = oz.oz_set_info(oz.OZ_SET_E)
+    assert (r, p) == (13, 33) and mods[-1] == 227
+    assert oz.oz_row_pitch(1) == 16 and oz.oz_row_pitch(5003) == 5008 and oz.oz_row_pitch(4096) == 4096
+    # planes of A and B + residues dominate the workspace
+    m, n, k = 16384, 16384, 1024
+    need = oz.oz_workspace_bytes(m, n, k, oz.OZ_SET_S, 0)
+    assert need >= 30 * (m + n) * k + 24 * m * n
+    assert need < 30 * (m + n) * k + 24 * m * n + (1 << 22)
+    assert oz.oz_workspace_bytes(m, n, k, 7, 0) == 0
+    assert "workspace" in oz.oz_status_string(oz.OZ_ERR_WORKSPACE)

@@ -1,0 +1,224 @@
+"""GPU parity: every stage entry point and the whole oz_dgemm, through the C-ABI, against the
+CPU oracle on the same seeded inputs.  Integer outputs (shifts, plane bytes, residues) must be
+bit-exact; FP64 outputs within 2 * 2^-53 * (|A||B|)_ij of the oracle and of a double-double GEMM."""
+import numpy as np
+import pytest
+
+import synth_inputs as syn
+from oracle import oz_oracle as ozo
+
+pytestmark = pytest.mark.gpu
+
+U = 2.0 ** -53
+OSET = {"S": ozo.SET_S, "E": ozo.SET_E}
+
+
+def _oracle_route(sub, quant, rule):
+    return (ozo.SUB_FP8 if sub == "fp8" else ozo.SUB_INT8,
+            ozo.QUANT_RN if quant == "RN" else ozo.QUANT_TZ,
+            ozo.SCALE_CS if rule == "CS" else ozo.SCALE_MAXEXP)
+
+
+def _oracle_deconstruct(side, X, set_name, sub, quant, rule):
+    osub, oq, orule = _oracle_route(sub, quant, rule)
+    k = X.shape[1] if side == 0 else X.shape[0]
+    tA, tB = ozo.budget_maxexp(OSET[set_name], max(k, 1))
+    sh = ozo.shifts(side, X, OSET[set_name], orule, tA if side == 0 else tB)
+    Q = ozo.quantise(side, X, sh, oq)
+    D = ozo.residues(Q, OSET[set_name])
+    return ozo.planes(D, OSET[set_name], osub), sh, D
+
+
+# ------------------------------------------------------------------ deconstruction (a1-a4)
+@pytest.mark.parametrize("side", [0, 1])
+@pytest.mark.parametrize("lines,k,dist", [(256, 256, "uniform"), (37, 129, "lognormal:2.0"),
+                                          (130, 1000, "normal"), (1, 1, "uniform"), (5, 17, "lognormal:0.5"),
+                                          (67, 4101, "lognormal:2.0"), (300, 16, "uniform")])
+@pytest.mark.parametrize("set_name,sub,quant,rule", [("S", "fp8", "RN", "CS"), ("S", "int8", "TZ", "MAXEXP"),
+                                                     ("E", "fp8", "TZ", "CS"), ("E", "int8", "RN", "MAXEXP")])
+def test_deconstruct_bit_exact(side, lines, k, dist, set_name, sub, quant, rule):
+    import tests.gpu_helpers as gh
+    rng = np.random.default_rng(100 + lines + k)
+    X = syn._draw(rng, lines, k, dist) if side == 0 else syn._draw(rng, k, lines, dist)
+    P, sh, st = gh.deconstruct(side, X, set_name, gh.route(sub, quant, rule))
+    Po, sho, _ = _oracle_deconstruct(side, X, set_name, sub, quant, rule)
+    assert st == 0
+    assert (sh == sho).all()
+    assert P.shape == Po.shape and (P == Po).all()
+
+
+@pytest.mark.parametrize("kind", ["zero_lines", "subnormal", "spike", "small_integers"])
+@pytest.mark.parametrize("rule", ["CS", "MAXEXP"])
+def test_deconstruct_edge_inputs(kind, rule):
+    import tests.gpu_helpers as gh
+    A, B = syn.special_operands(kind, 40, 24, 100)
+    for side, X in ((0, A), (1, B)):
+        P, sh, st = gh.deconstruct(side, X, "S", gh.route("fp8", "RN", rule))
+        Po, sho, _ = _oracle_deconstruct(side, X, "S", "fp8", "RN", rule)
+        assert st == 0 and (sh == sho).all() and (P == Po).all()
+
+
+def test_deconstruct_nonfinite_contract():
+    import tests.gpu_helpers as gh
+    import paper_2609_09095_b200 as oz
+    A, _ = syn.special_operands("spike", 16, 8, 40)
+    A[3, 7] = np.inf
+    A[9, 0] = np.nan
+    P, sh, st = gh.deconstruct(0, A, "S", gh.route())
+    Po, sho, _ = _oracle_deconstruct(0, A, "S", "fp8", "RN", "CS")
+    assert st == oz.OZ_ERR_NONFINITE_INPUT
+    assert sh[3] == oz.OZ_NONFINITE_SHIFT and sh[9] == oz.OZ_NONFINITE_SHIFT
+    assert (sh == sho).all() and (P == Po).all()
+    assert gh.sync_status() == 0   # the status word is cleared by the query
+
+
+# ------------------------------------------------------------------ residue GEMMs (a5-a6)
+def _random_planes(rng, set_name, sub, lines, k, extreme=False):
+    """Stored planes of random centred residues (or of the residues with the largest digits)."""
+    ms = ozo.modset(OSET[set_name])
+    D = np.zeros((len(ms), lines, k), dtype=np.int16)
+    for i, m in enumerate(ms):
+        lo, hi = -(m // 2), (m - 1) // 2
+        if extreme:
+            cand = sorted(range(lo, hi + 1), key=lambda d: -max(abs(v) for v in ozo.split(d, m)))[:4]
+            D[i] = rng.choice(cand, size=(lines, k))
+        else:
+            D[i] = rng.integers(lo, hi + 1, size=(lines, k))
+    osub = ozo.SUB_FP8 if sub == "fp8" else ozo.SUB_INT8
+    return ozo.planes(D, OSET[set_name], osub), D
+
+
+@pytest.mark.parametrize("m,n,k", [(128, 256, 128), (256, 512, 384), (200, 300, 200), (1, 1, 1),
+                                   (129, 257, 130), (3, 700, 17), (520, 40, 1000)])
+@pytest.mark.parametrize("set_name,sub", [("S", "fp8"), ("S", "int8"), ("E", "fp8")])
+def test_residue_gemm_bit_exact(m, n, k, set_name, sub):
+    import tests.gpu_helpers as gh
+    rng = np.random.default_rng(m * 7 + n * 3 + k)
+    PA, DA = _random_planes(rng, set_name, sub, m, k)
+    PB, DB = _random_planes(rng, set_name, sub, n, k)
+    R, st = gh.residue_gemm(PA, PB, k, set_name, gh.route(sub))
+    want = ozo.products(DA, DB, OSET[set_name])
+    assert st == 0
+    assert (R == want).all()
+
+
+@pytest.mark.parametrize("k", [4096, 5003, 32768])
+@pytest.mark.parametrize("sub", ["fp8", "int8"])
+def test_accumulation_is_exact_at_depth(k, sub):
+    """Planes made of the largest digits only: accumulators reach k*484 (non-square) and
+    k*512 (square, two K-loops in one accumulator) -- up to 2^24 at k = 32768."""
+    import tests.gpu_helpers as gh
+    rng = np.random.default_rng(k)
+    m, n = 130, 260
+    PA, DA = _random_planes(rng, "S", sub, m, k, extreme=True)
+    PB, DB = _random_planes(rng, "S", sub, n, k, extreme=True)
+    # make some rows all-equal so that terms do not cancel
+    PA[:, :8, :k] = PA[:, :1, :1]
+    PB[:, :8, :k] = PB[:, :1, :1]
+    want, worst = ozo.plane_products(PA, PB, k, ozo.SET_S, ozo.SUB_FP8 if sub == "fp8" else ozo.SUB_INT8)
+    assert worst > 0.9 * 256 * k
+    R, st = gh.residue_gemm(PA, PB, k, "S", gh.route(sub))
+    assert st == 0
+    assert (R == want).all()
+
+
+# ------------------------------------------------------------------ reconstruction (a7)
+@pytest.mark.parametrize("set_name", ["S", "E"])
+@pytest.mark.parametrize("m,n", [(256, 64), (1, 1), (7, 5), (130, 3)])
+def test_reconstruct_bit_exact(set_name, m, n):
+    import tests.gpu_helpers as gh
+    rng = np.random.default_rng(m + n)
+    ms = ozo.modset(OSET[set_name])
+    M = int(np.prod([int(v) for v in ms], dtype=object))
+    R = np.stack([rng.integers(0, mm, size=(n, m)) for mm in ms]).astype(np.uint16)
+    # boundary integers: -M/2, M/2-1, 0, +-1, and values whose conversion to double is a tie
+    special = [-(M // 2), M // 2 - 1, 0, 1, -1, 2**53 + 1, 2**54 + 2, -(2**60 + 2**7), 2**100 + 2**47,
+               2**100 + 3 * 2**47, -(2**100 + 2**47), 2**110 + 2**57 + 1]
+    flat = R.reshape(len(ms), -1)
+    for t, x in enumerate(special[: flat.shape[1]]):
+        flat[:, t] = [x % mm for mm in ms]
+    R = flat.reshape(len(ms), n, m)
+    sA = rng.integers(-60, 120, size=m).astype(np.int32)
+    sB = rng.integers(-60, 120, size=n).astype(np.int32)
+    C0 = np.asfortranarray(rng.standard_normal((m, n)))
+    CI = ozo.crt(R, OSET[set_name])
+    for alpha, beta in ((1.0, 0.0), (-1.0, 1.0), (-1.0, 0.0), (1.0, 1.0)):
+        got, st = gh.reconstruct(R, sA, sB, set_name, alpha, beta, C0)
+        want = ozo.output(CI, sA, sB, alpha, beta, C0)
+        assert st == 0
+        assert (got == want).all()
+
+
+# ------------------------------------------------------------------ whole method
+def _check_against_oracle_and_dd(A, B, got, want, C0=None, alpha=1.0, strict_dd=True):
+    hi, lo, ab = ozo.dd_gemm(A, B)
+    tol = 2 * U * ab
+    assert (np.abs(got - want) <= tol).all()
+    ref = alpha * hi if C0 is None else C0 + alpha * hi
+    err_dd = np.abs(got - ref) / np.maximum(tol + (0 if C0 is None else U * np.abs(ref)), 1e-300)
+    if strict_dd:
+        assert err_dd.max() <= 1.0
+    return float(err_dd.max())
+
+
+@pytest.mark.parametrize("cfg_id,m,n,k,sets", [(1, 256, 256, 256, ("S",)), (2, 300, 520, 4096, ("S",)),
+                                               (3, 384, 512, 1024, ("E", "S")), (4, 700, 128, 4096, ("S",)),
+                                               (5, 263, 301, 5003, ("S",))])
+def test_dgemm_configs_cut_down(cfg_id, m, n, k, sets):
+    import tests.gpu_helpers as gh
+    cfg = syn.CONFIGS[cfg_id]
+    A, B, C0 = syn.operands(cfg, m, n, k, want_c=True)
+    for set_name in sets:
+        for sub in cfg.substrates:
+            rt = gh.route(sub, "RN", "CS")
+            use_c0 = C0 if cfg.beta else None
+            got, st = gh.dgemm(A, B, set_name, rt, cfg.alpha, cfg.beta, use_c0)
+            want = ozo.dgemm(A, B, OSET[set_name], ozo.QUANT_RN, ozo.SCALE_CS, cfg.alpha, cfg.beta, use_c0)
+            assert st == 0
+            assert (got == want).all()      # the CRT is exact on both sides: bit-identical FP64
+            # cfg 5 (very wide exponent spread) is beyond what 12 moduli can deliver against the true product
+            _check_against_oracle_and_dd(A, B, got, want, use_c0, cfg.alpha, strict_dd=(cfg_id != 5))
+
+
+@pytest.mark.parametrize("quant,rule", [("TZ", "MAXEXP"), ("RN", "MAXEXP"), ("TZ", "CS")])
+def test_dgemm_variants(quant, rule):
+    import tests.gpu_helpers as gh
+    A, B = syn.operands(syn.CONFIGS[1], 130, 70, 200)
+    got, st = gh.dgemm(A, B, "S", gh.route("fp8", quant, rule))
+    _, oq, orule = _oracle_route("fp8", quant, rule)
+    want = ozo.dgemm(A, B, ozo.SET_S, oq, orule)
+    assert st == 0 and (got == want).all()
+
+
+def test_dgemm_edge_cases():
+    import tests.gpu_helpers as gh
+    import paper_2609_09095_b200 as oz
+    for kind in ("zero_lines", "subnormal", "spike", "small_integers"):
+        A, B = syn.special_operands(kind, 33, 17, 70)
+        got, st = gh.dgemm(A, B, "S", gh.route())
+        assert st == 0 and (got == ozo.dgemm(A, B)).all()
+    A, B = syn.special_operands("small_integers", 33, 17, 70)
+    assert (gh.dgemm(A, B, "E", gh.route())[0] == A @ B).all()          # exact integer product
+    A[4, 4] = np.nan
+    got, st = gh.dgemm(A, B, "S", gh.route())
+    want = ozo.dgemm(A, B)
+    assert st == oz.OZ_ERR_NONFINITE_INPUT
+    assert np.isnan(got[4, :]).all() and (np.isnan(got) == np.isnan(want)).all()
+    assert (got[~np.isnan(got)] == want[~np.isnan(want)]).all()
+    # k = 0: C = 0 (beta 0) or unchanged (beta 1); empty m or n: nothing to do
+    Z, st = gh.dgemm(np.zeros((5, 0), order="F"), np.zeros((0, 3), order="F"), "S", gh.route())
+    assert st == 0 and (Z == 0).all()
+
+
+def test_argument_errors_are_reported_on_the_host():
+    import torch
+    import paper_2609_09095_b200 as oz
+    t = torch.zeros(64, dtype=torch.float64, device="cuda")
+    assert oz.oz_dgemm(4, 4, 4, t, 2, t, 4, t, 4) == oz.OZ_ERR_INVALID_ARG          # lda < m
+    assert oz.oz_dgemm(4, 4, oz.OZ_K_MAX + 1, t, 4, t, oz.OZ_K_MAX + 1, t, 4) == oz.OZ_ERR_UNSUPPORTED
+    assert oz.oz_dgemm_ex(4, 4, 4, 2.0, t, 4, t, 4, 0.0, t, 4) == oz.OZ_ERR_UNSUPPORTED
+    assert oz.oz_dgemm(4, 4, 4, t, 4, t, 4, t, 4, 5, 0) == oz.OZ_ERR_INVALID_ARG        # unknown set
+    assert oz.oz_dgemm(4, 4, 4, t, 4, t, 4, t, 4, 0, 0x003) == oz.OZ_ERR_INVALID_ARG    # two substrates
+    oz.oz_set_workspace(None)
+    assert oz.oz_dgemm(4, 4, 4, t, 4, t, 4, t, 4) == oz.OZ_ERR_WORKSPACE
+    assert oz.oz_dgemm(0, 4, 4, t, 4, t, 4, t, 4) == oz.OZ_OK
