@@ -1,0 +1,317 @@
+#!/usr/bin/env python
+"""Benchmark of the emulated-FP64 GEMM hot path (deconstruct -> residue GEMMs -> reconstruct).
+
+One "step" is one oz_dgemm_ex call on the HPL trailing-update configuration
+(C(16384x16384) -= A(16384x1024) B(1024x16384), synthetic U(-1,1) operands), i.e. one pass of the
+whole hot path.  Prints ONE JSON line (rank 0):
+
+  value      emulated FP64 TFLOP/s = 2 m n k / time, inputs resident in HBM
+  e2e        same metric through oz_dgemm_host with pinned HOST buffers (copies timed)
+  roofline   the residue-GEMM kernel: 3 r plane products, low-precision FLOP/s against the
+             tensor peak (measured bf16 peak x 2 for 8-bit operands), timed with CUDA events
+             recorded on the launching stream between the stages
+  cpu_baseline  the CPU oracle, as it stands, on a bounded sample of the same workload
+
+`--impl reference` times the CPU oracle alone (there is no other implementation of the paper).
+N > 1 (torchrun): every rank runs the same independent problem (weak scaling, no collective in
+the data path); the time is the max over ranks, the value the sum of the work.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import synth_inputs as syn  # noqa: E402
+
+METRIC = "emulated FP64 TFLOPS (2mnk/s)"
+UNIT = "TFLOP/s"
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as fh:
+            d = json.load(fh)
+        return {"hbm_gbs": d["hbm_gbs"], "bf16": d["bf16_tflops"],
+                "bf16_sustained": d.get("bf16_tflops_sustained", d["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16": 1590.0, "bf16_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
+                 "-i", str(self.gpu), "-lms", "50"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, smax, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.lines:
+            f = [t.strip() for t in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1]))
+                smax.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, val in zip(names, f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        busy = [v for v in sm if v > 0.5 * max(sm)] or sm
+        return {"sm_mhz": statistics.median(busy), "sm_max_mhz": max(smax), "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+def aggregate_over_ranks(local_ms: float, local_work: float, world: int, reduce_max, reduce_sum):
+    """Whole-job numbers from per-rank ones: time = max over ranks, work = sum over ranks."""
+    ms = reduce_max(local_ms) if world > 1 else local_ms
+    work = reduce_sum(local_work) if world > 1 else local_work
+    return ms, work
+
+
+def oracle_sample_tflops(cfg, set_name: str, sample=(4096, 6144, 1024)):
+    """Times the CPU oracle (whole method) on a bounded sample of the workload."""
+    from oracle import oz_oracle as ozo
+    m, n, k = min(sample[0], cfg.m), min(sample[1], cfg.n), min(sample[2], cfg.k)
+    A, B, C0 = syn.operands(cfg, m, n, k, want_c=True)
+    oset = ozo.SET_S if set_name == "S" else ozo.SET_E
+    ozo.dgemm(np.asfortranarray(A[:32]), np.asfortranarray(B[:, :32]), oset)  # load the library, warm the threads
+    t0 = time.perf_counter()
+    ozo.dgemm(A, B, oset, ozo.QUANT_RN, ozo.SCALE_CS, cfg.alpha, cfg.beta, C0 if cfg.beta else None)
+    dt = time.perf_counter() - t0
+    return 2.0 * m * n * k / dt / 1e12, ozo.num_threads(), f"{m}x{n}x{k} block of the workload, {dt:.1f} s"
+
+
+def run_reference(args, cfg, set_name):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    vals = []
+    sample = (1024, 1536, 1024)
+    for i in range(args.warmup + args.steps):
+        v, cores, desc = oracle_sample_tflops(cfg, set_name, sample)
+        if i >= args.warmup:
+            vals.append(v)
+    value = len(vals) / sum(1.0 / v for v in vals)
+    ms = 2.0 * sample[0] * sample[1] * sample[2] / (value * 1e12) * 1e3
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "int64", "data": "synthetic",
+            "config": {"workload": cfg.name, "modulus_set": set_name, "m": cfg.m, "n": cfg.n, "k": cfg.k,
+                       "note": "CPU oracle; each step is a bounded sample of the workload"},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", type=int, default=3, help="synthetic configuration 1..5 (3 = HPL update)")
+    ap.add_argument("--set", dest="set_name", default="S", choices=["S", "E"])
+    ap.add_argument("--substrate", default="fp8", choices=["fp8", "int8"])
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3:
+        args.warmup = 3
+    cfg = syn.CONFIGS[args.config]
+    if args.impl == "reference":
+        run_reference(args, cfg, args.set_name)
+        return
+
+    import torch
+    import torch.distributed as dist
+    import paper_2609_09095_b200 as oz
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+
+    m, n, k = cfg.m, cfg.n, cfg.k
+    modset = oz.OZ_SET_S if args.set_name == "S" else oz.OZ_SET_E
+    route = (oz.OZ_SUB_FP8 if args.substrate == "fp8" else oz.OZ_SUB_INT8) | oz.OZ_QUANT_RN | oz.OZ_SCALE_CS
+    r, p_store, _ = oz.oz_set_info(modset)
+
+    # every rank owns an independent instance of the problem (weak scaling); seeds differ per rank
+    cfg_rank = syn.Config(**{**cfg.__dict__, "seed": cfg.seed + rank})
+    A, B, C0 = syn.operands(cfg_rank, want_c=True)
+    hA = torch.from_numpy(np.ascontiguousarray(A.T)).pin_memory()
+    hB = torch.from_numpy(np.ascontiguousarray(B.T)).pin_memory()
+    hC = torch.from_numpy(np.ascontiguousarray(C0.T)).pin_memory()
+    del A, B, C0
+    dA, dB, dC = hA.cuda(), hB.cuda(), hC.cuda()
+    core = oz.oz_workspace_bytes(m, n, k, modset, route)
+    ws_bytes = core + 8 * (m * k + k * n + m * n) + 4096
+    ws = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")
+    oz.check(oz.oz_set_workspace(ws, ws_bytes), "oz_set_workspace")
+    stream = torch.cuda.current_stream()
+
+    def step():
+        oz.check(oz.oz_dgemm_ex(m, n, k, cfg.alpha, dA, m, dB, k, cfg.beta, dC, m, modset, route, stream),
+                 "oz_dgemm_ex")
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        step()
+    oz.check(oz.oz_query_status(stream), "device status after warm-up")
+
+    # ---- timed region: K steps, per-stage events recorded by the library on the launching stream
+    stage_events = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(args.steps)]
+    for evs in stage_events:
+        for e in evs:
+            e.record(stream)  # materialise the handles
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler = ClockSampler(local_rank)
+    barrier()
+    sampler.start()
+    launches0 = oz.oz_launch_count()
+    ev0.record(stream)
+    for i in range(args.steps):
+        oz.oz_set_stage_events(stage_events[i])
+        step()
+    ev1.record(stream)
+    barrier()
+    launches = oz.oz_launch_count() - launches0
+    clocks = sampler.stop()
+    oz.oz_set_stage_events(None)
+    oz.check(oz.oz_query_status(stream), "device status after the timed steps")
+    local_ms = ev0.elapsed_time(ev1) / args.steps
+    stage_ms = np.array([[evs[i].elapsed_time(evs[i + 1]) for i in range(4)] for evs in stage_events]).mean(axis=0)
+
+    # ---- end to end through the host-buffer entry point (copies inside the timed region)
+    def e2e_step():
+        oz.check(oz.oz_dgemm_host(m, n, k, cfg.alpha, hA, m, hB, k, cfg.beta, hC, m, modset, route, stream),
+                 "oz_dgemm_host")
+
+    e2e_step()
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(args.e2e_steps):
+        e2e_step()
+    e1.record(stream)
+    barrier()
+    e2e_local_ms = e0.elapsed_time(e1) / args.e2e_steps
+    oz.check(oz.oz_query_status(stream), "device status after the end-to-end steps")
+
+    flops = 2.0 * m * n * k
+    if world > 1:
+        def rmax(v):
+            t = torch.tensor([v], dtype=torch.float64, device="cuda")
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            return float(t.item())
+
+        def rsum(v):
+            t = torch.tensor([v], dtype=torch.float64, device="cuda")
+            dist.all_reduce(t, op=dist.ReduceOp.SUM)
+            return float(t.item())
+    else:
+        rmax = rsum = None
+    ms, work = aggregate_over_ranks(local_ms, flops, world, rmax, rsum)
+    e2e_ms, _ = aggregate_over_ranks(e2e_local_ms, flops, world, rmax, rsum)
+
+    if rank == 0:
+        peaks = measured_peaks()
+        value = work / (ms * 1e-3) / 1e12
+        lowp_flops = 3.0 * r * flops                       # p_mma = 3r plane products
+        gemm_ms = float(stage_ms[2])
+        tensor_peak = 2.0 * peaks["bf16_sustained"]        # 8-bit operands: nominal 2x the bf16 rate
+        achieved = lowp_flops / (gemm_ms * 1e-3) / 1e12
+        roof_nominal = 4500.0 / (3 * r + 1)                # P_low/(3r+1) at B200's dense 8-bit rate
+        hbm = peaks["hbm_gbs"]
+        dec_bytes = (8 + 8 * 2 + p_store) * (m * k + k * n)   # max-exponent + sum-of-squares scans, convert read, planes written
+        rec_bytes = (2 * r + 8 + (8 if cfg.beta else 0)) * m * n
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "fp8_e4m3" if args.substrate == "fp8" else "int8",
+            "data": "synthetic",
+            "config": {"workload": cfg.name, "m": m, "n": n, "k": k, "alpha": cfg.alpha, "beta": cfg.beta,
+                       "modulus_set": args.set_name, "r": r, "substrate": args.substrate, "quantiser": "RN",
+                       "scale_rule": "CS",
+                       "l2": "inputs larger than L2 (126 MB): A+B %.0f MB, C %.0f MB, planes %.0f MB, residues %.0f MB"
+                             % (8e-6 * (m * k + k * n), 8e-6 * m * n, 1e-6 * p_store * (m + n) * k, 2e-6 * r * m * n),
+                       "parallelism": f"replicas x{world}" if world > 1 else "single GPU"},
+            "roof": {"definition": "P_low/(3r+1)", "nominal_tflops": roof_nominal,
+                     "frac_of_nominal": value / world / roof_nominal,
+                     "at_measured_peak_tflops": tensor_peak / (3 * r + 1),
+                     "frac_at_measured_peak": value / world / (tensor_peak / (3 * r + 1))},
+            "roofline": {"kernel": "residue_gemm_kernel (tcgen05)", "bound": "tensor", "achieved": achieved,
+                         "peak": tensor_peak, "unit": "TFLOP/s", "frac": achieved / tensor_peak,
+                         "peak_source": f"{peaks['source']} bf16 sustained x2 (8-bit operands)",
+                         "frac_of_nominal_4500": achieved / 4500.0, "traffic": None,
+                         "ms_per_launch": gemm_ms},
+            "stages": {
+                "deconstruct_A_ms": float(stage_ms[0]), "deconstruct_B_ms": float(stage_ms[1]),
+                "residue_gemm_ms": gemm_ms, "reconstruct_ms": float(stage_ms[3]),
+                "deconstruct_GBps": dec_bytes / ((stage_ms[0] + stage_ms[1]) * 1e-3) / 1e9,
+                "reconstruct_GBps": rec_bytes / (stage_ms[3] * 1e-3) / 1e9,
+                "hbm_peak_GBps": hbm, "hbm_peak_source": peaks["source"]},
+            "e2e": {"value": work / (e2e_ms * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": e2e_ms,
+                    "h2d_bytes_per_step": 8 * (m * k + k * n + (m * n if cfg.beta else 0)),
+                    "d2h_bytes_per_step": 8 * m * n, "steps": args.e2e_steps},
+            "gpu_launches": int(launches), "clocks": clocks,
+        }
+        if not args.no_cpu_baseline:
+            v, cores, desc = oracle_sample_tflops(cfg, args.set_name)
+            line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc}
+        print(json.dumps(line))
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

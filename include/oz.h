@@ -141,6 +141,13 @@ oz_status_t oz_reconstruct(int64_t m, int64_t n, const uint16_t *R, int64_t ldr,
  * (OZ_OK, OZ_ERR_NONFINITE_INPUT, OZ_ERR_RANGE, OZ_ERR_TIMEOUT or OZ_ERR_CUDA). */
 oz_status_t oz_query_status(void *stream);
 
+/* Optional per-stage timing hook for benchmarks (the paper's Algorithm 1 prices each stage
+ * separately).  `events` is a HOST array of 5 cudaEvent_t handles (as void*), or NULL to switch the
+ * hook off.  While set, oz_dgemm / oz_dgemm_ex record them on the call's stream: [0] before the
+ * first kernel, [1] after the deconstruction of A, [2] after the deconstruction of B, [3] after the
+ * residue GEMMs, [4] after the reconstruction.  The handles are copied; the caller owns the events. */
+oz_status_t oz_set_stage_events(void *const *events);
+
 /* Number of kernels launched by the library on this process since load (for benchmarks). */
 uint64_t oz_launch_count(void);
 

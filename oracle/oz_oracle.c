@@ -363,7 +363,10 @@ int ozo_planes(int64_t lines, int64_t k, const int16_t *D, int set, int substrat
 
 static int plane_digit(uint8_t byte, int substrate)
 {
-    if (substrate == OZO_SUB_FP8) return (int)ozo_e4m3_value(byte);
+    if (substrate == OZO_SUB_FP8) {
+        double v = ozo_e4m3_value(byte);
+        return (v == v) ? (int)v : 0; /* NaN codes never occur in stored planes */
+    }
     return (int)(int8_t)byte;
 }
 
@@ -401,6 +404,8 @@ int64_t ozo_plane_products(int64_t m, int64_t n, int64_t k, const uint8_t *PA,
 {
     int mod[16], r = ozo_modset(set, mod), plane = 0;
     int64_t worst = 0;
+    int digit_of[256]; /* value of every byte code on this substrate, decoded once */
+    for (int c = 0; c < 256; ++c) digit_of[c] = plane_digit((uint8_t)c, substrate);
     for (int i = 0; i < r; ++i) {
         int s = ozo_square_root(mod[i]);
         int np = s ? 2 : 3;
@@ -412,8 +417,8 @@ int64_t ozo_plane_products(int64_t m, int64_t n, int64_t k, const uint8_t *PA,
                 for (int64_t kk = 0; kk < k; ++kk) {
                     int a[3], b[3];
                     for (int q = 0; q < np; ++q) {
-                        a[q] = plane_digit(PA[(plane + q) * strideA + ii * pitchA + kk], substrate);
-                        b[q] = plane_digit(PB[(plane + q) * strideB + j * pitchB + kk], substrate);
+                        a[q] = digit_of[PA[(plane + q) * strideA + ii * pitchA + kk]];
+                        b[q] = digit_of[PB[(plane + q) * strideB + j * pitchB + kk]];
                     }
                     if (s) {
                         acc[0] += (int64_t)a[0] * b[0];

@@ -25,7 +25,7 @@ OZ_NONFINITE_SHIFT = -(2 ** 31)
 
 EXPORTS = ["oz_set_info", "oz_row_pitch", "oz_workspace_bytes", "oz_set_workspace", "oz_dgemm",
            "oz_dgemm_ex", "oz_dgemm_host", "oz_deconstruct", "oz_residue_gemm", "oz_reconstruct",
-           "oz_query_status", "oz_launch_count", "oz_status_string"]
+           "oz_query_status", "oz_set_stage_events", "oz_launch_count", "oz_status_string"]
 
 __all__ = EXPORTS + ["EXPORTS", "OzError", "load", "check", "LIB_PATH", "OZ_OK", "OZ_ERR_INVALID_ARG",
                      "OZ_ERR_UNSUPPORTED", "OZ_ERR_WORKSPACE", "OZ_ERR_CUDA",
@@ -66,6 +66,7 @@ def load() -> C.CDLL:
                                     i64, vp]
     lib.oz_reconstruct.argtypes = [i64, i64, vp, i64, i64, vp, vp, i32, dbl, dbl, vp, i64, vp]
     lib.oz_query_status.argtypes = [vp]
+    lib.oz_set_stage_events.argtypes = [C.POINTER(vp)]
     lib.oz_launch_count.restype = C.c_uint64
     lib.oz_status_string.argtypes = [i32]
     lib.oz_status_string.restype = C.c_char_p
@@ -162,6 +163,15 @@ def oz_reconstruct(m, n, R, ldr, mod_stride, shiftA, shiftB, modset, alpha, beta
 
 def oz_query_status(stream=None) -> int:
     return load().oz_query_status(_stream(stream))
+
+
+def oz_set_stage_events(events) -> int:
+    """events: five torch.cuda.Event objects (already recorded once, so their handles exist),
+    five raw cudaEvent_t addresses, or None."""
+    if events is None:
+        return load().oz_set_stage_events(None)
+    arr = (C.c_void_p * 5)(*[e if isinstance(e, int) else e.cuda_event for e in events])
+    return load().oz_set_stage_events(arr)
 
 
 def oz_launch_count() -> int:

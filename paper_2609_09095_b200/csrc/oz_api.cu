@@ -24,6 +24,8 @@ unsigned int *g_status_addr[kMaxDevices] = {};
 void *g_workspace[kMaxDevices] = {};
 size_t g_workspace_bytes[kMaxDevices] = {};
 std::atomic<uint64_t> g_launches{0};
+cudaEvent_t g_stage_events[5] = {};
+bool g_stage_events_on = false;
 
 // Is the integer v exactly representable in E4M3 (the set of Lemma 1)?  If so return its
 // byte code through *code.  OCP E4M3: bias 7, 3 mantissa bits, largest finite value 448.
@@ -244,15 +246,23 @@ oz_status_t dgemm_impl(int64_t m, int64_t n, int64_t k, double alpha, const doub
     uint8_t *PB = reinterpret_cast<uint8_t *>(ws + L.PB);
     uint16_t *R = reinterpret_cast<uint16_t *>(ws + L.R);
 
+    const bool ev = g_stage_events_on;
+    if (ev) OZ_CUDA_CHECK(cudaEventRecord(g_stage_events[0], stream));
     st = launch_deconstruct(0, m, k, A, lda, set, rt, PA, L.strideA, L.pitch, shiftA, ws + L.scrA, stream);
     if (st != OZ_OK) return st;
+    if (ev) OZ_CUDA_CHECK(cudaEventRecord(g_stage_events[1], stream));
     st = launch_deconstruct(1, n, k, B, ldb, set, rt, PB, L.strideB, L.pitch, shiftB, ws + L.scrB, stream);
     if (st != OZ_OK) return st;
+    if (ev) OZ_CUDA_CHECK(cudaEventRecord(g_stage_events[2], stream));
     st = launch_residue_gemm(m, n, k, PA, L.strideA, L.pitch, PB, L.strideB, L.pitch, set, rt, R,
                              L.ldr, L.mod_stride, stream);
     if (st != OZ_OK) return st;
-    return launch_reconstruct(m, n, R, L.ldr, L.mod_stride, shiftA, shiftB, set, alpha, beta, C,
-                              ldc, stream);
+    if (ev) OZ_CUDA_CHECK(cudaEventRecord(g_stage_events[3], stream));
+    st = launch_reconstruct(m, n, R, L.ldr, L.mod_stride, shiftA, shiftB, set, alpha, beta, C, ldc,
+                            stream);
+    if (st != OZ_OK) return st;
+    if (ev) OZ_CUDA_CHECK(cudaEventRecord(g_stage_events[4], stream));
+    return OZ_OK;
 }
 
 }  // namespace
@@ -420,6 +430,18 @@ oz_status_t oz_query_status(void *stream)
     if (word[0] & (1u << OZ_ERR_TIMEOUT)) return OZ_ERR_TIMEOUT;
     if (word[0] & (1u << OZ_ERR_RANGE)) return OZ_ERR_RANGE;
     if (word[0] & (1u << OZ_ERR_NONFINITE_INPUT)) return OZ_ERR_NONFINITE_INPUT;
+    return OZ_OK;
+}
+
+oz_status_t oz_set_stage_events(void *const *events)
+{
+    std::lock_guard<std::mutex> lock(g_mutex);
+    g_stage_events_on = events != nullptr;
+    for (int i = 0; i < 5; ++i)
+        g_stage_events[i] = events ? static_cast<cudaEvent_t>(events[i]) : nullptr;
+    if (events)
+        for (int i = 0; i < 5; ++i)
+            if (!events[i]) { g_stage_events_on = false; return OZ_ERR_INVALID_ARG; }
     return OZ_OK;
 }
 
