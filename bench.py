@@ -154,12 +154,16 @@ def main():
     ap.add_argument("--config", type=int, default=3, help="synthetic configuration 1..5 (3 = HPL update)")
     ap.add_argument("--set", dest="set_name", default="S", choices=["S", "E"])
     ap.add_argument("--substrate", default="fp8", choices=["fp8", "int8"])
+    ap.add_argument("--shape", default=None, help="m,n,k override (same distribution and seed as --config)")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
     cfg = syn.CONFIGS[args.config]
+    if args.shape:
+        sm_, sn_, sk_ = [int(v) for v in args.shape.split(",")]
+        cfg = syn.Config(**{**cfg.__dict__, "m": sm_, "n": sn_, "k": sk_, "name": cfg.name + "_shape_" + args.shape.replace(",", "x")})
     if args.impl == "reference":
         run_reference(args, cfg, args.set_name)
         return

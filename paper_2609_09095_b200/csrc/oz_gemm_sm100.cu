@@ -10,15 +10,21 @@
 //   non-square:  job 0 = D0.E0 (-15);  job 1 = DS.ES (16);  job 2 = D1.E1 (240)
 // Three MMA K-loops per modulus either way (p_mma = 3r).
 //
-// Kernel structure (one persistent CTA per SM, 320 threads):
-//   warp 0      TMA producer: 128-byte-swizzled K-major tiles of A (128 rows) and B (256 rows)
-//               into a 4-stage shared-memory ring, no multicast
-//   warp 1      MMA issuer: one lane issues tcgen05.mma (M=128, N=256, K=32, cta_group::1);
-//               accumulators live in TMEM, two slots of 256 columns used alternately per job
-//   warps 2..9  epilogue: tcgen05.ld the finished slot, reduce each accumulator modulo m_i in
-//               FP32 (all values are integers below 2^24, every step exact), fold it with the
-//               job's weight into a per-thread running combination held in registers, release
-//               the slot; after the last job reduce once more and store 16-bit residues
+// The tile is computed transposed: the MMA's M dimension (128 TMEM lanes) runs over 128 columns
+// j of C (planes of B), its N dimension (256 TMEM columns) over 256 rows i of C (planes of A).
+// An epilogue thread therefore owns one column j and a run of consecutive rows, which is
+// contiguous in the column-major residue array: 16-byte stores, no staging.
+//
+// Kernel structure (one persistent CTA per SM, 640 threads, 96 registers each):
+//   warp 0       TMA producer: 128-byte-swizzled K-major tiles of B (128 lines) and A (256 lines)
+//                into a 4-stage shared-memory ring, no multicast
+//   warp 1       MMA issuer: one lane issues tcgen05.mma (M=128, N=256, K=32, cta_group::1);
+//                accumulators live in TMEM, two slots of 256 columns used alternately per job
+//   warps 4..19  epilogue (4 per TMEM lane quarter, 64 columns each): tcgen05.ld the finished slot,
+//                reduce each accumulator modulo m_i in FP32 (all values are integers below 2^24,
+//                every step exact), fold it with the job's weight into a per-thread running
+//                combination held in registers, release the slot; after the last job reduce once
+//                more and store 16-bit residues
 // so the epilogue of one job overlaps the K-loop of the next, and TMEM never needs the three
 // accumulators of a non-square modulus at once.
 //
@@ -36,18 +42,19 @@
 namespace oz {
 namespace {
 
-constexpr int BLOCK_M = 128;
-constexpr int BLOCK_N = 256;
+constexpr int BLOCK_M = 128;                       // MMA M: columns j of C (lines of B)
+constexpr int BLOCK_N = 256;                       // MMA N: rows i of C (lines of A)
 constexpr int BLOCK_K = 128;                       // bytes = elements (8-bit operands)
 constexpr int UMMA_K = 32;                         // 8-bit operands: 32 elements per instruction
 constexpr int STAGES = 4;
-constexpr int A_BYTES = BLOCK_M * BLOCK_K;         // 16 KiB
-constexpr int B_BYTES = BLOCK_N * BLOCK_K;         // 32 KiB
+constexpr int A_BYTES = BLOCK_M * BLOCK_K;         // 16 KiB: MMA operand a = tile of B's planes
+constexpr int B_BYTES = BLOCK_N * BLOCK_K;         // 32 KiB: MMA operand b = tile of A's planes
 constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
 constexpr int TMEM_COLS = 512;                     // two accumulator slots of BLOCK_N columns
-constexpr int NUM_THREADS = 320;
-constexpr int EPI_WARPS = 8;
-constexpr int COLS_PER_WARP = BLOCK_N / 2;         // two warps share a TMEM lane quarter
+constexpr int NUM_THREADS = 640;
+constexpr int FIRST_EPI_WARP = 4;                  // warps 0..3: producer, MMA issuer, two idle
+constexpr int EPI_WARPS = 16;
+constexpr int COLS_PER_WARP = BLOCK_N / 4;         // four warps share a TMEM lane quarter
 constexpr size_t SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
 
 struct ModInfo {
@@ -59,7 +66,8 @@ struct ModInfo {
 
 struct GemmParams {
     int64_t m, n, k;
-    int tiles_m, tiles_n, nk;       // nk = K chunks of BLOCK_K
+    int tiles_m, tiles_n, nk;       // tiles of 256 rows / 128 columns of C; nk = K chunks of BLOCK_K
+    int vec_store;                  // R rows 16-byte aligned: use vector stores
     int r;
     int64_t total_items;
     uint16_t *R;
@@ -113,10 +121,13 @@ __device__ __forceinline__ unsigned long long global_timer_ns()
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s per wait
 
 // Bounded wait.  Returns false when the wait ran out or another role already gave up.
+// The timer is read only after a long run of failed polls: the common path never touches it.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag,
                                           unsigned int *status)
 {
-    if (mbar_try_wait(bar, parity)) return true;
+#pragma unroll 1
+    for (int it = 0; it < 4096; ++it)
+        if (mbar_try_wait(bar, parity)) return true;
     unsigned long long start = global_timer_ns();
     for (;;) {
 #pragma unroll 1
@@ -299,9 +310,9 @@ residue_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
     tc_fence_after();
     const uint32_t tmem_base = *tmem_base_ptr;
 
-    if (warp == 0) {
-        // ------------------------------------------------------------ TMA producer
-        if (lane == 0) {
+    if (warp < FIRST_EPI_WARP) {
+        if (warp == 0 && lane == 0) {
+            // -------------------------------------------------------- TMA producer
             int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
@@ -319,8 +330,8 @@ residue_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
                             uint32_t fb = full_bar + 8 * stage;
                             mbar_expect_tx(fb, STAGE_BYTES);
                             uint32_t sa = tiles + stage * STAGE_BYTES;
-                            tma_load_3d(sa, &mapA, fb, kc * BLOCK_K, it.tm * BLOCK_M, pa);
-                            tma_load_3d(sa + A_BYTES, &mapB, fb, kc * BLOCK_K, it.tn * BLOCK_N, pb);
+                            tma_load_3d(sa, &mapB, fb, kc * BLOCK_K, it.tn * BLOCK_M, pb);
+                            tma_load_3d(sa + A_BYTES, &mapA, fb, kc * BLOCK_K, it.tm * BLOCK_N, pa);
                             if (++stage == STAGES) { stage = 0; phase ^= 1u; }
                         }
                     }
@@ -331,10 +342,8 @@ residue_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
                 unsigned long long t0 = global_timer_ns();
                 while (global_timer_ns() - t0 < 2000000ull) { }
             }
-        }
-    } else if (warp == 1) {
-        // ------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
+        } else if (warp == 1 && lane == 0) {
+            // -------------------------------------------------------- MMA issuer
             constexpr uint32_t idesc = instr_desc<SUB>();
             int stage = 0;
             uint32_t phase = 0;
@@ -380,8 +389,8 @@ residue_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
         }
     } else {
         // ------------------------------------------------------------ epilogue
-        const int q = warp & 3;                       // TMEM lane quarter this warp may read
-        const int half = (warp - 2) >> 2;             // which half of the tile's columns
+        const int q = warp & 3;                              // TMEM lane quarter this warp may read
+        const int part = (warp - FIRST_EPI_WARP) >> 2;       // which 64 of the tile's 256 TMEM columns
         int slot = 0;
         uint32_t slot_phase = 0;   // bit s = phase of slot s
         bool ok = true;
@@ -398,7 +407,7 @@ residue_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
                 tc_fence_after();
                 const float wj = mi.w[job];
                 const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) +
-                                       static_cast<uint32_t>(slot * BLOCK_N + half * COLS_PER_WARP);
+                                       static_cast<uint32_t>(slot * BLOCK_N + part * COLS_PER_WARP);
 #pragma unroll
                 for (int c0 = 0; c0 < COLS_PER_WARP; c0 += 32) {
                     uint32_t v[32];
@@ -419,20 +428,35 @@ residue_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
                 slot ^= 1;
             }
             if (!ok) break;
-            const int64_t row = static_cast<int64_t>(it.tm) * BLOCK_M + q * 32 + lane;
-            const int64_t col0 = static_cast<int64_t>(it.tn) * BLOCK_N + half * COLS_PER_WARP;
-            if (row < p.m) {
-                uint16_t *dst = p.R + it.mod * p.mod_stride + col0 * p.ldr + row;
+            // this thread: column j of C, rows i0 .. i0+63 (contiguous in the residue array)
+            const int64_t j = static_cast<int64_t>(it.tn) * BLOCK_M + q * 32 + lane;
+            const int64_t i0 = static_cast<int64_t>(it.tm) * BLOCK_N + part * COLS_PER_WARP;
+            if (j < p.n && i0 < p.m) {
+                uint16_t *dst = p.R + it.mod * p.mod_stride + j * p.ldr + i0;
+                uint32_t packed[COLS_PER_WARP / 2];
 #pragma unroll
-                for (int c = 0; c < COLS_PER_WARP; ++c) {
-                    if (col0 + c < p.n) {
-                        float t = comb[c];
+                for (int c = 0; c < COLS_PER_WARP; c += 2) {
+                    uint32_t bits[2];
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        float t = comb[c + h];
                         float quot = fmaf(t, inv_m, 12582912.0f) - 12582912.0f;
                         float res = fmaf(-quot, mm, t);
-                        res = res < 0.0f ? res + mm : res;                           // canonical [0, m)
-                        uint32_t bits = __float_as_uint(res + 8388608.0f);           // integer in the low mantissa bits
-                        dst[c * p.ldr] = static_cast<uint16_t>(bits & 0xFFFFu);
+                        res = res < 0.0f ? res + mm : res;                       // canonical [0, m)
+                        bits[h] = __float_as_uint(res + 8388608.0f);             // integer in the low mantissa bits
                     }
+                    packed[c >> 1] = __byte_perm(bits[0], bits[1], 0x5410);
+                }
+                if (p.vec_store && i0 + COLS_PER_WARP <= p.m) {
+#pragma unroll
+                    for (int c = 0; c < COLS_PER_WARP / 8; ++c)
+                        *reinterpret_cast<uint4 *>(dst + 8 * c) =
+                            make_uint4(packed[4 * c], packed[4 * c + 1], packed[4 * c + 2], packed[4 * c + 3]);
+                } else {
+#pragma unroll
+                    for (int c = 0; c < COLS_PER_WARP; ++c)
+                        if (i0 + c < p.m)
+                            dst[c] = static_cast<uint16_t>((packed[c >> 1] >> (16 * (c & 1))) & 0xFFFFu);
                 }
             }
         }
@@ -492,8 +516,9 @@ oz_status_t launch_residue_gemm(int64_t m, int64_t n, int64_t k, const uint8_t *
 {
     GemmParams p{};
     p.m = m; p.n = n; p.k = k;
-    p.tiles_m = static_cast<int>((m + BLOCK_M - 1) / BLOCK_M);
-    p.tiles_n = static_cast<int>((n + BLOCK_N - 1) / BLOCK_N);
+    p.tiles_m = static_cast<int>((m + BLOCK_N - 1) / BLOCK_N);   // 256 rows of C per tile
+    p.tiles_n = static_cast<int>((n + BLOCK_M - 1) / BLOCK_M);   // 128 columns of C per tile
+    p.vec_store = ((ldr & 7) == 0 && (mod_stride & 7) == 0 && (reinterpret_cast<uintptr_t>(R) & 15u) == 0) ? 1 : 0;
     p.nk = static_cast<int>((k + BLOCK_K - 1) / BLOCK_K);
     p.r = set_r(set);
     p.total_items = static_cast<int64_t>(p.r) * p.tiles_m * p.tiles_n;
@@ -515,8 +540,8 @@ oz_status_t launch_residue_gemm(int64_t m, int64_t n, int64_t k, const uint8_t *
     if (k == 0) p.nk = 1;   // one all-zero chunk (the planes' padding) gives residues 0
 
     CUtensorMap mapA, mapB;
-    if (!make_plane_map(&mapA, PA, m, pitchA, strideA, p_store(set), BLOCK_M) ||
-        !make_plane_map(&mapB, PB, n, pitchB, strideB, p_store(set), BLOCK_N))
+    if (!make_plane_map(&mapA, PA, m, pitchA, strideA, p_store(set), BLOCK_N) ||
+        !make_plane_map(&mapB, PB, n, pitchB, strideB, p_store(set), BLOCK_M))
         return OZ_ERR_CUDA;
 
     int dev = 0, sms = 148;
