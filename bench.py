@@ -158,7 +158,7 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
-    if args.warmup < 3:
+    if args.warmup < 3 and args.impl != "reference":
         args.warmup = 3
     cfg = syn.CONFIGS[args.config]
     if args.shape:

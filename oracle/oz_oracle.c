@@ -339,23 +339,29 @@ int ozo_planes(int64_t lines, int64_t k, const int16_t *D, int set, int substrat
     int mod[16], r = ozo_modset(set, mod), plane = 0, bad = 0;
     for (int i = 0; i < r; ++i) {
         int np = ozo_planes_of(mod[i]);
-        for (int64_t l = 0; l < lines; ++l) {
-            for (int64_t kk = 0; kk < row_pitch; ++kk) {
-                int dg[3] = {0, 0, 0};
-                if (kk < k) ozo_split(D[((int64_t)i * lines + l) * k + kk], mod[i], dg);
-                for (int q = 0; q < np; ++q) {
-                    int byte;
-                    if (substrate == OZO_SUB_FP8) {
-                        byte = ozo_e4m3_encode(dg[q]);
-                        if (byte < 0) { bad = 1; byte = 0x7F; }
-                    } else {
-                        if (dg[q] < -128 || dg[q] > 127) bad = 1;
-                        byte = dg[q] & 0xFF;
-                    }
-                    P[(int64_t)(plane + q) * plane_stride + l * row_pitch + kk] = (uint8_t)byte;
+        /* bytes of every centred residue of this modulus, worked out once (index d + 1024) */
+        static uint8_t code[2048][3];
+        for (int d = -(mod[i] / 2); 2 * d < mod[i]; ++d) {
+            int dg[3] = {0, 0, 0};
+            ozo_split(d, mod[i], dg);
+            for (int q = 0; q < np; ++q) {
+                int byte;
+                if (substrate == OZO_SUB_FP8) {
+                    byte = ozo_e4m3_encode(dg[q]);
+                    if (byte < 0) { bad = 1; byte = 0x7F; }
+                } else {
+                    if (dg[q] < -128 || dg[q] > 127) bad = 1;
+                    byte = dg[q] & 0xFF;
                 }
+                code[d + 1024][q] = (uint8_t)byte;
             }
         }
+        for (int64_t l = 0; l < lines; ++l)
+            for (int64_t kk = 0; kk < row_pitch; ++kk)
+                for (int q = 0; q < np; ++q) {
+                    int d = kk < k ? D[((int64_t)i * lines + l) * k + kk] : 0;
+                    P[(int64_t)(plane + q) * plane_stride + l * row_pitch + kk] = code[d + 1024][q];
+                }
         plane += np;
     }
     return bad ? -1 : plane;
