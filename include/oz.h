@@ -118,6 +118,23 @@ oz_status_t oz_deconstruct(int side, int64_t lines, int64_t k, const double *X, 
                            int64_t plane_stride, int64_t row_pitch, int32_t *shift,
                            void *scratch, void *stream);
 
+/* oz_deconstruct for callers that cannot allocate device memory (no counterpart in the paper: it
+ * is a packaging variant, not a step of the method).  Identical to oz_deconstruct except that the
+ * scan scratch is a fixed array inside the library (16 * OZ_STATIC_MAX_LINES + 256 bytes, held by
+ * every GPU that loads the library until the process exits), so there is no `scratch` argument
+ * and the call performs no device allocation of any kind.
+ *   - lines > OZ_STATIC_MAX_LINES returns OZ_ERR_WORKSPACE with nothing enqueued.
+ *   - The first call on a device looks the array's device address up (a host-side query, once per
+ *     device, with that device current); make that first call before starting a stream capture.
+ *   - All calls on a device share the one array.  Each call clears what it uses before use, so
+ *     results never depend on an earlier call; but two calls whose kernels overlap on the GPU
+ *     (different streams, no ordering between them) race on it.  Serialise them. */
+#define OZ_STATIC_MAX_LINES 262144
+oz_status_t oz_deconstruct_static(int side, int64_t lines, int64_t k, const double *X, int64_t ldx,
+                                  oz_modset_t set, uint32_t route, uint8_t *planes,
+                                  int64_t plane_stride, int64_t row_pitch, int32_t *shift,
+                                  void *stream);
+
 /* Residue products (Eq. 3 through the plane identities of Sec. 2 "FP8 variant" and Eq. 8):
  * for every modulus i,  R_i = (A_i B_i) mod m_i  from the stored planes of A (lines = m) and
  * B (lines = n), on the tensor cores.  Output R[i*mod_stride + j*ldr + row], uint16 in [0, m_i).

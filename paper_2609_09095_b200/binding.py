@@ -22,16 +22,18 @@ OZ_QUANT_RN, OZ_QUANT_TZ = 0x010, 0x020
 OZ_SCALE_MAXEXP, OZ_SCALE_CS = 0x100, 0x200
 OZ_K_MAX = 32768
 OZ_NONFINITE_SHIFT = -(2 ** 31)
+OZ_STATIC_MAX_LINES = 262144
 
 EXPORTS = ["oz_set_info", "oz_row_pitch", "oz_workspace_bytes", "oz_set_workspace", "oz_dgemm",
-           "oz_dgemm_ex", "oz_dgemm_host", "oz_deconstruct", "oz_residue_gemm", "oz_reconstruct",
+           "oz_dgemm_ex", "oz_dgemm_host", "oz_deconstruct", "oz_deconstruct_static",
+           "oz_residue_gemm", "oz_reconstruct",
            "oz_query_status", "oz_set_stage_events", "oz_launch_count", "oz_status_string"]
 
 __all__ = EXPORTS + ["EXPORTS", "OzError", "load", "check", "LIB_PATH", "OZ_OK", "OZ_ERR_INVALID_ARG",
                      "OZ_ERR_UNSUPPORTED", "OZ_ERR_WORKSPACE", "OZ_ERR_CUDA",
                      "OZ_ERR_NONFINITE_INPUT", "OZ_ERR_RANGE", "OZ_ERR_TIMEOUT", "OZ_SET_S",
                      "OZ_SET_E", "OZ_SUB_FP8", "OZ_SUB_INT8", "OZ_QUANT_RN", "OZ_QUANT_TZ",
-                     "OZ_SCALE_MAXEXP", "OZ_SCALE_CS", "OZ_K_MAX", "OZ_NONFINITE_SHIFT"]
+                     "OZ_SCALE_MAXEXP", "OZ_SCALE_CS", "OZ_K_MAX", "OZ_NONFINITE_SHIFT", "OZ_STATIC_MAX_LINES"]
 
 _lib = None
 
@@ -62,6 +64,7 @@ def load() -> C.CDLL:
     lib.oz_dgemm_ex.argtypes = [i64, i64, i64, dbl, vp, i64, vp, i64, dbl, vp, i64, i32, u32, vp]
     lib.oz_dgemm_host.argtypes = lib.oz_dgemm_ex.argtypes
     lib.oz_deconstruct.argtypes = [i32, i64, i64, vp, i64, i32, u32, vp, i64, i64, vp, vp, vp]
+    lib.oz_deconstruct_static.argtypes = [i32, i64, i64, vp, i64, i32, u32, vp, i64, i64, vp, vp]
     lib.oz_residue_gemm.argtypes = [i64, i64, i64, vp, i64, i64, vp, i64, i64, i32, u32, vp, i64,
                                     i64, vp]
     lib.oz_reconstruct.argtypes = [i64, i64, vp, i64, i64, vp, vp, i32, dbl, dbl, vp, i64, vp]
@@ -147,6 +150,14 @@ def oz_deconstruct(side, lines, k, X, ldx, modset, route, planes, plane_stride, 
     return load().oz_deconstruct(side, lines, k, _ptr(X), ldx, modset, route, _ptr(planes),
                                  plane_stride, row_pitch, _ptr(shift), _ptr(scratch),
                                  _stream(stream))
+
+
+def oz_deconstruct_static(side, lines, k, X, ldx, modset, route, planes, plane_stride, row_pitch,
+                          shift, stream=None) -> int:
+    """oz_deconstruct with the scan scratch held inside the library: for callers that cannot
+    allocate device memory.  At most OZ_STATIC_MAX_LINES lines; calls must not overlap on the GPU."""
+    return load().oz_deconstruct_static(side, lines, k, _ptr(X), ldx, modset, route, _ptr(planes),
+                                        plane_stride, row_pitch, _ptr(shift), _stream(stream))
 
 
 def oz_residue_gemm(m, n, k, PA, strideA, pitchA, PB, strideB, pitchB, modset, route, R, ldr,
