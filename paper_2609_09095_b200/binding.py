@@ -11,7 +11,7 @@ import ctypes as C
 import os
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "liboz_b200.so")
+LIB_PATH = os.environ.get("OZ_B200_LIB") or os.path.join(_HERE, "liboz_b200.so")
 
 OZ_OK = 0
 OZ_ERR_INVALID_ARG, OZ_ERR_UNSUPPORTED, OZ_ERR_WORKSPACE, OZ_ERR_CUDA = 1, 2, 3, 4

@@ -55,7 +55,8 @@ constexpr int NUM_THREADS = 640;
 constexpr int FIRST_EPI_WARP = 4;                  // warps 0..3: producer, MMA issuer, two idle
 constexpr int EPI_WARPS = 16;
 constexpr int COLS_PER_WARP = BLOCK_N / 4;         // four warps share a TMEM lane quarter
-constexpr size_t SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr int XPOSE_BYTES = 16 * 128;                // per epilogue warp: 16 lines x 128 bytes
+constexpr size_t SMEM_BYTES = STAGES * STAGE_BYTES + EPI_WARPS * XPOSE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
 
 struct ModInfo {
     float m, inv_m;
@@ -280,13 +281,14 @@ residue_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
     extern __shared__ unsigned char smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t tiles = (raw + 1023u) & ~1023u;                     // 1024-byte aligned ring
-    const uint32_t bars = tiles + STAGES * STAGE_BYTES;
+    const uint32_t bars = tiles + STAGES * STAGE_BYTES + EPI_WARPS * XPOSE_BYTES;
     const uint32_t full_bar = bars;                                   // STAGES x 8 bytes
     const uint32_t empty_bar = bars + 8 * STAGES;
     const uint32_t tfull_bar = bars + 16 * STAGES;                    // 2 x 8
     const uint32_t tempty_bar = tfull_bar + 16;                       // 2 x 8
     const uint32_t tmem_slot = tempty_bar + 16;                       // 4 bytes: TMEM base address
-    unsigned char *gen = smem_raw + (tiles - raw) + STAGES * STAGE_BYTES;
+    unsigned char *xpose_base = smem_raw + (tiles - raw) + STAGES * STAGE_BYTES;
+    unsigned char *gen = xpose_base + EPI_WARPS * XPOSE_BYTES;
     volatile uint32_t *tmem_base_ptr = reinterpret_cast<volatile uint32_t *>(gen + 16 * STAGES + 32);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(gen + 16 * STAGES + 40);
 
@@ -429,35 +431,56 @@ residue_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
             }
             if (!ok) break;
             // this thread: column j of C, rows i0 .. i0+63 (contiguous in the residue array)
-            const int64_t j = static_cast<int64_t>(it.tn) * BLOCK_M + q * 32 + lane;
+            const int64_t jw = static_cast<int64_t>(it.tn) * BLOCK_M + q * 32;   // first column of the warp
+            const int64_t j = jw + lane;
             const int64_t i0 = static_cast<int64_t>(it.tm) * BLOCK_N + part * COLS_PER_WARP;
-            if (j < p.n && i0 < p.m) {
-                uint16_t *dst = p.R + it.mod * p.mod_stride + j * p.ldr + i0;
-                uint32_t packed[COLS_PER_WARP / 2];
+            if (i0 >= p.m || jw >= p.n) continue;                                 // warp-uniform
+            uint32_t packed[COLS_PER_WARP / 2];
 #pragma unroll
-                for (int c = 0; c < COLS_PER_WARP; c += 2) {
-                    uint32_t bits[2];
+            for (int c = 0; c < COLS_PER_WARP; c += 2) {
+                uint32_t bits[2];
 #pragma unroll
-                    for (int h = 0; h < 2; ++h) {
-                        float t = comb[c + h];
-                        float quot = fmaf(t, inv_m, 12582912.0f) - 12582912.0f;
-                        float res = fmaf(-quot, mm, t);
-                        res = res < 0.0f ? res + mm : res;                       // canonical [0, m)
-                        bits[h] = __float_as_uint(res + 8388608.0f);             // integer in the low mantissa bits
+                for (int h = 0; h < 2; ++h) {
+                    float t = comb[c + h];
+                    float quot = fmaf(t, inv_m, 12582912.0f) - 12582912.0f;
+                    float res = fmaf(-quot, mm, t);
+                    res = res < 0.0f ? res + mm : res;                       // canonical [0, m)
+                    bits[h] = __float_as_uint(res + 8388608.0f);             // integer in the low mantissa bits
+                }
+                packed[c >> 1] = __byte_perm(bits[0], bits[1], 0x5410);
+            }
+            uint16_t *rbase = p.R + it.mod * p.mod_stride;
+            if (p.vec_store && i0 + COLS_PER_WARP <= p.m) {
+                // Transpose through a per-warp shared buffer so that one store instruction writes
+                // four whole 128-byte lines (lane -> line lane/8 + 4t, 16-byte chunk lane%8)
+                // instead of 32 separate 16-byte pieces.  Chunks are XOR-swizzled by the line
+                // number: both the writes and the reads are free of bank conflicts.
+                unsigned char *xp = xpose_base + (warp - FIRST_EPI_WARP) * XPOSE_BYTES;
+#pragma unroll
+                for (int rho = 0; rho < 2; ++rho) {
+                    if ((lane >> 4) == rho) {
+                        const int lr = lane & 15;
+#pragma unroll
+                        for (int c = 0; c < 8; ++c)
+                            *reinterpret_cast<uint4 *>(xp + lr * 128 + ((c ^ (lr & 7)) << 4)) =
+                                make_uint4(packed[4 * c], packed[4 * c + 1], packed[4 * c + 2], packed[4 * c + 3]);
                     }
-                    packed[c >> 1] = __byte_perm(bits[0], bits[1], 0x5410);
-                }
-                if (p.vec_store && i0 + COLS_PER_WARP <= p.m) {
+                    __syncwarp();
 #pragma unroll
-                    for (int c = 0; c < COLS_PER_WARP / 8; ++c)
-                        *reinterpret_cast<uint4 *>(dst + 8 * c) =
-                            make_uint4(packed[4 * c], packed[4 * c + 1], packed[4 * c + 2], packed[4 * c + 3]);
-                } else {
-#pragma unroll
-                    for (int c = 0; c < COLS_PER_WARP; ++c)
-                        if (i0 + c < p.m)
-                            dst[c] = static_cast<uint16_t>((packed[c >> 1] >> (16 * (c & 1))) & 0xFFFFu);
+                    for (int t = 0; t < 4; ++t) {
+                        const int lr = (lane >> 3) + 4 * t, c = lane & 7;
+                        uint4 val = *reinterpret_cast<const uint4 *>(xp + lr * 128 + ((c ^ (lr & 7)) << 4));
+                        const int64_t jg = jw + 16 * rho + lr;
+                        if (jg < p.n) *reinterpret_cast<uint4 *>(rbase + jg * p.ldr + i0 + 8 * c) = val;
+                    }
+                    __syncwarp();
                 }
+            } else if (j < p.n) {
+                uint16_t *dst = rbase + j * p.ldr + i0;
+#pragma unroll
+                for (int c = 0; c < COLS_PER_WARP; ++c)
+                    if (i0 + c < p.m)
+                        dst[c] = static_cast<uint16_t>((packed[c >> 1] >> (16 * (c & 1))) & 0xFFFFu);
             }
         }
     }

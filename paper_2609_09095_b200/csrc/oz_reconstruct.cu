@@ -4,13 +4,13 @@
 // The paper's SIMT branch walks Garner's mixed-radix digits (r(r-1)/2 multiply-reduce steps).
 // CRT fixes c' uniquely, so any exact evaluation gives the same integer; this kernel uses the
 // weighted form
-//     c' = sum_i t_i (M/m_i)  -  kappa M,     t_i = (c_i (M/m_i)^-1) mod m_i  (balanced),
-// with every M/m_i and M cut into three 38-bit chunks.  |t_i| <= (m_i+1)/2 < 2^10, so each of
-// the three chunk sums is an integer below 2^52 and is formed EXACTLY by FP64 fused
-// multiply-adds (the FP64 pipe is otherwise idle in this kernel).  kappa = round(S/M) comes from
-// a floating estimate and is then made exact by a 128-bit range test, so the result is the
-// unique representative in [-M/2, M/2) in every case.  The final conversion of the 128-bit
-// integer to FP64 is a single round-to-nearest-even done in integer arithmetic.
+//     c' = sum_i c_i V_i  -  kappa M,     V_i = ((M/m_i)^-1 mod m_i) (M/m_i) mod M,
+// with every V_i and M cut into three 38-bit chunks.  c_i < 2^10.1, so each of the three chunk
+// sums is an integer below 2^52 and is formed EXACTLY by FP64 fused multiply-adds (about r MACs
+// per chunk, on a pipe that is otherwise idle here).  kappa = round(S/M) comes from a floating
+// estimate and is then made exact by a 128-bit range test, so the result is the unique
+// representative in [-M/2, M/2) in every case.  The final conversion of the 128-bit integer to
+// FP64 is a single round-to-nearest-even done in integer arithmetic.
 #include <utility>
 
 #include "oz_internal.h"
@@ -19,11 +19,8 @@ namespace oz {
 namespace {
 
 struct ReconConst {
-    float m[kMaxR];
-    float inv_m[kMaxR];
-    float q[kMaxR];            // (M/m_i)^-1 mod m_i
-    double W[kMaxR][3];        // M/m_i = W0 + W1 2^38 + W2 2^76
-    double Mc[3];              // M     = M0 + M1 2^38 + M2 2^76
+    double V[kMaxR][3];        // V_i = V0 + V1 2^38 + V2 2^76
+    double Mc[3];              // M   = M0 + M1 2^38 + M2 2^76
     double inv_M;              // 1/M (rounded)
     unsigned long long M_lo, M_hi;
 };
@@ -33,43 +30,27 @@ __constant__ ReconConst c_recon[2];
 constexpr double kTwo38 = 274877906944.0;             // 2^38
 constexpr double kTwoM38 = 1.0 / 274877906944.0;      // 2^-38
 constexpr double kTwo76 = kTwo38 * kTwo38;            // 2^76
+constexpr double kTwo52 = 4503599627370496.0;         // 2^52
 constexpr double kRint = 6755399441055744.0;          // 1.5 * 2^52: (x + kRint) - kRint = rint(x)
 
-// nearest double (ties to even) of a 128-bit integer times 2^scale
-__device__ __forceinline__ double i128_to_double(__int128 v, int scale)
+// x * 2^scale for a finite double x (exact unless the result leaves the normal range)
+__device__ __forceinline__ double scale_pow2(double x, int scale)
 {
-    bool neg = v < 0;
-    unsigned __int128 a = neg ? static_cast<unsigned __int128>(0) - static_cast<unsigned __int128>(v)
-                              : static_cast<unsigned __int128>(v);
-    unsigned long long hi = static_cast<unsigned long long>(a >> 64);
-    unsigned long long lo = static_cast<unsigned long long>(a);
-    double d;
-    if (hi == 0) {
-        d = __ull2double_rn(lo);
-    } else {
-        int lz = __clzll(static_cast<long long>(hi));
-        unsigned long long top = lz ? ((hi << lz) | (lo >> (64 - lz))) : hi;
-        unsigned long long rest = lz ? (lo << lz) : lo;
-        top |= (rest != 0ull) ? 1ull : 0ull;     // sticky bit, far below the rounding position
-        d = __ull2double_rn(top);
-        scale += 64 - lz;
-    }
-    d = scalbn(d, scale);
-    return neg ? -d : d;
+    int hi = __double2hiint(x);
+    int be = (hi >> 20) & 0x7FF;
+    int nb = be + scale;
+    if (be != 0 && nb >= 1 && nb <= 2046) return __hiloint2double(hi + (scale << 20), __double2loint(x));
+    return scalbn(x, scale);        // zero, or a result outside the normal range
 }
 
 template <int SET, int I>
 __device__ __forceinline__ void crt_term(uint32_t c, double &S0, double &S1, double &S2)
 {
     const ReconConst &K = c_recon[SET];
-    float cf = __uint_as_float(0x4B000000u | c) - 8388608.0f;          // exact: c < 2^16
-    float x = cf * K.q[I];                                              // < 2^21, exact
-    float quot = fmaf(x, K.inv_m[I], 12582912.0f) - 12582912.0f;        // rint(x / m) up to +-1
-    float t = fmaf(-quot, K.m[I], x);                                   // exact, |t| <= (m+1)/2
-    double td = static_cast<double>(t);
-    S0 = fma(td, K.W[I][0], S0);
-    S1 = fma(td, K.W[I][1], S1);
-    S2 = fma(td, K.W[I][2], S2);
+    double cd = __hiloint2double(0x43300000, static_cast<int>(c)) - kTwo52;   // exact u32 -> double
+    S0 = fma(cd, K.V[I][0], S0);
+    S1 = fma(cd, K.V[I][1], S1);
+    S2 = fma(cd, K.V[I][2], S2);
 }
 
 template <int SET, int... I>
@@ -87,7 +68,7 @@ __device__ __forceinline__ double reconstruct_one(const uint32_t (&c)[kMaxR], in
     crt_sum<SET>(std::make_integer_sequence<int, set_r(SET)>{}, c, S0, S1, S2);
     double val = fma(S2, kTwo76, fma(S1, kTwo38, S0));
     double kappa = (val * K.inv_M + kRint) - kRint;
-    double T0 = fma(-kappa, K.Mc[0], S0);
+    double T0 = fma(-kappa, K.Mc[0], S0);              // exact: integers below 2^53
     double T1 = fma(-kappa, K.Mc[1], S1);
     double T2 = fma(-kappa, K.Mc[2], S2);
     // carry-normalise so that the three chunks do not overlap
@@ -97,16 +78,36 @@ __device__ __forceinline__ double reconstruct_one(const uint32_t (&c)[kMaxR], in
     double c1 = (T1 * kTwoM38 + kRint) - kRint;
     T1 = fma(-c1, kTwo38, T1);
     T2 += c1;
-    const __int128 one = 1;
-    __int128 v = static_cast<__int128>(__double2ll_rn(T2)) * (one << 76);
-    v += static_cast<__int128>(__double2ll_rn(T1)) * (one << 38);
-    v += static_cast<__int128>(__double2ll_rn(T0));
-    // exact lift to [-M/2, M/2)  (M is even for both sets)
-    const __int128 M = static_cast<__int128>((static_cast<unsigned __int128>(K.M_hi) << 64) | K.M_lo);
-    const __int128 Mh = M >> 1;
-    if (v >= Mh) v -= M;
-    else if (v < -Mh) v += M;
-    return i128_to_double(v, -shift_sum);
+    const long long t0 = __double2ll_rn(T0), t1 = __double2ll_rn(T1), t2 = __double2ll_rn(T2);
+    // v = t0 + t1 2^38 + t2 2^76 as a two's-complement (hi:lo) pair
+    unsigned long long lo = static_cast<unsigned long long>(t0) + (static_cast<unsigned long long>(t1) << 38);
+    long long hi = (t0 >> 63) + (t1 >> 26) + (lo < static_cast<unsigned long long>(t0) ? 1 : 0) +
+                   static_cast<long long>(static_cast<unsigned long long>(t2) << 12);
+    // exact lift to [-M/2, M/2): only values within one part in 2^37 of +-M/2 can need it
+    const long long mh_hi = static_cast<long long>(K.M_hi >> 1);
+    if (hi >= mh_hi || hi <= -mh_hi) {
+        const __int128 M = static_cast<__int128>((static_cast<unsigned __int128>(K.M_hi) << 64) | K.M_lo);
+        const __int128 Mh = M >> 1;     // M is even for both sets
+        __int128 v = static_cast<__int128>((static_cast<unsigned __int128>(static_cast<unsigned long long>(hi)) << 64) | lo);
+        if (v >= Mh) v -= M;
+        else if (v < -Mh) v += M;
+        lo = static_cast<unsigned long long>(v);
+        hi = static_cast<long long>(v >> 64);
+    }
+    const bool neg = hi < 0;
+    if (neg) {
+        lo = 0ull - lo;
+        hi = ~hi + (lo == 0ull ? 1 : 0);
+    }
+    // nearest double, ties to even: top 64 bits with a sticky bit far below the rounding position
+    const unsigned long long uhi = static_cast<unsigned long long>(hi);
+    const int lz = __clzll(static_cast<long long>(uhi | 1ull));          // uhi < 2^48: lz in [16, 63]
+    const unsigned long long top = (uhi << lz) | (lo >> (64 - lz));
+    const unsigned long long rest = lo << lz;
+    unsigned long long mant = uhi ? (top | (rest ? 1ull : 0ull)) : lo;
+    int scale = (uhi ? 64 - lz : 0) - shift_sum;
+    double d = scale_pow2(__ull2double_rn(mant), scale);
+    return neg ? -d : d;
 }
 
 template <int SET>
@@ -175,22 +176,17 @@ oz_status_t upload_reconstruct_constants()
         for (int i = 0; i < set_r(set); ++i) M *= static_cast<unsigned>(modulus(set, i));
         const unsigned __int128 mask = (static_cast<unsigned __int128>(1) << 38) - 1;
         ReconConst &K = host[set];
-        for (int i = 0; i < kMaxR; ++i) {
-            K.m[i] = 1.0f; K.inv_m[i] = 1.0f; K.q[i] = 0.0f;
-            K.W[i][0] = K.W[i][1] = K.W[i][2] = 0.0;
-        }
+        for (int i = 0; i < kMaxR; ++i) K.V[i][0] = K.V[i][1] = K.V[i][2] = 0.0;
         for (int i = 0; i < set_r(set); ++i) {
             unsigned mi = static_cast<unsigned>(modulus(set, i));
             unsigned __int128 W = M / mi;
             unsigned wm = static_cast<unsigned>(W % mi), inv = 0;
             for (unsigned c = 1; c < mi; ++c)
                 if ((static_cast<unsigned long long>(wm) * c) % mi == 1) { inv = c; break; }
-            K.m[i] = static_cast<float>(mi);
-            K.inv_m[i] = 1.0f / static_cast<float>(mi);
-            K.q[i] = static_cast<float>(inv);
-            K.W[i][0] = static_cast<double>(static_cast<unsigned long long>(W & mask));
-            K.W[i][1] = static_cast<double>(static_cast<unsigned long long>((W >> 38) & mask));
-            K.W[i][2] = static_cast<double>(static_cast<unsigned long long>(W >> 76));
+            unsigned __int128 V = W * inv;          // < M, and V = 1 mod m_i, 0 mod the other moduli
+            K.V[i][0] = static_cast<double>(static_cast<unsigned long long>(V & mask));
+            K.V[i][1] = static_cast<double>(static_cast<unsigned long long>((V >> 38) & mask));
+            K.V[i][2] = static_cast<double>(static_cast<unsigned long long>(V >> 76));
         }
         K.Mc[0] = static_cast<double>(static_cast<unsigned long long>(M & mask));
         K.Mc[1] = static_cast<double>(static_cast<unsigned long long>((M >> 38) & mask));
