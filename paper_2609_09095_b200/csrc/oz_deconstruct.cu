@@ -275,13 +275,15 @@ convert_kernel(const double *__restrict__ X, int64_t ldx, int64_t lines, int64_t
     __syncthreads();
 
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int64_t nchunks = (row_pitch + kChunk - 1) / kChunk;
+    // work items are numbered in 32 bits (checked on the host): cheap division
+    const uint32_t nchunks = static_cast<uint32_t>((row_pitch + kChunk - 1) / kChunk);
 
     if (SIDE == 1) {
-        const int64_t items = lines * nchunks;
-        for (int64_t item = blockIdx.x * 8ll + warp; item < items; item += gridDim.x * 8ll) {
-            int64_t line = item / nchunks;
-            int64_t kb = (item - line * nchunks) * kChunk + lane * 4;
+        const uint32_t items = static_cast<uint32_t>(lines) * nchunks;
+        for (uint32_t item = blockIdx.x * 8u + warp; item < items; item += gridDim.x * 8u) {
+            const uint32_t uline = item / nchunks;
+            const int64_t line = uline;
+            int64_t kb = static_cast<int64_t>(item - uline * nchunks) * kChunk + lane * 4;
             if (kb >= row_pitch) continue;
             int sigma = shift[line];
             bool dead = sigma == OZ_NONFINITE_SHIFT;
@@ -293,11 +295,12 @@ convert_kernel(const double *__restrict__ X, int64_t ldx, int64_t lines, int64_t
         }
     } else {
         double *tile = reinterpret_cast<double *>(smem_raw + kLutWords * 4);
-        const int64_t ltiles = (lines + kTileLines - 1) / kTileLines;
-        const int64_t items = ltiles * nchunks;
-        for (int64_t item = blockIdx.x; item < items; item += gridDim.x) {
-            int64_t lt = item % ltiles;           // neighbouring blocks read neighbouring rows
-            int64_t kc = item / ltiles;
+        const uint32_t ltiles = static_cast<uint32_t>((lines + kTileLines - 1) / kTileLines);
+        const uint32_t items = ltiles * nchunks;
+        for (uint32_t item = blockIdx.x; item < items; item += gridDim.x) {
+            const uint32_t ukc = item / ltiles;
+            const int64_t kc = ukc;
+            const int64_t lt = item - ukc * ltiles;  // neighbouring blocks read neighbouring rows
             int64_t line_l = lt * kTileLines + lane;
             for (int kk = warp; kk < kChunk; kk += kConvThreads / 32) {
                 int64_t kg = kc * kChunk + kk;
@@ -332,6 +335,7 @@ oz_status_t launch_convert(const double *X, int64_t ldx, int64_t lines, int64_t 
                                        cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        static_cast<int>(smem)));
     int64_t nchunks = (row_pitch + kChunk - 1) / kChunk;
+    if (lines * nchunks >= 0x7FFFFFFFll) return OZ_ERR_UNSUPPORTED;   // item numbers are 32-bit
     int64_t need = SIDE == 1 ? (lines * nchunks + 7) / 8
                              : ((lines + kTileLines - 1) / kTileLines) * nchunks;
     int sms = 148;

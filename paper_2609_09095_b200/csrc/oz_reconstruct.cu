@@ -22,6 +22,7 @@ struct ReconConst {
     double V[kMaxR][3];        // V_i = V0 + V1 2^38 + V2 2^76
     double Mc[3];              // M   = M0 + M1 2^38 + M2 2^76
     double inv_M;              // 1/M (rounded)
+    double half_M_guard;       // (M/2) (1 - 2^-30): beyond it the lift is decided exactly
     unsigned long long M_lo, M_hi;
 };
 
@@ -60,6 +61,39 @@ __device__ __forceinline__ void crt_sum(std::integer_sequence<int, I...>, const 
     (crt_term<SET, I>(c[I], S0, S1, S2), ...);
 }
 
+// Exact tail (rare path): the normalised chunks as a 128-bit integer, exact lift to
+// [-M/2, M/2), round-to-nearest-even conversion in integer arithmetic, power-of-two scale.
+__device__ __noinline__ double finish_exact(double T0, double T1, double T2, int shift_sum, int set)
+{
+    const ReconConst &K = c_recon[set];
+    const long long t0 = __double2ll_rn(T0), t1 = __double2ll_rn(T1), t2 = __double2ll_rn(T2);
+    // v = t0 + t1 2^38 + t2 2^76 as a two's-complement (hi:lo) pair
+    unsigned long long lo = static_cast<unsigned long long>(t0) + (static_cast<unsigned long long>(t1) << 38);
+    long long hi = (t0 >> 63) + (t1 >> 26) + (lo < static_cast<unsigned long long>(t0) ? 1 : 0) +
+                   static_cast<long long>(static_cast<unsigned long long>(t2) << 12);
+    const __int128 M = static_cast<__int128>((static_cast<unsigned __int128>(K.M_hi) << 64) | K.M_lo);
+    const __int128 Mh = M >> 1;     // M is even for both sets
+    __int128 v = static_cast<__int128>((static_cast<unsigned __int128>(static_cast<unsigned long long>(hi)) << 64) | lo);
+    if (v >= Mh) v -= M;
+    else if (v < -Mh) v += M;
+    lo = static_cast<unsigned long long>(v);
+    hi = static_cast<long long>(v >> 64);
+    const bool neg = hi < 0;
+    if (neg) {
+        lo = 0ull - lo;
+        hi = ~hi + (lo == 0ull ? 1 : 0);
+    }
+    // nearest double, ties to even: top 64 bits with a sticky bit far below the rounding position
+    const unsigned long long uhi = static_cast<unsigned long long>(hi);
+    const int lz = __clzll(static_cast<long long>(uhi | 1ull));          // uhi < 2^49: lz in [15, 63]
+    const unsigned long long top = (uhi << lz) | (lo >> (64 - lz));
+    const unsigned long long rest = lo << lz;
+    unsigned long long mant = uhi ? (top | (rest ? 1ull : 0ull)) : lo;
+    int scale = (uhi ? 64 - lz : 0) - shift_sum;
+    double d = scale_pow2(__ull2double_rn(mant), scale);
+    return neg ? -d : d;
+}
+
 template <int SET>
 __device__ __forceinline__ double reconstruct_one(const uint32_t (&c)[kMaxR], int shift_sum)
 {
@@ -71,43 +105,33 @@ __device__ __forceinline__ double reconstruct_one(const uint32_t (&c)[kMaxR], in
     double T0 = fma(-kappa, K.Mc[0], S0);              // exact: integers below 2^53
     double T1 = fma(-kappa, K.Mc[1], S1);
     double T2 = fma(-kappa, K.Mc[2], S2);
-    // carry-normalise so that the three chunks do not overlap
+    // carry-normalise so that the three chunks do not overlap: |T0|, |T1| <= 2^37
     double c0 = (T0 * kTwoM38 + kRint) - kRint;
     T0 = fma(-c0, kTwo38, T0);
     T1 += c0;
     double c1 = (T1 * kTwoM38 + kRint) - kRint;
     T1 = fma(-c1, kTwo38, T1);
     T2 += c1;
-    const long long t0 = __double2ll_rn(T0), t1 = __double2ll_rn(T1), t2 = __double2ll_rn(T2);
-    // v = t0 + t1 2^38 + t2 2^76 as a two's-complement (hi:lo) pair
-    unsigned long long lo = static_cast<unsigned long long>(t0) + (static_cast<unsigned long long>(t1) << 38);
-    long long hi = (t0 >> 63) + (t1 >> 26) + (lo < static_cast<unsigned long long>(t0) ? 1 : 0) +
-                   static_cast<long long>(static_cast<unsigned long long>(t2) << 12);
-    // exact lift to [-M/2, M/2): only values within one part in 2^37 of +-M/2 can need it
-    const long long mh_hi = static_cast<long long>(K.M_hi >> 1);
-    if (hi >= mh_hi || hi <= -mh_hi) {
-        const __int128 M = static_cast<__int128>((static_cast<unsigned __int128>(K.M_hi) << 64) | K.M_lo);
-        const __int128 Mh = M >> 1;     // M is even for both sets
-        __int128 v = static_cast<__int128>((static_cast<unsigned __int128>(static_cast<unsigned long long>(hi)) << 64) | lo);
-        if (v >= Mh) v -= M;
-        else if (v < -Mh) v += M;
-        lo = static_cast<unsigned long long>(v);
-        hi = static_cast<long long>(v >> 64);
-    }
-    const bool neg = hi < 0;
-    if (neg) {
-        lo = 0ull - lo;
-        hi = ~hi + (lo == 0ull ? 1 : 0);
-    }
-    // nearest double, ties to even: top 64 bits with a sticky bit far below the rounding position
-    const unsigned long long uhi = static_cast<unsigned long long>(hi);
-    const int lz = __clzll(static_cast<long long>(uhi | 1ull));          // uhi < 2^48: lz in [16, 63]
-    const unsigned long long top = (uhi << lz) | (lo >> (64 - lz));
-    const unsigned long long rest = lo << lz;
-    unsigned long long mant = uhi ? (top | (rest ? 1ull : 0ull)) : lo;
-    int scale = (uhi ? 64 - lz : 0) - shift_sum;
-    double d = scale_pow2(__ull2double_rn(mant), scale);
-    return neg ? -d : d;
+    // c' = X2 + X1 + X0 exactly.  Fast path: two error-free additions give r = RN(s + t) and
+    // the exact residual rem of that last rounding; r is the correctly rounded value of c'
+    // unless c' lies within a hair of a rounding boundary (|rem| ~ half an ulp, or r a power
+    // of two) or within a hair of +-M/2 (where the symmetric lift could apply).  Those cases,
+    // a vanishing fraction of random data, take the exact integer path.
+    const double X2 = T2 * kTwo76, X1 = T1 * kTwo38;   // exact
+    const double s = X2 + X1;
+    const double err = X1 - (s - X2);                   // exact: s + err = X2 + X1
+    const double t = err + T0;
+    const double r = s + t;
+    const double rem = t - (r - s);                     // exact: r + rem = s + t
+    const long long rb = __double_as_longlong(r);
+    const int eb = static_cast<int>((rb >> 52) & 0x7FF);
+    if (eb == 0) return 0.0;                            // c' = 0 (r is an integer: never subnormal)
+    const double half_ulp = __longlong_as_double(static_cast<long long>(eb - 53) << 52);
+    const bool near_tie = fabs(rem) >= fma(-half_ulp, 9.313225746154785e-10, half_ulp);   // (1 - 2^-30)
+    const bool pow2 = (rb & 0xFFFFFFFFFFFFFll) == 0 && rem != 0.0;
+    const bool near_half_M = fabs(r) >= K.half_M_guard;
+    if (near_tie || pow2 || near_half_M) return finish_exact(T0, T1, T2, shift_sum, SET);
+    return scale_pow2(r, -shift_sum);
 }
 
 template <int SET>
@@ -116,13 +140,14 @@ reconstruct_kernel(const uint16_t *__restrict__ R, int64_t ldr, int64_t mod_stri
                    int64_t n, const int32_t *__restrict__ shiftA, const int32_t *__restrict__ shiftB,
                    double alpha, double beta, double *__restrict__ C, int64_t ldc, int vecR, int vecC)
 {
-    const int64_t pairs = (m + 1) >> 1;
-    int64_t idx = blockIdx.x * 256ll + threadIdx.x;
-    if (idx >= pairs * n) return;
-    int64_t j = idx / pairs;
-    int64_t row = (idx - j * pairs) * 2;
-    bool two = row + 1 < m;
+    // grid.x covers the row pairs of a column, grid.y (and .z beyond 65535) the columns: no division
+    const int64_t row = (blockIdx.x * 256ll + threadIdx.x) * 2;
+    if (row >= m) return;
+    const bool two = row + 1 < m;
     constexpr int r = set_r(SET);
+    const int64_t j = blockIdx.y + 65535ll * blockIdx.z;
+    if (j >= n) return;
+    {
 
     uint32_t c0[kMaxR], c1[kMaxR];
     const uint16_t *base = R + j * ldr + row;
@@ -164,6 +189,7 @@ reconstruct_kernel(const uint16_t *__restrict__ R, int64_t ldr, int64_t mod_stri
         out[0] = beta != 0.0 ? out[0] + p0 : p0;
         if (two) out[1] = beta != 0.0 ? out[1] + p1 : p1;
     }
+    }
 }
 
 }  // namespace
@@ -192,6 +218,7 @@ oz_status_t upload_reconstruct_constants()
         K.Mc[1] = static_cast<double>(static_cast<unsigned long long>((M >> 38) & mask));
         K.Mc[2] = static_cast<double>(static_cast<unsigned long long>(M >> 76));
         K.inv_M = 1.0 / static_cast<double>(M);
+        K.half_M_guard = 0.5 * static_cast<double>(M) * (1.0 - 9.313225746154785e-10);
         K.M_lo = static_cast<unsigned long long>(M);
         K.M_hi = static_cast<unsigned long long>(M >> 64);
     }
@@ -206,15 +233,17 @@ oz_status_t launch_reconstruct(int64_t m, int64_t n, const uint16_t *R, int64_t 
 {
     int vecR = ((ldr & 1) == 0 && (mod_stride & 1) == 0 && (reinterpret_cast<uintptr_t>(R) & 3u) == 0) ? 1 : 0;
     int vecC = ((ldc & 1) == 0 && (reinterpret_cast<uintptr_t>(C) & 15u) == 0) ? 1 : 0;
-    int64_t total = ((m + 1) >> 1) * n;
-    int64_t blocks = (total + 255) / 256;
-    if (blocks > 0x7FFFFFFFll) return OZ_ERR_UNSUPPORTED;
+    int64_t bx = (((m + 1) >> 1) + 255) / 256;
+    if (bx > 0x7FFFFFFFll) return OZ_ERR_UNSUPPORTED;
+    if (n > 65535ll * 65535ll) return OZ_ERR_UNSUPPORTED;
+    dim3 grid(static_cast<unsigned>(bx), static_cast<unsigned>(n < 65535 ? n : 65535),
+              static_cast<unsigned>((n + 65534) / 65535));
     if (set == 0)
-        reconstruct_kernel<0><<<static_cast<unsigned>(blocks), 256, 0, stream>>>(
-            R, ldr, mod_stride, m, n, shiftA, shiftB, alpha, beta, C, ldc, vecR, vecC);
+        reconstruct_kernel<0><<<grid, 256, 0, stream>>>(R, ldr, mod_stride, m, n, shiftA, shiftB, alpha,
+                                                        beta, C, ldc, vecR, vecC);
     else
-        reconstruct_kernel<1><<<static_cast<unsigned>(blocks), 256, 0, stream>>>(
-            R, ldr, mod_stride, m, n, shiftA, shiftB, alpha, beta, C, ldc, vecR, vecC);
+        reconstruct_kernel<1><<<grid, 256, 0, stream>>>(R, ldr, mod_stride, m, n, shiftA, shiftB, alpha,
+                                                        beta, C, ldc, vecR, vecC);
     count_launch();
     OZ_CUDA_CHECK(cudaGetLastError());
     return OZ_OK;
