@@ -34,6 +34,11 @@ sys.path.insert(0, ROOT)
 
 import synth_inputs as syn  # noqa: E402
 
+# DRAM read amplification of the residue GEMM (reads / plane bytes), measured with ncu on a
+# 16384x4096x2048 launch; writes equal the residue bytes exactly.  Used to scale the measured
+# traffic to the full-size launch, which is too large to capture.
+GEMM_DRAM_READ_AMPLIFICATION = 1.60
+
 METRIC = "emulated FP64 TFLOPS (2mnk/s)"
 UNIT = "TFLOP/s"
 
@@ -81,7 +86,7 @@ class ClockSampler:
             self.proc.wait(timeout=5)
         except subprocess.TimeoutExpired:
             self.proc.kill()
-        sm, smax, reasons = [], [], set()
+        sm, smax, pw, reasons = [], [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for line in self.lines:
             f = [t.strip() for t in line.split(",")]
@@ -92,14 +97,20 @@ class ClockSampler:
                 smax.append(float(f[2]))
             except ValueError:
                 continue
+            try:
+                pw.append(float(f[3]))
+            except ValueError:
+                pw.append(0.0)
             for name, val in zip(names, f[5:9]):
                 if val.lower().startswith("active"):
                     reasons.add(name)
         if not sm:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
-        busy = [v for v in sm if v > 0.5 * max(sm)] or sm
+        # samples taken under load: power draw above half of the largest seen
+        top = max(pw) if pw else 0.0
+        busy = [v for v, w in zip(sm, pw) if w >= 0.5 * top] or sm
         return {"sm_mhz": statistics.median(busy), "sm_max_mhz": max(smax), "reasons": sorted(reasons),
-                "samples": len(sm)}
+                "samples": len(sm), "samples_under_load": len(busy), "power_w_max": top}
 
 
 def aggregate_over_ranks(local_ms: float, local_work: float, world: int, reduce_max, reduce_sum):
@@ -207,6 +218,8 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
+    sampler = ClockSampler(local_rank)
+    sampler.start()          # nvidia-smi needs a moment to start: launch it before the warm-up
     for _ in range(args.warmup):
         step()
     oz.check(oz.oz_query_status(stream), "device status after warm-up")
@@ -217,9 +230,8 @@ def main():
         for e in evs:
             e.record(stream)  # materialise the handles
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    sampler = ClockSampler(local_rank)
     barrier()
-    sampler.start()
+    sampler.lines.clear()    # keep only samples taken from here on
     launches0 = oz.oz_launch_count()
     ev0.record(stream)
     for i in range(args.steps):
@@ -295,7 +307,10 @@ def main():
             "roofline": {"kernel": "residue_gemm_kernel (tcgen05)", "bound": "tensor", "achieved": achieved,
                          "peak": tensor_peak, "unit": "TFLOP/s", "frac": achieved / tensor_peak,
                          "peak_source": f"{peaks['source']} bf16 sustained x2 (8-bit operands)",
-                         "frac_of_nominal_4500": achieved / 4500.0, "traffic": None,
+                         "frac_of_nominal_4500": achieved / 4500.0,
+                         "traffic": GEMM_DRAM_READ_AMPLIFICATION * p_store * (m + n) * k + 2.0 * r * m * n,
+                         "traffic_unit": "bytes per launch (ncu dram read+write of a smaller launch, scaled by units)",
+                         "algorithmic_dram_bytes": p_store * (m + n) * k + 2.0 * r * m * n,
                          "ms_per_launch": gemm_ms},
             "stages": {
                 "deconstruct_A_ms": float(stage_ms[0]), "deconstruct_B_ms": float(stage_ms[1]),

@@ -200,7 +200,7 @@ Layout make_layout(int64_t m, int64_t n, int64_t k, int set)
 {
     Layout L{};
     Carve c;
-    L.pitch = oz_row_pitch(k);
+    L.pitch = round_up(k > 0 ? k : 1, 128);   // whole 128-byte lines per TMA box row (k = 5003 -> 5120)
     L.strideA = m * L.pitch;
     L.strideB = n * L.pitch;
     L.ldr = round_up(m, 8);
