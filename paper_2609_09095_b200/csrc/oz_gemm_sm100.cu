@@ -36,6 +36,7 @@
 // word, every role leaves its loops, in-flight copies are given a bounded time to land, TMEM is
 // freed and the kernel returns.
 #include <cuda.h>
+#include <cstdlib>
 
 #include "oz_internal.h"
 
@@ -46,21 +47,35 @@ constexpr int BLOCK_M = 128;                       // MMA M: columns j of C (lin
 constexpr int BLOCK_N = 256;                       // MMA N: rows i of C (lines of A)
 constexpr int BLOCK_K = 128;                       // bytes = elements (8-bit operands)
 constexpr int UMMA_K = 32;                         // 8-bit operands: 32 elements per instruction
-constexpr int STAGES = 4;
-constexpr int A_BYTES = BLOCK_M * BLOCK_K;         // 16 KiB: MMA operand a = tile of B's planes
-constexpr int B_BYTES = BLOCK_N * BLOCK_K;         // 32 KiB: MMA operand b = tile of A's planes
-constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+constexpr int A_BYTES = BLOCK_M * BLOCK_K;         // 16 KiB: MMA operand a = 128 lines of B's planes per CTA
+
+// CG = 1: one CTA per tile of 128 columns x 256 rows of C.
+// CG = 2: a pair of CTAs (cluster of 2) shares one tcgen05.mma.cta_group::2 of M = 256: the tile is
+//         256 columns x 256 rows; each CTA loads its own 128 lines of B's planes (operand a) and HALF
+//         of the 256 lines of A's planes (operand b), the tensor core reads both halves, and each
+//         CTA's TMEM holds the accumulators of its own 128 columns.  Per CTA this halves the
+//         shared-memory traffic of operand b and the TMA bytes per MMA.
+template <int CG>
+struct Tile {
+    static constexpr int B_LINES = BLOCK_N / CG;                 // lines of A's planes loaded per CTA
+    static constexpr int B_BYTES = B_LINES * BLOCK_K;            // 32 KiB / 16 KiB
+    static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;        // 48 KiB / 32 KiB
+    static constexpr int STAGES = CG == 1 ? 4 : 6;               // 192 KiB ring either way
+    static constexpr int TILE_J = BLOCK_M * CG;                  // columns of C per work item
+};
 constexpr int TMEM_COLS = 512;                     // two accumulator slots of BLOCK_N columns
 constexpr int NUM_THREADS = 640;
 constexpr int FIRST_EPI_WARP = 4;                  // warps 0..3: producer, MMA issuer, two idle
 constexpr int EPI_WARPS = 16;
 constexpr int COLS_PER_WARP = BLOCK_N / 4;         // four warps share a TMEM lane quarter
 constexpr int XPOSE_BYTES = 16 * 128;                // per epilogue warp: 16 lines x 128 bytes
-constexpr size_t SMEM_BYTES = STAGES * STAGE_BYTES + EPI_WARPS * XPOSE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr size_t SMEM_BYTES = 4 * 49152 + EPI_WARPS * XPOSE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+static_assert(Tile<1>::STAGES * Tile<1>::STAGE_BYTES == 4 * 49152 && Tile<2>::STAGES * Tile<2>::STAGE_BYTES == 4 * 49152, "ring size");
 
 struct ModInfo {
     float m, inv_m;
     float w[3];           // weight of each job
+    int reduce[3];        // reduce the accumulator modulo m before weighting (0: the exact FP32 range allows skipping it)
     int njobs;            // 2 (square) or 3
     int plane0;           // first stored plane of this modulus
 };
@@ -99,17 +114,45 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar)
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
 
+// cluster-scope acquire: the barriers of the CTA-pair variant are also signalled by the peer CTA
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
 {
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(ok)
         : "r"(bar), "r"(parity)
         : "memory");
     return ok != 0;
+}
+
+__device__ __forceinline__ uint32_t cluster_ctarank()
+{
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+
+// shared::cluster address of the same shared-memory location in CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank)
+{
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+    return r;
+}
+
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr)
+{
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+
+// all threads of both CTAs of the pair (no time limit: every thread reaches it on every path)
+__device__ __forceinline__ void cluster_sync_all()
+{
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
 
 __device__ __forceinline__ unsigned long long global_timer_ns()
@@ -153,47 +196,69 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map
         : "memory");
 }
 
-__device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t cols)
+// CTA-pair copy: same as tma_load_3d, but the mbarrier may live in the peer CTA (cluster address)
+__device__ __forceinline__ void tma_load_3d_pair(uint32_t dst, const CUtensorMap *map, uint32_t bar_cluster,
+                                                 int c0, int c1, int c2)
 {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem),
-                 "r"(cols)
-                 : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    asm volatile(
+        "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes "
+        "[%0], [%1, {%3, %4, %5}], [%2];"
+        ::"r"(dst), "l"(map), "r"(bar_cluster), "r"(c0), "r"(c1), "r"(c2)
+        : "memory");
 }
 
+// In the CTA-pair variant the same warp of BOTH CTAs executes the allocation / release.
+template <int CG>
+__device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t cols)
+{
+    if (CG == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    } else {
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    }
+}
+
+template <int CG>
 __device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols)
 {
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols)
-                 : "memory");
+    if (CG == 1)
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+    else
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
 }
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
-template <int SUB>
+template <int SUB, int CG>
 __device__ __forceinline__ void umma(uint32_t d_tmem, uint64_t da, uint64_t db, uint32_t idesc,
                                      uint32_t accumulate)
 {
-    if (SUB == 0) {
-        asm volatile(
-            "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-            "tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], %1, %2, %3, p;\n\t}"
-            ::"r"(d_tmem), "l"(da), "l"(db), "r"(idesc), "r"(accumulate)
-            : "memory");
-    } else {
-        asm volatile(
-            "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-            "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
-            ::"r"(d_tmem), "l"(da), "l"(db), "r"(idesc), "r"(accumulate)
-            : "memory");
-    }
+#define OZ_UMMA(GROUP, KIND)                                                                      \
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"                              \
+                 "tcgen05.mma.cta_group::" GROUP ".kind::" KIND " [%0], %1, %2, %3, p;\n\t}"      \
+                 ::"r"(d_tmem), "l"(da), "l"(db), "r"(idesc), "r"(accumulate) : "memory")
+    if (SUB == 0 && CG == 1) OZ_UMMA("1", "f8f6f4");
+    if (SUB == 0 && CG == 2) OZ_UMMA("2", "f8f6f4");
+    if (SUB == 1 && CG == 1) OZ_UMMA("1", "i8");
+    if (SUB == 1 && CG == 2) OZ_UMMA("2", "i8");
+#undef OZ_UMMA
 }
 
 // mbarrier arrives once every MMA issued so far by this thread has completed
+// (CTA pair: the arrive is delivered to the barrier at this offset in BOTH CTAs)
+template <int CG>
 __device__ __forceinline__ void umma_commit(uint32_t bar)
 {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar)
-                 : "memory");
+    if (CG == 1) {
+        asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+    } else {
+        const uint16_t both = 3;
+        asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                     ::"r"(bar), "h"(both) : "memory");
+    }
 }
 
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32])
@@ -225,13 +290,13 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr)
 }
 
 // instruction descriptor: D format, A/B formats, K-major both, N/8 at bit 17, M/16 at bit 24
-template <int SUB>
+template <int SUB, int CG>
 __host__ __device__ constexpr uint32_t instr_desc()
 {
     uint32_t cfmt = SUB == 0 ? 1u /*f32*/ : 2u /*s32*/;
     uint32_t abfmt = SUB == 0 ? 0u /*e4m3*/ : 1u /*s8*/;
     return (cfmt << 4) | (abfmt << 7) | (abfmt << 10) | (static_cast<uint32_t>(BLOCK_N >> 3) << 17) |
-           (static_cast<uint32_t>(BLOCK_M >> 4) << 24);
+           (static_cast<uint32_t>((BLOCK_M * CG) >> 4) << 24);
 }
 
 // work item -> (modulus, tile_m, tile_n): modulus-major so that one modulus' planes stay in L2;
@@ -273,11 +338,18 @@ __device__ __forceinline__ void job_planes(const ModInfo &mi, int job, int pair,
 
 __device__ __forceinline__ int job_pairs(const ModInfo &mi, int job) { return (mi.njobs == 2 && job == 1) ? 2 : 1; }
 
-template <int SUB>
+template <int SUB, int CG>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 residue_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB,
                     const __grid_constant__ GemmParams p)
 {
+    constexpr int STAGES = Tile<CG>::STAGES;
+    constexpr int STAGE_BYTES = Tile<CG>::STAGE_BYTES;
+    // CTA pair: rank 0 leads (issues the MMAs, owns the `full` and `tmem-empty` barriers that both
+    // CTAs signal); work items are dealt to pairs, so both CTAs walk the same item sequence.
+    const uint32_t rank = CG == 2 ? cluster_ctarank() : 0u;
+    const int64_t first_item = CG == 2 ? (blockIdx.x >> 1) : blockIdx.x;
+    const int64_t item_step = CG == 2 ? (gridDim.x >> 1) : gridDim.x;
     extern __shared__ unsigned char smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t tiles = (raw + 1023u) & ~1023u;                     // 1024-byte aligned ring
@@ -301,14 +373,15 @@ residue_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
         }
         for (int s = 0; s < 2; ++s) {
             mbar_init(tfull_bar + 8 * s, 1);
-            mbar_init(tempty_bar + 8 * s, EPI_WARPS);
+            mbar_init(tempty_bar + 8 * s, EPI_WARPS * CG);   // pair: the peer's epilogue warps arrive too
         }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == 1) tmem_alloc(tmem_slot, TMEM_COLS);
+    if (warp == 1) tmem_alloc<CG>(tmem_slot, TMEM_COLS);
     tc_fence_before();
     __syncthreads();
+    if (CG == 2) cluster_sync_all();      // the peer's barriers exist before anything signals them
     tc_fence_after();
     const uint32_t tmem_base = *tmem_base_ptr;
 
@@ -318,7 +391,7 @@ residue_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
             int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
-            for (int64_t item = blockIdx.x; ok && item < p.total_items; item += gridDim.x) {
+            for (int64_t item = first_item; ok && item < p.total_items; item += item_step) {
                 Item it = decode_item(item, p);
                 const ModInfo &mi = p.mod[it.mod];
                 for (int job = 0; ok && job < mi.njobs; ++job) {
@@ -330,10 +403,20 @@ residue_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
                             ok = mbar_wait(empty_bar + 8 * stage, phase ^ 1u, abort_flag, p.status);
                             if (!ok) break;
                             uint32_t fb = full_bar + 8 * stage;
-                            mbar_expect_tx(fb, STAGE_BYTES);
                             uint32_t sa = tiles + stage * STAGE_BYTES;
-                            tma_load_3d(sa, &mapB, fb, kc * BLOCK_K, it.tn * BLOCK_M, pb);
-                            tma_load_3d(sa + A_BYTES, &mapA, fb, kc * BLOCK_K, it.tm * BLOCK_N, pa);
+                            if (CG == 1) {
+                                mbar_expect_tx(fb, STAGE_BYTES);
+                                tma_load_3d(sa, &mapB, fb, kc * BLOCK_K, it.tn * BLOCK_M, pb);
+                                tma_load_3d(sa + A_BYTES, &mapA, fb, kc * BLOCK_K, it.tm * BLOCK_N, pa);
+                            } else {
+                                // both CTAs' copies complete on the leader's barrier
+                                if (rank == 0) mbar_expect_tx(fb, 2 * STAGE_BYTES);
+                                const uint32_t fb_leader = map_to_cta(fb, 0);
+                                tma_load_3d_pair(sa, &mapB, fb_leader, kc * BLOCK_K,
+                                                 it.tn * Tile<CG>::TILE_J + static_cast<int>(rank) * BLOCK_M, pb);
+                                tma_load_3d_pair(sa + A_BYTES, &mapA, fb_leader, kc * BLOCK_K,
+                                                 it.tm * BLOCK_N + static_cast<int>(rank) * Tile<CG>::B_LINES, pa);
+                            }
                             if (++stage == STAGES) { stage = 0; phase ^= 1u; }
                         }
                     }
@@ -344,15 +427,15 @@ residue_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
                 unsigned long long t0 = global_timer_ns();
                 while (global_timer_ns() - t0 < 2000000ull) { }
             }
-        } else if (warp == 1 && lane == 0) {
-            // -------------------------------------------------------- MMA issuer
-            constexpr uint32_t idesc = instr_desc<SUB>();
+        } else if (warp == 1 && lane == 0 && rank == 0) {
+            // -------------------------------------------------------- MMA issuer (pair: leader CTA only)
+            constexpr uint32_t idesc = instr_desc<SUB, CG>();
             int stage = 0;
             uint32_t phase = 0;
             int slot = 0;
             uint32_t slot_phase = 0;   // bit s = phase of slot s
             bool ok = true;
-            for (int64_t item = blockIdx.x; ok && item < p.total_items; item += gridDim.x) {
+            for (int64_t item = first_item; ok && item < p.total_items; item += item_step) {
                 Item it = decode_item(item, p);
                 const ModInfo &mi = p.mod[it.mod];
                 for (int job = 0; ok && job < mi.njobs; ++job) {
@@ -371,15 +454,15 @@ residue_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
 #pragma unroll
                         for (int ks = 0; ks < BLOCK_K / UMMA_K; ++ks) {
                             // advancing K inside the 128-byte swizzle atom: +32 bytes = +2 in the address field
-                            umma<SUB>(d_tmem, da + static_cast<uint64_t>(ks * (UMMA_K >> 4)),
+                            umma<SUB, CG>(d_tmem, da + static_cast<uint64_t>(ks * (UMMA_K >> 4)),
                                       db + static_cast<uint64_t>(ks * (UMMA_K >> 4)), idesc, accumulate);
                             accumulate = 1;
                         }
-                        umma_commit(empty_bar + 8 * stage);     // frees the stage when these MMAs finish
+                        umma_commit<CG>(empty_bar + 8 * stage);     // frees the stage when these MMAs finish
                         if (++stage == STAGES) { stage = 0; phase ^= 1u; }
                     }
                     if (!ok) break;
-                    umma_commit(tfull_bar + 8 * slot);           // accumulator complete
+                    umma_commit<CG>(tfull_bar + 8 * slot);           // accumulator complete
                     slot_phase ^= 1u << slot;
                     slot ^= 1;
                 }
@@ -396,7 +479,7 @@ residue_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
         int slot = 0;
         uint32_t slot_phase = 0;   // bit s = phase of slot s
         bool ok = true;
-        for (int64_t item = blockIdx.x; ok && item < p.total_items; item += gridDim.x) {
+        for (int64_t item = first_item; ok && item < p.total_items; item += item_step) {
             Item it = decode_item(item, p);
             const ModInfo &mi = p.mod[it.mod];
             const float mm = mi.m, inv_m = mi.inv_m;
@@ -408,30 +491,44 @@ residue_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
                 if (!ok) break;
                 tc_fence_after();
                 const float wj = mi.w[job];
+                const bool reduce_first = mi.reduce[job] != 0;
                 const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) +
                                        static_cast<uint32_t>(slot * BLOCK_N + part * COLS_PER_WARP);
 #pragma unroll
                 for (int c0 = 0; c0 < COLS_PER_WARP; c0 += 32) {
                     uint32_t v[32];
                     tmem_ld32(taddr + c0, v);
+                    if (reduce_first) {
 #pragma unroll
-                    for (int e = 0; e < 32; ++e) {
-                        float acc = SUB == 0 ? __uint_as_float(v[e])
-                                             : __int2float_rn(static_cast<int>(v[e]));
-                        float quot = fmaf(acc, inv_m, 12582912.0f) - 12582912.0f;   // rint(acc/m)
-                        float res = fmaf(-quot, mm, acc);                            // exact, |res| <= ~m/2
-                        comb[c0 + e] = fmaf(res, wj, comb[c0 + e]);                  // exact, < 2^24
+                        for (int e = 0; e < 32; ++e) {
+                            float acc = SUB == 0 ? __uint_as_float(v[e])
+                                                 : __int2float_rn(static_cast<int>(v[e]));
+                            float quot = fmaf(acc, inv_m, 12582912.0f) - 12582912.0f;   // rint(acc/m)
+                            float res = fmaf(-quot, mm, acc);                            // exact, |res| <= ~m/2
+                            comb[c0 + e] = fmaf(res, wj, comb[c0 + e]);                  // exact, < 2^24
+                        }
+                    } else {
+                        // the host has checked that w * acc stays below 2^24 for this k: no reduction needed
+#pragma unroll
+                        for (int e = 0; e < 32; ++e) {
+                            float acc = SUB == 0 ? __uint_as_float(v[e])
+                                                 : __int2float_rn(static_cast<int>(v[e]));
+                            comb[c0 + e] = fmaf(acc, wj, comb[c0 + e]);
+                        }
                     }
                 }
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(tempty_bar + 8 * slot);
+                if (lane == 0) {
+                    if (CG == 1) mbar_arrive(tempty_bar + 8 * slot);
+                    else mbar_arrive_cluster(map_to_cta(tempty_bar + 8 * slot, 0));   // the leader's barrier
+                }
                 slot_phase ^= 1u << slot;
                 slot ^= 1;
             }
             if (!ok) break;
             // this thread: column j of C, rows i0 .. i0+63 (contiguous in the residue array)
-            const int64_t jw = static_cast<int64_t>(it.tn) * BLOCK_M + q * 32;   // first column of the warp
+            const int64_t jw = static_cast<int64_t>(it.tn) * Tile<CG>::TILE_J + rank * BLOCK_M + q * 32;   // first column of the warp
             const int64_t j = jw + lane;
             const int64_t i0 = static_cast<int64_t>(it.tm) * BLOCK_N + part * COLS_PER_WARP;
             if (i0 >= p.m || jw >= p.n) continue;                                 // warp-uniform
@@ -487,9 +584,10 @@ residue_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
 
     tc_fence_before();
     __syncthreads();
+    if (CG == 2) cluster_sync_all();      // neither CTA leaves while the other may still touch it
     if (warp == 1) {
         tc_fence_after();
-        tmem_dealloc(tmem_base, TMEM_COLS);
+        tmem_dealloc<CG>(tmem_base, TMEM_COLS);
     }
 }
 
@@ -530,17 +628,57 @@ bool make_plane_map(CUtensorMap *map, const uint8_t *base, int64_t lines, int64_
     return rc == CUDA_SUCCESS;
 }
 
+template <int SUB, int CG>
+oz_status_t launch_variant(const CUtensorMap &mapA, const CUtensorMap &mapB, const GemmParams &p, int sms,
+                           cudaStream_t stream)
+{
+    auto kernel = residue_gemm_kernel<SUB, CG>;
+    OZ_CUDA_CHECK(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       static_cast<int>(SMEM_BYTES)));
+    int64_t groups = sms / CG;                                    // CTAs, or CTA pairs
+    if (p.total_items < groups) groups = p.total_items;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(groups * CG));
+    cfg.blockDim = dim3(NUM_THREADS);
+    cfg.dynamicSmemBytes = SMEM_BYTES;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = CG;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    OZ_CUDA_CHECK(cudaLaunchKernelEx(&cfg, kernel, mapA, mapB, p));
+    count_launch();
+    OZ_CUDA_CHECK(cudaGetLastError());
+    return OZ_OK;
+}
+
 }  // namespace
+
+// Which variant runs: CTA pairs (tcgen05 cta_group::2, tiles of 256 columns) unless that would pad
+// the column count noticeably more than 128-column tiles do (n = 128: one half-empty pair tile).
+// OZ_GEMM_CTA_GROUP=1|2 overrides the choice for experiments.
+static int cta_group_choice(int64_t n)
+{
+    const char *env = getenv("OZ_GEMM_CTA_GROUP");
+    if (env && env[0] == '2') return 2;
+    if (env && env[0] == '1') return 1;
+    const int64_t pad1 = round_up(n, BLOCK_M), pad2 = round_up(n, 2 * BLOCK_M);
+    return (pad2 * 20 <= pad1 * 21) ? 2 : 1;
+}
 
 oz_status_t launch_residue_gemm(int64_t m, int64_t n, int64_t k, const uint8_t *PA, int64_t strideA,
                                 int64_t pitchA, const uint8_t *PB, int64_t strideB, int64_t pitchB,
                                 int set, const Route &rt, uint16_t *R, int64_t ldr,
                                 int64_t mod_stride, cudaStream_t stream)
 {
+    const int cg = cta_group_choice(n);
     GemmParams p{};
     p.m = m; p.n = n; p.k = k;
-    p.tiles_m = static_cast<int>((m + BLOCK_N - 1) / BLOCK_N);   // 256 rows of C per tile
-    p.tiles_n = static_cast<int>((n + BLOCK_M - 1) / BLOCK_M);   // 128 columns of C per tile
+    p.tiles_m = static_cast<int>((m + BLOCK_N - 1) / BLOCK_N);             // 256 rows of C per tile
+    p.tiles_n = static_cast<int>((n + BLOCK_M * cg - 1) / (BLOCK_M * cg)); // 128 (256) columns of C per tile
     p.vec_store = ((ldr & 7) == 0 && (mod_stride & 7) == 0 && (reinterpret_cast<uintptr_t>(R) & 15u) == 0) ? 1 : 0;
     p.nk = static_cast<int>((k + BLOCK_K - 1) / BLOCK_K);
     p.r = set_r(set);
@@ -552,37 +690,41 @@ oz_status_t launch_residue_gemm(int64_t m, int64_t n, int64_t k, const uint8_t *
         p.mod[i].m = static_cast<float>(mi);
         p.mod[i].inv_m = 1.0f / static_cast<float>(mi);
         p.mod[i].plane0 = first_plane(set, i);
+        // Exact FP32 range of the running combination: digits are bounded by |d0| <= 14 (16 for
+        // squares), |d1| <= 16, |d0+d1| <= 22 (Lemma 1), a reduced accumulator by (m+1)/2 <= 545.
+        // A job's accumulator may be weighted without reducing it first while the worst-case sum
+        // stays below 2^24.
+        const int64_t lim = (1ll << 24) - 1, kk = k > 0 ? k : 1;
         if (s) {
             p.mod[i].njobs = 2;
             p.mod[i].w[0] = 1.0f; p.mod[i].w[1] = static_cast<float>(s); p.mod[i].w[2] = 0.0f;
+            p.mod[i].reduce[0] = (256 * kk + static_cast<int64_t>(s) * 545 <= lim) ? 0 : 1;
+            p.mod[i].reduce[1] = 1;
+            p.mod[i].reduce[2] = 1;
         } else {
             p.mod[i].njobs = 3;
             p.mod[i].w[0] = -15.0f; p.mod[i].w[1] = 16.0f; p.mod[i].w[2] = 240.0f;
+            const bool skip01 = (15 * 196 + 16 * 484) * kk + 240 * 545 <= lim;
+            p.mod[i].reduce[0] = skip01 ? 0 : 1;
+            p.mod[i].reduce[1] = skip01 ? 0 : 1;
+            p.mod[i].reduce[2] = 1;
         }
     }
     if (k == 0) p.nk = 1;   // one all-zero chunk (the planes' padding) gives residues 0
 
     CUtensorMap mapA, mapB;
-    if (!make_plane_map(&mapA, PA, m, pitchA, strideA, p_store(set), BLOCK_N) ||
+    if (!make_plane_map(&mapA, PA, m, pitchA, strideA, p_store(set), BLOCK_N / cg) ||
         !make_plane_map(&mapB, PB, n, pitchB, strideB, p_store(set), BLOCK_M))
         return OZ_ERR_CUDA;
 
     int dev = 0, sms = 148;
     OZ_CUDA_CHECK(cudaGetDevice(&dev));
     OZ_CUDA_CHECK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
-    int grid = static_cast<int>(p.total_items < sms ? p.total_items : sms);
-    if (rt.substrate == 0) {
-        OZ_CUDA_CHECK(cudaFuncSetAttribute(residue_gemm_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                           static_cast<int>(SMEM_BYTES)));
-        residue_gemm_kernel<0><<<grid, NUM_THREADS, SMEM_BYTES, stream>>>(mapA, mapB, p);
-    } else {
-        OZ_CUDA_CHECK(cudaFuncSetAttribute(residue_gemm_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                           static_cast<int>(SMEM_BYTES)));
-        residue_gemm_kernel<1><<<grid, NUM_THREADS, SMEM_BYTES, stream>>>(mapA, mapB, p);
-    }
-    count_launch();
-    OZ_CUDA_CHECK(cudaGetLastError());
-    return OZ_OK;
+    if (cg == 2)
+        return rt.substrate == 0 ? launch_variant<0, 2>(mapA, mapB, p, sms, stream)
+                                 : launch_variant<1, 2>(mapA, mapB, p, sms, stream);
+    return rt.substrate == 0 ? launch_variant<0, 1>(mapA, mapB, p, sms, stream)
+                             : launch_variant<1, 1>(mapA, mapB, p, sms, stream);
 }
 
 }  // namespace oz
