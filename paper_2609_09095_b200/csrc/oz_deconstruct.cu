@@ -13,8 +13,10 @@
 //
 // Residue of a 64-bit two's-complement integer a' modulo m (the paper's byte-plane identity of
 // paragraph "O2", applied to 16-bit limbs so that every partial sum stays below 2^32):
-//   a' mod m = (l0 + l1 (2^16 mod m) + l2 (2^32 mod m) + l3 (2^48 mod m) + [a'<0] ((-2^64) mod m)) mod m
-// followed by one Barrett step with floor(2^32/m).  The digit split, the Lemma 1 carry and the
+//   a' mod m = (l0 + l1 (2^16 mod m) + l2 (2^32 mod m) + l3 (2^48 mod m) + bias_m) mod m
+// with the top limb l3 taken SIGNED (this replaces the paper's (-2^64) mod m sign correction) and
+// bias_m a multiple of m that keeps the sum non-negative, followed by one exact multiply-high
+// division by m.  The digit split, the Lemma 1 carry and the
 // E4M3 / INT8 encoding are folded into a per-modulus table indexed by the canonical residue
 // (built on the host at set-up), held in shared memory.
 #include <utility>
@@ -104,27 +106,48 @@ scan_kernel(const double *__restrict__ X, int64_t ldx, int64_t lines, int64_t k,
     unsigned long long acc = 0;
     int E = 0;
     if (PASS == 1 && live) E = s.emax[line];
+    // 2^(9-E) as a double, when it is a normal number (not for lines of subnormals only)
+    const bool fast_scale = PASS == 1 && E != INT32_MIN && 9 - E >= -1000 && 9 - E <= 1000;
+    const double scale9 = __hiloint2double((1023 + (fast_scale ? 9 - E : 0)) << 20, 0);
     if (live && !(PASS == 1 && E == INT32_MIN)) {
-        for (int64_t kk = kstart; kk < k1; kk += kstep) {
-            double x = *element(X, ldx, SIDE, line, kk);
-            if (PASS == 0) {
-                int e;
-                int c = classify(x, &e);
-                if (c == 2) bad = 1;
-                if (c == 1 && e > emax) emax = e;
-            } else {
-                unsigned long long bits = static_cast<unsigned long long>(__double_as_longlong(x));
-                int be = static_cast<int>((bits >> 52) & 0x7FF);
-                unsigned long long frac = bits & 0xFFFFFFFFFFFFFull;
-                if (be == 0x7FF || (be == 0 && frac == 0)) continue;
-                unsigned long long sig = be ? (frac | (1ull << 52)) : frac;
-                int ex = be ? be - 1023 : -1022;
-                int sh = 43 + E - ex;                 // |x| 2^(9-E) = sig / 2^sh
-                unsigned long long abar;
-                if (sh >= 64) abar = 1;
-                else if (sh <= 0) abar = sig << (-sh);
-                else abar = (sig >> sh) + ((sig & ((1ull << sh) - 1)) ? 1ull : 0ull);
-                acc += abar * abar;
+        // batches of 8 independent loads keep enough bytes in flight to run at memory speed
+        for (int64_t kb = kstart; kb < k1; kb += 8 * kstep) {
+            double xs[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                int64_t kk = kb + u * kstep;
+                xs[u] = kk < k1 ? *element(X, ldx, SIDE, line, kk) : 0.0;
+            }
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                double x = xs[u];
+                if (PASS == 0) {
+                    int e;
+                    int c = classify(x, &e);
+                    if (c == 2) bad = 1;
+                    if (c == 1 && e > emax) emax = e;
+                } else if (fast_scale) {
+                    // ceil(|x| 2^(9-E)) through an exact FP64 scaling and a round-up conversion; a
+                    // non-zero x whose scaled value underflows to zero still counts as 1
+                    double y = fabs(x) * scale9;
+                    unsigned long long abar = static_cast<unsigned long long>(__double2ll_ru(y));
+                    if (abar == 0ull && x != 0.0) abar = 1ull;
+                    if (!(y < 2048.0)) abar = 0ull;       // Inf/NaN: the line is flagged, value unused
+                    acc += abar * abar;
+                } else {
+                    unsigned long long bits = static_cast<unsigned long long>(__double_as_longlong(x));
+                    int be = static_cast<int>((bits >> 52) & 0x7FF);
+                    unsigned long long frac = bits & 0xFFFFFFFFFFFFFull;
+                    if (be == 0x7FF || (be == 0 && frac == 0)) continue;
+                    unsigned long long sig = be ? (frac | (1ull << 52)) : frac;
+                    int ex = be ? be - 1023 : -1022;
+                    int sh = 43 + E - ex;                 // |x| 2^(9-E) = sig / 2^sh
+                    unsigned long long abar;
+                    if (sh >= 64) abar = 1;
+                    else if (sh <= 0) abar = sig << (-sh);
+                    else abar = (sig >> sh) + ((sig & ((1ull << sh) - 1)) ? 1ull : 0ull);
+                    acc += abar * abar;
+                }
             }
         }
     }
@@ -174,7 +197,16 @@ __global__ void scan_finalize_kernel(ScanScratch s, int64_t lines, int rule, int
     shift[i] = (top >> 1) + 9 - E;
 }
 
-// Eq. 1 for one element: a' = quant(x 2^sigma) as a 64-bit integer.
+// Eq. 1 for one element, fast form: multiplying by the power of two 2^sigma is exact in FP64 (a
+// product that underflows is far below 1/2 and rounds to zero either way), and the hardware
+// conversion rounds to nearest-even or toward zero.  Valid while 2^sigma is a normal double.
+__device__ __forceinline__ long long quantise_fp(double x, double scale, bool tz)
+{
+    double y = x * scale;
+    return tz ? __double2ll_rz(y) : __double2ll_rn(y);
+}
+
+// Eq. 1 for one element, integer form (any sigma): a' = quant(x 2^sigma) as a 64-bit integer.
 __device__ __forceinline__ long long quantise(double x, int sigma, bool tz)
 {
     unsigned long long bits = static_cast<unsigned long long>(__double_as_longlong(x));
@@ -199,24 +231,28 @@ __device__ __forceinline__ long long quantise(double x, int sigma, bool tz)
 template <int SET, int I>
 __device__ __forceinline__ void convert_modulus(const uint32_t (&l0)[4], const uint32_t (&l1)[4],
                                                 const uint32_t (&l2)[4], const uint32_t (&l3)[4],
-                                                const uint32_t (&neg)[4],
                                                 const uint32_t *__restrict__ lut, uint8_t *out,
                                                 int64_t plane_stride)
 {
     constexpr uint32_t m = modulus(SET, I);
     constexpr uint32_t c1 = pow2_mod(16, m), c2 = pow2_mod(32, m), c3 = pow2_mod(48, m);
-    constexpr uint32_t corr = (m - pow2_mod(64, m)) % m;     // (-2^64) mod m
-    constexpr uint32_t magic = barrett_magic(m);
+    // a' = l0 + l1 2^16 + l2 2^32 + l3 2^48 with the top limb SIGNED; `bias` (a multiple of m not
+    // below 2^15 c3) keeps the limb sum non-negative, so no separate sign correction is needed.
+    constexpr uint32_t bias = ((32768u * c3 + m - 1) / m) * m;
+    // floor(v / m) = (v * ceil(2^39 / m)) >> 39 exactly for v < 2^28
+    constexpr uint32_t magic = static_cast<uint32_t>(((1ull << 39) + m - 1) / m);
     constexpr int off = lut_offset(SET, I);
     constexpr int plane = first_plane(SET, I);
-    static_assert(65535ull * (1ull + c1 + c2 + c3) + corr < 0x100000000ull, "limb sum fits 32 bits");
+    static_assert(65535ull * (1ull + c1 + c2) + 32767ull * c3 + bias < (1ull << 28), "limb sum below 2^28");
     uint32_t w[4];
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
-        uint32_t v = l0[e] + l1[e] * c1 + l2[e] * c2 + l3[e] * c3 + neg[e] * corr;
-        uint32_t q = __umulhi(v, magic);
-        uint32_t r = v - q * m;                  // in [0, 2m)
-        r = min(r, r - m);                       // unsigned: picks r - m when r >= m
+        uint32_t v = l3[e] * c3 + bias;          // l3 holds the signed limb in two's complement
+        v = l2[e] * c2 + v;
+        v = l1[e] * c1 + v;
+        v += l0[e];
+        uint32_t q = __umulhi(v, magic) >> 7;
+        uint32_t r = v - q * m;                  // canonical residue in [0, m)
         w[e] = lut[off + r];
     }
     uint32_t t01 = __byte_perm(w[0], w[1], 0x5140);
@@ -234,11 +270,10 @@ template <int SET, int... I>
 __device__ __forceinline__ void convert_all_moduli(std::integer_sequence<int, I...>,
                                                    const uint32_t (&l0)[4], const uint32_t (&l1)[4],
                                                    const uint32_t (&l2)[4], const uint32_t (&l3)[4],
-                                                   const uint32_t (&neg)[4],
                                                    const uint32_t *__restrict__ lut, uint8_t *out,
                                                    int64_t plane_stride)
 {
-    (convert_modulus<SET, I>(l0, l1, l2, l3, neg, lut, out, plane_stride), ...);
+    (convert_modulus<SET, I>(l0, l1, l2, l3, lut, out, plane_stride), ...);
 }
 
 // Four consecutive inner-dimension elements of one line -> 4 bytes of every stored plane.
@@ -247,20 +282,22 @@ __device__ __forceinline__ void convert4(const double (&x)[4], int sigma, bool t
                                          const uint32_t *__restrict__ lut, uint8_t *out,
                                          int64_t plane_stride)
 {
-    uint32_t l0[4], l1[4], l2[4], l3[4], neg[4];
+    uint32_t l0[4], l1[4], l2[4], l3[4];
+    // 2^sigma as a double when it is a normal number (always, except for lines of subnormals)
+    const bool fast = sigma >= -1000 && sigma <= 1000;
+    const double scale = __hiloint2double((1023 + (fast ? sigma : 0)) << 20, 0);
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
-        long long a = quantise(x[e], sigma, tz);
+        long long a = fast ? quantise_fp(x[e], scale, tz) : quantise(x[e], sigma, tz);
         unsigned long long p = static_cast<unsigned long long>(a);
         uint32_t lo = static_cast<uint32_t>(p), hi = static_cast<uint32_t>(p >> 32);
         l0[e] = lo & 0xFFFFu;
         l1[e] = lo >> 16;
         l2[e] = hi & 0xFFFFu;
-        l3[e] = hi >> 16;
-        neg[e] = hi >> 31;
+        l3[e] = static_cast<uint32_t>(static_cast<int32_t>(hi) >> 16);   // signed top limb
     }
-    convert_all_moduli<SET>(std::make_integer_sequence<int, set_r(SET)>{}, l0, l1, l2, l3, neg, lut,
-                            out, plane_stride);
+    convert_all_moduli<SET>(std::make_integer_sequence<int, set_r(SET)>{}, l0, l1, l2, l3, lut, out,
+                            plane_stride);
 }
 
 template <int SET, int SIDE>
