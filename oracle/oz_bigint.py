@@ -15,6 +15,7 @@ from fractions import Fraction
 SETS = {
     "S": [1089, 1024, 961, 841, 625, 529, 511, 509, 503, 499, 491, 487],
     "E": [1089, 1024, 961, 841, 625, 529, 251, 247, 241, 239, 233, 229, 227],
+    "A": [256, 255, 253, 251, 247, 241, 239, 233, 229, 227, 223, 217, 211, 199, 197],
 }
 
 

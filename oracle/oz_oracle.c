@@ -38,10 +38,14 @@
 typedef __int128 i128;
 typedef unsigned __int128 u128;
 
-enum { OZO_SET_S = 0, OZO_SET_E = 1 };
+enum { OZO_SET_S = 0, OZO_SET_E = 1, OZO_SET_A = 2 };
 enum { OZO_QUANT_RN = 0, OZO_QUANT_TZ = 1 };
 enum { OZO_SCALE_MAXEXP = 0, OZO_SCALE_CS = 1 };
-enum { OZO_SUB_FP8 = 0, OZO_SUB_INT8 = 1 };
+/* FP8 / INT8: two-limb digit planes (Sec. 2 "FP8 variant").  INT8_NATIVE: one plane per modulus
+ * holding the centred residue itself as a signed byte -- possible for byte moduli only (Sec. 2,
+ * "The substrate transition": "the centred residue of a byte modulus (m <= 256) fits an INT8
+ * operand directly", alpha_INT8 = r + 1).                                                     */
+enum { OZO_SUB_FP8 = 0, OZO_SUB_INT8 = 1, OZO_SUB_INT8_NATIVE = 2 };
 
 #define OZO_NONFINITE_SHIFT INT32_MIN
 
@@ -50,12 +54,14 @@ enum { OZO_SUB_FP8 = 0, OZO_SUB_INT8 = 1 };
 /* ------------------------------------------------------------------ */
 static const int SET_S[12] = {1089, 1024, 961, 841, 625, 529, 511, 509, 503, 499, 491, 487};
 static const int SET_E[13] = {1089, 1024, 961, 841, 625, 529, 251, 247, 241, 239, 233, 229, 227};
+/* "Candidate A (all-byte)": fifteen coprime moduli, 117.8 bits */
+static const int SET_A[15] = {256, 255, 253, 251, 247, 241, 239, 233, 229, 227, 223, 217, 211, 199, 197};
 
 int ozo_modset(int set, int *moduli)
 {
-    const int *src = (set == OZO_SET_S) ? SET_S : SET_E;
-    int r = (set == OZO_SET_S) ? 12 : 13;
-    if (set != OZO_SET_S && set != OZO_SET_E) return 0;
+    const int *src = (set == OZO_SET_S) ? SET_S : (set == OZO_SET_E ? SET_E : SET_A);
+    int r = (set == OZO_SET_S) ? 12 : (set == OZO_SET_E ? 13 : 15);
+    if (set != OZO_SET_S && set != OZO_SET_E && set != OZO_SET_A) return 0;
     for (int i = 0; i < r; ++i) moduli[i] = src[i];
     return r;
 }
@@ -71,10 +77,23 @@ int ozo_square_root(int m)
 /* stored planes per modulus: 2 for a square, 3 otherwise (Sec. 2, FP8 variant) */
 int ozo_planes_of(int m) { return ozo_square_root(m) ? 2 : 3; }
 
+/* stored planes per modulus on a substrate: one for native INT8 residues, else 2 or 3 */
+int ozo_planes_of_sub(int m, int substrate)
+{
+    return substrate == OZO_SUB_INT8_NATIVE ? 1 : ozo_planes_of(m);
+}
+
 int ozo_pstore(int set)
 {
     int mod[16], r = ozo_modset(set, mod), p = 0;
     for (int i = 0; i < r; ++i) p += ozo_planes_of(mod[i]);
+    return p;
+}
+
+int ozo_pstore_sub(int set, int substrate)
+{
+    int mod[16], r = ozo_modset(set, mod), p = 0;
+    for (int i = 0; i < r; ++i) p += ozo_planes_of_sub(mod[i], substrate);
     return p;
 }
 
@@ -338,12 +357,13 @@ int ozo_planes(int64_t lines, int64_t k, const int16_t *D, int set, int substrat
 {
     int mod[16], r = ozo_modset(set, mod), plane = 0, bad = 0;
     for (int i = 0; i < r; ++i) {
-        int np = ozo_planes_of(mod[i]);
+        int np = ozo_planes_of_sub(mod[i], substrate);
         /* bytes of every centred residue of this modulus, worked out once (index d + 1024) */
         static uint8_t code[2048][3];
         for (int d = -(mod[i] / 2); 2 * d < mod[i]; ++d) {
             int dg[3] = {0, 0, 0};
-            ozo_split(d, mod[i], dg);
+            if (substrate == OZO_SUB_INT8_NATIVE) dg[0] = d; /* the residue is the operand */
+            else ozo_split(d, mod[i], dg);
             for (int q = 0; q < np; ++q) {
                 int byte;
                 if (substrate == OZO_SUB_FP8) {
@@ -414,7 +434,7 @@ int64_t ozo_plane_products(int64_t m, int64_t n, int64_t k, const uint8_t *PA,
     for (int c = 0; c < 256; ++c) digit_of[c] = plane_digit((uint8_t)c, substrate);
     for (int i = 0; i < r; ++i) {
         int s = ozo_square_root(mod[i]);
-        int np = s ? 2 : 3;
+        int np = substrate == OZO_SUB_INT8_NATIVE ? 1 : (s ? 2 : 3);
         int64_t worst_i = 0;
 #pragma omp parallel for schedule(static) reduction(max : worst_i)
         for (int64_t j = 0; j < n; ++j)
@@ -426,7 +446,9 @@ int64_t ozo_plane_products(int64_t m, int64_t n, int64_t k, const uint8_t *PA,
                         a[q] = digit_of[PA[(plane + q) * strideA + ii * pitchA + kk]];
                         b[q] = digit_of[PB[(plane + q) * strideB + j * pitchB + kk]];
                     }
-                    if (s) {
+                    if (np == 1) {
+                        acc[0] += (int64_t)a[0] * b[0];
+                    } else if (s) {
                         acc[0] += (int64_t)a[0] * b[0];
                         acc[1] += (int64_t)a[1] * b[0] + (int64_t)a[0] * b[1];
                     } else {
@@ -439,8 +461,9 @@ int64_t ozo_plane_products(int64_t m, int64_t n, int64_t k, const uint8_t *PA,
                     int64_t v = acc[q] < 0 ? -acc[q] : acc[q];
                     if (v > worst_i) worst_i = v;
                 }
-                int64_t t = s ? acc[0] + (int64_t)s * acc[1]
-                              : -15 * acc[0] + 16 * acc[1] + 240 * acc[2];
+                int64_t t = np == 1 ? acc[0]
+                            : s     ? acc[0] + (int64_t)s * acc[1]
+                                    : -15 * acc[0] + 16 * acc[1] + 240 * acc[2];
                 int64_t c = t % mod[i];
                 if (c < 0) c += mod[i];
                 R[((int64_t)i * n + j) * m + ii] = (uint16_t)c;

@@ -19,10 +19,10 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "oz_oracle.c")
 _LIB = os.path.join(_HERE, "liboz_oracle.so")
 
-SET_S, SET_E = 0, 1
+SET_S, SET_E, SET_A = 0, 1, 2
 QUANT_RN, QUANT_TZ = 0, 1
 SCALE_MAXEXP, SCALE_CS = 0, 1
-SUB_FP8, SUB_INT8 = 0, 1
+SUB_FP8, SUB_INT8, SUB_INT8_NATIVE = 0, 1, 2
 NONFINITE_SHIFT = -(2**31)
 
 _lib = None
@@ -76,8 +76,8 @@ def modset(s: int) -> list[int]:
     return [buf[i] for i in range(r)]
 
 
-def pstore(s: int) -> int:
-    return lib().ozo_pstore(s)
+def pstore(s: int, substrate: int = 0) -> int:
+    return lib().ozo_pstore_sub(s, substrate)
 
 
 def planes_of(m: int) -> int:
@@ -187,10 +187,10 @@ def residues(Q: np.ndarray, s: int) -> np.ndarray:
 def planes(D: np.ndarray, s: int, substrate: int, row_pitch: int | None = None) -> np.ndarray:
     r, lines, k = D.shape
     pitch = row_pitch if row_pitch is not None else (k + 15) // 16 * 16
-    P = np.full((pstore(s), lines, pitch), 0xAA, dtype=np.uint8)
+    P = np.full((pstore(s, substrate), lines, pitch), 0xAA, dtype=np.uint8)
     rc = lib().ozo_planes(_i64(lines), _i64(k), _p(np.ascontiguousarray(D)), s, substrate, _p(P),
                           _i64(lines * pitch), _i64(pitch))
-    assert rc == pstore(s), "a digit was not representable on the substrate"
+    assert rc == pstore(s, substrate), "a digit was not representable on the substrate"
     return P
 
 

@@ -27,7 +27,7 @@ def read_golden(name):
 
 
 PAPER = read_golden("paper_constants.txt")
-SETS = {"S": ozo.SET_S, "E": ozo.SET_E}
+SETS = {"S": ozo.SET_S, "E": ozo.SET_E, "A": ozo.SET_A}
 
 
 # ----------------------------------------------------------------- P1: the sets
@@ -36,9 +36,10 @@ def test_modulus_sets_match_paper():
     assert ozo.modset(ozo.SET_S) == S
     tail = [int(v) for v in PAPER["set_E_tail"].split()]
     assert ozo.modset(ozo.SET_E) == S[:6] + tail
+    assert ozo.modset(ozo.SET_A) == [int(v) for v in PAPER["set_A"].split()]
 
 
-@pytest.mark.parametrize("name", ["S", "E"])
+@pytest.mark.parametrize("name", ["S", "E", "A"])
 def test_set_counts_and_range(name):
     ms = ozo.modset(SETS[name])
     for i, a in enumerate(ms):
@@ -56,7 +57,7 @@ def test_set_counts_and_range(name):
 
 
 # ----------------------------------------------------------------- range budget
-@pytest.mark.parametrize("name", ["S", "E"])
+@pytest.mark.parametrize("name", ["S", "E", "A"])
 @pytest.mark.parametrize("k", [1, 7, 256, 1024, 4096, 5003, 32768])
 def test_budget_is_inside_crt_range(name, k):
     M = math.prod(ozo.modset(SETS[name]))
@@ -185,9 +186,32 @@ def test_lemma1_is_sharp_at_513():
         assert good == ok
 
 
+def test_all_byte_set_native_int8_planes():
+    """Set A: every reduction constant fits a byte (largest 243, dot products < 2^19), every
+    centred residue fits a signed byte (m = 256 reaches -128), one plane and one product per modulus."""
+    ms = ozo.modset(ozo.SET_A)
+    assert max(pow(256, j, m) for m in ms for j in range(8)) == int(PAPER["max_reduction_constant_A"])
+    assert 8 * 255 * int(PAPER["max_reduction_constant_A"]) < int(PAPER["byte_dot_bound"])
+    assert len(ms) + 1 == int(PAPER["alpha_A_int8_native"])
+    assert ozo.pstore(ozo.SET_A, ozo.SUB_INT8_NATIVE) == len(ms) == 15
+    assert ozo.pstore(ozo.SET_A, ozo.SUB_FP8) == int(PAPER["pstore_A"])
+    assert ozo.centred_residue(128, 256) == -128 and ozo.centred_residue(-129, 256) == 127
+    rng = np.random.default_rng(12)
+    Q = rng.integers(-2**52, 2**52, size=(3, 40))
+    Q[0, :15] = [m // 2 for m in ms]                    # the endpoint residues
+    Q[1, :15] = [-(m // 2) for m in ms]
+    D = ozo.residues(Q, ozo.SET_A)
+    P = ozo.planes(D, ozo.SET_A, ozo.SUB_INT8_NATIVE)
+    assert P.shape == (15, 3, 48)
+    assert (P[:, :, :40].view(np.int8) == D).all() and (P[:, :, 40:] == 0).all()
+    for i, m in enumerate(ms):
+        assert ((D[i].astype(np.int64) - Q) % m == 0).all()
+        assert D[i].min() >= -(m // 2) and D[i].max() <= (m - 1) // 2 and D[i].min() >= -128
+
+
 def test_byte_moduli_never_carry():
     lo_s, hi_s = [int(v) for v in PAPER["byte_modulus_sum_range"].split()]
-    for m in ozo.modset(ozo.SET_E)[6:]:
+    for m in ozo.modset(ozo.SET_E)[6:] + ozo.modset(ozo.SET_A)[1:]:
         for d in range(-(m // 2), (m - 1) // 2 + 1):
             d0, d1, ds = ozo.split(d, m)
             assert d0 == (d + 8) % 16 - 8 and d == d0 + 16 * d1
@@ -219,7 +243,7 @@ def test_square_split_exhaustive(m):
 
 
 # ----------------------------------------------------------------- P6: CRT round trip
-@pytest.mark.parametrize("name", ["S", "E"])
+@pytest.mark.parametrize("name", ["S", "E", "A"])
 def test_crt_round_trip(name):
     ms = ozo.modset(SETS[name])
     M = math.prod(ms)
@@ -299,7 +323,8 @@ def test_shifts_keep_product_in_range(rule, name):
 
 # ----------------------------------------------------------------- P7: brute force / big ints
 @pytest.mark.parametrize("name,quant,rule", [("S", "RN", "CS"), ("S", "TZ", "MAXEXP"),
-                                             ("E", "RN", "MAXEXP"), ("E", "TZ", "CS")])
+                                             ("E", "RN", "MAXEXP"), ("E", "TZ", "CS"),
+                                             ("A", "RN", "CS"), ("A", "TZ", "MAXEXP")])
 def test_whole_method_against_big_integers(name, quant, rule):
     rng = np.random.default_rng(21)
     m, n, k = 5, 4, 19
@@ -320,7 +345,8 @@ def test_whole_method_against_big_integers(name, quant, rule):
     assert ozo.direct(QA, QB, as_int=True).tolist() == Cint
 
 
-@pytest.mark.parametrize("name,sub", [("S", ozo.SUB_FP8), ("S", ozo.SUB_INT8), ("E", ozo.SUB_FP8)])
+@pytest.mark.parametrize("name,sub", [("S", ozo.SUB_FP8), ("S", ozo.SUB_INT8), ("E", ozo.SUB_FP8),
+                                      ("A", ozo.SUB_FP8), ("A", ozo.SUB_INT8_NATIVE)])
 def test_planes_reproduce_residue_products(name, sub):
     rng = np.random.default_rng(4)
     m, n, k = 6, 5, 37
@@ -333,10 +359,10 @@ def test_planes_reproduce_residue_products(name, sub):
         assert ((DA[i].astype(np.int64) - QA) % mm == 0).all()
         assert (2 * DA[i].astype(np.int64) >= -mm).all() and (2 * DA[i].astype(np.int64) < mm).all()
     PA, PB = ozo.planes(DA, SETS[name], sub), ozo.planes(DB, SETS[name], sub)
-    assert PA.shape == (ozo.pstore(SETS[name]), m, 48) and (PA[:, :, k:] == 0).all()
+    assert PA.shape == (ozo.pstore(SETS[name], sub), m, 48) and (PA[:, :, k:] == 0).all()
     R1 = ozo.products(DA, DB, SETS[name])
     R2, worst = ozo.plane_products(PA, PB, k, SETS[name], sub)
-    assert (R1 == R2).all() and worst <= 2 * 256 * k
+    assert (R1 == R2).all() and worst <= (128 * 128 if sub == ozo.SUB_INT8_NATIVE else 2 * 256) * k
     want = (QA.astype(object) @ QB.astype(object).T)
     for i, mm in enumerate(ms):
         assert (R1[i].T.astype(object) == want % mm).all()
@@ -346,7 +372,7 @@ def test_planes_reproduce_residue_products(name, sub):
 def test_exact_on_small_integers():
     A, B = syn.special_operands("small_integers", 12, 10, 64)
     want = (A.astype(np.int64).astype(object) @ B.astype(np.int64).astype(object))
-    for name in ("S", "E"):
+    for name in ("S", "E", "A"):
         for quant in (ozo.QUANT_RN, ozo.QUANT_TZ):
             for rule in (ozo.SCALE_MAXEXP, ozo.SCALE_CS):
                 Cm = ozo.dgemm(A, B, SETS[name], quant, rule)
