@@ -125,7 +125,7 @@ def oracle_sample_tflops(cfg, set_name: str, sample=(4096, 6144, 1024)):
     from oracle import oz_oracle as ozo
     m, n, k = min(sample[0], cfg.m), min(sample[1], cfg.n), min(sample[2], cfg.k)
     A, B, C0 = syn.operands(cfg, m, n, k, want_c=True)
-    oset = ozo.SET_S if set_name == "S" else ozo.SET_E
+    oset = {"S": ozo.SET_S, "E": ozo.SET_E, "A": ozo.SET_A}[set_name]
     ozo.dgemm(np.asfortranarray(A[:32]), np.asfortranarray(B[:, :32]), oset)  # load the library, warm the threads
     t0 = time.perf_counter()
     ozo.dgemm(A, B, oset, ozo.QUANT_RN, ozo.SCALE_CS, cfg.alpha, cfg.beta, C0 if cfg.beta else None)
@@ -163,8 +163,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", type=int, default=3, help="synthetic configuration 1..5 (3 = HPL update)")
-    ap.add_argument("--set", dest="set_name", default="S", choices=["S", "E"])
-    ap.add_argument("--substrate", default="fp8", choices=["fp8", "int8"])
+    ap.add_argument("--set", dest="set_name", default="S", choices=["S", "E", "A"])
+    ap.add_argument("--substrate", default="fp8", choices=["fp8", "int8", "int8n"],
+                    help="int8n = native INT8 residues, one plane per modulus (set A only)")
     ap.add_argument("--shape", default=None, help="m,n,k override (same distribution and seed as --config)")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -191,9 +192,14 @@ def main():
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
 
     m, n, k = cfg.m, cfg.n, cfg.k
-    modset = oz.OZ_SET_S if args.set_name == "S" else oz.OZ_SET_E
-    route = (oz.OZ_SUB_FP8 if args.substrate == "fp8" else oz.OZ_SUB_INT8) | oz.OZ_QUANT_RN | oz.OZ_SCALE_CS
-    r, p_store, _ = oz.oz_set_info(modset)
+    modset = {"S": oz.OZ_SET_S, "E": oz.OZ_SET_E, "A": oz.OZ_SET_A}[args.set_name]
+    sub = {"fp8": oz.OZ_SUB_FP8, "int8": oz.OZ_SUB_INT8, "int8n": oz.OZ_SUB_INT8_NATIVE}[args.substrate]
+    route = sub | oz.OZ_QUANT_RN | oz.OZ_SCALE_CS
+    r, _, _ = oz.oz_set_info(modset)
+    p_store = oz.oz_plane_count(modset, route)
+    if p_store == 0:
+        raise SystemExit("the native INT8 substrate needs the all-byte set: --set A --substrate int8n")
+    passes = r if args.substrate == "int8n" else 3 * r    # plane products per FP64 product
 
     # every rank owns an independent instance of the problem (weak scaling); seeds differ per rank
     cfg_rank = syn.Config(**{**cfg.__dict__, "seed": cfg.seed + rank})
@@ -281,11 +287,11 @@ def main():
     if rank == 0:
         peaks = measured_peaks()
         value = work / (ms * 1e-3) / 1e12
-        lowp_flops = 3.0 * r * flops                       # p_mma = 3r plane products
+        lowp_flops = float(passes) * flops                 # p_mma plane products (3r, or r on the native INT8 route)
         gemm_ms = float(stage_ms[2])
         tensor_peak = 2.0 * peaks["bf16_sustained"]        # 8-bit operands: nominal 2x the bf16 rate
         achieved = lowp_flops / (gemm_ms * 1e-3) / 1e12
-        roof_nominal = 4500.0 / (3 * r + 1)                # P_low/(3r+1) at B200's dense 8-bit rate
+        roof_nominal = 4500.0 / (passes + 1)               # P_low/(3r+1), or P_low/(r+1) native INT8, at B200's dense 8-bit rate
         hbm = peaks["hbm_gbs"]
         dec_bytes = (8 + 8 * 2 + p_store) * (m * k + k * n)   # max-exponent + sum-of-squares scans, convert read, planes written
         rec_bytes = (2 * r + 8 + (8 if cfg.beta else 0)) * m * n
@@ -300,10 +306,10 @@ def main():
                        "l2": "inputs larger than L2 (126 MB): A+B %.0f MB, C %.0f MB, planes %.0f MB, residues %.0f MB"
                              % (8e-6 * (m * k + k * n), 8e-6 * m * n, 1e-6 * p_store * (m + n) * k, 2e-6 * r * m * n),
                        "parallelism": f"replicas x{world}" if world > 1 else "single GPU"},
-            "roof": {"definition": "P_low/(3r+1)", "nominal_tflops": roof_nominal,
+            "roof": {"definition": "P_low/(3r+1)" if passes == 3 * r else "P_low/(r+1)", "nominal_tflops": roof_nominal,
                      "frac_of_nominal": value / world / roof_nominal,
-                     "at_measured_peak_tflops": tensor_peak / (3 * r + 1),
-                     "frac_at_measured_peak": value / world / (tensor_peak / (3 * r + 1))},
+                     "at_measured_peak_tflops": tensor_peak / (passes + 1),
+                     "frac_at_measured_peak": value / world / (tensor_peak / (passes + 1))},
             "roofline": {"kernel": "residue_gemm_kernel (tcgen05)", "bound": "tensor", "achieved": achieved,
                          "peak": tensor_peak, "unit": "TFLOP/s", "frac": achieved / tensor_peak,
                          "peak_source": f"{peaks['source']} bf16 sustained x2 (8-bit operands)",

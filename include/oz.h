@@ -53,12 +53,16 @@ typedef enum {
 } oz_status_t;
 
 /* Modulus sets: S = the published 12-modulus set (Sec. 2, step (ii));
- * E = the hybrid set, six squares of S plus seven byte moduli ("Candidate E"). */
-typedef enum { OZ_SET_S = 0, OZ_SET_E = 1 } oz_modset_t;
+ * E = the hybrid set, six squares of S plus seven byte moduli ("Candidate E");
+ * A = the all-byte set of fifteen moduli, 117.8 bits ("Candidate A"). */
+typedef enum { OZ_SET_S = 0, OZ_SET_E = 1, OZ_SET_A = 2 } oz_modset_t;
 
 /* route bit field: one substrate, one quantiser, one scale rule (0 picks the default) */
 #define OZ_SUB_FP8      0x001u  /* planes are E4M3 bytes, FP32 accumulation (default)          */
 #define OZ_SUB_INT8     0x002u  /* same digits as two's-complement bytes, INT32 accumulation   */
+#define OZ_SUB_INT8_NATIVE 0x004u /* set A only: the centred residue of a byte modulus IS the INT8
+                                   * operand -- one plane and one product per modulus (Sec. 2, "The
+                                   * substrate transition": alpha_INT8 = r + 1 = 16 passes)            */
 #define OZ_QUANT_RN     0x010u  /* round to nearest, ties to even (variant Ozaki-II-RN, default) */
 #define OZ_QUANT_TZ     0x020u  /* truncate toward zero (variant Ozaki-II-TZ)                  */
 #define OZ_SCALE_MAXEXP 0x100u  /* shift from the largest exponent of the line (Eq. 2 read literally) */
@@ -70,6 +74,10 @@ typedef enum { OZ_SET_S = 0, OZ_SET_E = 1 } oz_modset_t;
 /* Number of moduli r and of stored planes p_store of a set (Table "tuples": 12/30, 13/33).
  * Returns OZ_ERR_INVALID_ARG for an unknown set.  `moduli` (host, may be NULL) receives r ints. */
 oz_status_t oz_set_info(oz_modset_t set, int *r, int *p_store, int *moduli);
+
+/* Stored planes of a set on the substrate named by `route`: 30 / 33 / 44 for S / E / A with
+ * two-limb digits, 15 for set A with OZ_SUB_INT8_NATIVE; 0 for an invalid combination. */
+int oz_plane_count(oz_modset_t set, uint32_t route);
 
 /* Pitch in bytes of one plane row for inner dimension k: k rounded up to 16 (TMA stride rule). */
 int64_t oz_row_pitch(int64_t k);

@@ -16,15 +16,15 @@ LIB_PATH = os.environ.get("OZ_B200_LIB") or os.path.join(_HERE, "liboz_b200.so")
 OZ_OK = 0
 OZ_ERR_INVALID_ARG, OZ_ERR_UNSUPPORTED, OZ_ERR_WORKSPACE, OZ_ERR_CUDA = 1, 2, 3, 4
 OZ_ERR_NONFINITE_INPUT, OZ_ERR_RANGE, OZ_ERR_TIMEOUT = 5, 6, 7
-OZ_SET_S, OZ_SET_E = 0, 1
-OZ_SUB_FP8, OZ_SUB_INT8 = 0x001, 0x002
+OZ_SET_S, OZ_SET_E, OZ_SET_A = 0, 1, 2
+OZ_SUB_FP8, OZ_SUB_INT8, OZ_SUB_INT8_NATIVE = 0x001, 0x002, 0x004
 OZ_QUANT_RN, OZ_QUANT_TZ = 0x010, 0x020
 OZ_SCALE_MAXEXP, OZ_SCALE_CS = 0x100, 0x200
 OZ_K_MAX = 32768
 OZ_NONFINITE_SHIFT = -(2 ** 31)
 OZ_STATIC_MAX_LINES = 262144
 
-EXPORTS = ["oz_set_info", "oz_row_pitch", "oz_workspace_bytes", "oz_set_workspace", "oz_dgemm",
+EXPORTS = ["oz_set_info", "oz_plane_count", "oz_row_pitch", "oz_workspace_bytes", "oz_set_workspace", "oz_dgemm",
            "oz_dgemm_ex", "oz_dgemm_host", "oz_deconstruct", "oz_deconstruct_static",
            "oz_residue_gemm", "oz_reconstruct",
            "oz_query_status", "oz_set_stage_events", "oz_launch_count", "oz_status_string"]
@@ -32,7 +32,7 @@ EXPORTS = ["oz_set_info", "oz_row_pitch", "oz_workspace_bytes", "oz_set_workspac
 __all__ = EXPORTS + ["EXPORTS", "OzError", "load", "check", "LIB_PATH", "OZ_OK", "OZ_ERR_INVALID_ARG",
                      "OZ_ERR_UNSUPPORTED", "OZ_ERR_WORKSPACE", "OZ_ERR_CUDA",
                      "OZ_ERR_NONFINITE_INPUT", "OZ_ERR_RANGE", "OZ_ERR_TIMEOUT", "OZ_SET_S",
-                     "OZ_SET_E", "OZ_SUB_FP8", "OZ_SUB_INT8", "OZ_QUANT_RN", "OZ_QUANT_TZ",
+                     "OZ_SET_E", "OZ_SET_A", "OZ_SUB_FP8", "OZ_SUB_INT8", "OZ_SUB_INT8_NATIVE", "OZ_QUANT_RN", "OZ_QUANT_TZ",
                      "OZ_SCALE_MAXEXP", "OZ_SCALE_CS", "OZ_K_MAX", "OZ_NONFINITE_SHIFT", "OZ_STATIC_MAX_LINES"]
 
 _lib = None
@@ -55,6 +55,7 @@ def load() -> C.CDLL:
     lib = C.CDLL(LIB_PATH)
     i64, u32, vp, dbl, i32 = C.c_int64, C.c_uint32, C.c_void_p, C.c_double, C.c_int
     lib.oz_set_info.argtypes = [i32, C.POINTER(i32), C.POINTER(i32), C.POINTER(i32)]
+    lib.oz_plane_count.argtypes = [i32, u32]
     lib.oz_row_pitch.argtypes = [i64]
     lib.oz_row_pitch.restype = i64
     lib.oz_workspace_bytes.argtypes = [i64, i64, i64, i32, u32]
@@ -109,6 +110,10 @@ def oz_set_info(modset: int):
     mod = (C.c_int * 16)()
     check(load().oz_set_info(modset, C.byref(r), C.byref(p), mod), "oz_set_info")
     return r.value, p.value, [mod[i] for i in range(r.value)]
+
+
+def oz_plane_count(modset: int, route: int = 0) -> int:
+    return load().oz_plane_count(modset, route)
 
 
 def oz_row_pitch(k: int) -> int:

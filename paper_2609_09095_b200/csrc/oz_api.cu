@@ -11,7 +11,7 @@ namespace oz {
 // ------------------------------------------------------------------------------------------
 // per-device objects: plane lookup tables and the sticky status word
 // ------------------------------------------------------------------------------------------
-__device__ uint32_t g_lut[2][2][kLutWords];
+__device__ uint32_t g_lut[kNumSets][3][kLutWords];
 __device__ unsigned int g_status[4];
 
 namespace {
@@ -50,6 +50,7 @@ int floor_mod(int a, int b) { int r = a % b; return r < 0 ? r + b : r; }
 uint32_t lut_entry(int u, int m, int substrate)
 {
     int d = (2 * u >= m) ? u - m : u;        // centred, -m/2 included
+    if (substrate == 2) return static_cast<uint32_t>(d & 0xFF);   // native INT8: the residue is the operand
     int s = square_root(m);
     int dig[3] = {0, 0, 0};
     if (s) {
@@ -100,6 +101,7 @@ bool decode_route(uint32_t route, Route *out)
     if (route & ~0xFFFu) return false;
     if (sub == 0 || sub == OZ_SUB_FP8) out->substrate = 0;
     else if (sub == OZ_SUB_INT8) out->substrate = 1;
+    else if (sub == OZ_SUB_INT8_NATIVE) out->substrate = 2;
     else return false;
     if (q == 0 || q == OZ_QUANT_RN) out->quant = 0;
     else if (q == OZ_QUANT_TZ) out->quant = 1;
@@ -108,6 +110,13 @@ bool decode_route(uint32_t route, Route *out)
     else if (sc == OZ_SCALE_MAXEXP) out->rule = 0;
     else return false;
     return true;
+}
+
+// the native INT8 route needs every centred residue to fit a signed byte: all-byte set A only
+bool decode_route_for_set(int set, uint32_t route, Route *out)
+{
+    if (!decode_route(route, out)) return false;
+    return !(out->native() && set != OZ_SET_A);
 }
 
 void budget_maxexp(int set, int64_t k, int *tA, int *tB)
@@ -138,9 +147,9 @@ oz_status_t ensure_device_ready()
     if (dev < 0 || dev >= kMaxDevices) return OZ_ERR_CUDA;
     std::lock_guard<std::mutex> lock(g_mutex);
     if (g_ready[dev]) return OZ_OK;
-    static uint32_t host_lut[2][2][kLutWords];
-    for (int set = 0; set < 2; ++set)
-        for (int sub = 0; sub < 2; ++sub) {
+    static uint32_t host_lut[kNumSets][3][kLutWords];
+    for (int set = 0; set < kNumSets; ++set)
+        for (int sub = 0; sub < 3; ++sub) {
             int off = 0;
             for (int i = 0; i < set_r(set); ++i) {
                 int m = modulus(set, i);
@@ -167,7 +176,7 @@ const uint32_t *device_lut(int set, int substrate)
 {
     int dev = 0;
     cudaGetDevice(&dev);
-    return g_lut_addr[dev] + (static_cast<size_t>(set) * 2 + substrate) * kLutWords;
+    return g_lut_addr[dev] + (static_cast<size_t>(set) * 3 + substrate) * kLutWords;
 }
 
 unsigned int *device_status_word()
@@ -196,7 +205,7 @@ struct Layout {
     int64_t pitch, strideA, strideB, ldr, mod_stride;
 };
 
-Layout make_layout(int64_t m, int64_t n, int64_t k, int set)
+Layout make_layout(int64_t m, int64_t n, int64_t k, int set, bool native)
 {
     Layout L{};
     Carve c;
@@ -209,21 +218,21 @@ Layout make_layout(int64_t m, int64_t n, int64_t k, int set)
     L.shiftB = c.take(4 * static_cast<size_t>(n));
     L.scrA = c.take(16 * static_cast<size_t>(m) + 256);
     L.scrB = c.take(16 * static_cast<size_t>(n) + 256);
-    L.PA = c.take(static_cast<size_t>(p_store(set)) * L.strideA);
-    L.PB = c.take(static_cast<size_t>(p_store(set)) * L.strideB);
+    L.PA = c.take(static_cast<size_t>(p_store(set, native)) * L.strideA);
+    L.PB = c.take(static_cast<size_t>(p_store(set, native)) * L.strideB);
     L.R = c.take(2 * static_cast<size_t>(set_r(set)) * L.mod_stride);
     L.total = c.off;
     return L;
 }
 
-bool valid_set(int set) { return set == OZ_SET_S || set == OZ_SET_E; }
+bool valid_set(int set) { return set == OZ_SET_S || set == OZ_SET_E || set == OZ_SET_A; }
 
 oz_status_t dgemm_impl(int64_t m, int64_t n, int64_t k, double alpha, const double *A, int64_t lda,
                        const double *B, int64_t ldb, double beta, double *C, int64_t ldc, int set,
                        uint32_t route, cudaStream_t stream, char *ws, size_t ws_bytes)
 {
     Route rt;
-    if (!valid_set(set) || !decode_route(route, &rt)) return OZ_ERR_INVALID_ARG;
+    if (!valid_set(set) || !decode_route_for_set(set, route, &rt)) return OZ_ERR_INVALID_ARG;
     if (m < 0 || n < 0 || k < 0) return OZ_ERR_INVALID_ARG;
     if (!(alpha == 1.0 || alpha == -1.0) || !(beta == 0.0 || beta == 1.0)) return OZ_ERR_UNSUPPORTED;
     if (k > OZ_K_MAX) return OZ_ERR_UNSUPPORTED;
@@ -235,7 +244,7 @@ oz_status_t dgemm_impl(int64_t m, int64_t n, int64_t k, double alpha, const doub
         return OZ_OK;
     }
     if (!A || !B || lda < m || ldb < k) return OZ_ERR_INVALID_ARG;
-    Layout L = make_layout(m, n, k, set);
+    Layout L = make_layout(m, n, k, set, rt.native());
     if (!ws || ws_bytes < L.total) return OZ_ERR_WORKSPACE;
     oz_status_t st = ensure_device_ready();
     if (st != OZ_OK) return st;
@@ -282,13 +291,20 @@ oz_status_t oz_set_info(oz_modset_t set, int *r, int *pstore, int *moduli)
     return OZ_OK;
 }
 
+int oz_plane_count(oz_modset_t set, uint32_t route)
+{
+    Route rt;
+    if (!valid_set(set) || !decode_route_for_set(set, route, &rt)) return 0;
+    return p_store(set, rt.native());
+}
+
 int64_t oz_row_pitch(int64_t k) { return round_up(k > 0 ? k : 1, 16); }
 
 size_t oz_workspace_bytes(int64_t m, int64_t n, int64_t k, oz_modset_t set, uint32_t route)
 {
     Route rt;
-    if (!valid_set(set) || !decode_route(route, &rt) || m < 0 || n < 0 || k < 0) return 0;
-    return make_layout(m > 0 ? m : 1, n > 0 ? n : 1, k > 0 ? k : 1, set).total;
+    if (!valid_set(set) || !decode_route_for_set(set, route, &rt) || m < 0 || n < 0 || k < 0) return 0;
+    return make_layout(m > 0 ? m : 1, n > 0 ? n : 1, k > 0 ? k : 1, set, rt.native()).total;
 }
 
 oz_status_t oz_set_workspace(void *workspace, size_t bytes)
@@ -331,7 +347,7 @@ oz_status_t oz_dgemm_host(int64_t m, int64_t n, int64_t k, double alpha, const d
     OZ_CUDA_CHECK(cudaGetDevice(&dev));
     if (dev < 0 || dev >= kMaxDevices) return OZ_ERR_CUDA;
     Route rt;
-    if (!valid_set(set) || !decode_route(route, &rt)) return OZ_ERR_INVALID_ARG;
+    if (!valid_set(set) || !decode_route_for_set(set, route, &rt)) return OZ_ERR_INVALID_ARG;
     if (m < 0 || n < 0 || k < 0) return OZ_ERR_INVALID_ARG;
     if (m == 0 || n == 0) return OZ_OK;
     if (!C_host || ldc < m || (k > 0 && (!A_host || !B_host || lda < m || ldb < k)))
@@ -339,7 +355,7 @@ oz_status_t oz_dgemm_host(int64_t m, int64_t n, int64_t k, double alpha, const d
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     char *ws = static_cast<char *>(g_workspace[dev]);
     int64_t kk = k > 0 ? k : 1;
-    size_t core = make_layout(m, n, kk, set).total;
+    size_t core = make_layout(m, n, kk, set, rt.native()).total;
     size_t bytesA = 8 * static_cast<size_t>(m) * kk, bytesB = 8 * static_cast<size_t>(kk) * n;
     size_t bytesC = 8 * static_cast<size_t>(m) * n;
     size_t offA = core, offB = offA + round_up(bytesA, 256), offC = offB + round_up(bytesB, 256);
@@ -364,7 +380,7 @@ oz_status_t oz_deconstruct(int side, int64_t lines, int64_t k, const double *X, 
                            int64_t row_pitch, int32_t *shift, void *scratch, void *stream)
 {
     Route rt;
-    if (!valid_set(set) || !decode_route(route, &rt) || (side != 0 && side != 1))
+    if (!valid_set(set) || !decode_route_for_set(set, route, &rt) || (side != 0 && side != 1))
         return OZ_ERR_INVALID_ARG;
     if (lines < 0 || k < 0) return OZ_ERR_INVALID_ARG;
     if (k > OZ_K_MAX) return OZ_ERR_UNSUPPORTED;
@@ -387,7 +403,7 @@ oz_status_t oz_residue_gemm(int64_t m, int64_t n, int64_t k, const uint8_t *PA, 
                             int64_t mod_stride, void *stream)
 {
     Route rt;
-    if (!valid_set(set) || !decode_route(route, &rt)) return OZ_ERR_INVALID_ARG;
+    if (!valid_set(set) || !decode_route_for_set(set, route, &rt)) return OZ_ERR_INVALID_ARG;
     if (m < 0 || n < 0 || k < 0) return OZ_ERR_INVALID_ARG;
     if (k > OZ_K_MAX) return OZ_ERR_UNSUPPORTED;
     if (m == 0 || n == 0) return OZ_OK;

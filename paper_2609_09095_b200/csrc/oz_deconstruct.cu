@@ -228,7 +228,7 @@ __device__ __forceinline__ long long quantise(double x, int sigma, bool tz)
 
 // One modulus (compile-time index I of set SET) for four consecutive inner-dimension elements:
 // residues, table look-up, byte transposition, 2 or 3 four-byte plane stores.
-template <int SET, int I>
+template <int SET, bool NATIVE, int I>
 __device__ __forceinline__ void convert_modulus(const uint32_t (&l0)[4], const uint32_t (&l1)[4],
                                                 const uint32_t (&l2)[4], const uint32_t (&l3)[4],
                                                 const uint32_t *__restrict__ lut, uint8_t *out,
@@ -242,7 +242,7 @@ __device__ __forceinline__ void convert_modulus(const uint32_t (&l0)[4], const u
     // floor(v / m) = (v * ceil(2^39 / m)) >> 39 exactly for v < 2^28
     constexpr uint32_t magic = static_cast<uint32_t>(((1ull << 39) + m - 1) / m);
     constexpr int off = lut_offset(SET, I);
-    constexpr int plane = first_plane(SET, I);
+    constexpr int plane = first_plane(SET, I, NATIVE);
     static_assert(65535ull * (1ull + c1 + c2) + 32767ull * c3 + bias < (1ull << 28), "limb sum below 2^28");
     uint32_t w[4];
 #pragma unroll
@@ -258,6 +258,7 @@ __device__ __forceinline__ void convert_modulus(const uint32_t (&l0)[4], const u
     uint32_t t01 = __byte_perm(w[0], w[1], 0x5140);
     uint32_t t23 = __byte_perm(w[2], w[3], 0x5140);
     *reinterpret_cast<uint32_t *>(out + plane * plane_stride) = __byte_perm(t01, t23, 0x5410);
+    if (NATIVE) return;                       // one plane: the centred residue itself
     *reinterpret_cast<uint32_t *>(out + (plane + 1) * plane_stride) = __byte_perm(t01, t23, 0x7632);
     if (planes_of(m) == 3) {
         uint32_t u01 = __byte_perm(w[0], w[1], 0x0062);
@@ -266,18 +267,18 @@ __device__ __forceinline__ void convert_modulus(const uint32_t (&l0)[4], const u
     }
 }
 
-template <int SET, int... I>
+template <int SET, bool NATIVE, int... I>
 __device__ __forceinline__ void convert_all_moduli(std::integer_sequence<int, I...>,
                                                    const uint32_t (&l0)[4], const uint32_t (&l1)[4],
                                                    const uint32_t (&l2)[4], const uint32_t (&l3)[4],
                                                    const uint32_t *__restrict__ lut, uint8_t *out,
                                                    int64_t plane_stride)
 {
-    (convert_modulus<SET, I>(l0, l1, l2, l3, lut, out, plane_stride), ...);
+    (convert_modulus<SET, NATIVE, I>(l0, l1, l2, l3, lut, out, plane_stride), ...);
 }
 
 // Four consecutive inner-dimension elements of one line -> 4 bytes of every stored plane.
-template <int SET>
+template <int SET, bool NATIVE>
 __device__ __forceinline__ void convert4(const double (&x)[4], int sigma, bool tz,
                                          const uint32_t *__restrict__ lut, uint8_t *out,
                                          int64_t plane_stride)
@@ -296,11 +297,11 @@ __device__ __forceinline__ void convert4(const double (&x)[4], int sigma, bool t
         l2[e] = hi & 0xFFFFu;
         l3[e] = static_cast<uint32_t>(static_cast<int32_t>(hi) >> 16);   // signed top limb
     }
-    convert_all_moduli<SET>(std::make_integer_sequence<int, set_r(SET)>{}, l0, l1, l2, l3, lut, out,
+    convert_all_moduli<SET, NATIVE>(std::make_integer_sequence<int, set_r(SET)>{}, l0, l1, l2, l3, lut, out,
                             plane_stride);
 }
 
-template <int SET, int SIDE>
+template <int SET, int SIDE, bool NATIVE>
 __global__ void __launch_bounds__(kConvThreads)
 convert_kernel(const double *__restrict__ X, int64_t ldx, int64_t lines, int64_t k,
                const int32_t *__restrict__ shift, const uint32_t *__restrict__ lut_global,
@@ -328,7 +329,7 @@ convert_kernel(const double *__restrict__ X, int64_t ldx, int64_t lines, int64_t
 #pragma unroll
             for (int e = 0; e < 4; ++e)
                 x[e] = (!dead && kb + e < k) ? X[kb + e + line * ldx] : 0.0;
-            convert4<SET>(x, dead ? 0 : sigma, tz != 0, lut, planes + line * row_pitch + kb, plane_stride);
+            convert4<SET, NATIVE>(x, dead ? 0 : sigma, tz != 0, lut, planes + line * row_pitch + kb, plane_stride);
         }
     } else {
         double *tile = reinterpret_cast<double *>(smem_raw + kLutWords * 4);
@@ -355,20 +356,20 @@ convert_kernel(const double *__restrict__ X, int64_t ldx, int64_t lines, int64_t
                 double x[4];
 #pragma unroll
                 for (int e = 0; e < 4; ++e) x[e] = dead ? 0.0 : tile[li * kTilePitch + lane * 4 + e];
-                convert4<SET>(x, dead ? 0 : sigma, tz != 0, lut, planes + line * row_pitch + kb, plane_stride);
+                convert4<SET, NATIVE>(x, dead ? 0 : sigma, tz != 0, lut, planes + line * row_pitch + kb, plane_stride);
             }
             __syncthreads();
         }
     }
 }
 
-template <int SET, int SIDE>
+template <int SET, int SIDE, bool NATIVE>
 oz_status_t launch_convert(const double *X, int64_t ldx, int64_t lines, int64_t k,
                            const int32_t *shift, const uint32_t *lut, uint8_t *planes,
                            int64_t plane_stride, int64_t row_pitch, int tz, cudaStream_t stream)
 {
     size_t smem = kLutWords * 4 + (SIDE == 0 ? sizeof(double) * kTileLines * kTilePitch : 0);
-    OZ_CUDA_CHECK(cudaFuncSetAttribute(convert_kernel<SET, SIDE>,
+    OZ_CUDA_CHECK(cudaFuncSetAttribute(convert_kernel<SET, SIDE, NATIVE>,
                                        cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        static_cast<int>(smem)));
     int64_t nchunks = (row_pitch + kChunk - 1) / kChunk;
@@ -379,7 +380,7 @@ oz_status_t launch_convert(const double *X, int64_t ldx, int64_t lines, int64_t 
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, 0);
     int64_t cap = static_cast<int64_t>(sms) * (SIDE == 1 ? 6 : 3);
     int grid = static_cast<int>(need < cap ? need : cap);
-    convert_kernel<SET, SIDE><<<grid, kConvThreads, smem, stream>>>(
+    convert_kernel<SET, SIDE, NATIVE><<<grid, kConvThreads, smem, stream>>>(
         X, ldx, lines, k, shift, lut, planes, plane_stride, row_pitch, tz);
     count_launch();
     OZ_CUDA_CHECK(cudaGetLastError());
@@ -431,12 +432,15 @@ oz_status_t launch_deconstruct(int side, int64_t lines, int64_t k, const double 
     OZ_CUDA_CHECK(cudaGetLastError());
 
     const uint32_t *lut = device_lut(set, rt.substrate);
-    if (set == 0) {
-        return side == 0 ? launch_convert<0, 0>(X, ldx, lines, k, shift, lut, planes, plane_stride, row_pitch, rt.quant, stream)
-                         : launch_convert<0, 1>(X, ldx, lines, k, shift, lut, planes, plane_stride, row_pitch, rt.quant, stream);
-    }
-    return side == 0 ? launch_convert<1, 0>(X, ldx, lines, k, shift, lut, planes, plane_stride, row_pitch, rt.quant, stream)
-                     : launch_convert<1, 1>(X, ldx, lines, k, shift, lut, planes, plane_stride, row_pitch, rt.quant, stream);
+#define OZ_CONVERT(SET_, NATIVE_)                                                                        \
+    (side == 0 ? launch_convert<SET_, 0, NATIVE_>(X, ldx, lines, k, shift, lut, planes, plane_stride,    \
+                                                  row_pitch, rt.quant, stream)                           \
+               : launch_convert<SET_, 1, NATIVE_>(X, ldx, lines, k, shift, lut, planes, plane_stride,    \
+                                                  row_pitch, rt.quant, stream))
+    if (set == 0) return OZ_CONVERT(0, false);
+    if (set == 1) return OZ_CONVERT(1, false);
+    return rt.native() ? OZ_CONVERT(2, true) : OZ_CONVERT(2, false);
+#undef OZ_CONVERT
 }
 
 }  // namespace oz

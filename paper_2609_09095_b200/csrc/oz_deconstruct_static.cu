@@ -51,7 +51,8 @@ extern "C" oz_status_t oz_deconstruct_static(int side, int64_t lines, int64_t k,
                                              int64_t row_pitch, int32_t *shift, void *stream)
 {
     oz::Route rt;
-    if ((set != OZ_SET_S && set != OZ_SET_E) || !oz::decode_route(route, &rt) || (side != 0 && side != 1))
+    if ((set != OZ_SET_S && set != OZ_SET_E && set != OZ_SET_A) || !oz::decode_route_for_set(set, route, &rt) ||
+        (side != 0 && side != 1))
         return OZ_ERR_INVALID_ARG;
     if (lines < 0 || k < 0) return OZ_ERR_INVALID_ARG;
     if (k > OZ_K_MAX) return OZ_ERR_UNSUPPORTED;

@@ -29,8 +29,12 @@
 // accumulators of a non-square modulus at once.
 //
 // Exactness: the FP8 route relies on integer-valued partial sums below 2^24 being accumulated
-// without rounding (accumulation invariant of Algorithm 2, Lemma 1); the INT8 route accumulates in
-// INT32.  Both are converted to FP32 exactly because k <= OZ_K_MAX keeps |acc| < 2^24.
+// without rounding (accumulation invariant of Algorithm 2, Lemma 1) and its epilogue works in
+// exact FP32; the INT8 routes accumulate in INT32 and their epilogue is integer arithmetic
+// (weights by IMAD, `mod m` by a multiply-high division on a biased, non-negative value).
+//
+// Native INT8 route (all-byte set A only): the centred residue itself is the operand, so a modulus
+// is ONE job -- one plane, one K-loop, weight 1 -- and the schedule has r = 15 products.
 //
 // Every barrier wait is bounded: on expiry the CTA records OZ_ERR_TIMEOUT in the device status
 // word, every role leaves its loops, in-flight copies are given a bounded time to land, TMEM is
@@ -76,8 +80,13 @@ struct ModInfo {
     float m, inv_m;
     float w[3];           // weight of each job
     int reduce[3];        // reduce the accumulator modulo m before weighting (0: the exact FP32 range allows skipping it)
-    int njobs;            // 2 (square) or 3
+    int njobs;            // 2 (square), 3, or 1 (native INT8 residues)
     int plane0;           // first stored plane of this modulus
+    // integer epilogue of the INT8 routes (INT32 accumulators):
+    int iw[3];            // weights as integers
+    uint32_t mi;          // the modulus
+    uint32_t magic;       // floor(2^32 / m)
+    uint32_t bias;        // a multiple of m just above 2^31: makes a signed combination non-negative
 };
 
 struct GemmParams {
@@ -483,9 +492,11 @@ residue_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
             Item it = decode_item(item, p);
             const ModInfo &mi = p.mod[it.mod];
             const float mm = mi.m, inv_m = mi.inv_m;
-            float comb[COLS_PER_WARP];
+            const uint32_t im = mi.mi, imagic = mi.magic, ibias = mi.bias;
+            // running combination per element: FP32 (FP8 route) or INT32 (INT8 routes), as raw bits
+            uint32_t comb[COLS_PER_WARP];
 #pragma unroll
-            for (int c = 0; c < COLS_PER_WARP; ++c) comb[c] = 0.0f;
+            for (int c = 0; c < COLS_PER_WARP; ++c) comb[c] = 0u;
             for (int job = 0; ok && job < mi.njobs; ++job) {
                 ok = mbar_wait(tfull_bar + 8 * slot, (slot_phase >> slot) & 1u, abort_flag, p.status);
                 if (!ok) break;
@@ -498,22 +509,37 @@ residue_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
                 for (int c0 = 0; c0 < COLS_PER_WARP; c0 += 32) {
                     uint32_t v[32];
                     tmem_ld32(taddr + c0, v);
-                    if (reduce_first) {
+                    if (SUB == 0) {
+                        if (reduce_first) {
 #pragma unroll
-                        for (int e = 0; e < 32; ++e) {
-                            float acc = SUB == 0 ? __uint_as_float(v[e])
-                                                 : __int2float_rn(static_cast<int>(v[e]));
-                            float quot = fmaf(acc, inv_m, 12582912.0f) - 12582912.0f;   // rint(acc/m)
-                            float res = fmaf(-quot, mm, acc);                            // exact, |res| <= ~m/2
-                            comb[c0 + e] = fmaf(res, wj, comb[c0 + e]);                  // exact, < 2^24
+                            for (int e = 0; e < 32; ++e) {
+                                float acc = __uint_as_float(v[e]);
+                                float quot = fmaf(acc, inv_m, 12582912.0f) - 12582912.0f;   // rint(acc/m)
+                                float res = fmaf(-quot, mm, acc);                            // exact, |res| <= ~m/2
+                                comb[c0 + e] = __float_as_uint(fmaf(res, wj, __uint_as_float(comb[c0 + e])));
+                            }
+                        } else {
+                            // the host has checked that w * acc stays below 2^24 for this k
+#pragma unroll
+                            for (int e = 0; e < 32; ++e)
+                                comb[c0 + e] = __float_as_uint(fmaf(__uint_as_float(v[e]), wj, __uint_as_float(comb[c0 + e])));
                         }
                     } else {
-                        // the host has checked that w * acc stays below 2^24 for this k: no reduction needed
+                        // INT32 accumulators: exact integer arithmetic, no conversions
+                        const int iwj = mi.iw[job];
+                        if (reduce_first) {
 #pragma unroll
-                        for (int e = 0; e < 32; ++e) {
-                            float acc = SUB == 0 ? __uint_as_float(v[e])
-                                                 : __int2float_rn(static_cast<int>(v[e]));
-                            comb[c0 + e] = fmaf(acc, wj, comb[c0 + e]);
+                            for (int e = 0; e < 32; ++e) {
+                                uint32_t u = v[e] + ibias;                       // non-negative, same residue
+                                uint32_t r = u - __umulhi(u, imagic) * im;       // in [0, 2m)
+                                r = min(r, r - im);
+                                comb[c0 + e] = static_cast<uint32_t>(static_cast<int>(r) * iwj + static_cast<int>(comb[c0 + e]));
+                            }
+                        } else {
+                            // the host has checked that the weighted sum stays inside INT32 for this k
+#pragma unroll
+                            for (int e = 0; e < 32; ++e)
+                                comb[c0 + e] = static_cast<uint32_t>(static_cast<int>(v[e]) * iwj + static_cast<int>(comb[c0 + e]));
                         }
                     }
                 }
@@ -538,11 +564,17 @@ residue_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
                 uint32_t bits[2];
 #pragma unroll
                 for (int h = 0; h < 2; ++h) {
-                    float t = comb[c + h];
-                    float quot = fmaf(t, inv_m, 12582912.0f) - 12582912.0f;
-                    float res = fmaf(-quot, mm, t);
-                    res = res < 0.0f ? res + mm : res;                       // canonical [0, m)
-                    bits[h] = __float_as_uint(res + 8388608.0f);             // integer in the low mantissa bits
+                    if (SUB == 0) {
+                        float t = __uint_as_float(comb[c + h]);
+                        float quot = fmaf(t, inv_m, 12582912.0f) - 12582912.0f;
+                        float res = fmaf(-quot, mm, t);
+                        res = res < 0.0f ? res + mm : res;                   // canonical [0, m)
+                        bits[h] = __float_as_uint(res + 8388608.0f);         // integer in the low mantissa bits
+                    } else {
+                        uint32_t u = comb[c + h] + ibias;
+                        uint32_t r = u - __umulhi(u, imagic) * im;           // in [0, 2m)
+                        bits[h] = min(r, r - im);                            // canonical [0, m)
+                    }
                 }
                 packed[c >> 1] = __byte_perm(bits[0], bits[1], 0x5410);
             }
@@ -689,32 +721,47 @@ oz_status_t launch_residue_gemm(int64_t m, int64_t n, int64_t k, const uint8_t *
         int mi = modulus(set, i), s = square_root(mi);
         p.mod[i].m = static_cast<float>(mi);
         p.mod[i].inv_m = 1.0f / static_cast<float>(mi);
-        p.mod[i].plane0 = first_plane(set, i);
-        // Exact FP32 range of the running combination: digits are bounded by |d0| <= 14 (16 for
-        // squares), |d1| <= 16, |d0+d1| <= 22 (Lemma 1), a reduced accumulator by (m+1)/2 <= 545.
-        // A job's accumulator may be weighted without reducing it first while the worst-case sum
-        // stays below 2^24.
-        const int64_t lim = (1ll << 24) - 1, kk = k > 0 ? k : 1;
-        if (s) {
-            p.mod[i].njobs = 2;
-            p.mod[i].w[0] = 1.0f; p.mod[i].w[1] = static_cast<float>(s); p.mod[i].w[2] = 0.0f;
-            p.mod[i].reduce[0] = (256 * kk + static_cast<int64_t>(s) * 545 <= lim) ? 0 : 1;
-            p.mod[i].reduce[1] = 1;
-            p.mod[i].reduce[2] = 1;
+        // Exact range of the running combination.  Digits are bounded by |d0| <= 14 (16 for
+        // squares), |d1| <= 16, |d0+d1| <= 22 (Lemma 1), a reduced accumulator by (m+1)/2 <= 545
+        // (FP32 path, balanced) or m-1 <= 1088 (integer path, canonical).  A job's accumulator may
+        // be weighted without reducing it first while the worst-case sum stays inside the exact
+        // range: 2^24 for the FP32 epilogue, 2^31 (minus headroom for the bias) for the integer one.
+        const bool integer = rt.substrate != 0;
+        const int64_t lim = integer ? (1ll << 31) - 8192 : (1ll << 24) - 1, kk = k > 0 ? k : 1;
+        const int64_t red = integer ? 1088 : 545;
+        ModInfo &mo = p.mod[i];
+        mo.mi = static_cast<uint32_t>(mi);
+        mo.magic = barrett_magic(static_cast<uint32_t>(mi));
+        mo.bias = static_cast<uint32_t>((((1ull << 31) + mi - 1) / mi) * mi);
+        mo.plane0 = first_plane(set, i, rt.native());
+        if (rt.native()) {
+            mo.njobs = 1;
+            mo.w[0] = 1.0f; mo.w[1] = mo.w[2] = 0.0f;
+            mo.reduce[0] = (128 * 128 * kk <= lim) ? 0 : 1;
+            mo.reduce[1] = mo.reduce[2] = 1;
+        } else if (s) {
+            mo.njobs = 2;
+            mo.w[0] = 1.0f; mo.w[1] = static_cast<float>(s); mo.w[2] = 0.0f;
+            const bool skip_all = integer && (256 + 512 * static_cast<int64_t>(s)) * kk <= lim;
+            mo.reduce[0] = (skip_all || 256 * kk + static_cast<int64_t>(s) * red <= lim) ? 0 : 1;
+            mo.reduce[1] = skip_all ? 0 : 1;
+            mo.reduce[2] = 1;
         } else {
-            p.mod[i].njobs = 3;
-            p.mod[i].w[0] = -15.0f; p.mod[i].w[1] = 16.0f; p.mod[i].w[2] = 240.0f;
-            const bool skip01 = (15 * 196 + 16 * 484) * kk + 240 * 545 <= lim;
-            p.mod[i].reduce[0] = skip01 ? 0 : 1;
-            p.mod[i].reduce[1] = skip01 ? 0 : 1;
-            p.mod[i].reduce[2] = 1;
+            mo.njobs = 3;
+            mo.w[0] = -15.0f; mo.w[1] = 16.0f; mo.w[2] = 240.0f;
+            const bool skip_all = integer && (15 * 196 + 16 * 484 + 240 * 256) * kk <= lim;
+            const bool skip01 = skip_all || (15 * 196 + 16 * 484) * kk + 240 * red <= lim;
+            mo.reduce[0] = skip01 ? 0 : 1;
+            mo.reduce[1] = skip01 ? 0 : 1;
+            mo.reduce[2] = skip_all ? 0 : 1;
         }
+        for (int j = 0; j < 3; ++j) mo.iw[j] = static_cast<int>(mo.w[j]);
     }
     if (k == 0) p.nk = 1;   // one all-zero chunk (the planes' padding) gives residues 0
 
     CUtensorMap mapA, mapB;
-    if (!make_plane_map(&mapA, PA, m, pitchA, strideA, p_store(set), BLOCK_N / cg) ||
-        !make_plane_map(&mapB, PB, n, pitchB, strideB, p_store(set), BLOCK_M))
+    if (!make_plane_map(&mapA, PA, m, pitchA, strideA, p_store(set, rt.native()), BLOCK_N / cg) ||
+        !make_plane_map(&mapB, PB, n, pitchB, strideB, p_store(set, rt.native()), BLOCK_M))
         return OZ_ERR_CUDA;
 
     int dev = 0, sms = 148;
@@ -724,7 +771,7 @@ oz_status_t launch_residue_gemm(int64_t m, int64_t n, int64_t k, const uint8_t *
         return rt.substrate == 0 ? launch_variant<0, 2>(mapA, mapB, p, sms, stream)
                                  : launch_variant<1, 2>(mapA, mapB, p, sms, stream);
     return rt.substrate == 0 ? launch_variant<0, 1>(mapA, mapB, p, sms, stream)
-                             : launch_variant<1, 1>(mapA, mapB, p, sms, stream);
+                             : launch_variant<1, 1>(mapA, mapB, p, sms, stream);   // INT8 two-limb and native
 }
 
 }  // namespace oz

@@ -9,18 +9,20 @@
 
 namespace oz {
 
-constexpr int kMaxR = 13;          // moduli in the largest supported set (E)
-constexpr int kMaxPlanes = 33;     // stored planes of set E
+constexpr int kMaxR = 15;          // moduli in the largest supported set (A)
+constexpr int kMaxPlanes = 44;     // stored planes of set A on the two-limb substrates
 constexpr int kLutWords = 8208;    // >= sum of the moduli of either set (S: 8197, E: 6838)
 
-// ---- modulus sets (Sec. 2 step (ii) for S; "Candidate E" paragraph for E) ----------------
-__host__ __device__ constexpr int set_r(int set) { return set == 0 ? 12 : 13; }
+// ---- modulus sets (Sec. 2 step (ii) for S; "Candidate E" and "Candidate A" paragraphs) ---
+constexpr int kNumSets = 3;
+__host__ __device__ constexpr int set_r(int set) { return set == 0 ? 12 : (set == 1 ? 13 : 15); }
 
 __host__ __device__ constexpr int modulus(int set, int i)
 {
-    constexpr int S[13] = {1089, 1024, 961, 841, 625, 529, 511, 509, 503, 499, 491, 487, 1};
-    constexpr int E[13] = {1089, 1024, 961, 841, 625, 529, 251, 247, 241, 239, 233, 229, 227};
-    return set == 0 ? S[i] : E[i];
+    constexpr int S[15] = {1089, 1024, 961, 841, 625, 529, 511, 509, 503, 499, 491, 487, 1, 1, 1};
+    constexpr int E[15] = {1089, 1024, 961, 841, 625, 529, 251, 247, 241, 239, 233, 229, 227, 1, 1};
+    constexpr int A[15] = {256, 255, 253, 251, 247, 241, 239, 233, 229, 227, 223, 217, 211, 199, 197};
+    return set == 0 ? S[i] : (set == 1 ? E[i] : A[i]);
 }
 
 // square root of a square modulus, 0 otherwise
@@ -31,16 +33,24 @@ __host__ __device__ constexpr int square_root(int m)
     return 0;
 }
 
-__host__ __device__ constexpr int planes_of(int m) { return square_root(m) ? 2 : 3; }
+// stored planes of one modulus: 2 (square) or 3 digit planes; 1 when the centred residue itself is
+// the INT8 operand (native route, byte moduli only: Sec. 2 "The substrate transition")
+__host__ __device__ constexpr int planes_of(int m, bool native = false)
+{
+    return native ? 1 : (square_root(m) ? 2 : 3);
+}
 
-__host__ __device__ constexpr int first_plane(int set, int i)
+__host__ __device__ constexpr int first_plane(int set, int i, bool native = false)
 {
     int p = 0;
-    for (int j = 0; j < i; ++j) p += planes_of(modulus(set, j));
+    for (int j = 0; j < i; ++j) p += planes_of(modulus(set, j), native);
     return p;
 }
 
-__host__ __device__ constexpr int p_store(int set) { return first_plane(set, set_r(set)); }
+__host__ __device__ constexpr int p_store(int set, bool native = false)
+{
+    return first_plane(set, set_r(set), native);
+}
 
 __host__ __device__ constexpr int lut_offset(int set, int i)
 {
@@ -67,11 +77,13 @@ inline int64_t round_up(int64_t v, int64_t a) { return (v + a - 1) / a * a; }
 
 // ---- route decoding ----------------------------------------------------------------------
 struct Route {
-    int substrate;  // 0 fp8, 1 int8
+    int substrate;  // 0 fp8, 1 int8 (two-limb digits), 2 int8 native (one residue plane, set A only)
+    bool native() const { return substrate == 2; }
     int quant;      // 0 rn, 1 tz
     int rule;       // 0 maxexp, 1 cs
 };
 bool decode_route(uint32_t route, Route *out);
+bool decode_route_for_set(int set, uint32_t route, Route *out);   // also rejects native INT8 off set A
 
 // ---- per-device state --------------------------------------------------------------------
 // Builds the lookup tables and constant blocks on the current device the first time it is used.

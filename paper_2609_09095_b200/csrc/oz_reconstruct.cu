@@ -26,11 +26,12 @@ struct ReconConst {
     unsigned long long M_lo, M_hi;
 };
 
-__constant__ ReconConst c_recon[2];
+__constant__ ReconConst c_recon[kNumSets];
 
-constexpr double kTwo38 = 274877906944.0;             // 2^38
-constexpr double kTwoM38 = 1.0 / 274877906944.0;      // 2^-38
-constexpr double kTwo76 = kTwo38 * kTwo38;            // 2^76
+// Chunk width: 38 bits for S and E (residues < 2^10.1, 13 terms: sums < 2^52); 40 bits for the
+// 117.8-bit set A (residues < 2^8, 15 terms: sums < 2^52), so that three chunks cover M.
+__host__ __device__ constexpr int chunk_bits(int set) { return set == 2 ? 40 : 38; }
+__host__ __device__ constexpr double pow2d(int e) { double v = 1.0; for (int i = 0; i < e; ++i) v *= 2.0; return v; }
 constexpr double kTwo52 = 4503599627370496.0;         // 2^52
 constexpr double kRint = 6755399441055744.0;          // 1.5 * 2^52: (x + kRint) - kRint = rint(x)
 
@@ -44,21 +45,23 @@ __device__ __forceinline__ double scale_pow2(double x, int scale)
     return scalbn(x, scale);        // zero, or a result outside the normal range
 }
 
-template <int SET, int I>
-__device__ __forceinline__ void crt_term(uint32_t c, double &S0, double &S1, double &S2)
+// w packs the residues of two consecutive rows (low / high 16 bits); HALF selects the row
+template <int SET, int HALF, int I>
+__device__ __forceinline__ void crt_term(uint32_t w, double &S0, double &S1, double &S2)
 {
     const ReconConst &K = c_recon[SET];
+    const uint32_t c = HALF ? (w >> 16) : (w & 0xFFFFu);
     double cd = __hiloint2double(0x43300000, static_cast<int>(c)) - kTwo52;   // exact u32 -> double
     S0 = fma(cd, K.V[I][0], S0);
     S1 = fma(cd, K.V[I][1], S1);
     S2 = fma(cd, K.V[I][2], S2);
 }
 
-template <int SET, int... I>
+template <int SET, int HALF, int... I>
 __device__ __forceinline__ void crt_sum(std::integer_sequence<int, I...>, const uint32_t (&c)[kMaxR],
                                         double &S0, double &S1, double &S2)
 {
-    (crt_term<SET, I>(c[I], S0, S1, S2), ...);
+    (crt_term<SET, HALF, I>(c[I], S0, S1, S2), ...);
 }
 
 // Exact tail (rare path): the normalised chunks as a 128-bit integer, exact lift to
@@ -67,10 +70,11 @@ __device__ __noinline__ double finish_exact(double T0, double T1, double T2, int
 {
     const ReconConst &K = c_recon[set];
     const long long t0 = __double2ll_rn(T0), t1 = __double2ll_rn(T1), t2 = __double2ll_rn(T2);
-    // v = t0 + t1 2^38 + t2 2^76 as a two's-complement (hi:lo) pair
-    unsigned long long lo = static_cast<unsigned long long>(t0) + (static_cast<unsigned long long>(t1) << 38);
-    long long hi = (t0 >> 63) + (t1 >> 26) + (lo < static_cast<unsigned long long>(t0) ? 1 : 0) +
-                   static_cast<long long>(static_cast<unsigned long long>(t2) << 12);
+    // v = t0 + t1 2^cw + t2 2^(2cw) as a two's-complement (hi:lo) pair
+    const int cw = chunk_bits(set);
+    unsigned long long lo = static_cast<unsigned long long>(t0) + (static_cast<unsigned long long>(t1) << cw);
+    long long hi = (t0 >> 63) + (t1 >> (64 - cw)) + (lo < static_cast<unsigned long long>(t0) ? 1 : 0) +
+                   static_cast<long long>(static_cast<unsigned long long>(t2) << (2 * cw - 64));
     const __int128 M = static_cast<__int128>((static_cast<unsigned __int128>(K.M_hi) << 64) | K.M_lo);
     const __int128 Mh = M >> 1;     // M is even for both sets
     __int128 v = static_cast<__int128>((static_cast<unsigned __int128>(static_cast<unsigned long long>(hi)) << 64) | lo);
@@ -94,12 +98,15 @@ __device__ __noinline__ double finish_exact(double T0, double T1, double T2, int
     return neg ? -d : d;
 }
 
-template <int SET>
+template <int SET, int HALF>
 __device__ __forceinline__ double reconstruct_one(const uint32_t (&c)[kMaxR], int shift_sum)
 {
     const ReconConst &K = c_recon[SET];
     double S0 = 0.0, S1 = 0.0, S2 = 0.0;
-    crt_sum<SET>(std::make_integer_sequence<int, set_r(SET)>{}, c, S0, S1, S2);
+    crt_sum<SET, HALF>(std::make_integer_sequence<int, set_r(SET)>{}, c, S0, S1, S2);
+    constexpr double kTwo38 = pow2d(chunk_bits(SET));          // 2^cw  (names kept from the 38-bit case)
+    constexpr double kTwoM38 = 1.0 / pow2d(chunk_bits(SET));   // 2^-cw
+    constexpr double kTwo76 = kTwo38 * kTwo38;                 // 2^(2cw)
     double val = fma(S2, kTwo76, fma(S1, kTwo38, S0));
     double kappa = (val * K.inv_M + kRint) - kRint;
     double T0 = fma(-kappa, K.Mc[0], S0);              // exact: integers below 2^53
@@ -149,28 +156,29 @@ reconstruct_kernel(const uint16_t *__restrict__ R, int64_t ldr, int64_t mod_stri
     if (j >= n) return;
     {
 
-    uint32_t c0[kMaxR], c1[kMaxR];
+    // all residue loads are issued before any arithmetic: r independent requests in flight per
+    // thread, kept packed (two rows per word) so that they fit the register budget
+    uint32_t w[kMaxR];
     const uint16_t *base = R + j * ldr + row;
 #pragma unroll
     for (int i = 0; i < r; ++i) {
         if (vecR) {
-            uint32_t w = *reinterpret_cast<const uint32_t *>(base + i * mod_stride);
-            c0[i] = w & 0xFFFFu;
-            c1[i] = w >> 16;
+            w[i] = *reinterpret_cast<const uint32_t *>(base + i * mod_stride);
         } else {
-            c0[i] = base[i * mod_stride];
-            c1[i] = two ? base[i * mod_stride + 1] : 0u;
+            uint32_t lo = base[i * mod_stride];
+            uint32_t hi = two ? base[i * mod_stride + 1] : 0u;
+            w[i] = lo | (hi << 16);
         }
     }
     int sb = shiftB[j];
     int sa0 = shiftA[row], sa1 = two ? shiftA[row + 1] : 0;
     const double nan = __longlong_as_double(0x7FF8000000000000ll);
     double p0 = (sb == OZ_NONFINITE_SHIFT || sa0 == OZ_NONFINITE_SHIFT) ? nan
-                                                                         : reconstruct_one<SET>(c0, sa0 + sb);
+                                                                         : reconstruct_one<SET, 0>(w, sa0 + sb);
     double p1 = 0.0;
     if (two)
         p1 = (sb == OZ_NONFINITE_SHIFT || sa1 == OZ_NONFINITE_SHIFT) ? nan
-                                                                      : reconstruct_one<SET>(c1, sa1 + sb);
+                                                                      : reconstruct_one<SET, 1>(w, sa1 + sb);
     p0 *= alpha;
     p1 *= alpha;
     double *out = C + row + j * ldc;
@@ -196,11 +204,12 @@ reconstruct_kernel(const uint16_t *__restrict__ R, int64_t ldr, int64_t mod_stri
 
 oz_status_t upload_reconstruct_constants()
 {
-    static ReconConst host[2];
-    for (int set = 0; set < 2; ++set) {
+    static ReconConst host[kNumSets];
+    for (int set = 0; set < kNumSets; ++set) {
         unsigned __int128 M = 1;
         for (int i = 0; i < set_r(set); ++i) M *= static_cast<unsigned>(modulus(set, i));
-        const unsigned __int128 mask = (static_cast<unsigned __int128>(1) << 38) - 1;
+        const int cw = chunk_bits(set);
+        const unsigned __int128 mask = (static_cast<unsigned __int128>(1) << cw) - 1;
         ReconConst &K = host[set];
         for (int i = 0; i < kMaxR; ++i) K.V[i][0] = K.V[i][1] = K.V[i][2] = 0.0;
         for (int i = 0; i < set_r(set); ++i) {
@@ -211,12 +220,12 @@ oz_status_t upload_reconstruct_constants()
                 if ((static_cast<unsigned long long>(wm) * c) % mi == 1) { inv = c; break; }
             unsigned __int128 V = W * inv;          // < M, and V = 1 mod m_i, 0 mod the other moduli
             K.V[i][0] = static_cast<double>(static_cast<unsigned long long>(V & mask));
-            K.V[i][1] = static_cast<double>(static_cast<unsigned long long>((V >> 38) & mask));
-            K.V[i][2] = static_cast<double>(static_cast<unsigned long long>(V >> 76));
+            K.V[i][1] = static_cast<double>(static_cast<unsigned long long>((V >> cw) & mask));
+            K.V[i][2] = static_cast<double>(static_cast<unsigned long long>(V >> (2 * cw)));
         }
         K.Mc[0] = static_cast<double>(static_cast<unsigned long long>(M & mask));
-        K.Mc[1] = static_cast<double>(static_cast<unsigned long long>((M >> 38) & mask));
-        K.Mc[2] = static_cast<double>(static_cast<unsigned long long>(M >> 76));
+        K.Mc[1] = static_cast<double>(static_cast<unsigned long long>((M >> cw) & mask));
+        K.Mc[2] = static_cast<double>(static_cast<unsigned long long>(M >> (2 * cw)));
         K.inv_M = 1.0 / static_cast<double>(M);
         K.half_M_guard = 0.5 * static_cast<double>(M) * (1.0 - 9.313225746154785e-10);
         K.M_lo = static_cast<unsigned long long>(M);
@@ -238,7 +247,10 @@ oz_status_t launch_reconstruct(int64_t m, int64_t n, const uint16_t *R, int64_t 
     if (n > 65535ll * 65535ll) return OZ_ERR_UNSUPPORTED;
     dim3 grid(static_cast<unsigned>(bx), static_cast<unsigned>(n < 65535 ? n : 65535),
               static_cast<unsigned>((n + 65534) / 65535));
-    if (set == 0)
+    if (set == 2)
+        reconstruct_kernel<2><<<grid, 256, 0, stream>>>(R, ldr, mod_stride, m, n, shiftA, shiftB, alpha,
+                                                        beta, C, ldc, vecR, vecC);
+    else if (set == 0)
         reconstruct_kernel<0><<<grid, 256, 0, stream>>>(R, ldr, mod_stride, m, n, shiftA, shiftB, alpha,
                                                         beta, C, ldc, vecR, vecC);
     else

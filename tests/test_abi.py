@@ -30,6 +30,11 @@ def test_host_only_queries():
     assert (r, p) == (12, 30) and mods[0] == 1089 and mods[-1] == 487
     r, p, mods = oz.oz_set_info(oz.OZ_SET_E)
     assert (r, p) == (13, 33) and mods[-1] == 227
+    r, p, mods = oz.oz_set_info(oz.OZ_SET_A)
+    assert (r, p) == (15, 44) and mods[0] == 256 and mods[-1] == 197
+    assert oz.oz_plane_count(oz.OZ_SET_A, oz.OZ_SUB_INT8_NATIVE) == 15
+    assert oz.oz_plane_count(oz.OZ_SET_S, oz.OZ_SUB_INT8_NATIVE) == 0      # native INT8 needs byte moduli
+    assert oz.oz_plane_count(oz.OZ_SET_S, 0) == 30 and oz.oz_plane_count(oz.OZ_SET_E, oz.OZ_SUB_INT8) == 33
     assert oz.oz_row_pitch(1) == 16 and oz.oz_row_pitch(5003) == 5008 and oz.oz_row_pitch(4096) == 4096
     # planes of A and B + residues dominate the workspace
     m, n, k = 16384, 16384, 1024

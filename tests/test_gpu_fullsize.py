@@ -11,7 +11,8 @@ from oracle import oz_oracle as ozo
 
 pytestmark = pytest.mark.gpu
 U = 2.0 ** -53
-OSET = {"S": ozo.SET_S, "E": ozo.SET_E}
+OSET = {"S": ozo.SET_S, "E": ozo.SET_E, "A": ozo.SET_A}
+OSUB = {"fp8": ozo.SUB_FP8, "int8": ozo.SUB_INT8, "int8n": ozo.SUB_INT8_NATIVE}
 
 
 def _sample(n, rng, tile):
@@ -23,7 +24,8 @@ def _sample(n, rng, tile):
 
 
 @pytest.mark.parametrize("cfg_id,set_name,sub", [(2, "S", "fp8"), (3, "S", "fp8"), (3, "E", "fp8"),
-                                                 (5, "S", "fp8"), (4, "S", "int8"), (4, "S", "fp8")])
+                                                 (5, "S", "fp8"), (4, "S", "int8"), (4, "S", "fp8"),
+                                                 (3, "A", "int8n")])
 def test_full_size_sampled(cfg_id, set_name, sub):
     import paper_2609_09095_b200 as oz
     import tests.gpu_helpers as gh
@@ -34,7 +36,7 @@ def test_full_size_sampled(cfg_id, set_name, sub):
     rows, cols = _sample(m, rng, 256), _sample(n, rng, 128)
     As, Bs = np.asfortranarray(A[rows, :]), np.asfortranarray(B[:, cols])
     rt = gh.route(sub, "RN", "CS")
-    osub = ozo.SUB_FP8 if sub == "fp8" else ozo.SUB_INT8
+    osub = OSUB[sub]
     oset = OSET[set_name]
 
     # ---- oracle on the sampled sub-problem, stage by stage
@@ -49,7 +51,8 @@ def test_full_size_sampled(cfg_id, set_name, sub):
     Co = ozo.output(ozo.crt(Ro, oset), sA, sB, cfg.alpha, cfg.beta, Cs0)
 
     # ---- GPU, whole problem, stage entry points (the launchers oz_dgemm uses)
-    r, p, _ = oz.oz_set_info(gh.SETS[set_name])
+    r, _, _ = oz.oz_set_info(gh.SETS[set_name])
+    p = oz.oz_plane_count(gh.SETS[set_name], rt)
     pitch = oz.oz_row_pitch(k)
     dA, dB = gh.to_dev(A), gh.to_dev(B)
     PA = torch.empty((p, m, pitch), dtype=torch.uint8, device="cuda")

@@ -10,11 +10,12 @@ from oracle import oz_oracle as ozo
 pytestmark = pytest.mark.gpu
 
 U = 2.0 ** -53
-OSET = {"S": ozo.SET_S, "E": ozo.SET_E}
+OSET = {"S": ozo.SET_S, "E": ozo.SET_E, "A": ozo.SET_A}
+OSUB = {"fp8": ozo.SUB_FP8, "int8": ozo.SUB_INT8, "int8n": ozo.SUB_INT8_NATIVE}
 
 
 def _oracle_route(sub, quant, rule):
-    return (ozo.SUB_FP8 if sub == "fp8" else ozo.SUB_INT8,
+    return (OSUB[sub],
             ozo.QUANT_RN if quant == "RN" else ozo.QUANT_TZ,
             ozo.SCALE_CS if rule == "CS" else ozo.SCALE_MAXEXP)
 
@@ -35,7 +36,8 @@ def _oracle_deconstruct(side, X, set_name, sub, quant, rule):
                                           (130, 1000, "normal"), (1, 1, "uniform"), (5, 17, "lognormal:0.5"),
                                           (67, 4101, "lognormal:2.0"), (300, 16, "uniform")])
 @pytest.mark.parametrize("set_name,sub,quant,rule", [("S", "fp8", "RN", "CS"), ("S", "int8", "TZ", "MAXEXP"),
-                                                     ("E", "fp8", "TZ", "CS"), ("E", "int8", "RN", "MAXEXP")])
+                                                     ("E", "fp8", "TZ", "CS"), ("E", "int8", "RN", "MAXEXP"),
+                                                     ("A", "int8n", "RN", "CS"), ("A", "fp8", "TZ", "MAXEXP")])
 def test_deconstruct_bit_exact(side, lines, k, dist, set_name, sub, quant, rule):
     import tests.gpu_helpers as gh
     rng = np.random.default_rng(100 + lines + k)
@@ -80,17 +82,19 @@ def _random_planes(rng, set_name, sub, lines, k, extreme=False):
     for i, m in enumerate(ms):
         lo, hi = -(m // 2), (m - 1) // 2
         if extreme:
-            cand = sorted(range(lo, hi + 1), key=lambda d: -max(abs(v) for v in ozo.split(d, m)))[:4]
+            if sub == "int8n":
+                cand = [lo, hi, lo + 1, hi - 1]
+            else:
+                cand = sorted(range(lo, hi + 1), key=lambda d: -max(abs(v) for v in ozo.split(d, m)))[:4]
             D[i] = rng.choice(cand, size=(lines, k))
         else:
             D[i] = rng.integers(lo, hi + 1, size=(lines, k))
-    osub = ozo.SUB_FP8 if sub == "fp8" else ozo.SUB_INT8
-    return ozo.planes(D, OSET[set_name], osub), D
+    return ozo.planes(D, OSET[set_name], OSUB[sub]), D
 
 
 @pytest.mark.parametrize("m,n,k", [(128, 256, 128), (256, 512, 384), (200, 300, 200), (1, 1, 1),
                                    (129, 257, 130), (3, 700, 17), (520, 40, 1000)])
-@pytest.mark.parametrize("set_name,sub", [("S", "fp8"), ("S", "int8"), ("E", "fp8")])
+@pytest.mark.parametrize("set_name,sub", [("S", "fp8"), ("S", "int8"), ("E", "fp8"), ("A", "int8n"), ("A", "fp8")])
 def test_residue_gemm_bit_exact(m, n, k, set_name, sub):
     import tests.gpu_helpers as gh
     rng = np.random.default_rng(m * 7 + n * 3 + k)
@@ -103,27 +107,28 @@ def test_residue_gemm_bit_exact(m, n, k, set_name, sub):
 
 
 @pytest.mark.parametrize("k", [4096, 5003, 32768])
-@pytest.mark.parametrize("sub", ["fp8", "int8"])
+@pytest.mark.parametrize("sub", ["fp8", "int8", "int8n"])
 def test_accumulation_is_exact_at_depth(k, sub):
     """Planes made of the largest digits only: accumulators reach k*484 (non-square) and
     k*512 (square, two K-loops in one accumulator) -- up to 2^24 at k = 32768."""
     import tests.gpu_helpers as gh
     rng = np.random.default_rng(k)
     m, n = (130, 260) if k < 30000 else (40, 24)
-    PA, DA = _random_planes(rng, "S", sub, m, k, extreme=True)
-    PB, DB = _random_planes(rng, "S", sub, n, k, extreme=True)
+    set_name = "A" if sub == "int8n" else "S"
+    PA, DA = _random_planes(rng, set_name, sub, m, k, extreme=True)
+    PB, DB = _random_planes(rng, set_name, sub, n, k, extreme=True)
     # make some rows all-equal so that terms do not cancel
     PA[:, :8, :k] = PA[:, :1, :1]
     PB[:, :8, :k] = PB[:, :1, :1]
-    want, worst = ozo.plane_products(PA, PB, k, ozo.SET_S, ozo.SUB_FP8 if sub == "fp8" else ozo.SUB_INT8)
+    want, worst = ozo.plane_products(PA, PB, k, OSET[set_name], OSUB[sub])
     assert worst > 0.9 * 256 * k
-    R, st = gh.residue_gemm(PA, PB, k, "S", gh.route(sub))
+    R, st = gh.residue_gemm(PA, PB, k, set_name, gh.route(sub))
     assert st == 0
     assert (R == want).all()
 
 
 # ------------------------------------------------------------------ reconstruction (a7)
-@pytest.mark.parametrize("set_name", ["S", "E"])
+@pytest.mark.parametrize("set_name", ["S", "E", "A"])
 @pytest.mark.parametrize("m,n", [(256, 64), (1, 1), (7, 5), (130, 3)])
 def test_reconstruct_bit_exact(set_name, m, n):
     import tests.gpu_helpers as gh
@@ -163,13 +168,13 @@ def _check_against_oracle_and_dd(A, B, got, want, C0=None, alpha=1.0, strict_dd=
 
 @pytest.mark.parametrize("cfg_id,m,n,k,sets", [(1, 256, 256, 256, ("S",)), (2, 300, 520, 4096, ("S",)),
                                                (3, 384, 512, 1024, ("E", "S")), (4, 700, 128, 4096, ("S",)),
-                                               (5, 263, 301, 5003, ("S",))])
+                                               (5, 263, 301, 5003, ("S",)), (3, 300, 260, 1024, ("A",))])
 def test_dgemm_configs_cut_down(cfg_id, m, n, k, sets):
     import tests.gpu_helpers as gh
     cfg = syn.CONFIGS[cfg_id]
     A, B, C0 = syn.operands(cfg, m, n, k, want_c=True)
     for set_name in sets:
-        for sub in cfg.substrates:
+        for sub in (("int8n", "fp8") if set_name == "A" else cfg.substrates):
             rt = gh.route(sub, "RN", "CS")
             use_c0 = C0 if cfg.beta else None
             got, st = gh.dgemm(A, B, set_name, rt, cfg.alpha, cfg.beta, use_c0)
