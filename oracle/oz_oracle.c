@@ -475,6 +475,94 @@ int64_t ozo_plane_products(int64_t m, int64_t n, int64_t k, const uint8_t *PA,
 }
 
 /* ------------------------------------------------------------------ */
+/* Merged accumulators (discussion of Table "tuples": N_acc = 2)        */
+/* ------------------------------------------------------------------ */
+/* Regrouping Eq. 8 as  d e = -15 [ d0 e0 + (-16 d1) e1 ] + 16 (d0+d1)(e0+e1)  needs two
+ * accumulators per non-square modulus instead of three, at the price of one more stored plane,
+ * the pre-scaled -16*d1, on ONE operand (here: side 0, the rows of A).  The merged term reaches
+ * 4095 on the 9-bit tail of S (exact FP32 accumulation to K = 4097) and 1088 on byte moduli
+ * (K = 15 420).  Squares are unchanged.  FP8 substrate only (-256 does not fit a signed byte). */
+int ozo_planes_of_merged(int m, int side)
+{
+    if (ozo_square_root(m)) return 2;
+    return side == 0 ? 4 : 3;
+}
+
+int ozo_pstore_merged(int set, int side)
+{
+    int mod[16], r = ozo_modset(set, mod), p = 0;
+    for (int i = 0; i < r; ++i) p += ozo_planes_of_merged(mod[i], side);
+    return p;
+}
+
+/* plane order per non-square modulus on side 0: d0, d1, d0+d1, -16*d1 */
+int ozo_planes_merged(int side, int64_t lines, int64_t k, const int16_t *D, int set, uint8_t *P,
+                      int64_t plane_stride, int64_t row_pitch)
+{
+    int mod[16], r = ozo_modset(set, mod), plane = 0, bad = 0;
+    for (int i = 0; i < r; ++i) {
+        int np = ozo_planes_of_merged(mod[i], side);
+        for (int64_t l = 0; l < lines; ++l)
+            for (int64_t kk = 0; kk < row_pitch; ++kk) {
+                int dg[4] = {0, 0, 0, 0};
+                if (kk < k) {
+                    ozo_split(D[((int64_t)i * lines + l) * k + kk], mod[i], dg);
+                    dg[3] = -16 * dg[1];
+                }
+                for (int q = 0; q < np; ++q) {
+                    int byte = ozo_e4m3_encode(dg[q]);
+                    if (byte < 0) { bad = 1; byte = 0x7F; }
+                    P[(int64_t)(plane + q) * plane_stride + l * row_pitch + kk] = (uint8_t)byte;
+                }
+            }
+        plane += np;
+    }
+    return bad ? -1 : plane;
+}
+
+/* residues from the merged layout: PA in the side-0 layout (4 planes per non-square), PB plain */
+int64_t ozo_plane_products_merged(int64_t m, int64_t n, int64_t k, const uint8_t *PA,
+                                  int64_t strideA, int64_t pitchA, const uint8_t *PB,
+                                  int64_t strideB, int64_t pitchB, int set, uint16_t *R)
+{
+    int mod[16], r = ozo_modset(set, mod), pa = 0, pb = 0;
+    int64_t worst = 0;
+    int digit_of[256];
+    for (int c = 0; c < 256; ++c) digit_of[c] = plane_digit((uint8_t)c, OZO_SUB_FP8);
+    for (int i = 0; i < r; ++i) {
+        int s = ozo_square_root(mod[i]);
+        for (int64_t j = 0; j < n; ++j)
+            for (int64_t ii = 0; ii < m; ++ii) {
+                int64_t acc0 = 0, acc1 = 0;
+                for (int64_t kk = 0; kk < k; ++kk) {
+                    int a[4] = {0, 0, 0, 0}, b[3] = {0, 0, 0};
+                    for (int q = 0; q < ozo_planes_of_merged(mod[i], 0); ++q)
+                        a[q] = digit_of[PA[(pa + q) * strideA + ii * pitchA + kk]];
+                    for (int q = 0; q < ozo_planes_of_merged(mod[i], 1); ++q)
+                        b[q] = digit_of[PB[(pb + q) * strideB + j * pitchB + kk]];
+                    if (s) {
+                        acc0 += (int64_t)a[0] * b[0];
+                        acc1 += (int64_t)a[1] * b[0] + (int64_t)a[0] * b[1];
+                    } else {
+                        acc0 += (int64_t)a[0] * b[0] + (int64_t)a[3] * b[1];   /* d0 e0 - 16 d1 e1 */
+                        acc1 += (int64_t)a[2] * b[2];                           /* (d0+d1)(e0+e1)   */
+                    }
+                }
+                int64_t v0 = acc0 < 0 ? -acc0 : acc0, v1 = acc1 < 0 ? -acc1 : acc1;
+                if (v0 > worst) worst = v0;
+                if (v1 > worst) worst = v1;
+                int64_t t = s ? acc0 + (int64_t)s * acc1 : -15 * acc0 + 16 * acc1;
+                int64_t c = t % mod[i];
+                if (c < 0) c += mod[i];
+                R[((int64_t)i * n + j) * m + ii] = (uint16_t)c;
+            }
+        pa += ozo_planes_of_merged(mod[i], 0);
+        pb += ozo_planes_of_merged(mod[i], 1);
+    }
+    return worst;
+}
+
+/* ------------------------------------------------------------------ */
 /* Eq. 4-5 / Algorithm 3: Garner mixed-radix digits, Horner, lift       */
 /* ------------------------------------------------------------------ */
 /* w_j = (m_1 ... m_{j-1})^{-1} mod m_j, found by trial (w_1 unused = 0) */

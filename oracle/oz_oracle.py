@@ -49,6 +49,7 @@ def lib() -> C.CDLL:
         _lib.ozo_cs_bound.restype = C.c_uint64
         _lib.ozo_cs_bound.argtypes = [C.c_int, C.c_int64]
         _lib.ozo_plane_products.restype = C.c_int64
+        _lib.ozo_plane_products_merged.restype = C.c_int64
         _lib.ozo_centred_residue.argtypes = [C.c_int64, C.c_int]
     return _lib
 
@@ -192,6 +193,30 @@ def planes(D: np.ndarray, s: int, substrate: int, row_pitch: int | None = None) 
                           _i64(lines * pitch), _i64(pitch))
     assert rc == pstore(s, substrate), "a digit was not representable on the substrate"
     return P
+
+
+def pstore_merged(s: int, side: int) -> int:
+    return lib().ozo_pstore_merged(s, side)
+
+
+def planes_merged(side: int, D: np.ndarray, s: int, row_pitch: int | None = None) -> np.ndarray:
+    """FP8 planes of the merged-accumulator layout (side 0 carries the extra -16*d1 planes)."""
+    r, lines, k = D.shape
+    pitch = row_pitch if row_pitch is not None else (k + 15) // 16 * 16
+    P = np.full((pstore_merged(s, side), lines, pitch), 0xAA, dtype=np.uint8)
+    rc = lib().ozo_planes_merged(side, _i64(lines), _i64(k), _p(np.ascontiguousarray(D)), s, _p(P),
+                                 _i64(lines * pitch), _i64(pitch))
+    assert rc == pstore_merged(s, side), "a digit was not representable in E4M3"
+    return P
+
+
+def plane_products_merged(PA: np.ndarray, PB: np.ndarray, k: int, s: int):
+    _, m, pa = PA.shape
+    _, n, pb = PB.shape
+    R = np.zeros((len(modset(s)), n, m), dtype=np.uint16)
+    worst = lib().ozo_plane_products_merged(_i64(m), _i64(n), _i64(k), _p(PA), _i64(m * pa), _i64(pa),
+                                            _p(PB), _i64(n * pb), _i64(pb), s, _p(R))
+    return R, int(worst)
 
 
 def products(DA: np.ndarray, DB: np.ndarray, s: int) -> np.ndarray:

@@ -172,6 +172,45 @@ def test_lemma1_exhaustive(m):
     assert 2 ** 24 // int(PAPER["merged_term_max"]) == int(PAPER["merged_K_exact"])
 
 
+@pytest.mark.parametrize("name", ["S", "E", "A"])
+def test_merged_accumulator_layout(name):
+    """N_acc = 2 per modulus: regrouped Eq. 8 with the pre-scaled plane -16*d1 on one operand."""
+    ms = ozo.modset(SETS[name])
+    nonsq = [m for m in ms if math.isqrt(m) ** 2 != m]
+    # accumulators: 2 per modulus when merged (E and A rows of the table); S keeps 3 on its tail unmerged
+    assert 2 * len(ms) == {"S": 24, "E": int(PAPER["nacc_E"]), "A": int(PAPER["nacc_A"])}[name]
+    assert 2 * (len(ms) - len(nonsq)) + 3 * len(nonsq) == {"S": int(PAPER["nacc_S"]), "E": 33, "A": 44}[name]
+    assert ozo.pstore_merged(SETS[name], 0) == ozo.pstore(SETS[name]) + len(nonsq)
+    assert ozo.pstore_merged(SETS[name], 1) == ozo.pstore(SETS[name])
+    worst = 0
+    for m in nonsq:
+        lo, hi = -(m // 2), (m - 1) // 2
+        sp = {d: ozo.split(d, m) for d in range(lo, hi + 1)}
+        pre = [-16 * d1 for (_, d1, _) in sp.values()]
+        assert all(ozo.in_e4m3(v) for v in pre)
+        if m > 256:
+            assert min(pre) == int(PAPER["merged_prescaled_plane_extreme"])
+        a = max(abs(d0) for (d0, _, _) in sp.values())
+        b = max(abs(d1) for (_, d1, _) in sp.values())
+        here = max(abs(d0 * e0 - 16 * d1 * e1) for (d0, d1, _) in sp.values()
+                   for (e0, e1, _) in list(sp.values())[:: max(1, len(sp) // 97)] + [sp[lo], sp[hi]])
+        assert here <= a * a + 16 * b * b
+        worst = max(worst, here)
+    if name == "S":
+        assert worst <= int(PAPER["merged_term_max"])
+    else:
+        assert worst <= 1088 and 2 ** 24 // 1088 == int(PAPER["merged_K_exact_byte"])
+    rng = np.random.default_rng(31)
+    m_, n_, k = 5, 4, 41
+    QA = rng.integers(-2**50, 2**50, size=(m_, k))
+    QB = rng.integers(-2**50, 2**50, size=(n_, k))
+    DA, DB = ozo.residues(QA, SETS[name]), ozo.residues(QB, SETS[name])
+    PA, PB = ozo.planes_merged(0, DA, SETS[name]), ozo.planes_merged(1, DB, SETS[name])
+    assert (PB == ozo.planes(DB, SETS[name], ozo.SUB_FP8)).all()
+    R, w = ozo.plane_products_merged(PA, PB, k, SETS[name])
+    assert (R == ozo.products(DA, DB, SETS[name])).all() and w <= 4095 * k
+
+
 def test_lemma1_is_sharp_at_513():
     def rule(d):
         d0 = (d + 8) % 16 - 8
