@@ -68,6 +68,18 @@ typedef enum { OZ_SET_S = 0, OZ_SET_E = 1, OZ_SET_A = 2 } oz_modset_t;
 #define OZ_SCALE_MAXEXP 0x100u  /* shift from the largest exponent of the line (Eq. 2 read literally) */
 #define OZ_SCALE_CS     0x200u  /* shift from the 2-norm of the line, Cauchy-Schwarz bound (default) */
 
+/* Accumulator schedule of the residue GEMMs for non-square moduli on the FP8 substrate.
+ * MERGED: two accumulators per modulus, d e = -15 [d0 e0 + (-16 d1) e1] + 16 (d0+d1)(e0+e1)
+ * (discussion of Table "tuples", N_acc = 2).  The A operand then carries one more plane per
+ * non-square modulus, the pre-scaled -16*d1, after d0, d1, d0+d1.  Exact while the merged term
+ * stays below 2^24: k <= 4097 for set S, k <= 15420 for sets E and A; a larger k with this flag is
+ * OZ_ERR_UNSUPPORTED.  SEPARATE: the three accumulators of Eq. 8.  With neither bit, oz_dgemm /
+ * oz_dgemm_ex / oz_dgemm_host pick MERGED when it is exact and n >= 1024 (their planes are
+ * internal; for narrow C the extra planes of A cost more than the saved drains), and the stage entry
+ * points use SEPARATE. */
+#define OZ_ACC_MERGED   0x1000u
+#define OZ_ACC_SEPARATE 0x2000u
+
 #define OZ_K_MAX 32768
 #define OZ_NONFINITE_SHIFT INT32_MIN  /* value of shift[] for a line that holds Inf/NaN */
 
@@ -78,6 +90,10 @@ oz_status_t oz_set_info(oz_modset_t set, int *r, int *p_store, int *moduli);
 /* Stored planes of a set on the substrate named by `route`: 30 / 33 / 44 for S / E / A with
  * two-limb digits, 15 for set A with OZ_SUB_INT8_NATIVE; 0 for an invalid combination. */
 int oz_plane_count(oz_modset_t set, uint32_t route);
+
+/* Same, for the operand on `side` (0: A, 1: B): they differ only with OZ_ACC_MERGED, where A has
+ * one plane more per non-square modulus (S: 36 / 30, E: 40 / 33, A: 58 / 44). */
+int oz_plane_count_side(oz_modset_t set, uint32_t route, int side);
 
 /* Pitch in bytes of one plane row for inner dimension k: k rounded up to 16 (TMA stride rule). */
 int64_t oz_row_pitch(int64_t k);

@@ -502,19 +502,24 @@ int ozo_planes_merged(int side, int64_t lines, int64_t k, const int16_t *D, int 
     int mod[16], r = ozo_modset(set, mod), plane = 0, bad = 0;
     for (int i = 0; i < r; ++i) {
         int np = ozo_planes_of_merged(mod[i], side);
-        for (int64_t l = 0; l < lines; ++l)
-            for (int64_t kk = 0; kk < row_pitch; ++kk) {
-                int dg[4] = {0, 0, 0, 0};
-                if (kk < k) {
-                    ozo_split(D[((int64_t)i * lines + l) * k + kk], mod[i], dg);
-                    dg[3] = -16 * dg[1];
-                }
-                for (int q = 0; q < np; ++q) {
-                    int byte = ozo_e4m3_encode(dg[q]);
-                    if (byte < 0) { bad = 1; byte = 0x7F; }
-                    P[(int64_t)(plane + q) * plane_stride + l * row_pitch + kk] = (uint8_t)byte;
-                }
+        /* bytes of every centred residue of this modulus, worked out once (index d + 1024) */
+        static uint8_t code[2048][4];
+        for (int d = -(mod[i] / 2); 2 * d < mod[i]; ++d) {
+            int dg[4] = {0, 0, 0, 0};
+            ozo_split(d, mod[i], dg);
+            dg[3] = -16 * dg[1];
+            for (int q = 0; q < np; ++q) {
+                int byte = ozo_e4m3_encode(dg[q]);
+                if (byte < 0) { bad = 1; byte = 0x7F; }
+                code[d + 1024][q] = (uint8_t)byte;
             }
+        }
+        for (int64_t l = 0; l < lines; ++l)
+            for (int64_t kk = 0; kk < row_pitch; ++kk)
+                for (int q = 0; q < np; ++q) {
+                    int d = kk < k ? D[((int64_t)i * lines + l) * k + kk] : 0;
+                    P[(int64_t)(plane + q) * plane_stride + l * row_pitch + kk] = code[d + 1024][q];
+                }
         plane += np;
     }
     return bad ? -1 : plane;
@@ -531,14 +536,17 @@ int64_t ozo_plane_products_merged(int64_t m, int64_t n, int64_t k, const uint8_t
     for (int c = 0; c < 256; ++c) digit_of[c] = plane_digit((uint8_t)c, OZO_SUB_FP8);
     for (int i = 0; i < r; ++i) {
         int s = ozo_square_root(mod[i]);
+        const int npa = ozo_planes_of_merged(mod[i], 0), npb = ozo_planes_of_merged(mod[i], 1);
+        int64_t worst_i = 0;
+#pragma omp parallel for schedule(static) reduction(max : worst_i)
         for (int64_t j = 0; j < n; ++j)
             for (int64_t ii = 0; ii < m; ++ii) {
                 int64_t acc0 = 0, acc1 = 0;
                 for (int64_t kk = 0; kk < k; ++kk) {
                     int a[4] = {0, 0, 0, 0}, b[3] = {0, 0, 0};
-                    for (int q = 0; q < ozo_planes_of_merged(mod[i], 0); ++q)
+                    for (int q = 0; q < npa; ++q)
                         a[q] = digit_of[PA[(pa + q) * strideA + ii * pitchA + kk]];
-                    for (int q = 0; q < ozo_planes_of_merged(mod[i], 1); ++q)
+                    for (int q = 0; q < npb; ++q)
                         b[q] = digit_of[PB[(pb + q) * strideB + j * pitchB + kk]];
                     if (s) {
                         acc0 += (int64_t)a[0] * b[0];
@@ -549,15 +557,16 @@ int64_t ozo_plane_products_merged(int64_t m, int64_t n, int64_t k, const uint8_t
                     }
                 }
                 int64_t v0 = acc0 < 0 ? -acc0 : acc0, v1 = acc1 < 0 ? -acc1 : acc1;
-                if (v0 > worst) worst = v0;
-                if (v1 > worst) worst = v1;
+                if (v0 > worst_i) worst_i = v0;
+                if (v1 > worst_i) worst_i = v1;
                 int64_t t = s ? acc0 + (int64_t)s * acc1 : -15 * acc0 + 16 * acc1;
                 int64_t c = t % mod[i];
                 if (c < 0) c += mod[i];
                 R[((int64_t)i * n + j) * m + ii] = (uint16_t)c;
             }
-        pa += ozo_planes_of_merged(mod[i], 0);
-        pb += ozo_planes_of_merged(mod[i], 1);
+        if (worst_i > worst) worst = worst_i;
+        pa += npa;
+        pb += npb;
     }
     return worst;
 }

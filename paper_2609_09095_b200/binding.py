@@ -20,11 +20,12 @@ OZ_SET_S, OZ_SET_E, OZ_SET_A = 0, 1, 2
 OZ_SUB_FP8, OZ_SUB_INT8, OZ_SUB_INT8_NATIVE = 0x001, 0x002, 0x004
 OZ_QUANT_RN, OZ_QUANT_TZ = 0x010, 0x020
 OZ_SCALE_MAXEXP, OZ_SCALE_CS = 0x100, 0x200
+OZ_ACC_MERGED, OZ_ACC_SEPARATE = 0x1000, 0x2000
 OZ_K_MAX = 32768
 OZ_NONFINITE_SHIFT = -(2 ** 31)
 OZ_STATIC_MAX_LINES = 262144
 
-EXPORTS = ["oz_set_info", "oz_plane_count", "oz_row_pitch", "oz_workspace_bytes", "oz_set_workspace", "oz_dgemm",
+EXPORTS = ["oz_set_info", "oz_plane_count", "oz_plane_count_side", "oz_row_pitch", "oz_workspace_bytes", "oz_set_workspace", "oz_dgemm",
            "oz_dgemm_ex", "oz_dgemm_host", "oz_deconstruct", "oz_deconstruct_static",
            "oz_residue_gemm", "oz_reconstruct",
            "oz_query_status", "oz_set_stage_events", "oz_launch_count", "oz_status_string"]
@@ -33,7 +34,7 @@ __all__ = EXPORTS + ["EXPORTS", "OzError", "load", "check", "LIB_PATH", "OZ_OK",
                      "OZ_ERR_UNSUPPORTED", "OZ_ERR_WORKSPACE", "OZ_ERR_CUDA",
                      "OZ_ERR_NONFINITE_INPUT", "OZ_ERR_RANGE", "OZ_ERR_TIMEOUT", "OZ_SET_S",
                      "OZ_SET_E", "OZ_SET_A", "OZ_SUB_FP8", "OZ_SUB_INT8", "OZ_SUB_INT8_NATIVE", "OZ_QUANT_RN", "OZ_QUANT_TZ",
-                     "OZ_SCALE_MAXEXP", "OZ_SCALE_CS", "OZ_K_MAX", "OZ_NONFINITE_SHIFT", "OZ_STATIC_MAX_LINES"]
+                     "OZ_SCALE_MAXEXP", "OZ_SCALE_CS", "OZ_ACC_MERGED", "OZ_ACC_SEPARATE", "OZ_K_MAX", "OZ_NONFINITE_SHIFT", "OZ_STATIC_MAX_LINES"]
 
 _lib = None
 
@@ -56,6 +57,7 @@ def load() -> C.CDLL:
     i64, u32, vp, dbl, i32 = C.c_int64, C.c_uint32, C.c_void_p, C.c_double, C.c_int
     lib.oz_set_info.argtypes = [i32, C.POINTER(i32), C.POINTER(i32), C.POINTER(i32)]
     lib.oz_plane_count.argtypes = [i32, u32]
+    lib.oz_plane_count_side.argtypes = [i32, u32, i32]
     lib.oz_row_pitch.argtypes = [i64]
     lib.oz_row_pitch.restype = i64
     lib.oz_workspace_bytes.argtypes = [i64, i64, i64, i32, u32]
@@ -114,6 +116,10 @@ def oz_set_info(modset: int):
 
 def oz_plane_count(modset: int, route: int = 0) -> int:
     return load().oz_plane_count(modset, route)
+
+
+def oz_plane_count_side(modset: int, route: int, side: int) -> int:
+    return load().oz_plane_count_side(modset, route, side)
 
 
 def oz_row_pitch(k: int) -> int:

@@ -75,6 +75,11 @@ uint32_t lut_entry(int u, int m, int substrate)
         else byte = dig[q] & 0xFF;
         word |= static_cast<uint32_t>(byte) << (8 * q);
     }
+    if (substrate == 0 && !s) {              // byte 3: the pre-scaled plane -16*d1 of the merged schedule
+        int byte = 0;
+        e4m3_code(-16 * dig[1], &byte);
+        word |= static_cast<uint32_t>(byte) << 24;
+    }
     return word;
 }
 
@@ -97,8 +102,12 @@ uint64_t isqrt_u128(unsigned __int128 v)
 
 bool decode_route(uint32_t route, Route *out)
 {
-    uint32_t sub = route & 0x00Fu, q = route & 0x0F0u, sc = route & 0xF00u;
-    if (route & ~0xFFFu) return false;
+    uint32_t sub = route & 0x00Fu, q = route & 0x0F0u, sc = route & 0xF00u, ac = route & 0x3000u;
+    if (route & ~0x3FFFu) return false;
+    if (ac == 0) out->acc = 0;
+    else if (ac == OZ_ACC_MERGED) out->acc = 1;
+    else if (ac == OZ_ACC_SEPARATE) out->acc = 2;
+    else return false;
     if (sub == 0 || sub == OZ_SUB_FP8) out->substrate = 0;
     else if (sub == OZ_SUB_INT8) out->substrate = 1;
     else if (sub == OZ_SUB_INT8_NATIVE) out->substrate = 2;
@@ -116,7 +125,22 @@ bool decode_route(uint32_t route, Route *out)
 bool decode_route_for_set(int set, uint32_t route, Route *out)
 {
     if (!decode_route(route, out)) return false;
+    if (out->merged() && out->substrate != 0) return false;   // -16*d1 reaches -256: FP8 planes only
     return !(out->native() && set != OZ_SET_A);
+}
+
+// Fixes the accumulator schedule of a call.  `automatic`: the whole-method entry points, whose
+// planes are internal, take the merged schedule whenever it is exact; the stage entry points
+// default to separate accumulators because their plane layout is part of the interface.
+// The merged schedule saves one accumulator drain per non-square modulus but adds planes to A:
+// it pays when each plane of A is reused by many columns (n >= 1024), not for tall-skinny shapes
+// whose cost is writing and reading A's planes once.
+oz_status_t resolve_schedule(int set, int64_t k, int64_t n, bool automatic, Route *rt)
+{
+    if (rt->acc == 0)
+        rt->acc = (automatic && rt->substrate == 0 && k > 0 && k <= merged_k_limit(set) && n >= 1024) ? 1 : 2;
+    if (rt->acc == 1 && k > merged_k_limit(set)) return OZ_ERR_UNSUPPORTED;
+    return OZ_OK;
 }
 
 void budget_maxexp(int set, int64_t k, int *tA, int *tB)
@@ -205,7 +229,7 @@ struct Layout {
     int64_t pitch, strideA, strideB, ldr, mod_stride;
 };
 
-Layout make_layout(int64_t m, int64_t n, int64_t k, int set, bool native)
+Layout make_layout(int64_t m, int64_t n, int64_t k, int set, const Route &rt)
 {
     Layout L{};
     Carve c;
@@ -218,8 +242,8 @@ Layout make_layout(int64_t m, int64_t n, int64_t k, int set, bool native)
     L.shiftB = c.take(4 * static_cast<size_t>(n));
     L.scrA = c.take(16 * static_cast<size_t>(m) + 256);
     L.scrB = c.take(16 * static_cast<size_t>(n) + 256);
-    L.PA = c.take(static_cast<size_t>(p_store(set, native)) * L.strideA);
-    L.PB = c.take(static_cast<size_t>(p_store(set, native)) * L.strideB);
+    L.PA = c.take(static_cast<size_t>(p_store(set, rt.layout(0))) * L.strideA);
+    L.PB = c.take(static_cast<size_t>(p_store(set, rt.layout(1))) * L.strideB);
     L.R = c.take(2 * static_cast<size_t>(set_r(set)) * L.mod_stride);
     L.total = c.off;
     return L;
@@ -236,6 +260,7 @@ oz_status_t dgemm_impl(int64_t m, int64_t n, int64_t k, double alpha, const doub
     if (m < 0 || n < 0 || k < 0) return OZ_ERR_INVALID_ARG;
     if (!(alpha == 1.0 || alpha == -1.0) || !(beta == 0.0 || beta == 1.0)) return OZ_ERR_UNSUPPORTED;
     if (k > OZ_K_MAX) return OZ_ERR_UNSUPPORTED;
+    if (resolve_schedule(set, k, n, true, &rt) != OZ_OK) return OZ_ERR_UNSUPPORTED;
     if (m == 0 || n == 0) return OZ_OK;
     if (!C || ldc < m) return OZ_ERR_INVALID_ARG;
     if (k == 0) {
@@ -244,7 +269,7 @@ oz_status_t dgemm_impl(int64_t m, int64_t n, int64_t k, double alpha, const doub
         return OZ_OK;
     }
     if (!A || !B || lda < m || ldb < k) return OZ_ERR_INVALID_ARG;
-    Layout L = make_layout(m, n, k, set, rt.native());
+    Layout L = make_layout(m, n, k, set, rt);
     if (!ws || ws_bytes < L.total) return OZ_ERR_WORKSPACE;
     oz_status_t st = ensure_device_ready();
     if (st != OZ_OK) return st;
@@ -295,7 +320,14 @@ int oz_plane_count(oz_modset_t set, uint32_t route)
 {
     Route rt;
     if (!valid_set(set) || !decode_route_for_set(set, route, &rt)) return 0;
-    return p_store(set, rt.native());
+    return p_store(set, rt.layout(1));
+}
+
+int oz_plane_count_side(oz_modset_t set, uint32_t route, int side)
+{
+    Route rt;
+    if (!valid_set(set) || !decode_route_for_set(set, route, &rt) || (side != 0 && side != 1)) return 0;
+    return p_store(set, rt.layout(side));
 }
 
 int64_t oz_row_pitch(int64_t k) { return round_up(k > 0 ? k : 1, 16); }
@@ -304,7 +336,8 @@ size_t oz_workspace_bytes(int64_t m, int64_t n, int64_t k, oz_modset_t set, uint
 {
     Route rt;
     if (!valid_set(set) || !decode_route_for_set(set, route, &rt) || m < 0 || n < 0 || k < 0) return 0;
-    return make_layout(m > 0 ? m : 1, n > 0 ? n : 1, k > 0 ? k : 1, set, rt.native()).total;
+    if (resolve_schedule(set, k, n, true, &rt) != OZ_OK) return 0;
+    return make_layout(m > 0 ? m : 1, n > 0 ? n : 1, k > 0 ? k : 1, set, rt).total;
 }
 
 oz_status_t oz_set_workspace(void *workspace, size_t bytes)
@@ -349,13 +382,14 @@ oz_status_t oz_dgemm_host(int64_t m, int64_t n, int64_t k, double alpha, const d
     Route rt;
     if (!valid_set(set) || !decode_route_for_set(set, route, &rt)) return OZ_ERR_INVALID_ARG;
     if (m < 0 || n < 0 || k < 0) return OZ_ERR_INVALID_ARG;
+    if (k > OZ_K_MAX || resolve_schedule(set, k, n, true, &rt) != OZ_OK) return OZ_ERR_UNSUPPORTED;
     if (m == 0 || n == 0) return OZ_OK;
     if (!C_host || ldc < m || (k > 0 && (!A_host || !B_host || lda < m || ldb < k)))
         return OZ_ERR_INVALID_ARG;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     char *ws = static_cast<char *>(g_workspace[dev]);
     int64_t kk = k > 0 ? k : 1;
-    size_t core = make_layout(m, n, kk, set, rt.native()).total;
+    size_t core = make_layout(m, n, kk, set, rt).total;
     size_t bytesA = 8 * static_cast<size_t>(m) * kk, bytesB = 8 * static_cast<size_t>(kk) * n;
     size_t bytesC = 8 * static_cast<size_t>(m) * n;
     size_t offA = core, offB = offA + round_up(bytesA, 256), offC = offB + round_up(bytesB, 256);
@@ -384,6 +418,7 @@ oz_status_t oz_deconstruct(int side, int64_t lines, int64_t k, const double *X, 
         return OZ_ERR_INVALID_ARG;
     if (lines < 0 || k < 0) return OZ_ERR_INVALID_ARG;
     if (k > OZ_K_MAX) return OZ_ERR_UNSUPPORTED;
+    if (resolve_schedule(set, k, 0, false, &rt) != OZ_OK) return OZ_ERR_UNSUPPORTED;
     if (lines == 0) return OZ_OK;
     if (!planes || !shift || !scratch || (k > 0 && !X)) return OZ_ERR_INVALID_ARG;
     if (row_pitch < k || row_pitch < 16 || (row_pitch & 15) || (plane_stride & 15) ||
@@ -406,6 +441,7 @@ oz_status_t oz_residue_gemm(int64_t m, int64_t n, int64_t k, const uint8_t *PA, 
     if (!valid_set(set) || !decode_route_for_set(set, route, &rt)) return OZ_ERR_INVALID_ARG;
     if (m < 0 || n < 0 || k < 0) return OZ_ERR_INVALID_ARG;
     if (k > OZ_K_MAX) return OZ_ERR_UNSUPPORTED;
+    if (resolve_schedule(set, k, 0, false, &rt) != OZ_OK) return OZ_ERR_UNSUPPORTED;
     if (m == 0 || n == 0) return OZ_OK;
     if (!PA || !PB || !R || ldr < m || mod_stride < n * ldr) return OZ_ERR_INVALID_ARG;
     if ((pitchA & 15) || (pitchB & 15) || (strideA & 15) || (strideB & 15) || pitchA < k ||

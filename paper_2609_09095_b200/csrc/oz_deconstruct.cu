@@ -228,7 +228,7 @@ __device__ __forceinline__ long long quantise(double x, int sigma, bool tz)
 
 // One modulus (compile-time index I of set SET) for four consecutive inner-dimension elements:
 // residues, table look-up, byte transposition, 2 or 3 four-byte plane stores.
-template <int SET, bool NATIVE, int I>
+template <int SET, int LAYOUT, int I>
 __device__ __forceinline__ void convert_modulus(const uint32_t (&l0)[4], const uint32_t (&l1)[4],
                                                 const uint32_t (&l2)[4], const uint32_t (&l3)[4],
                                                 const uint32_t *__restrict__ lut, uint8_t *out,
@@ -242,7 +242,7 @@ __device__ __forceinline__ void convert_modulus(const uint32_t (&l0)[4], const u
     // floor(v / m) = (v * ceil(2^39 / m)) >> 39 exactly for v < 2^28
     constexpr uint32_t magic = static_cast<uint32_t>(((1ull << 39) + m - 1) / m);
     constexpr int off = lut_offset(SET, I);
-    constexpr int plane = first_plane(SET, I, NATIVE);
+    constexpr int plane = first_plane(SET, I, LAYOUT);
     static_assert(65535ull * (1ull + c1 + c2) + 32767ull * c3 + bias < (1ull << 28), "limb sum below 2^28");
     uint32_t w[4];
 #pragma unroll
@@ -258,27 +258,30 @@ __device__ __forceinline__ void convert_modulus(const uint32_t (&l0)[4], const u
     uint32_t t01 = __byte_perm(w[0], w[1], 0x5140);
     uint32_t t23 = __byte_perm(w[2], w[3], 0x5140);
     *reinterpret_cast<uint32_t *>(out + plane * plane_stride) = __byte_perm(t01, t23, 0x5410);
-    if (NATIVE) return;                       // one plane: the centred residue itself
+    if (LAYOUT == kLayoutNative) return;      // one plane: the centred residue itself
     *reinterpret_cast<uint32_t *>(out + (plane + 1) * plane_stride) = __byte_perm(t01, t23, 0x7632);
     if (planes_of(m) == 3) {
-        uint32_t u01 = __byte_perm(w[0], w[1], 0x0062);
-        uint32_t u23 = __byte_perm(w[2], w[3], 0x0062);
+        // bytes 2 and 3 of the table words: d0+d1 and the pre-scaled -16*d1
+        uint32_t u01 = __byte_perm(w[0], w[1], 0x7362);
+        uint32_t u23 = __byte_perm(w[2], w[3], 0x7362);
         *reinterpret_cast<uint32_t *>(out + (plane + 2) * plane_stride) = __byte_perm(u01, u23, 0x5410);
+        if (LAYOUT == kLayoutMerged)
+            *reinterpret_cast<uint32_t *>(out + (plane + 3) * plane_stride) = __byte_perm(u01, u23, 0x7632);
     }
 }
 
-template <int SET, bool NATIVE, int... I>
+template <int SET, int LAYOUT, int... I>
 __device__ __forceinline__ void convert_all_moduli(std::integer_sequence<int, I...>,
                                                    const uint32_t (&l0)[4], const uint32_t (&l1)[4],
                                                    const uint32_t (&l2)[4], const uint32_t (&l3)[4],
                                                    const uint32_t *__restrict__ lut, uint8_t *out,
                                                    int64_t plane_stride)
 {
-    (convert_modulus<SET, NATIVE, I>(l0, l1, l2, l3, lut, out, plane_stride), ...);
+    (convert_modulus<SET, LAYOUT, I>(l0, l1, l2, l3, lut, out, plane_stride), ...);
 }
 
 // Four consecutive inner-dimension elements of one line -> 4 bytes of every stored plane.
-template <int SET, bool NATIVE>
+template <int SET, int LAYOUT>
 __device__ __forceinline__ void convert4(const double (&x)[4], int sigma, bool tz,
                                          const uint32_t *__restrict__ lut, uint8_t *out,
                                          int64_t plane_stride)
@@ -297,11 +300,11 @@ __device__ __forceinline__ void convert4(const double (&x)[4], int sigma, bool t
         l2[e] = hi & 0xFFFFu;
         l3[e] = static_cast<uint32_t>(static_cast<int32_t>(hi) >> 16);   // signed top limb
     }
-    convert_all_moduli<SET, NATIVE>(std::make_integer_sequence<int, set_r(SET)>{}, l0, l1, l2, l3, lut, out,
+    convert_all_moduli<SET, LAYOUT>(std::make_integer_sequence<int, set_r(SET)>{}, l0, l1, l2, l3, lut, out,
                             plane_stride);
 }
 
-template <int SET, int SIDE, bool NATIVE>
+template <int SET, int SIDE, int LAYOUT>
 __global__ void __launch_bounds__(kConvThreads)
 convert_kernel(const double *__restrict__ X, int64_t ldx, int64_t lines, int64_t k,
                const int32_t *__restrict__ shift, const uint32_t *__restrict__ lut_global,
@@ -329,7 +332,7 @@ convert_kernel(const double *__restrict__ X, int64_t ldx, int64_t lines, int64_t
 #pragma unroll
             for (int e = 0; e < 4; ++e)
                 x[e] = (!dead && kb + e < k) ? X[kb + e + line * ldx] : 0.0;
-            convert4<SET, NATIVE>(x, dead ? 0 : sigma, tz != 0, lut, planes + line * row_pitch + kb, plane_stride);
+            convert4<SET, LAYOUT>(x, dead ? 0 : sigma, tz != 0, lut, planes + line * row_pitch + kb, plane_stride);
         }
     } else {
         double *tile = reinterpret_cast<double *>(smem_raw + kLutWords * 4);
@@ -356,20 +359,20 @@ convert_kernel(const double *__restrict__ X, int64_t ldx, int64_t lines, int64_t
                 double x[4];
 #pragma unroll
                 for (int e = 0; e < 4; ++e) x[e] = dead ? 0.0 : tile[li * kTilePitch + lane * 4 + e];
-                convert4<SET, NATIVE>(x, dead ? 0 : sigma, tz != 0, lut, planes + line * row_pitch + kb, plane_stride);
+                convert4<SET, LAYOUT>(x, dead ? 0 : sigma, tz != 0, lut, planes + line * row_pitch + kb, plane_stride);
             }
             __syncthreads();
         }
     }
 }
 
-template <int SET, int SIDE, bool NATIVE>
+template <int SET, int SIDE, int LAYOUT>
 oz_status_t launch_convert(const double *X, int64_t ldx, int64_t lines, int64_t k,
                            const int32_t *shift, const uint32_t *lut, uint8_t *planes,
                            int64_t plane_stride, int64_t row_pitch, int tz, cudaStream_t stream)
 {
     size_t smem = kLutWords * 4 + (SIDE == 0 ? sizeof(double) * kTileLines * kTilePitch : 0);
-    OZ_CUDA_CHECK(cudaFuncSetAttribute(convert_kernel<SET, SIDE, NATIVE>,
+    OZ_CUDA_CHECK(cudaFuncSetAttribute(convert_kernel<SET, SIDE, LAYOUT>,
                                        cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        static_cast<int>(smem)));
     int64_t nchunks = (row_pitch + kChunk - 1) / kChunk;
@@ -380,7 +383,7 @@ oz_status_t launch_convert(const double *X, int64_t ldx, int64_t lines, int64_t 
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, 0);
     int64_t cap = static_cast<int64_t>(sms) * (SIDE == 1 ? 6 : 3);
     int grid = static_cast<int>(need < cap ? need : cap);
-    convert_kernel<SET, SIDE, NATIVE><<<grid, kConvThreads, smem, stream>>>(
+    convert_kernel<SET, SIDE, LAYOUT><<<grid, kConvThreads, smem, stream>>>(
         X, ldx, lines, k, shift, lut, planes, plane_stride, row_pitch, tz);
     count_launch();
     OZ_CUDA_CHECK(cudaGetLastError());
@@ -432,14 +435,18 @@ oz_status_t launch_deconstruct(int side, int64_t lines, int64_t k, const double 
     OZ_CUDA_CHECK(cudaGetLastError());
 
     const uint32_t *lut = device_lut(set, rt.substrate);
-#define OZ_CONVERT(SET_, NATIVE_)                                                                        \
-    (side == 0 ? launch_convert<SET_, 0, NATIVE_>(X, ldx, lines, k, shift, lut, planes, plane_stride,    \
-                                                  row_pitch, rt.quant, stream)                           \
-               : launch_convert<SET_, 1, NATIVE_>(X, ldx, lines, k, shift, lut, planes, plane_stride,    \
-                                                  row_pitch, rt.quant, stream))
-    if (set == 0) return OZ_CONVERT(0, false);
-    if (set == 1) return OZ_CONVERT(1, false);
-    return rt.native() ? OZ_CONVERT(2, true) : OZ_CONVERT(2, false);
+#define OZ_CONVERT(SET_, SIDE_, LAYOUT_)                                                                 \
+    launch_convert<SET_, SIDE_, LAYOUT_>(X, ldx, lines, k, shift, lut, planes, plane_stride, row_pitch, \
+                                         rt.quant, stream)
+#define OZ_CONVERT_SET(SET_)                                                                             \
+    (side == 1 ? OZ_CONVERT(SET_, 1, kLayoutDigits)                                                      \
+               : (layout == kLayoutMerged ? OZ_CONVERT(SET_, 0, kLayoutMerged) : OZ_CONVERT(SET_, 0, kLayoutDigits)))
+    const int layout = rt.layout(side);
+    if (layout == kLayoutNative) return side == 0 ? OZ_CONVERT(2, 0, kLayoutNative) : OZ_CONVERT(2, 1, kLayoutNative);
+    if (set == 0) return OZ_CONVERT_SET(0);
+    if (set == 1) return OZ_CONVERT_SET(1);
+    return OZ_CONVERT_SET(2);
+#undef OZ_CONVERT_SET
 #undef OZ_CONVERT
 }
 

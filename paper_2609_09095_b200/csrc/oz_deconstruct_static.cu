@@ -56,6 +56,7 @@ extern "C" oz_status_t oz_deconstruct_static(int side, int64_t lines, int64_t k,
         return OZ_ERR_INVALID_ARG;
     if (lines < 0 || k < 0) return OZ_ERR_INVALID_ARG;
     if (k > OZ_K_MAX) return OZ_ERR_UNSUPPORTED;
+    if (oz::resolve_schedule(set, k, 0, false, &rt) != OZ_OK) return OZ_ERR_UNSUPPORTED;
     if (lines > kStaticMaxLines) return OZ_ERR_WORKSPACE;   // beyond the built-in scratch
     if (lines == 0) return OZ_OK;
     if (!planes || !shift || (k > 0 && !X)) return OZ_ERR_INVALID_ARG;

@@ -8,6 +8,9 @@
 // of tcgen05.mma instructions into one TMEM accumulator:
 //   square:      job 0 = D0.E0 (weight 1);  job 1 = [D1|D0].[E0|E1] (two K-loops, weight s)
 //   non-square:  job 0 = D0.E0 (-15);  job 1 = DS.ES (16);  job 2 = D1.E1 (240)
+//   non-square, merged accumulators (FP8, k <= 4097 / 15420): job 0 = [D0|-16 D1].[E0|E1] (-15);
+//                job 1 = DS.ES (16) -- the regrouping discussed under Table "tuples" (N_acc = 2);
+//                one TMEM drain fewer per modulus, which is what bounds the epilogue at small k
 // Three MMA K-loops per modulus either way (p_mma = 3r).
 //
 // The tile is computed transposed: the MMA's M dimension (128 TMEM lanes) runs over 128 columns
@@ -80,8 +83,9 @@ struct ModInfo {
     float m, inv_m;
     float w[3];           // weight of each job
     int reduce[3];        // reduce the accumulator modulo m before weighting (0: the exact FP32 range allows skipping it)
-    int njobs;            // 2 (square), 3, or 1 (native INT8 residues)
-    int plane0;           // first stored plane of this modulus
+    int njobs;            // 2 (square), 3, 1 (native INT8 residues) or 2 (non-square, merged accumulators)
+    int kind;             // 0 square, 1 non-square separate, 2 native, 3 non-square merged
+    int planeA0, planeB0; // first stored plane of this modulus in A's and in B's plane arrays
     // integer epilogue of the INT8 routes (INT32 accumulators):
     int iw[3];            // weights as integers
     uint32_t mi;          // the modulus
@@ -331,21 +335,29 @@ __device__ __forceinline__ Item decode_item(int64_t item, const GemmParams &p)
 // plane pair (A plane, B plane) of K-loop `pair` of job `job`
 __device__ __forceinline__ void job_planes(const ModInfo &mi, int job, int pair, int *pa, int *pb)
 {
-    if (mi.njobs == 3) {
-        // non-square: stored order d0, d1, dS; jobs d0e0, dSeS, d1e1
-        int sel = job == 0 ? 0 : (job == 1 ? 2 : 1);
-        *pa = mi.plane0 + sel;
-        *pb = mi.plane0 + sel;
-    } else if (job == 0) {
-        *pa = mi.plane0;
-        *pb = mi.plane0;
+    int oa, ob;
+    if (mi.kind == 1) {
+        // non-square, stored order d0, d1, dS; jobs d0 e0, dS eS, d1 e1
+        oa = ob = job == 0 ? 0 : (job == 1 ? 2 : 1);
+    } else if (mi.kind == 3) {
+        // non-square merged: job 0 = [d0 | -16 d1] . [e0 | e1] (two K-loops), job 1 = dS eS
+        oa = job == 0 ? (pair == 0 ? 0 : 3) : 2;
+        ob = job == 0 ? (pair == 0 ? 0 : 1) : 2;
+    } else if (mi.kind == 0 && job == 1) {
+        // square: job 1 = [d1 | d0] . [e0 | e1]
+        oa = pair == 0 ? 1 : 0;
+        ob = pair == 0 ? 0 : 1;
     } else {
-        *pa = mi.plane0 + (pair == 0 ? 1 : 0);
-        *pb = mi.plane0 + (pair == 0 ? 0 : 1);
+        oa = ob = 0;            // square job 0, native
     }
+    *pa = mi.planeA0 + oa;
+    *pb = mi.planeB0 + ob;
 }
 
-__device__ __forceinline__ int job_pairs(const ModInfo &mi, int job) { return (mi.njobs == 2 && job == 1) ? 2 : 1; }
+__device__ __forceinline__ int job_pairs(const ModInfo &mi, int job)
+{
+    return ((mi.kind == 0 && job == 1) || (mi.kind == 3 && job == 0)) ? 2 : 1;
+}
 
 template <int SUB, int CG>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
@@ -733,21 +745,35 @@ oz_status_t launch_residue_gemm(int64_t m, int64_t n, int64_t k, const uint8_t *
         mo.mi = static_cast<uint32_t>(mi);
         mo.magic = barrett_magic(static_cast<uint32_t>(mi));
         mo.bias = static_cast<uint32_t>((((1ull << 31) + mi - 1) / mi) * mi);
-        mo.plane0 = first_plane(set, i, rt.native());
+        mo.planeA0 = first_plane(set, i, rt.layout(0));
+        mo.planeB0 = first_plane(set, i, rt.layout(1));
         if (rt.native()) {
             mo.njobs = 1;
+            mo.kind = 2;
             mo.w[0] = 1.0f; mo.w[1] = mo.w[2] = 0.0f;
             mo.reduce[0] = (128 * 128 * kk <= lim) ? 0 : 1;
             mo.reduce[1] = mo.reduce[2] = 1;
         } else if (s) {
             mo.njobs = 2;
+            mo.kind = 0;
             mo.w[0] = 1.0f; mo.w[1] = static_cast<float>(s); mo.w[2] = 0.0f;
             const bool skip_all = integer && (256 + 512 * static_cast<int64_t>(s)) * kk <= lim;
             mo.reduce[0] = (skip_all || 256 * kk + static_cast<int64_t>(s) * red <= lim) ? 0 : 1;
             mo.reduce[1] = skip_all ? 0 : 1;
             mo.reduce[2] = 1;
+        } else if (rt.merged()) {
+            // d e = -15 [d0 e0 - 16 d1 e1] + 16 dS eS; merged term <= 4095 (9-bit tail) or 1088 (bytes)
+            mo.njobs = 2;
+            mo.kind = 3;
+            mo.w[0] = -15.0f; mo.w[1] = 16.0f; mo.w[2] = 0.0f;
+            const int64_t merged_term = mi > 256 ? 4095 : 1088;
+            const bool skip_all = (15 * merged_term + 16 * 484) * kk <= lim;
+            mo.reduce[0] = skip_all ? 0 : 1;
+            mo.reduce[1] = (skip_all || 16 * 484 * kk + 15 * red <= lim) ? 0 : 1;
+            mo.reduce[2] = 1;
         } else {
             mo.njobs = 3;
+            mo.kind = 1;
             mo.w[0] = -15.0f; mo.w[1] = 16.0f; mo.w[2] = 240.0f;
             const bool skip_all = integer && (15 * 196 + 16 * 484 + 240 * 256) * kk <= lim;
             const bool skip01 = skip_all || (15 * 196 + 16 * 484) * kk + 240 * red <= lim;
@@ -760,8 +786,8 @@ oz_status_t launch_residue_gemm(int64_t m, int64_t n, int64_t k, const uint8_t *
     if (k == 0) p.nk = 1;   // one all-zero chunk (the planes' padding) gives residues 0
 
     CUtensorMap mapA, mapB;
-    if (!make_plane_map(&mapA, PA, m, pitchA, strideA, p_store(set, rt.native()), BLOCK_N / cg) ||
-        !make_plane_map(&mapB, PB, n, pitchB, strideB, p_store(set, rt.native()), BLOCK_M))
+    if (!make_plane_map(&mapA, PA, m, pitchA, strideA, p_store(set, rt.layout(0)), BLOCK_N / cg) ||
+        !make_plane_map(&mapB, PB, n, pitchB, strideB, p_store(set, rt.layout(1)), BLOCK_M))
         return OZ_ERR_CUDA;
 
     int dev = 0, sms = 148;

@@ -10,7 +10,7 @@
 namespace oz {
 
 constexpr int kMaxR = 15;          // moduli in the largest supported set (A)
-constexpr int kMaxPlanes = 44;     // stored planes of set A on the two-limb substrates
+constexpr int kMaxPlanes = 58;     // stored planes of set A in the merged-accumulator layout
 constexpr int kLutWords = 8208;    // >= sum of the moduli of either set (S: 8197, E: 6838)
 
 // ---- modulus sets (Sec. 2 step (ii) for S; "Candidate E" and "Candidate A" paragraphs) ---
@@ -33,24 +33,34 @@ __host__ __device__ constexpr int square_root(int m)
     return 0;
 }
 
-// stored planes of one modulus: 2 (square) or 3 digit planes; 1 when the centred residue itself is
-// the INT8 operand (native route, byte moduli only: Sec. 2 "The substrate transition")
-__host__ __device__ constexpr int planes_of(int m, bool native = false)
+// Plane layouts of one operand:
+//   kLayoutDigits  2 (square) or 3 digit planes per modulus: d0, d1[, d0+d1]   (Sec. 2 "FP8 variant")
+//   kLayoutNative  1 plane: the centred residue itself as an INT8 operand (byte moduli only;
+//                  Sec. 2 "The substrate transition")
+//   kLayoutMerged  digits plus a fourth plane -16*d1 for every non-square modulus: the A operand of
+//                  the merged-accumulator schedule (discussion of Table "tuples", N_acc = 2)
+constexpr int kLayoutDigits = 0, kLayoutNative = 1, kLayoutMerged = 2;
+
+__host__ __device__ constexpr int planes_of(int m, int layout = kLayoutDigits)
 {
-    return native ? 1 : (square_root(m) ? 2 : 3);
+    return layout == kLayoutNative ? 1 : (square_root(m) ? 2 : (layout == kLayoutMerged ? 4 : 3));
 }
 
-__host__ __device__ constexpr int first_plane(int set, int i, bool native = false)
+__host__ __device__ constexpr int first_plane(int set, int i, int layout = kLayoutDigits)
 {
     int p = 0;
-    for (int j = 0; j < i; ++j) p += planes_of(modulus(set, j), native);
+    for (int j = 0; j < i; ++j) p += planes_of(modulus(set, j), layout);
     return p;
 }
 
-__host__ __device__ constexpr int p_store(int set, bool native = false)
+__host__ __device__ constexpr int p_store(int set, int layout = kLayoutDigits)
 {
-    return first_plane(set, set_r(set), native);
+    return first_plane(set, set_r(set), layout);
 }
+
+// largest k for which the merged accumulator d0 e0 - 16 d1 e1 stays exact in FP32: the merged term
+// reaches 4095 on the 9-bit tail of S and 1088 on byte moduli
+__host__ __device__ constexpr int64_t merged_k_limit(int set) { return set == 0 ? 4097 : 15420; }
 
 __host__ __device__ constexpr int lut_offset(int set, int i)
 {
@@ -78,12 +88,20 @@ inline int64_t round_up(int64_t v, int64_t a) { return (v + a - 1) / a * a; }
 // ---- route decoding ----------------------------------------------------------------------
 struct Route {
     int substrate;  // 0 fp8, 1 int8 (two-limb digits), 2 int8 native (one residue plane, set A only)
+    int acc;        // 0 unspecified, 1 merged accumulators, 2 separate accumulators
     bool native() const { return substrate == 2; }
+    bool merged() const { return acc == 1; }
+    // plane layout of the operand on `side` (0: rows of A, 1: columns of B)
+    int layout(int side) const
+    {
+        return native() ? kLayoutNative : ((merged() && side == 0) ? kLayoutMerged : kLayoutDigits);
+    }
     int quant;      // 0 rn, 1 tz
     int rule;       // 0 maxexp, 1 cs
 };
 bool decode_route(uint32_t route, Route *out);
-bool decode_route_for_set(int set, uint32_t route, Route *out);   // also rejects native INT8 off set A
+bool decode_route_for_set(int set, uint32_t route, Route *out);
+oz_status_t resolve_schedule(int set, int64_t k, int64_t n, bool automatic, Route *rt);   // merged or separate accumulators   // also rejects native INT8 off set A
 
 // ---- per-device state --------------------------------------------------------------------
 // Builds the lookup tables and constant blocks on the current device the first time it is used.

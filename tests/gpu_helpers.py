@@ -10,10 +10,12 @@ import paper_2609_09095_b200 as oz
 SETS = {"S": oz.OZ_SET_S, "E": oz.OZ_SET_E, "A": oz.OZ_SET_A}
 
 
-def route(sub="fp8", quant="RN", rule="CS") -> int:
+def route(sub="fp8", quant="RN", rule="CS", acc=None) -> int:
     r = {"fp8": oz.OZ_SUB_FP8, "int8": oz.OZ_SUB_INT8, "int8n": oz.OZ_SUB_INT8_NATIVE}[sub]
     r |= oz.OZ_QUANT_RN if quant == "RN" else oz.OZ_QUANT_TZ
     r |= oz.OZ_SCALE_CS if rule == "CS" else oz.OZ_SCALE_MAXEXP
+    if acc is not None:
+        r |= oz.OZ_ACC_MERGED if acc == "merged" else oz.OZ_ACC_SEPARATE
     return r
 
 
@@ -35,7 +37,7 @@ def deconstruct(side: int, X: np.ndarray, set_name: str, rt: int):
     lines = X.shape[0] if side == 0 else X.shape[1]
     k = X.shape[1] if side == 0 else X.shape[0]
     ldx = max(X.shape[0], 1)
-    p = oz.oz_plane_count(SETS[set_name], rt)
+    p = oz.oz_plane_count_side(SETS[set_name], rt, side)
     pitch = oz.oz_row_pitch(k)
     dX = to_dev(X) if X.size else torch.zeros(1, dtype=torch.float64, device="cuda")
     planes = torch.full((p, lines, pitch), 0xAA, dtype=torch.uint8, device="cuda")

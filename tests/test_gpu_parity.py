@@ -49,6 +49,60 @@ def test_deconstruct_bit_exact(side, lines, k, dist, set_name, sub, quant, rule)
     assert P.shape == Po.shape and (P == Po).all()
 
 
+@pytest.mark.parametrize("set_name,lines,k", [("S", 130, 1000), ("E", 67, 4101), ("A", 37, 129), ("S", 5, 4097)])
+def test_merged_schedule_stages_bit_exact(set_name, lines, k):
+    """Merged accumulators: the A operand carries the pre-scaled -16*d1 planes, B is unchanged, and
+    the two-accumulator GEMM gives the same residues."""
+    import tests.gpu_helpers as gh
+    rng = np.random.default_rng(lines + k)
+    A = syn._draw(rng, lines, k, "lognormal:0.5")
+    B = syn._draw(rng, k, 150, "normal")
+    rt = gh.route("fp8", "RN", "CS", acc="merged")
+    PA, shA, st = gh.deconstruct(0, A, set_name, rt)
+    PB, shB, st2 = gh.deconstruct(1, B, set_name, rt)
+    _, shAo, DA = _oracle_deconstruct(0, A, set_name, "fp8", "RN", "CS")
+    _, shBo, DB = _oracle_deconstruct(1, B, set_name, "fp8", "RN", "CS")
+    PAo, PBo = ozo.planes_merged(0, DA, OSET[set_name]), ozo.planes_merged(1, DB, OSET[set_name])
+    assert st == 0 and st2 == 0 and (shA == shAo).all() and (shB == shBo).all()
+    assert PA.shape == PAo.shape and (PA == PAo).all() and (PB == PBo).all()
+    R, st3 = gh.residue_gemm(PA, PB, k, set_name, rt)
+    assert st3 == 0 and (R == ozo.products(DA, DB, OSET[set_name])).all()
+
+
+def test_merged_schedule_limits():
+    import torch
+    import paper_2609_09095_b200 as oz
+    import tests.gpu_helpers as gh
+    assert oz.oz_plane_count_side(oz.OZ_SET_S, oz.OZ_ACC_MERGED, 0) == 36
+    assert oz.oz_plane_count_side(oz.OZ_SET_S, oz.OZ_ACC_MERGED, 1) == 30
+    assert oz.oz_plane_count_side(oz.OZ_SET_E, oz.OZ_ACC_MERGED, 0) == 40
+    assert oz.oz_plane_count_side(oz.OZ_SET_S, oz.OZ_ACC_MERGED | oz.OZ_SUB_INT8, 0) == 0   # FP8 planes only
+    t = torch.zeros(8, dtype=torch.float64, device="cuda")
+    u = torch.zeros(64, dtype=torch.uint8, device="cuda")
+    s32 = torch.zeros(4, dtype=torch.int32, device="cuda")
+    scr = torch.zeros(1024, dtype=torch.uint8, device="cuda")
+    rt = gh.route("fp8", "RN", "CS", acc="merged")
+    # beyond the exact depth of the merged accumulator the flag is refused, not silently dropped
+    assert oz.oz_deconstruct(0, 1, 4098, t, 1, oz.OZ_SET_S, rt, u, 4112, 4112, s32, scr) == oz.OZ_ERR_UNSUPPORTED
+    assert oz.oz_dgemm(4, 4, 4098, t, 4, t, 4098, t, 4, oz.OZ_SET_S, rt) == oz.OZ_ERR_UNSUPPORTED
+
+
+def test_merged_accumulator_exact_at_its_depth():
+    """k = 4097 on set S with the largest digits: the merged accumulator reaches 4095 * 4097 < 2^24."""
+    import tests.gpu_helpers as gh
+    rng = np.random.default_rng(4097)
+    m, n, k = 70, 140, 4097
+    _, DA = _random_planes(rng, "S", "fp8", m, k, extreme=True)
+    _, DB = _random_planes(rng, "S", "fp8", n, k, extreme=True)
+    DA[:, :8, :] = DA[:, :1, :1]
+    DB[:, :8, :] = DB[:, :1, :1]
+    PA, PB = ozo.planes_merged(0, DA, ozo.SET_S), ozo.planes_merged(1, DB, ozo.SET_S)
+    want, worst = ozo.plane_products_merged(PA, PB, k, ozo.SET_S)
+    assert worst < 2 ** 24 and worst > 0.5 * 4095 * k and (want == ozo.products(DA, DB, ozo.SET_S)).all()
+    R, st = gh.residue_gemm(PA, PB, k, "S", gh.route("fp8", acc="merged"))
+    assert st == 0 and (R == want).all()
+
+
 @pytest.mark.parametrize("kind", ["zero_lines", "subnormal", "spike", "small_integers"])
 @pytest.mark.parametrize("rule", ["CS", "MAXEXP"])
 def test_deconstruct_edge_inputs(kind, rule):
@@ -185,11 +239,12 @@ def test_dgemm_configs_cut_down(cfg_id, m, n, k, sets):
             _check_against_oracle_and_dd(A, B, got, want, use_c0, cfg.alpha, strict_dd=(cfg_id != 5))
 
 
-@pytest.mark.parametrize("quant,rule", [("TZ", "MAXEXP"), ("RN", "MAXEXP"), ("TZ", "CS")])
-def test_dgemm_variants(quant, rule):
+@pytest.mark.parametrize("quant,rule,acc", [("TZ", "MAXEXP", None), ("RN", "MAXEXP", "separate"),
+                                            ("TZ", "CS", "merged"), ("RN", "CS", "separate")])
+def test_dgemm_variants(quant, rule, acc):
     import tests.gpu_helpers as gh
     A, B = syn.operands(syn.CONFIGS[1], 130, 70, 200)
-    got, st = gh.dgemm(A, B, "S", gh.route("fp8", quant, rule))
+    got, st = gh.dgemm(A, B, "S", gh.route("fp8", quant, rule, acc))
     _, oq, orule = _oracle_route("fp8", quant, rule)
     want = ozo.dgemm(A, B, ozo.SET_S, oq, orule)
     assert st == 0 and (got == want).all()
