@@ -34,10 +34,11 @@ sys.path.insert(0, ROOT)
 
 import synth_inputs as syn  # noqa: E402
 
-# DRAM read amplification of the residue GEMM (reads / plane bytes), measured with ncu on a
-# 16384x4096x2048 launch; writes equal the residue bytes exactly.  Used to scale the measured
-# traffic to the full-size launch, which is too large to capture.
-GEMM_DRAM_READ_AMPLIFICATION = 1.60
+# DRAM traffic of the residue GEMM relative to its algorithmic bytes (reads / plane bytes, writes /
+# residue bytes), measured with ncu on a 16384x4096x2048 launch.  Used to scale the measured traffic
+# to the full-size launch, which is too large to capture.
+GEMM_DRAM_READ_AMPLIFICATION = 2.44
+GEMM_DRAM_WRITE_AMPLIFICATION = 1.10
 
 METRIC = "emulated FP64 TFLOPS (2mnk/s)"
 UNIT = "TFLOP/s"
@@ -197,6 +198,9 @@ def main():
     route = sub | oz.OZ_QUANT_RN | oz.OZ_SCALE_CS
     r, _, _ = oz.oz_set_info(modset)
     p_store = oz.oz_plane_count(modset, route)
+    # planes of A: six more in the merged-accumulator layout that oz_dgemm picks when it is exact
+    merged = args.substrate == "fp8" and n >= 1024 and k <= (4097 if args.set_name == "S" else 15420)
+    p_store_a = oz.oz_plane_count_side(modset, route | oz.OZ_ACC_MERGED, 0) if merged else p_store
     if p_store == 0:
         raise SystemExit("the native INT8 substrate needs the all-byte set: --set A --substrate int8n")
     passes = r if args.substrate == "int8n" else 3 * r    # plane products per FP64 product
@@ -293,7 +297,7 @@ def main():
         achieved = lowp_flops / (gemm_ms * 1e-3) / 1e12
         roof_nominal = 4500.0 / (passes + 1)               # P_low/(3r+1), or P_low/(r+1) native INT8, at B200's dense 8-bit rate
         hbm = peaks["hbm_gbs"]
-        dec_bytes = (8 + 8 * 2 + p_store) * (m * k + k * n)   # max-exponent + sum-of-squares scans, convert read, planes written
+        dec_bytes = 24 * (m * k + k * n) + (p_store_a * m + p_store * n) * k   # two scan passes + convert read; planes written
         rec_bytes = (2 * r + 8 + (8 if cfg.beta else 0)) * m * n
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -314,9 +318,10 @@ def main():
                          "peak": tensor_peak, "unit": "TFLOP/s", "frac": achieved / tensor_peak,
                          "peak_source": f"{peaks['source']} bf16 sustained x2 (8-bit operands)",
                          "frac_of_nominal_4500": achieved / 4500.0,
-                         "traffic": GEMM_DRAM_READ_AMPLIFICATION * p_store * (m + n) * k + 2.0 * r * m * n,
+                         "traffic": GEMM_DRAM_READ_AMPLIFICATION * (p_store_a * m + p_store * n) * k
+                                    + GEMM_DRAM_WRITE_AMPLIFICATION * 2.0 * r * m * n,
                          "traffic_unit": "bytes per launch (ncu dram read+write of a smaller launch, scaled by units)",
-                         "algorithmic_dram_bytes": p_store * (m + n) * k + 2.0 * r * m * n,
+                         "algorithmic_dram_bytes": (p_store_a * m + p_store * n) * k + 2.0 * r * m * n,
                          "ms_per_launch": gemm_ms},
             "stages": {
                 "deconstruct_A_ms": float(stage_ms[0]), "deconstruct_B_ms": float(stage_ms[1]),

@@ -43,8 +43,8 @@ enum { OZO_QUANT_RN = 0, OZO_QUANT_TZ = 1 };
 enum { OZO_SCALE_MAXEXP = 0, OZO_SCALE_CS = 1 };
 /* FP8 / INT8: two-limb digit planes (Sec. 2 "FP8 variant").  INT8_NATIVE: one plane per modulus
  * holding the centred residue itself as a signed byte -- possible for byte moduli only (Sec. 2,
- * "The substrate transition": "the centred residue of a byte modulus (m <= 256) fits an INT8
- * operand directly", alpha_INT8 = r + 1).                                                     */
+ * paragraph "The substrate transition": byte-modulus residues need no digit split on the INT8
+ * substrate, alpha_INT8 = r + 1).                                                             */
 enum { OZO_SUB_FP8 = 0, OZO_SUB_INT8 = 1, OZO_SUB_INT8_NATIVE = 2 };
 
 #define OZO_NONFINITE_SHIFT INT32_MIN
