@@ -71,12 +71,13 @@ typedef enum { OZ_SET_S = 0, OZ_SET_E = 1, OZ_SET_A = 2 } oz_modset_t;
 /* Accumulator schedule of the residue GEMMs for non-square moduli on the FP8 substrate.
  * MERGED: two accumulators per modulus, d e = -15 [d0 e0 + (-16 d1) e1] + 16 (d0+d1)(e0+e1)
  * (discussion of Table "tuples", N_acc = 2).  The A operand then carries one more plane per
- * non-square modulus, the pre-scaled -16*d1, after d0, d1, d0+d1.  Exact while the merged term
- * stays below 2^24: k <= 4097 for set S, k <= 15420 for sets E and A; a larger k with this flag is
- * OZ_ERR_UNSUPPORTED.  SEPARATE: the three accumulators of Eq. 8.  With neither bit, oz_dgemm /
- * oz_dgemm_ex / oz_dgemm_host pick MERGED when it is exact and n >= 1024 (their planes are
- * internal; for narrow C the extra planes of A cost more than the saved drains), and the stage entry
- * points use SEPARATE. */
+ * non-square modulus, the pre-scaled -16*d1, after d0, d1, d0+d1.  One merged accumulator is exact
+ * while its term stays below 2^24: k <= 4097 for set S, k <= 15420 for sets E and A.  A longer k is
+ * cut into equal K segments no longer than that, each with an accumulator of its own that is reduced
+ * modulo m_i before the segments are added (split-K inside the kernel; the residues are the same).
+ * SEPARATE: the three accumulators of Eq. 8.  With neither bit, oz_dgemm / oz_dgemm_ex /
+ * oz_dgemm_host pick MERGED when n >= 1024 (their planes are internal; for narrow C the extra planes
+ * of A cost more than the saved products), and the stage entry points use SEPARATE. */
 #define OZ_ACC_MERGED   0x1000u
 #define OZ_ACC_SEPARATE 0x2000u
 

@@ -130,7 +130,8 @@ bool decode_route_for_set(int set, uint32_t route, Route *out)
 }
 
 // Fixes the accumulator schedule of a call.  `automatic`: the whole-method entry points, whose
-// planes are internal, take the merged schedule whenever it is exact; the stage entry points
+// planes are internal, take the merged schedule (the GEMM cuts a long k into segments that each
+// stay exact); the stage entry points
 // default to separate accumulators because their plane layout is part of the interface.
 // The merged schedule saves one accumulator drain per non-square modulus but adds planes to A:
 // it pays when each plane of A is reused by many columns (n >= 1024), not for tall-skinny shapes
@@ -138,8 +139,7 @@ bool decode_route_for_set(int set, uint32_t route, Route *out)
 oz_status_t resolve_schedule(int set, int64_t k, int64_t n, bool automatic, Route *rt)
 {
     if (rt->acc == 0)
-        rt->acc = (automatic && rt->substrate == 0 && k > 0 && k <= merged_k_limit(set) && n >= 1024) ? 1 : 2;
-    if (rt->acc == 1 && k > merged_k_limit(set)) return OZ_ERR_UNSUPPORTED;
+        rt->acc = (automatic && rt->substrate == 0 && k > 0 && n >= 1024) ? 1 : 2;
     return OZ_OK;
 }
 

@@ -86,6 +86,8 @@ struct ModInfo {
     int njobs;            // 2 (square), 3, 1 (native INT8 residues) or 2 (non-square, merged accumulators)
     int kind;             // 0 square, 1 non-square separate, 2 native, 3 non-square merged
     int planeA0, planeB0; // first stored plane of this modulus in A's and in B's plane arrays
+    int nseg, seg_len;    // merged job 0 only: the K range is cut into nseg segments of seg_len chunks, each
+                          // with an accumulator of its own, so that every FP32 accumulator stays exact
     // integer epilogue of the INT8 routes (INT32 accumulators):
     int iw[3];            // weights as integers
     uint32_t mi;          // the modulus
@@ -359,6 +361,24 @@ __device__ __forceinline__ int job_pairs(const ModInfo &mi, int job)
     return ((mi.kind == 0 && job == 1) || (mi.kind == 3 && job == 0)) ? 2 : 1;
 }
 
+// accumulators (K segments) of job `job`
+__device__ __forceinline__ int job_segments(const ModInfo &mi, int job)
+{
+    return (mi.kind == 3 && job == 0) ? mi.nseg : 1;
+}
+
+// chunk range [kc0, kc1) of segment `seg`
+__device__ __forceinline__ void segment_range(const ModInfo &mi, int job, int seg, int nk, int *kc0, int *kc1)
+{
+    if (mi.kind == 3 && job == 0) {
+        *kc0 = seg * mi.seg_len;
+        *kc1 = min(nk, *kc0 + mi.seg_len);
+    } else {
+        *kc0 = 0;
+        *kc1 = nk;
+    }
+}
+
 template <int SUB, int CG>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 residue_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB,
@@ -415,12 +435,14 @@ residue_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
             for (int64_t item = first_item; ok && item < p.total_items; item += item_step) {
                 Item it = decode_item(item, p);
                 const ModInfo &mi = p.mod[it.mod];
-                for (int job = 0; ok && job < mi.njobs; ++job) {
-                    int npairs = job_pairs(mi, job);
+                for (int job = 0; ok && job < mi.njobs; ++job)
+                for (int seg = 0, nseg = job_segments(mi, job); ok && seg < nseg; ++seg) {
+                    int npairs = job_pairs(mi, job), kc0, kc1;
+                    segment_range(mi, job, seg, p.nk, &kc0, &kc1);
                     for (int pair = 0; ok && pair < npairs; ++pair) {
                         int pa, pb;
                         job_planes(mi, job, pair, &pa, &pb);
-                        for (int kc = 0; kc < p.nk; ++kc) {
+                        for (int kc = kc0; kc < kc1; ++kc) {
                             ok = mbar_wait(empty_bar + 8 * stage, phase ^ 1u, abort_flag, p.status);
                             if (!ok) break;
                             uint32_t fb = full_bar + 8 * stage;
@@ -459,13 +481,16 @@ residue_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
             for (int64_t item = first_item; ok && item < p.total_items; item += item_step) {
                 Item it = decode_item(item, p);
                 const ModInfo &mi = p.mod[it.mod];
-                for (int job = 0; ok && job < mi.njobs; ++job) {
+                for (int job = 0; ok && job < mi.njobs; ++job)
+                for (int seg = 0, nseg = job_segments(mi, job); ok && seg < nseg; ++seg) {
                     ok = mbar_wait(tempty_bar + 8 * slot, ((slot_phase >> slot) & 1u) ^ 1u, abort_flag, p.status);
                     if (!ok) break;
                     tc_fence_after();
                     const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(slot * BLOCK_N);
                     uint32_t accumulate = 0;
-                    int steps = job_pairs(mi, job) * p.nk;
+                    int kc0, kc1;
+                    segment_range(mi, job, seg, p.nk, &kc0, &kc1);
+                    int steps = job_pairs(mi, job) * (kc1 - kc0);
                     for (int st = 0; st < steps; ++st) {
                         ok = mbar_wait(full_bar + 8 * stage, phase, abort_flag, p.status);
                         if (!ok) break;
@@ -509,7 +534,8 @@ residue_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
             uint32_t comb[COLS_PER_WARP];
 #pragma unroll
             for (int c = 0; c < COLS_PER_WARP; ++c) comb[c] = 0u;
-            for (int job = 0; ok && job < mi.njobs; ++job) {
+            for (int job = 0; ok && job < mi.njobs; ++job)
+            for (int seg = 0, nseg = job_segments(mi, job); ok && seg < nseg; ++seg) {
                 ok = mbar_wait(tfull_bar + 8 * slot, (slot_phase >> slot) & 1u, abort_flag, p.status);
                 if (!ok) break;
                 tc_fence_after();
@@ -725,6 +751,7 @@ oz_status_t launch_residue_gemm(int64_t m, int64_t n, int64_t k, const uint8_t *
     p.tiles_n = static_cast<int>((n + BLOCK_M * cg - 1) / (BLOCK_M * cg)); // 128 (256) columns of C per tile
     p.vec_store = ((ldr & 7) == 0 && (mod_stride & 7) == 0 && (reinterpret_cast<uintptr_t>(R) & 15u) == 0) ? 1 : 0;
     p.nk = static_cast<int>((k + BLOCK_K - 1) / BLOCK_K);
+    if (k == 0) p.nk = 1;   // one all-zero chunk (the planes' padding) gives residues 0
     p.r = set_r(set);
     p.total_items = static_cast<int64_t>(p.r) * p.tiles_m * p.tiles_n;
     p.R = R; p.ldr = ldr; p.mod_stride = mod_stride;
@@ -747,6 +774,8 @@ oz_status_t launch_residue_gemm(int64_t m, int64_t n, int64_t k, const uint8_t *
         mo.bias = static_cast<uint32_t>((((1ull << 31) + mi - 1) / mi) * mi);
         mo.planeA0 = first_plane(set, i, rt.layout(0));
         mo.planeB0 = first_plane(set, i, rt.layout(1));
+        mo.nseg = 1;
+        mo.seg_len = p.nk;
         if (rt.native()) {
             mo.njobs = 1;
             mo.kind = 2;
@@ -766,10 +795,16 @@ oz_status_t launch_residue_gemm(int64_t m, int64_t n, int64_t k, const uint8_t *
             mo.njobs = 2;
             mo.kind = 3;
             mo.w[0] = -15.0f; mo.w[1] = 16.0f; mo.w[2] = 0.0f;
+            // K longer than the exact range of one merged accumulator is cut into equal segments,
+            // each drained and reduced on its own (the residues add modulo m).
             const int64_t merged_term = mi > 256 ? 4095 : 1088;
-            const bool skip_all = (15 * merged_term + 16 * 484) * kk <= lim;
+            const int seg_max = static_cast<int>(merged_k_limit(set) / BLOCK_K);
+            mo.nseg = (p.nk + seg_max - 1) / seg_max;
+            if (mo.nseg < 1) mo.nseg = 1;
+            mo.seg_len = (p.nk + mo.nseg - 1) / mo.nseg;
+            const bool skip_all = mo.nseg == 1 && (15 * merged_term + 16 * 484) * kk <= lim;
             mo.reduce[0] = skip_all ? 0 : 1;
-            mo.reduce[1] = (skip_all || 16 * 484 * kk + 15 * red <= lim) ? 0 : 1;
+            mo.reduce[1] = (skip_all || 16 * 484 * kk + 15 * red * mo.nseg <= lim) ? 0 : 1;
             mo.reduce[2] = 1;
         } else {
             mo.njobs = 3;
@@ -783,7 +818,6 @@ oz_status_t launch_residue_gemm(int64_t m, int64_t n, int64_t k, const uint8_t *
         }
         for (int j = 0; j < 3; ++j) mo.iw[j] = static_cast<int>(mo.w[j]);
     }
-    if (k == 0) p.nk = 1;   // one all-zero chunk (the planes' padding) gives residues 0
 
     CUtensorMap mapA, mapB;
     if (!make_plane_map(&mapA, PA, m, pitchA, strideA, p_store(set, rt.layout(0)), BLOCK_N / cg) ||

@@ -77,14 +77,24 @@ def test_merged_schedule_limits():
     assert oz.oz_plane_count_side(oz.OZ_SET_S, oz.OZ_ACC_MERGED, 1) == 30
     assert oz.oz_plane_count_side(oz.OZ_SET_E, oz.OZ_ACC_MERGED, 0) == 40
     assert oz.oz_plane_count_side(oz.OZ_SET_S, oz.OZ_ACC_MERGED | oz.OZ_SUB_INT8, 0) == 0   # FP8 planes only
-    t = torch.zeros(8, dtype=torch.float64, device="cuda")
-    u = torch.zeros(64, dtype=torch.uint8, device="cuda")
-    s32 = torch.zeros(4, dtype=torch.int32, device="cuda")
-    scr = torch.zeros(1024, dtype=torch.uint8, device="cuda")
-    rt = gh.route("fp8", "RN", "CS", acc="merged")
-    # beyond the exact depth of the merged accumulator the flag is refused, not silently dropped
-    assert oz.oz_deconstruct(0, 1, 4098, t, 1, oz.OZ_SET_S, rt, u, 4112, 4112, s32, scr) == oz.OZ_ERR_UNSUPPORTED
-    assert oz.oz_dgemm(4, 4, 4098, t, 4, t, 4098, t, 4, oz.OZ_SET_S, rt) == oz.OZ_ERR_UNSUPPORTED
+
+
+@pytest.mark.parametrize("set_name,k", [("S", 4224), ("S", 8321), ("S", 12289), ("E", 16640), ("A", 16640)])
+def test_merged_schedule_segments_long_k(set_name, k):
+    """k beyond the exact depth of one merged accumulator (4097 / 15420): the kernel cuts K into
+    segments, each with its own accumulator; extreme digits make a single accumulator overflow 2^24."""
+    import tests.gpu_helpers as gh
+    rng = np.random.default_rng(k)
+    m, n = 70, 140
+    _, DA = _random_planes(rng, set_name, "fp8", m, k, extreme=True)
+    _, DB = _random_planes(rng, set_name, "fp8", n, k, extreme=True)
+    for i, mod in enumerate(ozo.modset(OSET[set_name])):
+        DA[i, :8, :] = DB[i, :8, :] = (mod - 1) // 2      # largest residue: merged term 4095 (1088 on bytes)
+    PA, PB = ozo.planes_merged(0, DA, OSET[set_name]), ozo.planes_merged(1, DB, OSET[set_name])
+    _, worst = ozo.plane_products_merged(PA, PB, k, OSET[set_name])
+    assert worst >= 2 ** 24            # one accumulator over all of K would not be exact
+    R, st = gh.residue_gemm(PA, PB, k, set_name, gh.route("fp8", acc="merged"))
+    assert st == 0 and (R == ozo.products(DA, DB, OSET[set_name])).all()
 
 
 def test_merged_accumulator_exact_at_its_depth():
