@@ -199,7 +199,7 @@ def main():
     r, _, _ = oz.oz_set_info(modset)
     p_store = oz.oz_plane_count(modset, route)
     # planes of A: six more in the merged-accumulator layout that oz_dgemm picks when it is exact
-    merged = args.substrate == "fp8" and n >= 1024 and k <= (4097 if args.set_name == "S" else 15420)
+    merged = args.substrate == "fp8" and n >= 1024          # the library's default schedule
     p_store_a = oz.oz_plane_count_side(modset, route | oz.OZ_ACC_MERGED, 0) if merged else p_store
     if p_store == 0:
         raise SystemExit("the native INT8 substrate needs the all-byte set: --set A --substrate int8n")
@@ -298,7 +298,8 @@ def main():
         roof_nominal = 4500.0 / (passes + 1)               # P_low/(3r+1), or P_low/(r+1) native INT8, at B200's dense 8-bit rate
         hbm = peaks["hbm_gbs"]
         dec_bytes = 24 * (m * k + k * n) + (p_store_a * m + p_store * n) * k   # two scan passes + convert read; planes written
-        rec_bytes = (2 * r + 8 + (8 if cfg.beta else 0)) * m * n
+        rb = oz.oz_residue_elem_bytes(modset)                 # bytes per stored residue
+        rec_bytes = (rb * r + 8 + (8 if cfg.beta else 0)) * m * n
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
@@ -308,7 +309,7 @@ def main():
                        "modulus_set": args.set_name, "r": r, "substrate": args.substrate, "quantiser": "RN",
                        "scale_rule": "CS",
                        "l2": "inputs larger than L2 (126 MB): A+B %.0f MB, C %.0f MB, planes %.0f MB, residues %.0f MB"
-                             % (8e-6 * (m * k + k * n), 8e-6 * m * n, 1e-6 * p_store * (m + n) * k, 2e-6 * r * m * n),
+                             % (8e-6 * (m * k + k * n), 8e-6 * m * n, 1e-6 * p_store * (m + n) * k, 1e-6 * rb * r * m * n),
                        "parallelism": f"replicas x{world}" if world > 1 else "single GPU"},
             "roof": {"definition": "P_low/(3r+1)" if passes == 3 * r else "P_low/(r+1)", "nominal_tflops": roof_nominal,
                      "frac_of_nominal": value / world / roof_nominal,
@@ -319,9 +320,9 @@ def main():
                          "peak_source": f"{peaks['source']} bf16 sustained x2 (8-bit operands)",
                          "frac_of_nominal_4500": achieved / 4500.0,
                          "traffic": GEMM_DRAM_READ_AMPLIFICATION * (p_store_a * m + p_store * n) * k
-                                    + GEMM_DRAM_WRITE_AMPLIFICATION * 2.0 * r * m * n,
+                                    + GEMM_DRAM_WRITE_AMPLIFICATION * float(rb) * r * m * n,
                          "traffic_unit": "bytes per launch (ncu dram read+write of a smaller launch, scaled by units)",
-                         "algorithmic_dram_bytes": (p_store_a * m + p_store * n) * k + 2.0 * r * m * n,
+                         "algorithmic_dram_bytes": (p_store_a * m + p_store * n) * k + float(rb) * r * m * n,
                          "ms_per_launch": gemm_ms},
             "stages": {
                 "deconstruct_A_ms": float(stage_ms[0]), "deconstruct_B_ms": float(stage_ms[1]),

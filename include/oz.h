@@ -96,6 +96,11 @@ int oz_plane_count(oz_modset_t set, uint32_t route);
  * one plane more per non-square modulus (S: 36 / 30, E: 40 / 33, A: 58 / 44). */
 int oz_plane_count_side(oz_modset_t set, uint32_t route, int side);
 
+/* Bytes of one stored residue: 2 (uint16) for sets S and E, 1 (uint8) for the all-byte set A, whose
+ * moduli do not exceed 256; 0 for an unknown set.  This is the element type of the array R of
+ * oz_residue_gemm and oz_reconstruct. */
+size_t oz_residue_elem_bytes(oz_modset_t set);
+
 /* Pitch in bytes of one plane row for inner dimension k: k rounded up to 16 (TMA stride rule). */
 int64_t oz_row_pitch(int64_t k);
 
@@ -162,19 +167,24 @@ oz_status_t oz_deconstruct_static(int side, int64_t lines, int64_t k, const doub
 
 /* Residue products (Eq. 3 through the plane identities of Sec. 2 "FP8 variant" and Eq. 8):
  * for every modulus i,  R_i = (A_i B_i) mod m_i  from the stored planes of A (lines = m) and
- * B (lines = n), on the tensor cores.  Output R[i*mod_stride + j*ldr + row], uint16 in [0, m_i).
- * ldr >= m, mod_stride >= n*ldr (in elements).  Planes as written by oz_deconstruct with the
- * same set and substrate; plane bases 16-byte aligned, pitches and strides multiples of 16. */
+ * B (lines = n), on the tensor cores.  Output R[i*mod_stride + j*ldr + row], the canonical residue
+ * in [0, m_i) as an unsigned integer of oz_residue_elem_bytes(set) bytes (uint16 for S and E, uint8
+ * for A; device memory).  ldr >= m, mod_stride >= n*ldr (in elements); rows whose byte offset is a
+ * multiple of 16 (R 16-byte aligned, ldr and mod_stride multiples of 8 resp. 16 elements) take the
+ * fast vector stores, anything else a slower element-wise path with the same result.  Planes as
+ * written by oz_deconstruct with the same set and substrate; plane bases 16-byte aligned, pitches
+ * and strides multiples of 16. */
 oz_status_t oz_residue_gemm(int64_t m, int64_t n, int64_t k, const uint8_t *PA,
                             int64_t plane_strideA, int64_t row_pitchA, const uint8_t *PB,
                             int64_t plane_strideB, int64_t row_pitchB, oz_modset_t set,
-                            uint32_t route, uint16_t *R, int64_t ldr, int64_t mod_stride,
+                            uint32_t route, void *R, int64_t ldr, int64_t mod_stride,
                             void *stream);
 
 /* Reconstruction (Algorithm 3; Eq. 4-5 and the final step of Sec. 2 (iv)): the integer
  * c'_ij in [-M/2, M/2) congruent to the residues, times 2^-(shiftA[i]+shiftB[j]), rounded once;
- * C = alpha P (beta = 0) or C = C + alpha P (beta = 1).  The CRT is evaluated exactly. */
-oz_status_t oz_reconstruct(int64_t m, int64_t n, const uint16_t *R, int64_t ldr,
+ * C = alpha P (beta = 0) or C = C + alpha P (beta = 1).  The CRT is evaluated exactly.  R has the
+ * layout and element type that oz_residue_gemm writes for `set`. */
+oz_status_t oz_reconstruct(int64_t m, int64_t n, const void *R, int64_t ldr,
                            int64_t mod_stride, const int32_t *shiftA, const int32_t *shiftB,
                            oz_modset_t set, double alpha, double beta, double *C, int64_t ldc,
                            void *stream);

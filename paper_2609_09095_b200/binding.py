@@ -25,7 +25,7 @@ OZ_K_MAX = 32768
 OZ_NONFINITE_SHIFT = -(2 ** 31)
 OZ_STATIC_MAX_LINES = 262144
 
-EXPORTS = ["oz_set_info", "oz_plane_count", "oz_plane_count_side", "oz_row_pitch", "oz_workspace_bytes", "oz_set_workspace", "oz_dgemm",
+EXPORTS = ["oz_set_info", "oz_plane_count", "oz_plane_count_side", "oz_row_pitch", "oz_residue_elem_bytes", "oz_workspace_bytes", "oz_set_workspace", "oz_dgemm",
            "oz_dgemm_ex", "oz_dgemm_host", "oz_deconstruct", "oz_deconstruct_static",
            "oz_residue_gemm", "oz_reconstruct",
            "oz_query_status", "oz_set_stage_events", "oz_launch_count", "oz_status_string"]
@@ -60,6 +60,8 @@ def load() -> C.CDLL:
     lib.oz_plane_count_side.argtypes = [i32, u32, i32]
     lib.oz_row_pitch.argtypes = [i64]
     lib.oz_row_pitch.restype = i64
+    lib.oz_residue_elem_bytes.argtypes = [i32]
+    lib.oz_residue_elem_bytes.restype = C.c_size_t
     lib.oz_workspace_bytes.argtypes = [i64, i64, i64, i32, u32]
     lib.oz_workspace_bytes.restype = C.c_size_t
     lib.oz_set_workspace.argtypes = [vp, C.c_size_t]
@@ -124,6 +126,10 @@ def oz_plane_count_side(modset: int, route: int, side: int) -> int:
 
 def oz_row_pitch(k: int) -> int:
     return load().oz_row_pitch(k)
+
+
+def oz_residue_elem_bytes(modset: int) -> int:
+    return load().oz_residue_elem_bytes(modset)
 
 
 def oz_workspace_bytes(m, n, k, modset, route=0) -> int:

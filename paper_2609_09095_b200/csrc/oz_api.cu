@@ -236,7 +236,7 @@ Layout make_layout(int64_t m, int64_t n, int64_t k, int set, const Route &rt)
     L.pitch = round_up(k > 0 ? k : 1, 128);   // whole 128-byte lines per TMA box row (k = 5003 -> 5120)
     L.strideA = m * L.pitch;
     L.strideB = n * L.pitch;
-    L.ldr = round_up(m, 8);
+    L.ldr = round_up(m, 16 / residue_bytes(set));      // residue rows start on 16-byte boundaries
     L.mod_stride = n * L.ldr;
     L.shiftA = c.take(4 * static_cast<size_t>(m));
     L.shiftB = c.take(4 * static_cast<size_t>(n));
@@ -244,7 +244,7 @@ Layout make_layout(int64_t m, int64_t n, int64_t k, int set, const Route &rt)
     L.scrB = c.take(16 * static_cast<size_t>(n) + 256);
     L.PA = c.take(static_cast<size_t>(p_store(set, rt.layout(0))) * L.strideA);
     L.PB = c.take(static_cast<size_t>(p_store(set, rt.layout(1))) * L.strideB);
-    L.R = c.take(2 * static_cast<size_t>(set_r(set)) * L.mod_stride);
+    L.R = c.take(static_cast<size_t>(residue_bytes(set)) * set_r(set) * L.mod_stride);
     L.total = c.off;
     return L;
 }
@@ -278,7 +278,7 @@ oz_status_t dgemm_impl(int64_t m, int64_t n, int64_t k, double alpha, const doub
     int32_t *shiftB = reinterpret_cast<int32_t *>(ws + L.shiftB);
     uint8_t *PA = reinterpret_cast<uint8_t *>(ws + L.PA);
     uint8_t *PB = reinterpret_cast<uint8_t *>(ws + L.PB);
-    uint16_t *R = reinterpret_cast<uint16_t *>(ws + L.R);
+    void *R = ws + L.R;
 
     const bool ev = g_stage_events_on;
     if (ev) OZ_CUDA_CHECK(cudaEventRecord(g_stage_events[0], stream));
@@ -331,6 +331,11 @@ int oz_plane_count_side(oz_modset_t set, uint32_t route, int side)
 }
 
 int64_t oz_row_pitch(int64_t k) { return round_up(k > 0 ? k : 1, 16); }
+
+size_t oz_residue_elem_bytes(oz_modset_t set)
+{
+    return valid_set(set) ? static_cast<size_t>(residue_bytes(set)) : 0;
+}
 
 size_t oz_workspace_bytes(int64_t m, int64_t n, int64_t k, oz_modset_t set, uint32_t route)
 {
@@ -434,7 +439,7 @@ oz_status_t oz_deconstruct(int side, int64_t lines, int64_t k, const double *X, 
 
 oz_status_t oz_residue_gemm(int64_t m, int64_t n, int64_t k, const uint8_t *PA, int64_t strideA,
                             int64_t pitchA, const uint8_t *PB, int64_t strideB, int64_t pitchB,
-                            oz_modset_t set, uint32_t route, uint16_t *R, int64_t ldr,
+                            oz_modset_t set, uint32_t route, void *R, int64_t ldr,
                             int64_t mod_stride, void *stream)
 {
     Route rt;
@@ -454,7 +459,7 @@ oz_status_t oz_residue_gemm(int64_t m, int64_t n, int64_t k, const uint8_t *PA, 
                                mod_stride, static_cast<cudaStream_t>(stream));
 }
 
-oz_status_t oz_reconstruct(int64_t m, int64_t n, const uint16_t *R, int64_t ldr, int64_t mod_stride,
+oz_status_t oz_reconstruct(int64_t m, int64_t n, const void *R, int64_t ldr, int64_t mod_stride,
                            const int32_t *shiftA, const int32_t *shiftB, oz_modset_t set,
                            double alpha, double beta, double *C, int64_t ldc, void *stream)
 {

@@ -101,7 +101,7 @@ struct GemmParams {
     int vec_store;                  // R rows 16-byte aligned: use vector stores
     int r;
     int64_t total_items;
-    uint16_t *R;
+    void *R;                        // residues: uint16 (RB = 2) or uint8 (RB = 1, byte moduli)
     int64_t ldr, mod_stride;
     unsigned int *status;
     ModInfo mod[kMaxR];
@@ -122,11 +122,6 @@ __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
 {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes)
                  : "memory");
-}
-
-__device__ __forceinline__ void mbar_arrive(uint32_t bar)
-{
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
 
 // cluster-scope acquire: the barriers of the CTA-pair variant are also signalled by the peer CTA
@@ -158,9 +153,17 @@ __device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank)
     return r;
 }
 
-__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr)
+// Arrivals that hand a drained accumulator back to the MMA issuer.  The TMEM reads they follow have
+// already completed (tcgen05.wait::ld) and no memory written by this thread is read by the waiter,
+// so the arrive carries no release: a release would first wait for the residue stores in flight.
+__device__ __forceinline__ void mbar_arrive_relaxed(uint32_t bar)
 {
-    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+    asm volatile("mbarrier.arrive.relaxed.cta.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+
+__device__ __forceinline__ void mbar_arrive_cluster_relaxed(uint32_t cluster_addr)
+{
+    asm volatile("mbarrier.arrive.relaxed.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
 
 // all threads of both CTAs of the pair (no time limit: every thread reaches it on every path)
@@ -318,19 +321,24 @@ __host__ __device__ constexpr uint32_t instr_desc()
 // inside a modulus, bands of 16 tile rows are swept column by column.
 struct Item { int mod, tm, tn; };
 
-__device__ __forceinline__ Item decode_item(int64_t item, const GemmParams &p)
+__device__ __forceinline__ Item decode_item(int64_t item64, const GemmParams &p)
 {
-    constexpr int BAND = 16;
-    int64_t per_mod = static_cast<int64_t>(p.tiles_m) * p.tiles_n;
+    // the host refuses launches with 2^31 or more items: 32-bit divisions are enough
+    constexpr uint32_t BAND = 16;
+    const uint32_t item = static_cast<uint32_t>(item64);
+    const uint32_t tiles_m = static_cast<uint32_t>(p.tiles_m), tiles_n = static_cast<uint32_t>(p.tiles_n);
+    const uint32_t per_mod = tiles_m * tiles_n;
     Item it;
-    it.mod = static_cast<int>(item / per_mod);
-    int64_t t = item - it.mod * per_mod;
-    int64_t band_size = static_cast<int64_t>(BAND) * p.tiles_n;
-    int band = static_cast<int>(t / band_size);
-    int64_t in_band = t - band * band_size;
-    int rows = p.tiles_m - band * BAND < BAND ? p.tiles_m - band * BAND : BAND;
-    it.tn = static_cast<int>(in_band / rows);
-    it.tm = band * BAND + static_cast<int>(in_band - static_cast<int64_t>(it.tn) * rows);
+    const uint32_t mod = item / per_mod;
+    const uint32_t t = item - mod * per_mod;
+    const uint32_t band_size = BAND * tiles_n;
+    const uint32_t band = t / band_size;
+    const uint32_t in_band = t - band * band_size;
+    const uint32_t rows = tiles_m - band * BAND < BAND ? tiles_m - band * BAND : BAND;
+    const uint32_t tn = in_band / rows;
+    it.mod = static_cast<int>(mod);
+    it.tn = static_cast<int>(tn);
+    it.tm = static_cast<int>(band * BAND + (in_band - tn * rows));
     return it;
 }
 
@@ -379,7 +387,8 @@ __device__ __forceinline__ void segment_range(const ModInfo &mi, int job, int se
     }
 }
 
-template <int SUB, int CG>
+// RB: bytes of one stored residue (2: uint16, 1: uint8 for the all-byte modulus set)
+template <int SUB, int CG, int RB>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 residue_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB,
                     const __grid_constant__ GemmParams p)
@@ -584,8 +593,8 @@ residue_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) {
-                    if (CG == 1) mbar_arrive(tempty_bar + 8 * slot);
-                    else mbar_arrive_cluster(map_to_cta(tempty_bar + 8 * slot, 0));   // the leader's barrier
+                    if (CG == 1) mbar_arrive_relaxed(tempty_bar + 8 * slot);
+                    else mbar_arrive_cluster_relaxed(map_to_cta(tempty_bar + 8 * slot, 0));   // the leader's barrier
                 }
                 slot_phase ^= 1u << slot;
                 slot ^= 1;
@@ -596,12 +605,13 @@ residue_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
             const int64_t j = jw + lane;
             const int64_t i0 = static_cast<int64_t>(it.tm) * BLOCK_N + part * COLS_PER_WARP;
             if (i0 >= p.m || jw >= p.n) continue;                                 // warp-uniform
-            uint32_t packed[COLS_PER_WARP / 2];
+            // canonical residues in [0, m), packed 4 / RB to a word in row order
+            uint32_t packed[COLS_PER_WARP * RB / 4];
 #pragma unroll
-            for (int c = 0; c < COLS_PER_WARP; c += 2) {
-                uint32_t bits[2];
+            for (int c = 0; c < COLS_PER_WARP; c += 4) {
+                uint32_t bits[4];
 #pragma unroll
-                for (int h = 0; h < 2; ++h) {
+                for (int h = 0; h < 4; ++h) {
                     if (SUB == 0) {
                         float t = __uint_as_float(comb[c + h]);
                         float quot = fmaf(t, inv_m, 12582912.0f) - 12582912.0f;
@@ -614,40 +624,69 @@ residue_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
                         bits[h] = min(r, r - im);                            // canonical [0, m)
                     }
                 }
-                packed[c >> 1] = __byte_perm(bits[0], bits[1], 0x5410);
+                if constexpr (RB == 2) {
+                    packed[c >> 1] = __byte_perm(bits[0], bits[1], 0x5410);
+                    packed[(c >> 1) + 1] = __byte_perm(bits[2], bits[3], 0x5410);
+                } else {
+                    packed[c >> 2] = __byte_perm(__byte_perm(bits[0], bits[1], 0x0040),
+                                                 __byte_perm(bits[2], bits[3], 0x0040), 0x5410);
+                }
             }
-            uint16_t *rbase = p.R + it.mod * p.mod_stride;
+            unsigned char *rbase = static_cast<unsigned char *>(p.R) + it.mod * p.mod_stride * RB;
             if (p.vec_store && i0 + COLS_PER_WARP <= p.m) {
                 // Transpose through a per-warp shared buffer so that one store instruction writes
-                // four whole 128-byte lines (lane -> line lane/8 + 4t, 16-byte chunk lane%8)
+                // whole lines of the residue array (128 bytes per column for uint16, 64 for uint8)
                 // instead of 32 separate 16-byte pieces.  Chunks are XOR-swizzled by the line
                 // number: both the writes and the reads are free of bank conflicts.
                 unsigned char *xp = xpose_base + (warp - FIRST_EPI_WARP) * XPOSE_BYTES;
+                if constexpr (RB == 2) {
+                    // 16 lines x 128 bytes per pass; lane -> line lane/8 + 4t, 16-byte chunk lane%8
 #pragma unroll
-                for (int rho = 0; rho < 2; ++rho) {
-                    if ((lane >> 4) == rho) {
-                        const int lr = lane & 15;
+                    for (int rho = 0; rho < 2; ++rho) {
+                        if ((lane >> 4) == rho) {
+                            const int lr = lane & 15;
 #pragma unroll
-                        for (int c = 0; c < 8; ++c)
-                            *reinterpret_cast<uint4 *>(xp + lr * 128 + ((c ^ (lr & 7)) << 4)) =
-                                make_uint4(packed[4 * c], packed[4 * c + 1], packed[4 * c + 2], packed[4 * c + 3]);
+                            for (int c = 0; c < 8; ++c)
+                                *reinterpret_cast<uint4 *>(xp + lr * 128 + ((c ^ (lr & 7)) << 4)) =
+                                    make_uint4(packed[4 * c], packed[4 * c + 1], packed[4 * c + 2], packed[4 * c + 3]);
+                        }
+                        __syncwarp();
+#pragma unroll
+                        for (int t = 0; t < 4; ++t) {
+                            const int lr = (lane >> 3) + 4 * t, c = lane & 7;
+                            uint4 val = *reinterpret_cast<const uint4 *>(xp + lr * 128 + ((c ^ (lr & 7)) << 4));
+                            const int64_t jg = jw + 16 * rho + lr;
+                            if (jg < p.n) *reinterpret_cast<uint4 *>(rbase + (jg * p.ldr + i0 + 8 * c) * 2) = val;
+                        }
+                        __syncwarp();
                     }
+                } else {
+                    // 32 lines x 64 bytes in one pass; lane -> line lane/4 + 8t, 16-byte chunk lane%4
+                    constexpr int NCH = COLS_PER_WARP * RB / 16;     // 16-byte chunks per line
+#pragma unroll
+                    for (int c = 0; c < NCH; ++c)
+                        *reinterpret_cast<uint4 *>(xp + lane * 64 + (((c ^ (lane >> 1)) & 3) << 4)) =
+                            make_uint4(packed[4 * c], packed[4 * c + 1], packed[4 * c + 2], packed[4 * c + 3]);
                     __syncwarp();
 #pragma unroll
                     for (int t = 0; t < 4; ++t) {
-                        const int lr = (lane >> 3) + 4 * t, c = lane & 7;
-                        uint4 val = *reinterpret_cast<const uint4 *>(xp + lr * 128 + ((c ^ (lr & 7)) << 4));
-                        const int64_t jg = jw + 16 * rho + lr;
-                        if (jg < p.n) *reinterpret_cast<uint4 *>(rbase + jg * p.ldr + i0 + 8 * c) = val;
+                        const int lr = (lane >> 2) + 8 * t, c = lane & 3;
+                        uint4 val = *reinterpret_cast<const uint4 *>(xp + lr * 64 + (((c ^ (lr >> 1)) & 3) << 4));
+                        const int64_t jg = jw + lr;
+                        if (jg < p.n) *reinterpret_cast<uint4 *>(rbase + jg * p.ldr + i0 + 16 * c) = val;
                     }
                     __syncwarp();
                 }
             } else if (j < p.n) {
-                uint16_t *dst = rbase + j * p.ldr + i0;
+                unsigned char *dst = rbase + (j * p.ldr + i0) * RB;
 #pragma unroll
                 for (int c = 0; c < COLS_PER_WARP; ++c)
-                    if (i0 + c < p.m)
-                        dst[c] = static_cast<uint16_t>((packed[c >> 1] >> (16 * (c & 1))) & 0xFFFFu);
+                    if (i0 + c < p.m) {
+                        if constexpr (RB == 2)
+                            reinterpret_cast<uint16_t *>(dst)[c] = static_cast<uint16_t>((packed[c >> 1] >> (16 * (c & 1))) & 0xFFFFu);
+                        else
+                            dst[c] = static_cast<unsigned char>((packed[c >> 2] >> (8 * (c & 3))) & 0xFFu);
+                    }
             }
         }
     }
@@ -698,11 +737,11 @@ bool make_plane_map(CUtensorMap *map, const uint8_t *base, int64_t lines, int64_
     return rc == CUDA_SUCCESS;
 }
 
-template <int SUB, int CG>
+template <int SUB, int CG, int RB>
 oz_status_t launch_variant(const CUtensorMap &mapA, const CUtensorMap &mapB, const GemmParams &p, int sms,
                            cudaStream_t stream)
 {
-    auto kernel = residue_gemm_kernel<SUB, CG>;
+    auto kernel = residue_gemm_kernel<SUB, CG, RB>;
     OZ_CUDA_CHECK(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        static_cast<int>(SMEM_BYTES)));
     int64_t groups = sms / CG;                                    // CTAs, or CTA pairs
@@ -741,7 +780,7 @@ static int cta_group_choice(int64_t n)
 
 oz_status_t launch_residue_gemm(int64_t m, int64_t n, int64_t k, const uint8_t *PA, int64_t strideA,
                                 int64_t pitchA, const uint8_t *PB, int64_t strideB, int64_t pitchB,
-                                int set, const Route &rt, uint16_t *R, int64_t ldr,
+                                int set, const Route &rt, void *R, int64_t ldr,
                                 int64_t mod_stride, cudaStream_t stream)
 {
     const int cg = cta_group_choice(n);
@@ -749,11 +788,13 @@ oz_status_t launch_residue_gemm(int64_t m, int64_t n, int64_t k, const uint8_t *
     p.m = m; p.n = n; p.k = k;
     p.tiles_m = static_cast<int>((m + BLOCK_N - 1) / BLOCK_N);             // 256 rows of C per tile
     p.tiles_n = static_cast<int>((n + BLOCK_M * cg - 1) / (BLOCK_M * cg)); // 128 (256) columns of C per tile
-    p.vec_store = ((ldr & 7) == 0 && (mod_stride & 7) == 0 && (reinterpret_cast<uintptr_t>(R) & 15u) == 0) ? 1 : 0;
+    const int rb = residue_bytes(set);
+    p.vec_store = ((ldr * rb) % 16 == 0 && (mod_stride * rb) % 16 == 0 && (reinterpret_cast<uintptr_t>(R) & 15u) == 0) ? 1 : 0;
     p.nk = static_cast<int>((k + BLOCK_K - 1) / BLOCK_K);
     if (k == 0) p.nk = 1;   // one all-zero chunk (the planes' padding) gives residues 0
     p.r = set_r(set);
     p.total_items = static_cast<int64_t>(p.r) * p.tiles_m * p.tiles_n;
+    if (p.total_items >= 0x7FFFFFFFll) return OZ_ERR_UNSUPPORTED;        // item numbers are 32-bit in the kernel
     p.R = R; p.ldr = ldr; p.mod_stride = mod_stride;
     p.status = device_status_word();
     for (int i = 0; i < p.r; ++i) {
@@ -827,11 +868,19 @@ oz_status_t launch_residue_gemm(int64_t m, int64_t n, int64_t k, const uint8_t *
     int dev = 0, sms = 148;
     OZ_CUDA_CHECK(cudaGetDevice(&dev));
     OZ_CUDA_CHECK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    // substrate 0: FP8 planes; otherwise INT8 planes (two-limb digits or native residues)
+    if (rb == 1) {
+        if (cg == 2)
+            return rt.substrate == 0 ? launch_variant<0, 2, 1>(mapA, mapB, p, sms, stream)
+                                     : launch_variant<1, 2, 1>(mapA, mapB, p, sms, stream);
+        return rt.substrate == 0 ? launch_variant<0, 1, 1>(mapA, mapB, p, sms, stream)
+                                 : launch_variant<1, 1, 1>(mapA, mapB, p, sms, stream);
+    }
     if (cg == 2)
-        return rt.substrate == 0 ? launch_variant<0, 2>(mapA, mapB, p, sms, stream)
-                                 : launch_variant<1, 2>(mapA, mapB, p, sms, stream);
-    return rt.substrate == 0 ? launch_variant<0, 1>(mapA, mapB, p, sms, stream)
-                             : launch_variant<1, 1>(mapA, mapB, p, sms, stream);   // INT8 two-limb and native
+        return rt.substrate == 0 ? launch_variant<0, 2, 2>(mapA, mapB, p, sms, stream)
+                                 : launch_variant<1, 2, 2>(mapA, mapB, p, sms, stream);
+    return rt.substrate == 0 ? launch_variant<0, 1, 2>(mapA, mapB, p, sms, stream)
+                             : launch_variant<1, 1, 2>(mapA, mapB, p, sms, stream);
 }
 
 }  // namespace oz

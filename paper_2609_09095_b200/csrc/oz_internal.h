@@ -25,6 +25,9 @@ __host__ __device__ constexpr int modulus(int set, int i)
     return set == 0 ? S[i] : (set == 1 ? E[i] : A[i]);
 }
 
+// bytes of one stored residue in [0, m): the moduli of set A fit a byte
+__host__ __device__ constexpr int residue_bytes(int set) { return set == 2 ? 1 : 2; }
+
 // square root of a square modulus, 0 otherwise
 __host__ __device__ constexpr int square_root(int m)
 {
@@ -126,10 +129,10 @@ oz_status_t launch_deconstruct(int side, int64_t lines, int64_t k, const double 
 oz_status_t launch_residue_gemm(int64_t m, int64_t n, int64_t k, const uint8_t *PA,
                                 int64_t strideA, int64_t pitchA, const uint8_t *PB,
                                 int64_t strideB, int64_t pitchB, int set, const Route &rt,
-                                uint16_t *R, int64_t ldr, int64_t mod_stride,
+                                void *R, int64_t ldr, int64_t mod_stride,
                                 cudaStream_t stream);
 
-oz_status_t launch_reconstruct(int64_t m, int64_t n, const uint16_t *R, int64_t ldr,
+oz_status_t launch_reconstruct(int64_t m, int64_t n, const void *R, int64_t ldr,
                                int64_t mod_stride, const int32_t *shiftA, const int32_t *shiftB,
                                int set, double alpha, double beta, double *C, int64_t ldc,
                                cudaStream_t stream);

@@ -45,12 +45,13 @@ __device__ __forceinline__ double scale_pow2(double x, int scale)
     return scalbn(x, scale);        // zero, or a result outside the normal range
 }
 
-// w packs the residues of two consecutive rows (low / high 16 bits); HALF selects the row
+// w packs the residues of consecutive rows (two uint16 or four uint8); HALF selects the row
 template <int SET, int HALF, int I>
 __device__ __forceinline__ void crt_term(uint32_t w, double &S0, double &S1, double &S2)
 {
     const ReconConst &K = c_recon[SET];
-    const uint32_t c = HALF ? (w >> 16) : (w & 0xFFFFu);
+    constexpr int BITS = 8 * residue_bytes(SET);
+    const uint32_t c = (w >> (BITS * HALF)) & ((1u << BITS) - 1u);
     double cd = __hiloint2double(0x43300000, static_cast<int>(c)) - kTwo52;   // exact u32 -> double
     S0 = fma(cd, K.V[I][0], S0);
     S1 = fma(cd, K.V[I][1], S1);
@@ -141,48 +142,18 @@ __device__ __forceinline__ double reconstruct_one(const uint32_t (&c)[kMaxR], in
     return scale_pow2(r, -shift_sum);
 }
 
-template <int SET>
-__global__ void __launch_bounds__(256)
-reconstruct_kernel(const uint16_t *__restrict__ R, int64_t ldr, int64_t mod_stride, int64_t m,
-                   int64_t n, const int32_t *__restrict__ shiftA, const int32_t *__restrict__ shiftB,
-                   double alpha, double beta, double *__restrict__ C, int64_t ldc, int vecR, int vecC)
+// one row of the thread's group: reconstruct, scale by alpha
+template <int SET, int H>
+__device__ __forceinline__ double row_value(const uint32_t (&w)[kMaxR], int sa, int sb, double alpha)
 {
-    // grid.x covers the row pairs of a column, grid.y (and .z beyond 65535) the columns: no division
-    const int64_t row = (blockIdx.x * 256ll + threadIdx.x) * 2;
-    if (row >= m) return;
-    const bool two = row + 1 < m;
-    constexpr int r = set_r(SET);
-    const int64_t j = blockIdx.y + 65535ll * blockIdx.z;
-    if (j >= n) return;
-    {
-
-    // all residue loads are issued before any arithmetic: r independent requests in flight per
-    // thread, kept packed (two rows per word) so that they fit the register budget
-    uint32_t w[kMaxR];
-    const uint16_t *base = R + j * ldr + row;
-#pragma unroll
-    for (int i = 0; i < r; ++i) {
-        if (vecR) {
-            w[i] = *reinterpret_cast<const uint32_t *>(base + i * mod_stride);
-        } else {
-            uint32_t lo = base[i * mod_stride];
-            uint32_t hi = two ? base[i * mod_stride + 1] : 0u;
-            w[i] = lo | (hi << 16);
-        }
-    }
-    int sb = shiftB[j];
-    int sa0 = shiftA[row], sa1 = two ? shiftA[row + 1] : 0;
     const double nan = __longlong_as_double(0x7FF8000000000000ll);
-    double p0 = (sb == OZ_NONFINITE_SHIFT || sa0 == OZ_NONFINITE_SHIFT) ? nan
-                                                                         : reconstruct_one<SET, 0>(w, sa0 + sb);
-    double p1 = 0.0;
-    if (two)
-        p1 = (sb == OZ_NONFINITE_SHIFT || sa1 == OZ_NONFINITE_SHIFT) ? nan
-                                                                      : reconstruct_one<SET, 1>(w, sa1 + sb);
-    p0 *= alpha;
-    p1 *= alpha;
-    double *out = C + row + j * ldc;
-    if (vecC && two) {
+    double p = (sb == OZ_NONFINITE_SHIFT || sa == OZ_NONFINITE_SHIFT) ? nan : reconstruct_one<SET, H>(w, sa + sb);
+    return p * alpha;
+}
+
+__device__ __forceinline__ void store_pair(double *out, double p0, double p1, bool two, bool vec, double beta)
+{
+    if (vec && two) {
         double2 o;
         if (beta != 0.0) {
             double2 old = *reinterpret_cast<const double2 *>(out);
@@ -197,6 +168,61 @@ reconstruct_kernel(const uint16_t *__restrict__ R, int64_t ldr, int64_t mod_stri
         out[0] = beta != 0.0 ? out[0] + p0 : p0;
         if (two) out[1] = beta != 0.0 ? out[1] + p1 : p1;
     }
+}
+
+// Each thread reconstructs ROWS consecutive rows of one column: the residues of those rows are one
+// 32-bit word per modulus (two uint16 for S and E, four uint8 for the all-byte set A).
+template <int SET>
+__global__ void __launch_bounds__(256)
+reconstruct_kernel(const void *__restrict__ Rv, int64_t ldr, int64_t mod_stride, int64_t m,
+                   int64_t n, const int32_t *__restrict__ shiftA, const int32_t *__restrict__ shiftB,
+                   double alpha, double beta, double *__restrict__ C, int64_t ldc, int vecR, int vecC)
+{
+    constexpr int RB = residue_bytes(SET), ROWS = 4 / RB, r = set_r(SET);
+    // grid.x covers the row groups of a column, grid.y (and .z beyond 65535) the columns: no division
+    const int64_t row = (blockIdx.x * 256ll + threadIdx.x) * ROWS;
+    if (row >= m) return;
+    const int64_t j = blockIdx.y + 65535ll * blockIdx.z;
+    if (j >= n) return;
+    const int nrows = m - row < ROWS ? static_cast<int>(m - row) : ROWS;
+
+    // all residue loads are issued before any arithmetic: r independent requests in flight per
+    // thread, kept packed so that they fit the register budget
+    uint32_t w[kMaxR];
+    const unsigned char *base = static_cast<const unsigned char *>(Rv) + (j * ldr + row) * RB;
+#pragma unroll
+    for (int i = 0; i < r; ++i) {
+        const unsigned char *src = base + i * mod_stride * RB;
+        if (vecR) {
+            w[i] = *reinterpret_cast<const uint32_t *>(src);       // ldr is a multiple of ROWS: in bounds
+        } else {
+            uint32_t v = 0;
+#pragma unroll
+            for (int h = 0; h < ROWS; ++h) {
+                if (h < nrows) {
+                    uint32_t e = RB == 2 ? reinterpret_cast<const uint16_t *>(src)[h] : src[h];
+                    v |= e << (8 * RB * h);
+                }
+            }
+            w[i] = v;
+        }
+    }
+    const int sb = shiftB[j];
+    int sa[ROWS];
+#pragma unroll
+    for (int h = 0; h < ROWS; ++h) sa[h] = h < nrows ? shiftA[row + h] : 0;
+    double *out = C + row + j * ldc;
+    {
+        double p0 = row_value<SET, 0>(w, sa[0], sb, alpha);
+        double p1 = nrows > 1 ? row_value<SET, 1>(w, sa[1], sb, alpha) : 0.0;
+        store_pair(out, p0, p1, nrows > 1, vecC != 0, beta);
+    }
+    if constexpr (ROWS == 4) {
+        if (nrows > 2) {
+            double p2 = row_value<SET, 2>(w, sa[2], sb, alpha);
+            double p3 = nrows > 3 ? row_value<SET, 3>(w, sa[3], sb, alpha) : 0.0;
+            store_pair(out + 2, p2, p3, nrows > 3, vecC != 0, beta);
+        }
     }
 }
 
@@ -235,14 +261,16 @@ oz_status_t upload_reconstruct_constants()
     return OZ_OK;
 }
 
-oz_status_t launch_reconstruct(int64_t m, int64_t n, const uint16_t *R, int64_t ldr,
+oz_status_t launch_reconstruct(int64_t m, int64_t n, const void *R, int64_t ldr,
                                int64_t mod_stride, const int32_t *shiftA, const int32_t *shiftB,
                                int set, double alpha, double beta, double *C, int64_t ldc,
                                cudaStream_t stream)
 {
-    int vecR = ((ldr & 1) == 0 && (mod_stride & 1) == 0 && (reinterpret_cast<uintptr_t>(R) & 3u) == 0) ? 1 : 0;
+    // one 32-bit load per modulus covers a thread's rows when every row group starts on a 4-byte boundary
+    const int rows = 4 / residue_bytes(set);
+    int vecR = (ldr % rows == 0 && mod_stride % rows == 0 && (reinterpret_cast<uintptr_t>(R) & 3u) == 0) ? 1 : 0;
     int vecC = ((ldc & 1) == 0 && (reinterpret_cast<uintptr_t>(C) & 15u) == 0) ? 1 : 0;
-    int64_t bx = (((m + 1) >> 1) + 255) / 256;
+    int64_t bx = ((m + rows - 1) / rows + 255) / 256;
     if (bx > 0x7FFFFFFFll) return OZ_ERR_UNSUPPORTED;
     if (n > 65535ll * 65535ll) return OZ_ERR_UNSUPPORTED;
     dim3 grid(static_cast<unsigned>(bx), static_cast<unsigned>(n < 65535 ? n : 65535),

@@ -19,6 +19,11 @@ def route(sub="fp8", quant="RN", rule="CS", acc=None) -> int:
     return r
 
 
+def residue_dtype(set_name: str):
+    """torch / numpy element types of the residue array of a set (uint16, or uint8 for byte moduli)."""
+    return (torch.uint8, np.uint8) if oz.oz_residue_elem_bytes(SETS[set_name]) == 1 else (torch.uint16, np.uint16)
+
+
 def to_dev(X: np.ndarray) -> torch.Tensor:
     """Column-major numpy matrix -> device tensor with the same memory image."""
     assert X.flags.f_contiguous
@@ -55,7 +60,8 @@ def residue_gemm(PA: np.ndarray, PB: np.ndarray, k: int, set_name: str, rt: int,
     r, _, _ = oz.oz_set_info(SETS[set_name])
     ldr = m if ldr is None else ldr
     dA, dB = torch.from_numpy(PA).cuda(), torch.from_numpy(PB).cuda()
-    R = torch.full((r, n, ldr), 0xFFFF, dtype=torch.uint16, device="cuda")
+    tdt, _ = residue_dtype(set_name)
+    R = torch.full((r, n, ldr), 0xFF if tdt == torch.uint8 else 0xFFFF, dtype=tdt, device="cuda")
     oz.check(oz.oz_residue_gemm(m, n, k, dA, m * pa, pa, dB, n * pb, pb, SETS[set_name], rt, R, ldr,
                                 n * ldr), "oz_residue_gemm")
     st = sync_status()
@@ -63,9 +69,17 @@ def residue_gemm(PA: np.ndarray, PB: np.ndarray, k: int, set_name: str, rt: int,
 
 
 def reconstruct(R: np.ndarray, sA: np.ndarray, sB: np.ndarray, set_name: str, alpha=1.0, beta=0.0,
-                C0: np.ndarray | None = None):
+                C0: np.ndarray | None = None, ldr=None):
     r, n, m = R.shape
-    dR = torch.from_numpy(np.ascontiguousarray(R)).cuda()
+    if ldr is not None and ldr != m:
+        Rp = np.full((r, n, ldr), 0xFF, dtype=R.dtype)      # padding rows hold junk that must be ignored
+        Rp[:, :, :m] = R
+        dR = torch.from_numpy(Rp.astype(residue_dtype(set_name)[1])).cuda()
+        dC = to_dev(np.asfortranarray(C0)) if C0 is not None else torch.zeros((n, m), dtype=torch.float64, device="cuda")
+        oz.check(oz.oz_reconstruct(m, n, dR, ldr, n * ldr, torch.from_numpy(sA).cuda(), torch.from_numpy(sB).cuda(),
+                                   SETS[set_name], alpha, beta, dC, m), "oz_reconstruct")
+        return from_dev(dC), sync_status()
+    dR = torch.from_numpy(np.ascontiguousarray(R.astype(residue_dtype(set_name)[1]))).cuda()
     dC = to_dev(np.asfortranarray(C0)) if C0 is not None else torch.zeros((n, m), dtype=torch.float64, device="cuda")
     oz.check(oz.oz_reconstruct(m, n, dR, m, n * m, torch.from_numpy(sA).cuda(), torch.from_numpy(sB).cuda(),
                                SETS[set_name], alpha, beta, dC, m), "oz_reconstruct")

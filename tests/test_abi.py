@@ -36,12 +36,15 @@ def test_host_only_queries():
     assert oz.oz_plane_count(oz.OZ_SET_S, oz.OZ_SUB_INT8_NATIVE) == 0      # native INT8 needs byte moduli
     assert oz.oz_plane_count(oz.OZ_SET_S, 0) == 30 and oz.oz_plane_count(oz.OZ_SET_E, oz.OZ_SUB_INT8) == 33
     assert oz.oz_row_pitch(1) == 16 and oz.oz_row_pitch(5003) == 5008 and oz.oz_row_pitch(4096) == 4096
+    # residues of the all-byte set are stored as bytes
+    assert [oz.oz_residue_elem_bytes(s) for s in (oz.OZ_SET_S, oz.OZ_SET_E, oz.OZ_SET_A, 7)] == [2, 2, 1, 0]
+    assert oz.oz_workspace_bytes(4096, 4096, 512, oz.OZ_SET_A, oz.OZ_SUB_INT8_NATIVE) < 15 * (8192 * 512 + 4096 * 4096) + (1 << 22)
     # planes of A and B + residues dominate the workspace
     m, n, k = 16384, 16384, 1024
     need = oz.oz_workspace_bytes(m, n, k, oz.OZ_SET_S, oz.OZ_ACC_SEPARATE)
     assert need >= 30 * (m + n) * k + 24 * m * n
     assert need < 30 * (m + n) * k + 24 * m * n + (1 << 22)
-    # default route at k <= 4097: merged accumulators, six more planes on the A operand
+    # default route: merged accumulators, six more planes on the A operand
     assert oz.oz_workspace_bytes(m, n, k, oz.OZ_SET_S, 0) == need + 6 * m * k
     assert oz.oz_workspace_bytes(m, n, k, 7, 0) == 0
     assert "workspace" in oz.oz_status_string(oz.OZ_ERR_WORKSPACE)

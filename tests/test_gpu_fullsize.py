@@ -62,8 +62,8 @@ def test_full_size_sampled(cfg_id, set_name, sub):
     scr = torch.empty(16 * max(m, n) + 256, dtype=torch.uint8, device="cuda")
     oz.check(oz.oz_deconstruct(0, m, k, dA, m, gh.SETS[set_name], rt, PA, m * pitch, pitch, shA, scr), "deconstruct A")
     oz.check(oz.oz_deconstruct(1, n, k, dB, k, gh.SETS[set_name], rt, PB, n * pitch, pitch, shB, scr), "deconstruct B")
-    ldr = (m + 7) // 8 * 8
-    R = torch.empty((r, n, ldr), dtype=torch.uint16, device="cuda")
+    ldr = (m + 15) // 16 * 16
+    R = torch.empty((r, n, ldr), dtype=gh.residue_dtype(set_name)[0], device="cuda")
     oz.check(oz.oz_residue_gemm(m, n, k, PA, m * pitch, pitch, PB, n * pitch, pitch, gh.SETS[set_name], rt, R,
                                 ldr, n * ldr), "residue gemm")
     assert gh.sync_status() == 0
@@ -71,7 +71,10 @@ def test_full_size_sampled(cfg_id, set_name, sub):
     assert (shA[ri].cpu().numpy() == sA).all() and (shB[ci].cpu().numpy() == sB).all()
     assert (PA[:, ri, :].cpu().numpy() == PAo).all()
     assert (PB[:, ci, :].cpu().numpy() == PBo).all()
-    Rs = R.view(torch.int16)[:, ci, :][:, :, ri].cpu().numpy().view(np.uint16)   # torch cannot index uint16
+    if R.dtype == torch.uint8:
+        Rs = R[:, ci, :][:, :, ri].cpu().numpy()
+    else:
+        Rs = R.view(torch.int16)[:, ci, :][:, :, ri].cpu().numpy().view(np.uint16)   # torch cannot index uint16
     assert (Rs == Ro).all()
     del PA, PB, R
     torch.cuda.empty_cache()

@@ -191,10 +191,36 @@ def test_accumulation_is_exact_at_depth(k, sub):
     assert (R == want).all()
 
 
+@pytest.mark.parametrize("set_name,sub", [("S", "fp8"), ("A", "int8n"), ("A", "fp8"), ("E", "int8")])
+@pytest.mark.parametrize("m,ldr", [(200, 208), (130, 144), (64, 80), (300, 301)])
+def test_residue_gemm_padded_rows(m, ldr, set_name, sub):
+    """Leading dimension larger than m: aligned paddings take the vector stores with a ragged last
+    tile, an odd one the element-wise path; the padding itself must stay untouched."""
+    import tests.gpu_helpers as gh
+    rng = np.random.default_rng(m + ldr)
+    n, k = 70, 160
+    PA, DA = _random_planes(rng, set_name, sub, m, k)
+    PB, DB = _random_planes(rng, set_name, sub, n, k)
+    import torch
+    import paper_2609_09095_b200 as oz
+    r = len(ozo.modset(OSET[set_name]))
+    tdt, _ = gh.residue_dtype(set_name)
+    fill = 0xFF if tdt == torch.uint8 else 0xFFFF
+    R = torch.full((r, n, ldr), fill, dtype=tdt, device="cuda")
+    dA, dB = torch.from_numpy(PA).cuda(), torch.from_numpy(PB).cuda()
+    oz.check(oz.oz_residue_gemm(m, n, k, dA, m * PA.shape[2], PA.shape[2], dB, n * PB.shape[2], PB.shape[2],
+                                gh.SETS[set_name], gh.route(sub), R, ldr, n * ldr), "oz_residue_gemm")
+    assert gh.sync_status() == 0
+    Rh = R.cpu().numpy()
+    assert (Rh[:, :, :m] == ozo.products(DA, DB, OSET[set_name])).all()
+    assert (Rh[:, :, m:] == fill).all()
+
+
 # ------------------------------------------------------------------ reconstruction (a7)
 @pytest.mark.parametrize("set_name", ["S", "E", "A"])
-@pytest.mark.parametrize("m,n", [(256, 64), (1, 1), (7, 5), (130, 3)])
-def test_reconstruct_bit_exact(set_name, m, n):
+@pytest.mark.parametrize("m,n,ldr", [(256, 64, None), (1, 1, None), (7, 5, None), (130, 3, None), (258, 9, 272),
+                                     (131, 4, 132), (5, 3, 8), (259, 2, 261)])
+def test_reconstruct_bit_exact(set_name, m, n, ldr):
     import tests.gpu_helpers as gh
     rng = np.random.default_rng(m + n)
     ms = ozo.modset(OSET[set_name])
@@ -212,7 +238,7 @@ def test_reconstruct_bit_exact(set_name, m, n):
     C0 = np.asfortranarray(rng.standard_normal((m, n)))
     CI = ozo.crt(R, OSET[set_name])
     for alpha, beta in ((1.0, 0.0), (-1.0, 1.0), (-1.0, 0.0), (1.0, 1.0)):
-        got, st = gh.reconstruct(R, sA, sB, set_name, alpha, beta, C0)
+        got, st = gh.reconstruct(R, sA, sB, set_name, alpha, beta, C0, ldr=ldr)
         want = ozo.output(CI, sA, sB, alpha, beta, C0)
         assert st == 0
         assert (got == want).all()
