@@ -295,6 +295,25 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32])
     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
 
+// same load without the wait, into v[OFF .. OFF+31]
+template <int OFF>
+__device__ __forceinline__ void tmem_ld32_issue(uint32_t taddr, uint32_t (&v)[64])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(v[OFF + 0]), "=r"(v[OFF + 1]), "=r"(v[OFF + 2]), "=r"(v[OFF + 3]), "=r"(v[OFF + 4]),
+          "=r"(v[OFF + 5]), "=r"(v[OFF + 6]), "=r"(v[OFF + 7]), "=r"(v[OFF + 8]), "=r"(v[OFF + 9]),
+          "=r"(v[OFF + 10]), "=r"(v[OFF + 11]), "=r"(v[OFF + 12]), "=r"(v[OFF + 13]), "=r"(v[OFF + 14]),
+          "=r"(v[OFF + 15]), "=r"(v[OFF + 16]), "=r"(v[OFF + 17]), "=r"(v[OFF + 18]), "=r"(v[OFF + 19]),
+          "=r"(v[OFF + 20]), "=r"(v[OFF + 21]), "=r"(v[OFF + 22]), "=r"(v[OFF + 23]), "=r"(v[OFF + 24]),
+          "=r"(v[OFF + 25]), "=r"(v[OFF + 26]), "=r"(v[OFF + 27]), "=r"(v[OFF + 28]), "=r"(v[OFF + 29]),
+          "=r"(v[OFF + 30]), "=r"(v[OFF + 31])
+        : "r"(taddr)
+        : "memory");
+}
+
 // shared-memory matrix descriptor: K-major operand, 128-byte swizzle, 8-row groups 1024 B apart
 __device__ __forceinline__ uint64_t smem_desc(uint32_t addr)
 {
@@ -388,7 +407,9 @@ __device__ __forceinline__ void segment_range(const ModInfo &mi, int job, int se
 }
 
 // RB: bytes of one stored residue (2: uint16, 1: uint8 for the all-byte modulus set)
-template <int SUB, int CG, int RB>
+// DIRECT: native INT8 residues -- one accumulator per modulus, loaded straight into the registers
+//         that otherwise hold the running combination of several accumulators
+template <int SUB, int CG, int RB, bool DIRECT>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 residue_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB,
                     const __grid_constant__ GemmParams p)
@@ -541,8 +562,12 @@ residue_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
             const uint32_t im = mi.mi, imagic = mi.magic, ibias = mi.bias;
             // running combination per element: FP32 (FP8 route) or INT32 (INT8 routes), as raw bits
             uint32_t comb[COLS_PER_WARP];
+            if constexpr (!DIRECT) {
 #pragma unroll
-            for (int c = 0; c < COLS_PER_WARP; ++c) comb[c] = 0u;
+                for (int c = 0; c < COLS_PER_WARP; ++c) comb[c] = 0u;
+            }
+            // canonical residues in [0, m), packed 4 / RB to a word in row order
+            uint32_t packed[COLS_PER_WARP * RB / 4];
             for (int job = 0; ok && job < mi.njobs; ++job)
             for (int seg = 0, nseg = job_segments(mi, job); ok && seg < nseg; ++seg) {
                 ok = mbar_wait(tfull_bar + 8 * slot, (slot_phase >> slot) & 1u, abort_flag, p.status);
@@ -552,11 +577,17 @@ residue_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
                 const bool reduce_first = mi.reduce[job] != 0;
                 const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) +
                                        static_cast<uint32_t>(slot * BLOCK_N + part * COLS_PER_WARP);
+                if constexpr (DIRECT) {
+                    // the only accumulator of this modulus lands in the combination registers as it is
+                    tmem_ld32_issue<0>(taddr, comb);
+                    tmem_ld32_issue<32>(taddr + 32, comb);
+                    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                } else
 #pragma unroll
                 for (int c0 = 0; c0 < COLS_PER_WARP; c0 += 32) {
                     uint32_t v[32];
                     tmem_ld32(taddr + c0, v);
-                    if (SUB == 0) {
+                    if constexpr (SUB == 0) {
                         if (reduce_first) {
 #pragma unroll
                             for (int e = 0; e < 32; ++e) {
@@ -605,8 +636,6 @@ residue_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
             const int64_t j = jw + lane;
             const int64_t i0 = static_cast<int64_t>(it.tm) * BLOCK_N + part * COLS_PER_WARP;
             if (i0 >= p.m || jw >= p.n) continue;                                 // warp-uniform
-            // canonical residues in [0, m), packed 4 / RB to a word in row order
-            uint32_t packed[COLS_PER_WARP * RB / 4];
 #pragma unroll
             for (int c = 0; c < COLS_PER_WARP; c += 4) {
                 uint32_t bits[4];
@@ -737,11 +766,11 @@ bool make_plane_map(CUtensorMap *map, const uint8_t *base, int64_t lines, int64_
     return rc == CUDA_SUCCESS;
 }
 
-template <int SUB, int CG, int RB>
+template <int SUB, int CG, int RB, bool DIRECT = false>
 oz_status_t launch_variant(const CUtensorMap &mapA, const CUtensorMap &mapB, const GemmParams &p, int sms,
                            cudaStream_t stream)
 {
-    auto kernel = residue_gemm_kernel<SUB, CG, RB>;
+    auto kernel = residue_gemm_kernel<SUB, CG, RB, DIRECT>;
     OZ_CUDA_CHECK(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        static_cast<int>(SMEM_BYTES)));
     int64_t groups = sms / CG;                                    // CTAs, or CTA pairs
@@ -869,6 +898,9 @@ oz_status_t launch_residue_gemm(int64_t m, int64_t n, int64_t k, const uint8_t *
     OZ_CUDA_CHECK(cudaGetDevice(&dev));
     OZ_CUDA_CHECK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
     // substrate 0: FP8 planes; otherwise INT8 planes (two-limb digits or native residues)
+    if (rt.native())
+        return cg == 2 ? launch_variant<1, 2, 1, true>(mapA, mapB, p, sms, stream)
+                       : launch_variant<1, 1, 1, true>(mapA, mapB, p, sms, stream);
     if (rb == 1) {
         if (cg == 2)
             return rt.substrate == 0 ? launch_variant<0, 2, 1>(mapA, mapB, p, sms, stream)
