@@ -172,8 +172,10 @@ __device__ __forceinline__ void store_pair(double *out, double p0, double p1, bo
 
 // Each thread reconstructs ROWS consecutive rows of one column: the residues of those rows are one
 // 32-bit word per modulus (two uint16 for S and E, four uint8 for the all-byte set A).
+// Six blocks per SM (40 registers) for the two-byte sets: the kernel is bound by instruction issue
+// and gains from the extra warps; the four-row variant of set A would spill at that budget.
 template <int SET>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(256, residue_bytes(SET) == 2 ? 6 : 5)
 reconstruct_kernel(const void *__restrict__ Rv, int64_t ldr, int64_t mod_stride, int64_t m,
                    int64_t n, const int32_t *__restrict__ shiftA, const int32_t *__restrict__ shiftB,
                    double alpha, double beta, double *__restrict__ C, int64_t ldc, int vecR, int vecC)
