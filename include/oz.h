@@ -125,10 +125,15 @@ oz_status_t oz_dgemm_ex(int64_t m, int64_t n, int64_t k, double alpha, const dou
                         int64_t lda, const double *B, int64_t ldb, double beta, double *C,
                         int64_t ldc, oz_modset_t set, uint32_t route, void *stream);
 
-/* Same as oz_dgemm_ex but A, B, C are HOST pointers (pinned memory recommended).  The operands
- * are copied to staging areas inside the registered workspace, which must hold
- * oz_workspace_bytes() + 8 (m k + k n + m n) bytes, and C is copied back; the call returns after
- * enqueueing (the host buffers must stay valid until the stream has drained). */
+/* Same as oz_dgemm_ex but A, B, C are HOST pointers (pinned memory recommended: copies from
+ * pageable memory do not overlap anything).  The operands are copied to staging areas inside the
+ * registered workspace, which must hold oz_workspace_bytes() + 8 (m k + k n + m n) bytes, and C is
+ * copied back; the call returns after enqueueing (the host buffers must stay valid until the stream
+ * has drained).  When C is 128 MiB or more it travels in up to 16 column panels on two internal
+ * streams: its upload overlaps the deconstruction and the residue GEMMs, and each panel is downloaded
+ * while later ones are still uploaded and reconstructed.  `stream` waits for those internal streams,
+ * so work enqueued on it afterwards, or a synchronisation of it, sees the finished C.  The internal
+ * streams and events are created on a device's first such call (not inside a stream capture). */
 oz_status_t oz_dgemm_host(int64_t m, int64_t n, int64_t k, double alpha, const double *A_host,
                           int64_t lda, const double *B_host, int64_t ldb, double beta,
                           double *C_host, int64_t ldc, oz_modset_t set, uint32_t route,

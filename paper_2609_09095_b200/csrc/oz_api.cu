@@ -251,9 +251,21 @@ Layout make_layout(int64_t m, int64_t n, int64_t k, int set, const Route &rt)
 
 bool valid_set(int set) { return set == OZ_SET_S || set == OZ_SET_E || set == OZ_SET_A; }
 
+// Optional split of the reconstruction into column panels, used by the host-buffer entry point to
+// overlap the transfers of C with the computation: before panel p the stream waits for before[p]
+// (when wait_before), after it the stream records after[p].
+constexpr int kMaxPanels = 16;
+struct PanelPlan {
+    int np;
+    int64_t col0[kMaxPanels + 1];
+    bool wait_before;
+    cudaEvent_t *before, *after;
+};
+
 oz_status_t dgemm_impl(int64_t m, int64_t n, int64_t k, double alpha, const double *A, int64_t lda,
                        const double *B, int64_t ldb, double beta, double *C, int64_t ldc, int set,
-                       uint32_t route, cudaStream_t stream, char *ws, size_t ws_bytes)
+                       uint32_t route, cudaStream_t stream, char *ws, size_t ws_bytes,
+                       const PanelPlan *plan = nullptr)
 {
     Route rt;
     if (!valid_set(set) || !decode_route_for_set(set, route, &rt)) return OZ_ERR_INVALID_ARG;
@@ -292,10 +304,49 @@ oz_status_t dgemm_impl(int64_t m, int64_t n, int64_t k, double alpha, const doub
                              L.ldr, L.mod_stride, stream);
     if (st != OZ_OK) return st;
     if (ev) OZ_CUDA_CHECK(cudaEventRecord(g_stage_events[3], stream));
-    st = launch_reconstruct(m, n, R, L.ldr, L.mod_stride, shiftA, shiftB, set, alpha, beta, C, ldc,
-                            stream);
-    if (st != OZ_OK) return st;
+    if (!plan) {
+        st = launch_reconstruct(m, n, R, L.ldr, L.mod_stride, shiftA, shiftB, set, alpha, beta, C, ldc,
+                                stream);
+        if (st != OZ_OK) return st;
+    } else {
+        for (int p = 0; p < plan->np; ++p) {
+            const int64_t j0 = plan->col0[p], cols = plan->col0[p + 1] - j0;
+            if (plan->wait_before) OZ_CUDA_CHECK(cudaStreamWaitEvent(stream, plan->before[p], 0));
+            st = launch_reconstruct(m, cols, static_cast<char *>(R) + j0 * L.ldr * residue_bytes(set), L.ldr,
+                                    L.mod_stride, shiftA, shiftB + j0, set, alpha, beta, C + j0 * ldc, ldc,
+                                    stream);
+            if (st != OZ_OK) return st;
+            OZ_CUDA_CHECK(cudaEventRecord(plan->after[p], stream));
+        }
+    }
     if (ev) OZ_CUDA_CHECK(cudaEventRecord(g_stage_events[4], stream));
+    return OZ_OK;
+}
+
+// Side streams and events of the host-buffer entry point, created once per device.
+struct HostPipe {
+    bool ready;
+    cudaStream_t in, out;
+    cudaEvent_t start, ab, done, c[kMaxPanels], r[kMaxPanels];
+};
+HostPipe g_pipe[kMaxDevices];
+
+oz_status_t ensure_pipe(int dev, HostPipe **out)
+{
+    std::lock_guard<std::mutex> lock(g_mutex);
+    HostPipe &hp = g_pipe[dev];
+    if (!hp.ready) {
+        OZ_CUDA_CHECK(cudaStreamCreateWithFlags(&hp.in, cudaStreamNonBlocking));
+        OZ_CUDA_CHECK(cudaStreamCreateWithFlags(&hp.out, cudaStreamNonBlocking));
+        cudaEvent_t *single[3] = {&hp.start, &hp.ab, &hp.done};
+        for (cudaEvent_t *e : single) OZ_CUDA_CHECK(cudaEventCreateWithFlags(e, cudaEventDisableTiming));
+        for (int p = 0; p < kMaxPanels; ++p) {
+            OZ_CUDA_CHECK(cudaEventCreateWithFlags(&hp.c[p], cudaEventDisableTiming));
+            OZ_CUDA_CHECK(cudaEventCreateWithFlags(&hp.r[p], cudaEventDisableTiming));
+        }
+        hp.ready = true;
+    }
+    *out = &hp;
     return OZ_OK;
 }
 
@@ -402,6 +453,49 @@ oz_status_t oz_dgemm_host(int64_t m, int64_t n, int64_t k, double alpha, const d
     double *dA = reinterpret_cast<double *>(ws + offA);
     double *dB = reinterpret_cast<double *>(ws + offB);
     double *dC = reinterpret_cast<double *>(ws + offC);
+    // Large outputs: C travels in column panels on two side streams, so that its upload overlaps
+    // the deconstruction and the residue GEMMs, and the download of a finished panel overlaps the
+    // upload and the reconstruction of the next ones (PCIe is full duplex).  The caller's stream
+    // waits for both side streams before the call's work counts as done on it.
+    int np = static_cast<int>(bytesC >> 26);                 // panels of at least 64 MiB
+    if (np > kMaxPanels) np = kMaxPanels;
+    if (np > n) np = static_cast<int>(n);
+    if (k > 0 && np >= 2) {
+        HostPipe *hp = nullptr;
+        oz_status_t pst = ensure_pipe(dev, &hp);
+        if (pst != OZ_OK) return pst;
+        PanelPlan plan{};
+        plan.np = np;
+        for (int p = 0; p <= np; ++p) plan.col0[p] = n * p / np;
+        plan.wait_before = beta != 0.0;
+        plan.before = hp->c;
+        plan.after = hp->r;
+        OZ_CUDA_CHECK(cudaEventRecord(hp->start, s));          // the workspace may still be in use on s
+        OZ_CUDA_CHECK(cudaStreamWaitEvent(hp->in, hp->start, 0));
+        OZ_CUDA_CHECK(cudaStreamWaitEvent(hp->out, hp->start, 0));
+        OZ_CUDA_CHECK(cudaMemcpy2DAsync(dA, 8 * m, A_host, 8 * lda, 8 * m, k, cudaMemcpyHostToDevice, hp->in));
+        OZ_CUDA_CHECK(cudaMemcpy2DAsync(dB, 8 * k, B_host, 8 * ldb, 8 * k, n, cudaMemcpyHostToDevice, hp->in));
+        OZ_CUDA_CHECK(cudaEventRecord(hp->ab, hp->in));
+        if (beta != 0.0)
+            for (int p = 0; p < np; ++p) {
+                const int64_t j0 = plan.col0[p], cols = plan.col0[p + 1] - j0;
+                OZ_CUDA_CHECK(cudaMemcpy2DAsync(dC + j0 * m, 8 * m, C_host + j0 * ldc, 8 * ldc, 8 * m, cols,
+                                                cudaMemcpyHostToDevice, hp->in));
+                OZ_CUDA_CHECK(cudaEventRecord(hp->c[p], hp->in));
+            }
+        OZ_CUDA_CHECK(cudaStreamWaitEvent(s, hp->ab, 0));
+        oz_status_t st = dgemm_impl(m, n, k, alpha, dA, m, dB, kk, beta, dC, m, set, route, s, ws, core, &plan);
+        if (st != OZ_OK) return st;
+        for (int p = 0; p < np; ++p) {
+            const int64_t j0 = plan.col0[p], cols = plan.col0[p + 1] - j0;
+            OZ_CUDA_CHECK(cudaStreamWaitEvent(hp->out, hp->r[p], 0));
+            OZ_CUDA_CHECK(cudaMemcpy2DAsync(C_host + j0 * ldc, 8 * ldc, dC + j0 * m, 8 * m, 8 * m, cols,
+                                            cudaMemcpyDeviceToHost, hp->out));
+        }
+        OZ_CUDA_CHECK(cudaEventRecord(hp->done, hp->out));
+        OZ_CUDA_CHECK(cudaStreamWaitEvent(s, hp->done, 0));
+        return OZ_OK;
+    }
     if (k > 0) {
         OZ_CUDA_CHECK(cudaMemcpy2DAsync(dA, 8 * m, A_host, 8 * lda, 8 * m, k, cudaMemcpyHostToDevice, s));
         OZ_CUDA_CHECK(cudaMemcpy2DAsync(dB, 8 * k, B_host, 8 * ldb, 8 * k, n, cudaMemcpyHostToDevice, s));

@@ -318,3 +318,46 @@ def test_argument_errors_are_reported_on_the_host():
     oz.oz_set_workspace(None)
     assert oz.oz_dgemm(4, 4, 4, t, 4, t, 4, t, 4) == oz.OZ_ERR_WORKSPACE
     assert oz.oz_dgemm(0, 4, 4, t, 4, t, 4, t, 4) == oz.OZ_OK
+
+
+# ------------------------------------------------------------------ host-buffer entry point
+@pytest.mark.parametrize("m,n,k,alpha,beta,set_name,sub", [
+    (200, 300, 260, 1.0, 0.0, "S", "fp8"),          # small: one sequential upload / download
+    (4096, 4224, 96, -1.0, 1.0, "S", "fp8"),        # 138 MB of C: two column panels on side streams
+    (4100, 8200, 40, 1.0, 0.0, "A", "int8n"),       # four panels, ragged, no upload of C
+    (3000, 11200, 24, 1.0, 1.0, "E", "fp8"),        # four panels of unequal width
+])
+def test_dgemm_host_buffers(m, n, k, alpha, beta, set_name, sub):
+    """oz_dgemm_host (pinned host operands, copies inside, C in column panels when it is large) against
+    the oracle on sampled rows and columns and bit for bit against the device-pointer entry point."""
+    import torch
+    import paper_2609_09095_b200 as oz
+    import tests.gpu_helpers as gh
+    rng = np.random.default_rng(m + n + k)
+    A = np.asfortranarray(rng.uniform(-1, 1, size=(m, k)))
+    B = np.asfortranarray(rng.standard_normal((k, n)))
+    C0 = np.asfortranarray(rng.standard_normal((m, n)))
+    lda, ldb, ldc = m + 3, k + 1, m + 5
+    hA = torch.zeros((k, lda), dtype=torch.float64).pin_memory()
+    hB = torch.zeros((n, ldb), dtype=torch.float64).pin_memory()
+    hC = torch.full((n, ldc), 5.0, dtype=torch.float64).pin_memory()
+    hA[:, :m] = torch.from_numpy(np.ascontiguousarray(A.T))
+    hB[:, :k] = torch.from_numpy(np.ascontiguousarray(B.T))
+    hC[:, :m] = torch.from_numpy(np.ascontiguousarray(C0.T))
+    rt = gh.route(sub)
+    need = oz.oz_workspace_bytes(m, n, k, gh.SETS[set_name], rt) + 8 * (m * k + k * n + m * n) + 1024
+    gh.ensure_workspace(need)
+    for _ in range(2):                                  # twice: the side streams and events are reused
+        hC[:, :m] = torch.from_numpy(np.ascontiguousarray(C0.T))
+        oz.check(oz.oz_dgemm_host(m, n, k, alpha, hA, lda, hB, ldb, beta, hC, ldc, gh.SETS[set_name], rt),
+                 "oz_dgemm_host")
+        assert gh.sync_status() == 0
+        got = hC.numpy().T
+        assert (got[m:, :] == 5.0).all()                # rows beyond m of the host array are untouched
+        dev, st = gh.dgemm(A, B, set_name, rt, alpha, beta, C0 if beta else None)
+        assert st == 0 and (got[:m, :] == dev).all()
+    rows = np.unique(rng.integers(0, m, size=48))
+    cols = np.unique(np.concatenate([rng.integers(0, n, size=48), [0, n - 1, n // 2 - 1, n // 2]]))
+    want = ozo.dgemm(np.asfortranarray(A[rows, :]), np.asfortranarray(B[:, cols]), OSET[set_name], ozo.QUANT_RN,
+                     ozo.SCALE_CS, alpha, beta, np.asfortranarray(C0[np.ix_(rows, cols)]) if beta else None)
+    assert (got[np.ix_(rows, cols)] == want).all()
