@@ -28,8 +28,11 @@
  *   - m, n or k equal to zero is OZ_OK (k = 0 gives C = 0, or C unchanged for beta = 1).
  *   - Non-finite contract: an Inf or NaN anywhere in row i of A (column j of B)
  *     makes every C(i,:) (C(:,j)) NaN and sets OZ_ERR_NONFINITE_INPUT.
- *   - k is limited to OZ_K_MAX, the depth to which the FP32 accumulators of the FP8
- *     route stay exact (Lemma 1 and the accumulation invariant of Algorithm 2).
+ *   - One FP32 accumulator of the FP8 route stays exact to k = 32768 (Lemma 1 and the accumulation
+ *     invariant of Algorithm 2), an INT32 one to 131071 (native residues) or 4 million (digits).
+ *     A longer k is split inside the residue-GEMM kernel into K segments with an accumulator each,
+ *     reduced modulo m_i and added in the residue domain; the shifts are those of the whole k.
+ *     k is limited to OZ_K_MAX.
  */
 #ifndef OZ_H_
 #define OZ_H_
@@ -81,7 +84,7 @@ typedef enum { OZ_SET_S = 0, OZ_SET_E = 1, OZ_SET_A = 2 } oz_modset_t;
 #define OZ_ACC_MERGED   0x1000u
 #define OZ_ACC_SEPARATE 0x2000u
 
-#define OZ_K_MAX 32768
+#define OZ_K_MAX 1048576
 #define OZ_NONFINITE_SHIFT INT32_MIN  /* value of shift[] for a line that holds Inf/NaN */
 
 /* Number of moduli r and of stored planes p_store of a set (Table "tuples": 12/30, 13/33).

@@ -21,7 +21,7 @@ OZ_SUB_FP8, OZ_SUB_INT8, OZ_SUB_INT8_NATIVE = 0x001, 0x002, 0x004
 OZ_QUANT_RN, OZ_QUANT_TZ = 0x010, 0x020
 OZ_SCALE_MAXEXP, OZ_SCALE_CS = 0x100, 0x200
 OZ_ACC_MERGED, OZ_ACC_SEPARATE = 0x1000, 0x2000
-OZ_K_MAX = 32768
+OZ_K_MAX = 1048576
 OZ_NONFINITE_SHIFT = -(2 ** 31)
 OZ_STATIC_MAX_LINES = 262144
 

@@ -86,8 +86,12 @@ struct ModInfo {
     int njobs;            // 2 (square), 3, 1 (native INT8 residues) or 2 (non-square, merged accumulators)
     int kind;             // 0 square, 1 non-square separate, 2 native, 3 non-square merged
     int planeA0, planeB0; // first stored plane of this modulus in A's and in B's plane arrays
-    int nseg, seg_len;    // merged job 0 only: the K range is cut into nseg segments of seg_len chunks, each
-                          // with an accumulator of its own, so that every FP32 accumulator stays exact
+    // Split-K inside the kernel: the K range of a job is cut into segments of whole chunks, each with
+    // an accumulator of its own that is reduced before the next is added, so that every accumulator
+    // stays exact.  nseg / seg_len: job 0 of the merged schedule (depth 4097 or 15420);
+    // nseg_all / seg_len_all: every other job (depth 32768 in FP32; 2^31 / term size in INT32).
+    int nseg, seg_len;
+    int nseg_all, seg_len_all;
     // integer epilogue of the INT8 routes (INT32 accumulators):
     int iw[3];            // weights as integers
     uint32_t mi;          // the modulus
@@ -391,19 +395,15 @@ __device__ __forceinline__ int job_pairs(const ModInfo &mi, int job)
 // accumulators (K segments) of job `job`
 __device__ __forceinline__ int job_segments(const ModInfo &mi, int job)
 {
-    return (mi.kind == 3 && job == 0) ? mi.nseg : 1;
+    return (mi.kind == 3 && job == 0) ? mi.nseg : mi.nseg_all;
 }
 
 // chunk range [kc0, kc1) of segment `seg`
 __device__ __forceinline__ void segment_range(const ModInfo &mi, int job, int seg, int nk, int *kc0, int *kc1)
 {
-    if (mi.kind == 3 && job == 0) {
-        *kc0 = seg * mi.seg_len;
-        *kc1 = min(nk, *kc0 + mi.seg_len);
-    } else {
-        *kc0 = 0;
-        *kc1 = nk;
-    }
+    const int len = (mi.kind == 3 && job == 0) ? mi.seg_len : mi.seg_len_all;
+    *kc0 = seg * len;
+    *kc1 = min(nk, *kc0 + len);
 }
 
 // RB: bytes of one stored residue (2: uint16, 1: uint8 for the all-byte modulus set)
@@ -846,18 +846,25 @@ oz_status_t launch_residue_gemm(int64_t m, int64_t n, int64_t k, const uint8_t *
         mo.planeB0 = first_plane(set, i, rt.layout(1));
         mo.nseg = 1;
         mo.seg_len = p.nk;
+        // exact depth of one accumulator, in chunks of BLOCK_K: the largest term is 2 * 16 * 16 (the
+        // two-product job of a square), 128 * 128 for native residues
+        const int seg_max_all = !integer ? (1 << 24) / 512 / BLOCK_K
+                                         : static_cast<int>(((1ll << 31) - 1) / (rt.native() ? 16384 : 512) / BLOCK_K);
+        mo.nseg_all = (p.nk + seg_max_all - 1) / seg_max_all;
+        mo.seg_len_all = (p.nk + mo.nseg_all - 1) / mo.nseg_all;
+        const bool split = mo.nseg_all > 1;       // then every accumulator is reduced before it is weighted
         if (rt.native()) {
             mo.njobs = 1;
             mo.kind = 2;
             mo.w[0] = 1.0f; mo.w[1] = mo.w[2] = 0.0f;
-            mo.reduce[0] = (128 * 128 * kk <= lim) ? 0 : 1;
+            mo.reduce[0] = split ? 1 : 0;
             mo.reduce[1] = mo.reduce[2] = 1;
         } else if (s) {
             mo.njobs = 2;
             mo.kind = 0;
             mo.w[0] = 1.0f; mo.w[1] = static_cast<float>(s); mo.w[2] = 0.0f;
-            const bool skip_all = integer && (256 + 512 * static_cast<int64_t>(s)) * kk <= lim;
-            mo.reduce[0] = (skip_all || 256 * kk + static_cast<int64_t>(s) * red <= lim) ? 0 : 1;
+            const bool skip_all = !split && integer && (256 + 512 * static_cast<int64_t>(s)) * kk <= lim;
+            mo.reduce[0] = (skip_all || (!split && 256 * kk + static_cast<int64_t>(s) * red <= lim)) ? 0 : 1;
             mo.reduce[1] = skip_all ? 0 : 1;
             mo.reduce[2] = 1;
         } else if (rt.merged()) {
@@ -872,16 +879,16 @@ oz_status_t launch_residue_gemm(int64_t m, int64_t n, int64_t k, const uint8_t *
             mo.nseg = (p.nk + seg_max - 1) / seg_max;
             if (mo.nseg < 1) mo.nseg = 1;
             mo.seg_len = (p.nk + mo.nseg - 1) / mo.nseg;
-            const bool skip_all = mo.nseg == 1 && (15 * merged_term + 16 * 484) * kk <= lim;
+            const bool skip_all = !split && mo.nseg == 1 && (15 * merged_term + 16 * 484) * kk <= lim;
             mo.reduce[0] = skip_all ? 0 : 1;
-            mo.reduce[1] = (skip_all || 16 * 484 * kk + 15 * red * mo.nseg <= lim) ? 0 : 1;
+            mo.reduce[1] = (skip_all || (!split && 16 * 484 * kk + 15 * red * mo.nseg <= lim)) ? 0 : 1;
             mo.reduce[2] = 1;
         } else {
             mo.njobs = 3;
             mo.kind = 1;
             mo.w[0] = -15.0f; mo.w[1] = 16.0f; mo.w[2] = 240.0f;
-            const bool skip_all = integer && (15 * 196 + 16 * 484 + 240 * 256) * kk <= lim;
-            const bool skip01 = skip_all || (15 * 196 + 16 * 484) * kk + 240 * red <= lim;
+            const bool skip_all = !split && integer && (15 * 196 + 16 * 484 + 240 * 256) * kk <= lim;
+            const bool skip01 = skip_all || (!split && (15 * 196 + 16 * 484) * kk + 240 * red <= lim);
             mo.reduce[0] = skip01 ? 0 : 1;
             mo.reduce[1] = skip01 ? 0 : 1;
             mo.reduce[2] = skip_all ? 0 : 1;
@@ -898,7 +905,7 @@ oz_status_t launch_residue_gemm(int64_t m, int64_t n, int64_t k, const uint8_t *
     OZ_CUDA_CHECK(cudaGetDevice(&dev));
     OZ_CUDA_CHECK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
     // substrate 0: FP8 planes; otherwise INT8 planes (two-limb digits or native residues)
-    if (rt.native())
+    if (rt.native() && p.mod[0].nseg_all == 1)      // one accumulator per modulus: the direct drain
         return cg == 2 ? launch_variant<1, 2, 1, true>(mapA, mapB, p, sms, stream)
                        : launch_variant<1, 1, 1, true>(mapA, mapB, p, sms, stream);
     if (rb == 1) {

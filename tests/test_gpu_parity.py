@@ -216,6 +216,39 @@ def test_residue_gemm_padded_rows(m, ldr, set_name, sub):
     assert (Rh[:, :, m:] == fill).all()
 
 
+@pytest.mark.parametrize("k,set_name,sub,acc", [(40000, "S", "fp8", "separate"), (70001, "E", "fp8", "separate"),
+                                                (40000, "S", "fp8", "merged"), (140000, "A", "int8n", None),
+                                                (66000, "S", "int8", None)])
+def test_split_k_beyond_one_accumulator(k, set_name, sub, acc):
+    """k beyond the exact depth of one accumulator (32768 in FP32, 131071 for native INT8 residues): the
+    kernel cuts K into segments and adds their reduced results modulo m.  Largest digits, constant
+    rows: a single accumulator over all of K would overflow."""
+    import tests.gpu_helpers as gh
+    rng = np.random.default_rng(k)
+    m, n = 40, 24
+    _, DA = _random_planes(rng, set_name, sub, m, k, extreme=True)
+    _, DB = _random_planes(rng, set_name, sub, n, k, extreme=True)
+    DA[:, :8, :] = DA[:, :1, :1]
+    DB[:, :8, :] = DB[:, :1, :1]
+    if acc == "merged":
+        PA, PB = ozo.planes_merged(0, DA, OSET[set_name]), ozo.planes_merged(1, DB, OSET[set_name])
+    else:
+        PA, PB = ozo.planes(DA, OSET[set_name], OSUB[sub]), ozo.planes(DB, OSET[set_name], OSUB[sub])
+    R, st = gh.residue_gemm(PA, PB, k, set_name, gh.route(sub, acc=acc))
+    assert st == 0 and (R == ozo.products(DA, DB, OSET[set_name])).all()
+
+
+def test_dgemm_long_k():
+    """The whole method at k = 33000 > 32768 (shifts from the whole k, split-K inside the GEMM)."""
+    import tests.gpu_helpers as gh
+    A, B = syn.operands(syn.CONFIGS[2], 48, 1030, 33000)
+    for set_name, sub in (("S", "fp8"), ("A", "int8n")):
+        got, st = gh.dgemm(A, B, set_name, gh.route(sub))
+        want = ozo.dgemm(A, B, OSET[set_name])
+        assert st == 0
+        _check_against_oracle_and_dd(A, B, got, want)
+
+
 # ------------------------------------------------------------------ reconstruction (a7)
 @pytest.mark.parametrize("set_name", ["S", "E", "A"])
 @pytest.mark.parametrize("m,n,ldr", [(256, 64, None), (1, 1, None), (7, 5, None), (130, 3, None), (258, 9, 272),
