@@ -32,7 +32,6 @@ __constant__ ReconConst c_recon[kNumSets];
 // 117.8-bit set A (residues < 2^8, 15 terms: sums < 2^52), so that three chunks cover M.
 __host__ __device__ constexpr int chunk_bits(int set) { return set == 2 ? 40 : 38; }
 __host__ __device__ constexpr double pow2d(int e) { double v = 1.0; for (int i = 0; i < e; ++i) v *= 2.0; return v; }
-constexpr double kTwo52 = 4503599627370496.0;         // 2^52
 constexpr double kRint = 6755399441055744.0;          // 1.5 * 2^52: (x + kRint) - kRint = rint(x)
 
 // x * 2^scale for a finite double x (exact unless the result leaves the normal range)
@@ -52,7 +51,8 @@ __device__ __forceinline__ void crt_term(uint32_t w, double &S0, double &S1, dou
     const ReconConst &K = c_recon[SET];
     constexpr int BITS = 8 * residue_bytes(SET);
     const uint32_t c = (w >> (BITS * HALF)) & ((1u << BITS) - 1u);
-    double cd = __hiloint2double(0x43300000, static_cast<int>(c)) - kTwo52;   // exact u32 -> double
+    // exact; the hardware conversion keeps this off the FP64 pipe, which bounds the kernel
+    double cd = __uint2double_rn(c);
     S0 = fma(cd, K.V[I][0], S0);
     S1 = fma(cd, K.V[I][1], S1);
     S2 = fma(cd, K.V[I][2], S2);
