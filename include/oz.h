@@ -20,7 +20,9 @@
  *     "host".  The library never allocates or frees device memory; scratch comes
  *     from the workspace registered with oz_set_workspace().
  *   - All work is enqueued on `stream` (a cudaStream_t passed as void*; NULL is the
- *     default stream).  No call synchronises the host except oz_query_status().
+ *     default stream), or on internal streams that fork from it and join it again inside the
+ *     call, so that ordering on `stream` is all a caller needs.  No call synchronises the host
+ *     except oz_query_status().
  *   - Host-detectable errors return at once with nothing enqueued.  Conditions
  *     found on the device (non-finite input, a bounded wait that ran out) set a
  *     sticky per-device status word that oz_query_status() returns and clears.
@@ -204,8 +206,10 @@ oz_status_t oz_query_status(void *stream);
 /* Optional per-stage timing hook for benchmarks (the paper's Algorithm 1 prices each stage
  * separately).  `events` is a HOST array of 5 cudaEvent_t handles (as void*), or NULL to switch the
  * hook off.  While set, oz_dgemm / oz_dgemm_ex record them on the call's stream: [0] before the
- * first kernel, [1] after the deconstruction of A, [2] after the deconstruction of B, [3] after the
- * residue GEMMs, [4] after the reconstruction.  The handles are copied; the caller owns the events. */
+ * first kernel, [1] after the deconstruction of A, [2] once the deconstruction of B -- which runs
+ * next to A's on an internal stream that forks from and joins the call's stream -- has finished
+ * too, [3] after the residue GEMMs, [4] after the reconstruction.  The handles are copied; the
+ * caller owns the events. */
 oz_status_t oz_set_stage_events(void *const *events);
 
 /* Number of kernels launched by the library on this process since load (for benchmarks). */

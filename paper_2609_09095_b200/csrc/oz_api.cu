@@ -21,6 +21,9 @@ std::mutex g_mutex;
 bool g_ready[kMaxDevices] = {};
 const uint32_t *g_lut_addr[kMaxDevices] = {};
 unsigned int *g_status_addr[kMaxDevices] = {};
+// side stream on which the whole-method calls deconstruct B while A is deconstructed on the caller's
+cudaStream_t g_side_stream[kMaxDevices] = {};
+cudaEvent_t g_fork[kMaxDevices] = {}, g_join[kMaxDevices] = {};
 void *g_workspace[kMaxDevices] = {};
 size_t g_workspace_bytes[kMaxDevices] = {};
 std::atomic<uint64_t> g_launches{0};
@@ -192,6 +195,9 @@ oz_status_t ensure_device_ready()
     g_status_addr[dev] = static_cast<unsigned int *>(p);
     oz_status_t st = upload_reconstruct_constants();
     if (st != OZ_OK) return st;
+    OZ_CUDA_CHECK(cudaStreamCreateWithFlags(&g_side_stream[dev], cudaStreamNonBlocking));
+    OZ_CUDA_CHECK(cudaEventCreateWithFlags(&g_fork[dev], cudaEventDisableTiming));
+    OZ_CUDA_CHECK(cudaEventCreateWithFlags(&g_join[dev], cudaEventDisableTiming));
     g_ready[dev] = true;
     return OZ_OK;
 }
@@ -292,13 +298,23 @@ oz_status_t dgemm_impl(int64_t m, int64_t n, int64_t k, double alpha, const doub
     uint8_t *PB = reinterpret_cast<uint8_t *>(ws + L.PB);
     void *R = ws + L.R;
 
+    // The two operands are deconstructed side by side: B's chain of five short kernels runs on an
+    // internal stream that forks from and joins the caller's (their scratch, planes and shifts are
+    // disjoint).  Stage event [1] marks the end of A's chain, [2] the join.
+    int dev = 0;
+    OZ_CUDA_CHECK(cudaGetDevice(&dev));
+    cudaStream_t side = g_side_stream[dev];
     const bool ev = g_stage_events_on;
     if (ev) OZ_CUDA_CHECK(cudaEventRecord(g_stage_events[0], stream));
+    OZ_CUDA_CHECK(cudaEventRecord(g_fork[dev], stream));
+    OZ_CUDA_CHECK(cudaStreamWaitEvent(side, g_fork[dev], 0));
+    st = launch_deconstruct(1, n, k, B, ldb, set, rt, PB, L.strideB, L.pitch, shiftB, ws + L.scrB, side);
+    if (st != OZ_OK) return st;
+    OZ_CUDA_CHECK(cudaEventRecord(g_join[dev], side));
     st = launch_deconstruct(0, m, k, A, lda, set, rt, PA, L.strideA, L.pitch, shiftA, ws + L.scrA, stream);
     if (st != OZ_OK) return st;
     if (ev) OZ_CUDA_CHECK(cudaEventRecord(g_stage_events[1], stream));
-    st = launch_deconstruct(1, n, k, B, ldb, set, rt, PB, L.strideB, L.pitch, shiftB, ws + L.scrB, stream);
-    if (st != OZ_OK) return st;
+    OZ_CUDA_CHECK(cudaStreamWaitEvent(stream, g_join[dev], 0));
     if (ev) OZ_CUDA_CHECK(cudaEventRecord(g_stage_events[2], stream));
     st = launch_residue_gemm(m, n, k, PA, L.strideA, L.pitch, PB, L.strideB, L.pitch, set, rt, R,
                              L.ldr, L.mod_stride, stream);
