@@ -103,6 +103,7 @@ struct GemmParams {
     int64_t m, n, k;
     int tiles_m, tiles_n, nk;       // tiles of 256 rows / 128 columns of C; nk = K chunks of BLOCK_K
     int vec_store;                  // R rows 16-byte aligned: use vector stores
+    int stall_producer;             // test hook: the producer issues no copy, so every wait runs out
     int r;
     int64_t total_items;
     void *R;                        // residues: uint16 (RB = 2) or uint8 (RB = 1, byte moduli)
@@ -462,7 +463,7 @@ residue_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
             int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
-            for (int64_t item = first_item; ok && item < p.total_items; item += item_step) {
+            for (int64_t item = first_item; ok && !p.stall_producer && item < p.total_items; item += item_step) {
                 Item it = decode_item(item, p);
                 const ModInfo &mi = p.mod[it.mod];
                 for (int job = 0; ok && job < mi.njobs; ++job)
@@ -825,6 +826,12 @@ oz_status_t launch_residue_gemm(int64_t m, int64_t n, int64_t k, const uint8_t *
     p.total_items = static_cast<int64_t>(p.r) * p.tiles_m * p.tiles_n;
     if (p.total_items >= 0x7FFFFFFFll) return OZ_ERR_UNSUPPORTED;        // item numbers are 32-bit in the kernel
     p.R = R; p.ldr = ldr; p.mod_stride = mod_stride;
+    // Test hook for the bounded waits: with OZ_TEST_STALL_PRODUCER=1 no operand is ever loaded, every
+    // role's wait runs into its time limit, the kernel sets OZ_ERR_TIMEOUT and returns cleanly.
+    {
+        const char *env = getenv("OZ_TEST_STALL_PRODUCER");
+        p.stall_producer = (env && env[0] == '1') ? 1 : 0;
+    }
     p.status = device_status_word();
     for (int i = 0; i < p.r; ++i) {
         int mi = modulus(set, i), s = square_root(mi);

@@ -394,3 +394,27 @@ def test_dgemm_host_buffers(m, n, k, alpha, beta, set_name, sub):
     want = ozo.dgemm(np.asfortranarray(A[rows, :]), np.asfortranarray(B[:, cols]), OSET[set_name], ozo.QUANT_RN,
                      ozo.SCALE_CS, alpha, beta, np.asfortranarray(C0[np.ix_(rows, cols)]) if beta else None)
     assert (got[np.ix_(rows, cols)] == want).all()
+
+
+@pytest.mark.parametrize("n", [520, 512])        # single-CTA variant, CTA-pair variant
+def test_bounded_waits_time_out_cleanly(monkeypatch, n):
+    """No wait in the GEMM kernel is unbounded: with the producer told to load nothing (a test hook read
+    from the environment at launch), every role's wait runs into its 2 s limit, the kernel records
+    OZ_ERR_TIMEOUT, frees its tensor memory and returns; the context stays usable and the next call is
+    correct."""
+    import time
+    import paper_2609_09095_b200 as oz
+    import tests.gpu_helpers as gh
+    rng = np.random.default_rng(5)
+    m, k = 300, 256
+    PA, DA = _random_planes(rng, "S", "fp8", m, k)
+    PB, DB = _random_planes(rng, "S", "fp8", n, k)
+    monkeypatch.setenv("OZ_TEST_STALL_PRODUCER", "1")
+    t0 = time.time()
+    R, st = gh.residue_gemm(PA, PB, k, "S", gh.route("fp8"))
+    elapsed = time.time() - t0
+    assert st == oz.OZ_ERR_TIMEOUT
+    assert 1.5 < elapsed < 120.0
+    monkeypatch.delenv("OZ_TEST_STALL_PRODUCER")
+    R, st = gh.residue_gemm(PA, PB, k, "S", gh.route("fp8"))
+    assert st == 0 and (R == ozo.products(DA, DB, OSET["S"])).all()
