@@ -8,26 +8,34 @@
 // of tcgen05.mma instructions into one TMEM accumulator:
 //   square:      job 0 = D0.E0 (weight 1);  job 1 = [D1|D0].[E0|E1] (two K-loops, weight s)
 //   non-square:  job 0 = D0.E0 (-15);  job 1 = DS.ES (16);  job 2 = D1.E1 (240)
-//   non-square, merged accumulators (FP8, k <= 4097 / 15420): job 0 = [D0|-16 D1].[E0|E1] (-15);
-//                job 1 = DS.ES (16) -- the regrouping discussed under Table "tuples" (N_acc = 2);
-//                one TMEM drain fewer per modulus, which is what bounds the epilogue at small k
+//   non-square, merged accumulators (FP8): job 0 = [D0|-16 D1].[E0|E1] (-15); job 1 = DS.ES (16)
+//                -- the regrouping discussed under Table "tuples" (N_acc = 2); one TMEM drain
+//                fewer per modulus, and the drains are what the epilogue pays for at small k
 // Three MMA K-loops per modulus either way (p_mma = 3r).
+//
+// Split-K inside the kernel: a job whose K range exceeds the exact depth of its accumulator (4097
+// or 15420 for the merged job 0, 32768 for every other FP32 accumulator, 2^31 / term size in
+// INT32) is cut into segments of whole K chunks; each segment has an accumulator of its own that
+// is reduced modulo m_i before it is weighted and added, so the residues are those of the whole K.
 //
 // The tile is computed transposed: the MMA's M dimension (128 TMEM lanes) runs over 128 columns
 // j of C (planes of B), its N dimension (256 TMEM columns) over 256 rows i of C (planes of A).
-// An epilogue thread therefore owns one column j and a run of consecutive rows, which is
-// contiguous in the column-major residue array: 16-byte stores, no staging.
+// An epilogue thread therefore owns one column j and a run of 64 consecutive rows, which is
+// contiguous in the column-major residue array; a warp transposes its 32 x 64 block through a
+// small swizzled shared-memory buffer so that each store instruction writes whole lines.
 //
-// Kernel structure (one persistent CTA per SM, 640 threads, 96 registers each):
-//   warp 0       TMA producer: 128-byte-swizzled K-major tiles of B (128 lines) and A (256 lines)
-//                into a 4-stage shared-memory ring, no multicast
-//   warp 1       MMA issuer: one lane issues tcgen05.mma (M=128, N=256, K=32, cta_group::1);
-//                accumulators live in TMEM, two slots of 256 columns used alternately per job
+// Kernel structure (one persistent CTA per SM, 640 threads, 96 registers each; launched as
+// clusters of two CTAs that share one tcgen05.mma.cta_group::2 unless n pads badly to 256):
+//   warp 0       TMA producer: 128-byte-swizzled K-major tiles of B (128 lines) and A (256 lines,
+//                or this CTA's half of them in a pair) into a shared-memory ring of 192 KiB
+//                (4 stages of 48 KiB, or 6 of 32 KiB in a pair), no multicast
+//   warp 1       MMA issuer: one lane issues tcgen05.mma (M=128 or 256 across the pair, N=256,
+//                K=32); accumulators live in TMEM, two slots of 256 columns used alternately per job
 //   warps 4..19  epilogue (4 per TMEM lane quarter, 64 columns each): tcgen05.ld the finished slot,
 //                reduce each accumulator modulo m_i in FP32 (all values are integers below 2^24,
 //                every step exact), fold it with the job's weight into a per-thread running
 //                combination held in registers, release the slot; after the last job reduce once
-//                more and store 16-bit residues
+//                more and store the residues (uint16, or uint8 for the all-byte set)
 // so the epilogue of one job overlaps the K-loop of the next, and TMEM never needs the three
 // accumulators of a non-square modulus at once.
 //
@@ -37,7 +45,8 @@
 // (weights by IMAD, `mod m` by a multiply-high division on a biased, non-negative value).
 //
 // Native INT8 route (all-byte set A only): the centred residue itself is the operand, so a modulus
-// is ONE job -- one plane, one K-loop, weight 1 -- and the schedule has r = 15 products.
+// is ONE job -- one plane, one K-loop, weight 1 -- and the schedule has r = 15 products; its
+// accumulator is loaded straight into the combination registers and the slot released at once.
 //
 // Every barrier wait is bounded: on expiry the CTA records OZ_ERR_TIMEOUT in the device status
 // word, every role leaves its loops, in-flight copies are given a bounded time to land, TMEM is

@@ -5,12 +5,15 @@
 // CRT fixes c' uniquely, so any exact evaluation gives the same integer; this kernel uses the
 // weighted form
 //     c' = sum_i c_i V_i  -  kappa M,     V_i = ((M/m_i)^-1 mod m_i) (M/m_i) mod M,
-// with every V_i and M cut into three 38-bit chunks.  c_i < 2^10.1, so each of the three chunk
-// sums is an integer below 2^52 and is formed EXACTLY by FP64 fused multiply-adds (about r MACs
-// per chunk, on a pipe that is otherwise idle here).  kappa = round(S/M) comes from a floating
-// estimate and is then made exact by a 128-bit range test, so the result is the unique
-// representative in [-M/2, M/2) in every case.  The final conversion of the 128-bit integer to
-// FP64 is a single round-to-nearest-even done in integer arithmetic.
+// with every V_i and M cut into three 38-bit chunks (40-bit for the all-byte set).  c_i < 2^10.1
+// (2^8), so each of the three chunk sums is an integer below 2^52 and is formed EXACTLY by FP64
+// fused multiply-adds (r MACs per chunk).  kappa = round(S/M) comes from a floating estimate; the
+// carry-normalised chunks are then summed with error-free additions, which give the correctly
+// rounded FP64 value directly unless c' lies within a hair of a rounding boundary, of a power of
+// two or of +-M/2 -- those rare outputs take an exact path: the 128-bit integer, an exact range
+// test for the lift to [-M/2, M/2), and one round-to-nearest-even done in integer arithmetic.
+// A thread handles the consecutive rows whose residues share one 32-bit word per modulus (two
+// uint16, or four uint8 for the all-byte set).
 #include <utility>
 
 #include "oz_internal.h"
