@@ -22,7 +22,9 @@
  *   - All work is enqueued on `stream` (a cudaStream_t passed as void*; NULL is the
  *     default stream), or on internal streams that fork from it and join it again inside the
  *     call, so that ordering on `stream` is all a caller needs.  No call synchronises the host
- *     except oz_query_status().
+ *     except oz_query_status().  The whole-method entry points (oz_dgemm, oz_dgemm_ex,
+ *     oz_dgemm_host) create their internal stream and events on a device's first such call:
+ *     make that call outside a stream capture.  The stage entry points use `stream` only.
  *   - Host-detectable errors return at once with nothing enqueued.  Conditions
  *     found on the device (non-finite input, a bounded wait that ran out) set a
  *     sticky per-device status word that oz_query_status() returns and clears.

@@ -195,10 +195,21 @@ oz_status_t ensure_device_ready()
     g_status_addr[dev] = static_cast<unsigned int *>(p);
     oz_status_t st = upload_reconstruct_constants();
     if (st != OZ_OK) return st;
-    OZ_CUDA_CHECK(cudaStreamCreateWithFlags(&g_side_stream[dev], cudaStreamNonBlocking));
+    g_ready[dev] = true;
+    return OZ_OK;
+}
+
+// The side stream and its two events exist only for the whole-method calls and are created on a
+// device's first such call; the stage entry points (the allocation-free one among them) never get here.
+oz_status_t ensure_side_stream(int dev)
+{
+    std::lock_guard<std::mutex> lock(g_mutex);
+    if (g_side_stream[dev]) return OZ_OK;
+    cudaStream_t st = nullptr;
+    OZ_CUDA_CHECK(cudaStreamCreateWithFlags(&st, cudaStreamNonBlocking));
     OZ_CUDA_CHECK(cudaEventCreateWithFlags(&g_fork[dev], cudaEventDisableTiming));
     OZ_CUDA_CHECK(cudaEventCreateWithFlags(&g_join[dev], cudaEventDisableTiming));
-    g_ready[dev] = true;
+    g_side_stream[dev] = st;
     return OZ_OK;
 }
 
@@ -303,6 +314,8 @@ oz_status_t dgemm_impl(int64_t m, int64_t n, int64_t k, double alpha, const doub
     // disjoint).  Stage event [1] marks the end of A's chain, [2] the join.
     int dev = 0;
     OZ_CUDA_CHECK(cudaGetDevice(&dev));
+    st = ensure_side_stream(dev);
+    if (st != OZ_OK) return st;
     cudaStream_t side = g_side_stream[dev];
     const bool ev = g_stage_events_on;
     if (ev) OZ_CUDA_CHECK(cudaEventRecord(g_stage_events[0], stream));
