@@ -478,14 +478,16 @@ int64_t ozo_plane_products(int64_t m, int64_t n, int64_t k, const uint8_t *PA,
 /* Merged accumulators (discussion of Table "tuples": N_acc = 2)        */
 /* ------------------------------------------------------------------ */
 /* Regrouping Eq. 8 as  d e = -15 [ d0 e0 + (-16 d1) e1 ] + 16 (d0+d1)(e0+e1)  needs two
- * accumulators per non-square modulus instead of three, at the price of one more stored plane,
- * the pre-scaled -16*d1, on ONE operand (here: side 0, the rows of A).  The merged term reaches
- * 4095 on the 9-bit tail of S (exact FP32 accumulation to K = 4097) and 1088 on byte moduli
- * (K = 15 420).  Squares are unchanged.  FP8 substrate only (-256 does not fit a signed byte). */
+ * accumulators per non-square modulus instead of three.  The plane d1 enters only through the
+ * product d1 e1, so on ONE operand (here: side 0, the rows of A) the stored plane holds the
+ * pre-scaled -16*d1 in place of d1; the plane count does not change (Table "tuples": p_store
+ * stays 3 per non-square where N_acc = 2).  The merged term reaches 4095 on the 9-bit tail of S
+ * (exact FP32 accumulation to K = 4097) and 1088 on byte moduli (K = 15 420).  Squares are
+ * unchanged.  FP8 substrate only (-256 does not fit a signed byte). */
 int ozo_planes_of_merged(int m, int side)
 {
-    if (ozo_square_root(m)) return 2;
-    return side == 0 ? 4 : 3;
+    (void)side;
+    return ozo_square_root(m) ? 2 : 3;
 }
 
 int ozo_pstore_merged(int set, int side)
@@ -495,7 +497,7 @@ int ozo_pstore_merged(int set, int side)
     return p;
 }
 
-/* plane order per non-square modulus on side 0: d0, d1, d0+d1, -16*d1 */
+/* plane order per non-square modulus on side 0: d0, -16*d1, d0+d1; on side 1: d0, d1, d0+d1 */
 int ozo_planes_merged(int side, int64_t lines, int64_t k, const int16_t *D, int set, uint8_t *P,
                       int64_t plane_stride, int64_t row_pitch)
 {
@@ -507,7 +509,7 @@ int ozo_planes_merged(int side, int64_t lines, int64_t k, const int16_t *D, int 
         for (int d = -(mod[i] / 2); 2 * d < mod[i]; ++d) {
             int dg[4] = {0, 0, 0, 0};
             ozo_split(d, mod[i], dg);
-            dg[3] = -16 * dg[1];
+            if (side == 0 && np == 3) dg[1] = -16 * dg[1];
             for (int q = 0; q < np; ++q) {
                 int byte = ozo_e4m3_encode(dg[q]);
                 if (byte < 0) { bad = 1; byte = 0x7F; }
@@ -525,7 +527,7 @@ int ozo_planes_merged(int side, int64_t lines, int64_t k, const int16_t *D, int 
     return bad ? -1 : plane;
 }
 
-/* residues from the merged layout: PA in the side-0 layout (4 planes per non-square), PB plain */
+/* residues from the merged layout: PA in the side-0 layout (-16*d1 in place of d1), PB plain */
 int64_t ozo_plane_products_merged(int64_t m, int64_t n, int64_t k, const uint8_t *PA,
                                   int64_t strideA, int64_t pitchA, const uint8_t *PB,
                                   int64_t strideB, int64_t pitchB, int set, uint16_t *R)
@@ -543,7 +545,7 @@ int64_t ozo_plane_products_merged(int64_t m, int64_t n, int64_t k, const uint8_t
             for (int64_t ii = 0; ii < m; ++ii) {
                 int64_t acc0 = 0, acc1 = 0;
                 for (int64_t kk = 0; kk < k; ++kk) {
-                    int a[4] = {0, 0, 0, 0}, b[3] = {0, 0, 0};
+                    int a[3] = {0, 0, 0}, b[3] = {0, 0, 0};
                     for (int q = 0; q < npa; ++q)
                         a[q] = digit_of[PA[(pa + q) * strideA + ii * pitchA + kk]];
                     for (int q = 0; q < npb; ++q)
@@ -552,7 +554,7 @@ int64_t ozo_plane_products_merged(int64_t m, int64_t n, int64_t k, const uint8_t
                         acc0 += (int64_t)a[0] * b[0];
                         acc1 += (int64_t)a[1] * b[0] + (int64_t)a[0] * b[1];
                     } else {
-                        acc0 += (int64_t)a[0] * b[0] + (int64_t)a[3] * b[1];   /* d0 e0 - 16 d1 e1 */
+                        acc0 += (int64_t)a[0] * b[0] + (int64_t)a[1] * b[1];   /* d0 e0 - 16 d1 e1 */
                         acc1 += (int64_t)a[2] * b[2];                           /* (d0+d1)(e0+e1)   */
                     }
                 }

@@ -200,7 +200,7 @@ def pstore_merged(s: int, side: int) -> int:
 
 
 def planes_merged(side: int, D: np.ndarray, s: int, row_pitch: int | None = None) -> np.ndarray:
-    """FP8 planes of the merged-accumulator layout (side 0 carries the extra -16*d1 planes)."""
+    """FP8 planes of the merged-accumulator layout (side 0 stores -16*d1 in place of d1)."""
     r, lines, k = D.shape
     pitch = row_pitch if row_pitch is not None else (k + 15) // 16 * 16
     P = np.full((pstore_merged(s, side), lines, pitch), 0xAA, dtype=np.uint8)

@@ -180,8 +180,8 @@ def test_merged_accumulator_layout(name):
     # accumulators: 2 per modulus when merged (E and A rows of the table); S keeps 3 on its tail unmerged
     assert 2 * len(ms) == {"S": 24, "E": int(PAPER["nacc_E"]), "A": int(PAPER["nacc_A"])}[name]
     assert 2 * (len(ms) - len(nonsq)) + 3 * len(nonsq) == {"S": int(PAPER["nacc_S"]), "E": 33, "A": 44}[name]
-    assert ozo.pstore_merged(SETS[name], 0) == ozo.pstore(SETS[name]) + len(nonsq)
-    assert ozo.pstore_merged(SETS[name], 1) == ozo.pstore(SETS[name])
+    # the pre-scaled plane takes the place of d1 on one operand: the table's p_store is unchanged
+    assert ozo.pstore_merged(SETS[name], 0) == ozo.pstore_merged(SETS[name], 1) == int(PAPER["pstore_" + name])
     worst = 0
     for m in nonsq:
         lo, hi = -(m // 2), (m - 1) // 2
@@ -207,6 +207,18 @@ def test_merged_accumulator_layout(name):
     DA, DB = ozo.residues(QA, SETS[name]), ozo.residues(QB, SETS[name])
     PA, PB = ozo.planes_merged(0, DA, SETS[name]), ozo.planes_merged(1, DB, SETS[name])
     assert (PB == ozo.planes(DB, SETS[name], ozo.SUB_FP8)).all()
+    # side 0 differs from the plain layout in exactly the d1 planes of the non-square moduli
+    plain, p0 = ozo.planes(DA, SETS[name], ozo.SUB_FP8), 0
+    for m in ms:
+        np_ = 2 if math.isqrt(m) ** 2 == m else 3
+        for q in range(np_):
+            same = (PA[p0 + q] == plain[p0 + q]).all()
+            assert same or (np_ == 3 and q == 1)
+        if np_ == 3:
+            d1 = np.array([[ozo.split(int(d), m)[1] for d in row] for row in DA[ms.index(m)]])
+            want = np.array([[ozo.e4m3_encode(-16 * int(v)) for v in row] for row in d1], dtype=np.uint8)
+            assert (PA[p0 + 1][:, :k] == want).all()
+        p0 += np_
     R, w = ozo.plane_products_merged(PA, PB, k, SETS[name])
     assert (R == ozo.products(DA, DB, SETS[name])).all() and w <= 4095 * k
 
