@@ -198,9 +198,7 @@ def main():
     route = sub | oz.OZ_QUANT_RN | oz.OZ_SCALE_CS
     r, _, _ = oz.oz_set_info(modset)
     p_store = oz.oz_plane_count(modset, route)
-    # planes of A: six more in the merged-accumulator layout that oz_dgemm picks when it is exact
-    merged = args.substrate == "fp8" and n >= 1024          # the library's default schedule
-    p_store_a = oz.oz_plane_count_side(modset, route | oz.OZ_ACC_MERGED, 0) if merged else p_store
+    p_store_a = oz.oz_plane_count_side(modset, route, 0)    # same count on both operands
     if p_store == 0:
         raise SystemExit("the native INT8 substrate needs the all-byte set: --set A --substrate int8n")
     passes = r if args.substrate == "int8n" else 3 * r    # plane products per FP64 product

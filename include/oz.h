@@ -77,14 +77,15 @@ typedef enum { OZ_SET_S = 0, OZ_SET_E = 1, OZ_SET_A = 2 } oz_modset_t;
 
 /* Accumulator schedule of the residue GEMMs for non-square moduli on the FP8 substrate.
  * MERGED: two accumulators per modulus, d e = -15 [d0 e0 + (-16 d1) e1] + 16 (d0+d1)(e0+e1)
- * (discussion of Table "tuples", N_acc = 2).  The A operand then carries one more plane per
- * non-square modulus, the pre-scaled -16*d1, after d0, d1, d0+d1.  One merged accumulator is exact
- * while its term stays below 2^24: k <= 4097 for set S, k <= 15420 for sets E and A.  A longer k is
- * cut into equal K segments no longer than that, each with an accumulator of its own that is reduced
- * modulo m_i before the segments are added (split-K inside the kernel; the residues are the same).
+ * (discussion of Table "tuples", N_acc = 2).  The A operand then stores the pre-scaled -16*d1 in
+ * the place of d1 (plane order d0, -16*d1, d0+d1; d1 enters only through d1 e1), B is unchanged,
+ * and the plane counts stay those of the table.  One merged accumulator is exact while its term
+ * stays below 2^24: k <= 4097 for set S, k <= 15420 for sets E and A.  A longer k is cut into equal
+ * K segments no longer than that, each with an accumulator of its own that is reduced modulo m_i
+ * before the segments are added (split-K inside the kernel; the residues are the same).
  * SEPARATE: the three accumulators of Eq. 8.  With neither bit, oz_dgemm / oz_dgemm_ex /
- * oz_dgemm_host pick MERGED when n >= 1024 (their planes are internal; for narrow C the extra planes
- * of A cost more than the saved products), and the stage entry points use SEPARATE. */
+ * oz_dgemm_host pick MERGED on the FP8 substrate (their planes are internal), and the stage entry
+ * points use SEPARATE.  Planes of A written with MERGED must be multiplied with MERGED. */
 #define OZ_ACC_MERGED   0x1000u
 #define OZ_ACC_SEPARATE 0x2000u
 
@@ -99,8 +100,9 @@ oz_status_t oz_set_info(oz_modset_t set, int *r, int *p_store, int *moduli);
  * two-limb digits, 15 for set A with OZ_SUB_INT8_NATIVE; 0 for an invalid combination. */
 int oz_plane_count(oz_modset_t set, uint32_t route);
 
-/* Same, for the operand on `side` (0: A, 1: B): they differ only with OZ_ACC_MERGED, where A has
- * one plane more per non-square modulus (S: 36 / 30, E: 40 / 33, A: 58 / 44). */
+/* Same, for the operand on `side` (0: A, 1: B).  The counts of the two sides are equal on every
+ * route (with OZ_ACC_MERGED the pre-scaled plane takes the place of d1 on A); the function remains
+ * for callers that size the two plane arrays separately. */
 int oz_plane_count_side(oz_modset_t set, uint32_t route, int side);
 
 /* Bytes of one stored residue: 2 (uint16) for sets S and E, 1 (uint8) for the all-byte set A, whose

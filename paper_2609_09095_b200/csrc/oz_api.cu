@@ -133,16 +133,14 @@ bool decode_route_for_set(int set, uint32_t route, Route *out)
 }
 
 // Fixes the accumulator schedule of a call.  `automatic`: the whole-method entry points, whose
-// planes are internal, take the merged schedule (the GEMM cuts a long k into segments that each
-// stay exact); the stage entry points
-// default to separate accumulators because their plane layout is part of the interface.
-// The merged schedule saves one accumulator drain per non-square modulus but adds planes to A:
-// it pays when each plane of A is reused by many columns (n >= 1024), not for tall-skinny shapes
-// whose cost is writing and reading A's planes once.
+// planes are internal, take the merged schedule on the FP8 substrate (one accumulator drain fewer per
+// non-square modulus at no extra plane; the GEMM cuts a long k into segments that each stay exact);
+// the stage entry points default to separate accumulators because what their d1 plane holds is part
+// of the interface.
 oz_status_t resolve_schedule(int set, int64_t k, int64_t n, bool automatic, Route *rt)
 {
     if (rt->acc == 0)
-        rt->acc = (automatic && rt->substrate == 0 && k > 0 && n >= 1024) ? 1 : 2;
+        rt->acc = (automatic && rt->substrate == 0 && k > 0) ? 1 : 2;
     return OZ_OK;
 }
 

@@ -259,14 +259,16 @@ __device__ __forceinline__ void convert_modulus(const uint32_t (&l0)[4], const u
     uint32_t t23 = __byte_perm(w[2], w[3], 0x5140);
     *reinterpret_cast<uint32_t *>(out + plane * plane_stride) = __byte_perm(t01, t23, 0x5410);
     if (LAYOUT == kLayoutNative) return;      // one plane: the centred residue itself
-    *reinterpret_cast<uint32_t *>(out + (plane + 1) * plane_stride) = __byte_perm(t01, t23, 0x7632);
     if (planes_of(m) == 3) {
-        // bytes 2 and 3 of the table words: d0+d1 and the pre-scaled -16*d1
+        // bytes 2 and 3 of the table words: d0+d1 and the pre-scaled -16*d1, which takes the
+        // place of d1 in the merged layout
         uint32_t u01 = __byte_perm(w[0], w[1], 0x7362);
         uint32_t u23 = __byte_perm(w[2], w[3], 0x7362);
+        *reinterpret_cast<uint32_t *>(out + (plane + 1) * plane_stride) =
+            LAYOUT == kLayoutMerged ? __byte_perm(u01, u23, 0x7632) : __byte_perm(t01, t23, 0x7632);
         *reinterpret_cast<uint32_t *>(out + (plane + 2) * plane_stride) = __byte_perm(u01, u23, 0x5410);
-        if (LAYOUT == kLayoutMerged)
-            *reinterpret_cast<uint32_t *>(out + (plane + 3) * plane_stride) = __byte_perm(u01, u23, 0x7632);
+    } else {
+        *reinterpret_cast<uint32_t *>(out + (plane + 1) * plane_stride) = __byte_perm(t01, t23, 0x7632);
     }
 }
 

@@ -383,9 +383,9 @@ __device__ __forceinline__ void job_planes(const ModInfo &mi, int job, int pair,
         // non-square, stored order d0, d1, dS; jobs d0 e0, dS eS, d1 e1
         oa = ob = job == 0 ? 0 : (job == 1 ? 2 : 1);
     } else if (mi.kind == 3) {
-        // non-square merged: job 0 = [d0 | -16 d1] . [e0 | e1] (two K-loops), job 1 = dS eS
-        oa = job == 0 ? (pair == 0 ? 0 : 3) : 2;
-        ob = job == 0 ? (pair == 0 ? 0 : 1) : 2;
+        // non-square merged (A stores d0, -16 d1, dS): job 0 = [d0 | -16 d1] . [e0 | e1] (two K-loops),
+        // job 1 = dS eS
+        oa = ob = job == 0 ? pair : 2;
     } else if (mi.kind == 0 && job == 1) {
         // square: job 1 = [d1 | d0] . [e0 | e1]
         oa = pair == 0 ? 1 : 0;

@@ -10,7 +10,7 @@
 namespace oz {
 
 constexpr int kMaxR = 15;          // moduli in the largest supported set (A)
-constexpr int kMaxPlanes = 58;     // stored planes of set A in the merged-accumulator layout
+constexpr int kMaxPlanes = 44;     // stored planes of set A with two-limb digits
 constexpr int kLutWords = 8208;    // >= sum of the moduli of either set (S: 8197, E: 6838)
 
 // ---- modulus sets (Sec. 2 step (ii) for S; "Candidate E" and "Candidate A" paragraphs) ---
@@ -40,13 +40,14 @@ __host__ __device__ constexpr int square_root(int m)
 //   kLayoutDigits  2 (square) or 3 digit planes per modulus: d0, d1[, d0+d1]   (Sec. 2 "FP8 variant")
 //   kLayoutNative  1 plane: the centred residue itself as an INT8 operand (byte moduli only;
 //                  Sec. 2 "The substrate transition")
-//   kLayoutMerged  digits plus a fourth plane -16*d1 for every non-square modulus: the A operand of
-//                  the merged-accumulator schedule (discussion of Table "tuples", N_acc = 2)
+//   kLayoutMerged  the A operand of the merged-accumulator schedule (discussion of Table "tuples",
+//                  N_acc = 2): the d1 plane of every non-square modulus holds the pre-scaled -16*d1
+//                  (d1 enters only through d1*e1); same plane count as kLayoutDigits
 constexpr int kLayoutDigits = 0, kLayoutNative = 1, kLayoutMerged = 2;
 
 __host__ __device__ constexpr int planes_of(int m, int layout = kLayoutDigits)
 {
-    return layout == kLayoutNative ? 1 : (square_root(m) ? 2 : (layout == kLayoutMerged ? 4 : 3));
+    return layout == kLayoutNative ? 1 : (square_root(m) ? 2 : 3);
 }
 
 __host__ __device__ constexpr int first_plane(int set, int i, int layout = kLayoutDigits)

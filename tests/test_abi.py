@@ -44,7 +44,7 @@ def test_host_only_queries():
     need = oz.oz_workspace_bytes(m, n, k, oz.OZ_SET_S, oz.OZ_ACC_SEPARATE)
     assert need >= 30 * (m + n) * k + 24 * m * n
     assert need < 30 * (m + n) * k + 24 * m * n + (1 << 22)
-    # default route: merged accumulators, six more planes on the A operand
-    assert oz.oz_workspace_bytes(m, n, k, oz.OZ_SET_S, 0) == need + 6 * m * k
+    # default route: merged accumulators; the pre-scaled plane takes the place of d1, same workspace
+    assert oz.oz_workspace_bytes(m, n, k, oz.OZ_SET_S, 0) == need
     assert oz.oz_workspace_bytes(m, n, k, 7, 0) == 0
     assert "workspace" in oz.oz_status_string(oz.OZ_ERR_WORKSPACE)

@@ -73,9 +73,10 @@ def test_merged_schedule_limits():
     import torch
     import paper_2609_09095_b200 as oz
     import tests.gpu_helpers as gh
-    assert oz.oz_plane_count_side(oz.OZ_SET_S, oz.OZ_ACC_MERGED, 0) == 36
+    # the pre-scaled plane takes the place of d1: counts as in the paper's table
+    assert oz.oz_plane_count_side(oz.OZ_SET_S, oz.OZ_ACC_MERGED, 0) == 30
     assert oz.oz_plane_count_side(oz.OZ_SET_S, oz.OZ_ACC_MERGED, 1) == 30
-    assert oz.oz_plane_count_side(oz.OZ_SET_E, oz.OZ_ACC_MERGED, 0) == 40
+    assert oz.oz_plane_count_side(oz.OZ_SET_E, oz.OZ_ACC_MERGED, 0) == 33
     assert oz.oz_plane_count_side(oz.OZ_SET_S, oz.OZ_ACC_MERGED | oz.OZ_SUB_INT8, 0) == 0   # FP8 planes only
 
 
