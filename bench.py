@@ -35,10 +35,11 @@ sys.path.insert(0, ROOT)
 import synth_inputs as syn  # noqa: E402
 
 # DRAM traffic of the residue GEMM relative to its algorithmic bytes (reads / plane bytes, writes /
-# residue bytes), measured with ncu on a 16384x4096x2048 launch.  Used to scale the measured traffic
-# to the full-size launch, which is too large to capture.
-GEMM_DRAM_READ_AMPLIFICATION = 2.44
-GEMM_DRAM_WRITE_AMPLIFICATION = 1.10
+# residue bytes), measured with ncu on a 16384x4096x2048 launch (3.67 GB read for 1.26 GB of planes,
+# 1.72 GB written for 1.61 GB of residues; other captures of the same launch gave 2.4-3.1 and
+# 1.05-1.10).  Used to scale the measured traffic to the full-size launch, which is too large to capture.
+GEMM_DRAM_READ_AMPLIFICATION = 2.92
+GEMM_DRAM_WRITE_AMPLIFICATION = 1.07
 
 METRIC = "emulated FP64 TFLOPS (2mnk/s)"
 UNIT = "TFLOP/s"
