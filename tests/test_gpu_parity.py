@@ -320,6 +320,29 @@ def test_dgemm_variants(quant, rule, acc):
     assert st == 0 and (got == want).all()
 
 
+@pytest.mark.parametrize("seed", range(24))
+def test_dgemm_random_shapes(seed):
+    """Seeded random shapes, routes and scalars: ragged tiles in every dimension, every modulus set and
+    substrate, both quantisers and scale rules, alpha / beta in their four combinations."""
+    import tests.gpu_helpers as gh
+    rng = np.random.default_rng(9000 + seed)
+    m, n = int(rng.integers(1, 700)), int(rng.integers(1, 700))
+    k = int(rng.integers(1, 640)) if seed % 6 else int(rng.integers(4000, 9000))
+    if seed % 6 == 0:
+        m, n = min(m, 150), min(n, 150) + (1024 if seed % 12 == 0 else 0)
+    set_name, sub = [("S", "fp8"), ("S", "int8"), ("E", "fp8"), ("E", "int8"), ("A", "int8n"), ("A", "fp8"),
+                     ("A", "int8")][seed % 7]
+    quant, rule = ("RN", "TZ")[int(rng.integers(2))], ("CS", "MAXEXP")[int(rng.integers(2))]
+    alpha, beta = (1.0, -1.0)[int(rng.integers(2))], (0.0, 1.0)[int(rng.integers(2))]
+    dist = ("uniform", "normal", "lognormal:0.5", "lognormal:2.0")[int(rng.integers(4))]
+    A, B = syn._draw(rng, m, k, dist), syn._draw(rng, k, n, dist)
+    C0 = np.asfortranarray(rng.standard_normal((m, n))) if beta else None
+    got, st = gh.dgemm(A, B, set_name, gh.route(sub, quant, rule), alpha, beta, C0)
+    _, oq, orule = _oracle_route(sub, quant, rule)
+    want = ozo.dgemm(A, B, OSET[set_name], oq, orule, alpha, beta, C0)
+    assert st == 0 and (got == want).all()
+
+
 def test_dgemm_edge_cases():
     import tests.gpu_helpers as gh
     import paper_2609_09095_b200 as oz
