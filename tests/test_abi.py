@@ -48,3 +48,20 @@ def test_host_only_queries():
     assert oz.oz_workspace_bytes(m, n, k, oz.OZ_SET_S, 0) == need
     assert oz.oz_workspace_bytes(m, n, k, 7, 0) == 0
     assert "workspace" in oz.oz_status_string(oz.OZ_ERR_WORKSPACE)
+
+
+def test_header_is_plain_c(tmp_path):
+    """include/oz.h is a C header: it compiles as C99 with no C++ or CUDA types, and a C program can
+    name every entry point."""
+    import shutil
+    import subprocess
+    gcc = shutil.which("gcc")
+    if gcc is None:
+        pytest.skip("no C compiler")
+    import paper_2609_09095_b200 as oz
+    src = tmp_path / "use_oz.c"
+    calls = "\n".join(f"    p[{i}] = (fn_t)&{name};" for i, name in enumerate(oz.EXPORTS))
+    src.write_text('#include "oz.h"\ntypedef void (*fn_t)(void);\nint main(void)\n{\n    fn_t p[%d];\n%s\n'
+                   '    return p[0] == 0;\n}\n' % (len(oz.EXPORTS), calls))
+    inc = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "include")
+    subprocess.run([gcc, "-std=c99", "-Wall", "-Werror", "-pedantic", "-fsyntax-only", "-I", inc, str(src)], check=True)
