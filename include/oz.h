@@ -197,7 +197,9 @@ oz_status_t oz_residue_gemm(int64_t m, int64_t n, int64_t k, const uint8_t *PA,
 /* Reconstruction (Algorithm 3; Eq. 4-5 and the final step of Sec. 2 (iv)): the integer
  * c'_ij in [-M/2, M/2) congruent to the residues, times 2^-(shiftA[i]+shiftB[j]), rounded once;
  * C = alpha P (beta = 0) or C = C + alpha P (beta = 1).  The CRT is evaluated exactly.  R has the
- * layout and element type that oz_residue_gemm writes for `set`. */
+ * layout and element type that oz_residue_gemm writes for `set`; an entry may be any representative
+ * of its residue class below 2 m_i that fits the element type, not only the canonical one (adding
+ * m_i to c_i changes the CRT sum by a multiple of M). */
 oz_status_t oz_reconstruct(int64_t m, int64_t n, const void *R, int64_t ldr,
                            int64_t mod_stride, const int32_t *shiftA, const int32_t *shiftB,
                            oz_modset_t set, double alpha, double beta, double *C, int64_t ldc,

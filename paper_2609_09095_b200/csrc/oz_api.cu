@@ -327,8 +327,9 @@ oz_status_t dgemm_impl(int64_t m, int64_t n, int64_t k, double alpha, const doub
     if (ev) OZ_CUDA_CHECK(cudaEventRecord(g_stage_events[1], stream));
     OZ_CUDA_CHECK(cudaStreamWaitEvent(stream, g_join[dev], 0));
     if (ev) OZ_CUDA_CHECK(cudaEventRecord(g_stage_events[2], stream));
+    // the residues stay inside this call: the two-byte sets skip the canonicalisation
     st = launch_residue_gemm(m, n, k, PA, L.strideA, L.pitch, PB, L.strideB, L.pitch, set, rt, R,
-                             L.ldr, L.mod_stride, stream);
+                             L.ldr, L.mod_stride, residue_bytes(set) == 2, stream);
     if (st != OZ_OK) return st;
     if (ev) OZ_CUDA_CHECK(cudaEventRecord(g_stage_events[3], stream));
     if (!plan) {
@@ -577,7 +578,7 @@ oz_status_t oz_residue_gemm(int64_t m, int64_t n, int64_t k, const uint8_t *PA, 
     oz_status_t st = ensure_device_ready();
     if (st != OZ_OK) return st;
     return launch_residue_gemm(m, n, k, PA, strideA, pitchA, PB, strideB, pitchB, set, rt, R, ldr,
-                               mod_stride, static_cast<cudaStream_t>(stream));
+                               mod_stride, false, static_cast<cudaStream_t>(stream));
 }
 
 oz_status_t oz_reconstruct(int64_t m, int64_t n, const void *R, int64_t ldr, int64_t mod_stride,

@@ -419,7 +419,11 @@ __device__ __forceinline__ void segment_range(const ModInfo &mi, int job, int se
 // RB: bytes of one stored residue (2: uint16, 1: uint8 for the all-byte modulus set)
 // DIRECT: native INT8 residues -- one accumulator per modulus, loaded straight into the registers
 //         that otherwise hold the running combination of several accumulators
-template <int SUB, int CG, int RB, bool DIRECT>
+// LOOSE: the stored residue is some representative in [0, 2 m_i) instead of the canonical one in
+//         [0, m_i) (two-byte residues only).  The reconstruction is indifferent to it -- the CRT
+//         weight of m_i is a multiple of M -- and the epilogue saves the canonicalisation; used for
+//         the residues that stay inside the whole-method calls.
+template <int SUB, int CG, int RB, bool DIRECT, bool LOOSE>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 residue_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB,
                     const __grid_constant__ GemmParams p)
@@ -569,6 +573,7 @@ residue_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
             Item it = decode_item(item, p);
             const ModInfo &mi = p.mod[it.mod];
             const float mm = mi.m, inv_m = mi.inv_m;
+            const float loose_offset = mm + 8388608.0f;          // exact: m < 2^11
             const uint32_t im = mi.mi, imagic = mi.magic, ibias = mi.bias;
             // running combination per element: FP32 (FP8 route) or INT32 (INT8 routes), as raw bits
             uint32_t comb[COLS_PER_WARP];
@@ -654,13 +659,17 @@ residue_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
                     if (SUB == 0) {
                         float t = __uint_as_float(comb[c + h]);
                         float quot = fmaf(t, inv_m, 12582912.0f) - 12582912.0f;
-                        float res = fmaf(-quot, mm, t);
-                        res = res < 0.0f ? res + mm : res;                   // canonical [0, m)
-                        bits[h] = __float_as_uint(res + 8388608.0f);         // integer in the low mantissa bits
+                        float res = fmaf(-quot, mm, t);                      // |res| <= ~m/2
+                        if constexpr (LOOSE) {
+                            bits[h] = __float_as_uint(res + loose_offset);   // res + m in (0, 2m), low mantissa bits
+                        } else {
+                            res = res < 0.0f ? res + mm : res;               // canonical [0, m)
+                            bits[h] = __float_as_uint(res + 8388608.0f);     // integer in the low mantissa bits
+                        }
                     } else {
                         uint32_t u = comb[c + h] + ibias;
                         uint32_t r = u - __umulhi(u, imagic) * im;           // in [0, 2m)
-                        bits[h] = min(r, r - im);                            // canonical [0, m)
+                        bits[h] = LOOSE ? r : min(r, r - im);                // canonical [0, m) unless LOOSE
                     }
                 }
                 if constexpr (RB == 2) {
@@ -776,11 +785,12 @@ bool make_plane_map(CUtensorMap *map, const uint8_t *base, int64_t lines, int64_
     return rc == CUDA_SUCCESS;
 }
 
-template <int SUB, int CG, int RB, bool DIRECT = false>
+template <int SUB, int CG, int RB, bool DIRECT = false, bool LOOSE = false>
 oz_status_t launch_variant(const CUtensorMap &mapA, const CUtensorMap &mapB, const GemmParams &p, int sms,
                            cudaStream_t stream)
 {
-    auto kernel = residue_gemm_kernel<SUB, CG, RB, DIRECT>;
+    static_assert(!LOOSE || RB == 2, "a representative below 2m needs the two-byte element");
+    auto kernel = residue_gemm_kernel<SUB, CG, RB, DIRECT, LOOSE>;
     OZ_CUDA_CHECK(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        static_cast<int>(SMEM_BYTES)));
     int64_t groups = sms / CG;                                    // CTAs, or CTA pairs
@@ -820,7 +830,7 @@ static int cta_group_choice(int64_t n)
 oz_status_t launch_residue_gemm(int64_t m, int64_t n, int64_t k, const uint8_t *PA, int64_t strideA,
                                 int64_t pitchA, const uint8_t *PB, int64_t strideB, int64_t pitchB,
                                 int set, const Route &rt, void *R, int64_t ldr,
-                                int64_t mod_stride, cudaStream_t stream)
+                                int64_t mod_stride, bool loose, cudaStream_t stream)
 {
     const int cg = cta_group_choice(n);
     GemmParams p{};
@@ -930,6 +940,13 @@ oz_status_t launch_residue_gemm(int64_t m, int64_t n, int64_t k, const uint8_t *
                                      : launch_variant<1, 2, 1>(mapA, mapB, p, sms, stream);
         return rt.substrate == 0 ? launch_variant<0, 1, 1>(mapA, mapB, p, sms, stream)
                                  : launch_variant<1, 1, 1>(mapA, mapB, p, sms, stream);
+    }
+    if (loose) {
+        if (cg == 2)
+            return rt.substrate == 0 ? launch_variant<0, 2, 2, false, true>(mapA, mapB, p, sms, stream)
+                                     : launch_variant<1, 2, 2, false, true>(mapA, mapB, p, sms, stream);
+        return rt.substrate == 0 ? launch_variant<0, 1, 2, false, true>(mapA, mapB, p, sms, stream)
+                                 : launch_variant<1, 1, 2, false, true>(mapA, mapB, p, sms, stream);
     }
     if (cg == 2)
         return rt.substrate == 0 ? launch_variant<0, 2, 2>(mapA, mapB, p, sms, stream)

@@ -130,8 +130,8 @@ oz_status_t launch_deconstruct(int side, int64_t lines, int64_t k, const double 
 oz_status_t launch_residue_gemm(int64_t m, int64_t n, int64_t k, const uint8_t *PA,
                                 int64_t strideA, int64_t pitchA, const uint8_t *PB,
                                 int64_t strideB, int64_t pitchB, int set, const Route &rt,
-                                void *R, int64_t ldr, int64_t mod_stride,
-                                cudaStream_t stream);
+                                void *R, int64_t ldr, int64_t mod_stride, bool loose,
+                                cudaStream_t stream);   // loose: residues in [0, 2 m_i), two-byte sets
 
 oz_status_t launch_reconstruct(int64_t m, int64_t n, const void *R, int64_t ldr,
                                int64_t mod_stride, const int32_t *shiftA, const int32_t *shiftB,

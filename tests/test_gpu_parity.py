@@ -276,6 +276,15 @@ def test_reconstruct_bit_exact(set_name, m, n, ldr):
         want = ozo.output(CI, sA, sB, alpha, beta, C0)
         assert st == 0
         assert (got == want).all()
+    # any representative below 2 m_i that fits the element type gives the same integer
+    top = 255 if set_name == "A" else 65535
+    R2 = R.astype(np.int64)
+    for i, mm in enumerate(ms):
+        bump = (rng.integers(0, 2, size=R2[i].shape) == 1) & (R2[i] + mm <= top)
+        R2[i] = R2[i] + bump * mm
+    assert R.size < 64 or (R2 != R).any()
+    got, st = gh.reconstruct(R2.astype(np.uint16), sA, sB, set_name, 1.0, 0.0, None, ldr=ldr)
+    assert st == 0 and (got == ozo.output(CI, sA, sB, 1.0, 0.0, None)).all()
 
 
 # ------------------------------------------------------------------ whole method
