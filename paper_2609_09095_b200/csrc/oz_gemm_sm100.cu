@@ -106,6 +106,9 @@ struct ModInfo {
     uint32_t mi;          // the modulus
     uint32_t magic;       // floor(2^32 / m)
     uint32_t bias;        // a multiple of m just above 2^31: makes a signed combination non-negative
+    // native INT8 residues, one accumulator of at most 2^30 in magnitude (k <= 65536): exact division
+    uint32_t magic39;     // ceil(2^39 / m): floor(u / m) = (u * magic39) >> 39 exactly for u < 2^31 + 256, m in (128, 256]
+    uint32_t bias30;      // the multiple of m just above 2^30
 };
 
 struct GemmParams {
@@ -666,6 +669,9 @@ residue_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
                             res = res < 0.0f ? res + mm : res;               // canonical [0, m)
                             bits[h] = __float_as_uint(res + 8388608.0f);     // integer in the low mantissa bits
                         }
+                    } else if constexpr (DIRECT) {
+                        uint32_t u = comb[c + h] + mi.bias30;                 // in (0, 2^31 + 256)
+                        bits[h] = u - (__umulhi(u, mi.magic39) >> 7) * im;   // exact quotient: canonical [0, m)
                     } else {
                         uint32_t u = comb[c + h] + ibias;
                         uint32_t r = u - __umulhi(u, imagic) * im;           // in [0, 2m)
@@ -868,6 +874,8 @@ oz_status_t launch_residue_gemm(int64_t m, int64_t n, int64_t k, const uint8_t *
         mo.mi = static_cast<uint32_t>(mi);
         mo.magic = barrett_magic(static_cast<uint32_t>(mi));
         mo.bias = static_cast<uint32_t>((((1ull << 31) + mi - 1) / mi) * mi);
+        mo.magic39 = mi > 128 ? static_cast<uint32_t>(((1ull << 39) + mi - 1) / mi) : 0u;
+        mo.bias30 = static_cast<uint32_t>((((1ull << 30) + mi - 1) / mi) * mi);
         mo.planeA0 = first_plane(set, i, rt.layout(0));
         mo.planeB0 = first_plane(set, i, rt.layout(1));
         mo.nseg = 1;
@@ -931,7 +939,8 @@ oz_status_t launch_residue_gemm(int64_t m, int64_t n, int64_t k, const uint8_t *
     OZ_CUDA_CHECK(cudaGetDevice(&dev));
     OZ_CUDA_CHECK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
     // substrate 0: FP8 planes; otherwise INT8 planes (two-limb digits or native residues)
-    if (rt.native() && p.mod[0].nseg_all == 1)      // one accumulator per modulus: the direct drain
+    // one accumulator per modulus of at most 128 * 128 * k <= 2^30: the direct drain with the exact division
+    if (rt.native() && p.mod[0].nseg_all == 1 && k <= 65536)
         return cg == 2 ? launch_variant<1, 2, 1, true>(mapA, mapB, p, sms, stream)
                        : launch_variant<1, 1, 1, true>(mapA, mapB, p, sms, stream);
     if (rb == 1) {

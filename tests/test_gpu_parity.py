@@ -219,11 +219,13 @@ def test_residue_gemm_padded_rows(m, ldr, set_name, sub):
 
 @pytest.mark.parametrize("k,set_name,sub,acc", [(40000, "S", "fp8", "separate"), (70001, "E", "fp8", "separate"),
                                                 (40000, "S", "fp8", "merged"), (140000, "A", "int8n", None),
-                                                (66000, "S", "int8", None)])
+                                                (66000, "S", "int8", None), (65536, "A", "int8n", None),
+                                                (65537, "A", "int8n", None)])
 def test_split_k_beyond_one_accumulator(k, set_name, sub, acc):
     """k beyond the exact depth of one accumulator (32768 in FP32, 131071 for native INT8 residues): the
     kernel cuts K into segments and adds their reduced results modulo m.  Largest digits, constant
-    rows: a single accumulator over all of K would overflow."""
+    rows: a single accumulator over all of K would overflow.  k = 65536 / 65537 straddle the largest
+    depth served by the native route's direct drain (accumulators up to 2^30 in magnitude)."""
     import tests.gpu_helpers as gh
     rng = np.random.default_rng(k)
     m, n = 40, 24
