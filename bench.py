@@ -8,13 +8,18 @@ whole hot path.  Prints ONE JSON line (rank 0):
   value      emulated FP64 TFLOP/s = 2 m n k / time, inputs resident in HBM
   e2e        same metric through oz_dgemm_host with pinned HOST buffers (copies timed)
   roofline   the residue-GEMM kernel: 3 r plane products, low-precision FLOP/s against the
-             tensor peak (measured bf16 peak x 2 for 8-bit operands), timed with CUDA events
-             recorded on the launching stream between the stages
+             tensor peak (measured bf16 burst peak x 2 for 8-bit operands; the fractions of the
+             sustained figure, of the nominal 4.5 PFLOP/s and of a library 8-bit GEMM timed in the
+             same run stand beside it), timed with CUDA events recorded on the launching stream
+             between the stages
+  also       the same workload on the other routes (set E, INT8 digits, set A native INT8) and
+             with the operands' planes prepared once (oz_dgemm_prepared), a few steps each
   cpu_baseline  the CPU oracle, as it stands, on a bounded sample of the same workload
 
 `--impl reference` times the CPU oracle alone (there is no other implementation of the paper).
-N > 1 (torchrun): every rank runs the same independent problem (weak scaling, no collective in
-the data path); the time is the max over ranks, the value the sum of the work.
+N > 1: every rank runs the same independent problem (weak scaling, no collective in the data
+path); the time is the max over ranks, the value the sum of the work.  Under torchrun the ranks are
+given; run plainly with --gpus N, the script starts its own N ranks (one process per GPU).
 """
 from __future__ import annotations
 
@@ -35,11 +40,26 @@ sys.path.insert(0, ROOT)
 import synth_inputs as syn  # noqa: E402
 
 # DRAM traffic of the residue GEMM relative to its algorithmic bytes (reads / plane bytes, writes /
-# residue bytes), measured with ncu on a 16384x4096x2048 launch (3.67 GB read for 1.26 GB of planes,
-# 1.72 GB written for 1.61 GB of residues; other captures of the same launch gave 2.4-3.1 and
-# 1.05-1.10).  Used to scale the measured traffic to the full-size launch, which is too large to capture.
-GEMM_DRAM_READ_AMPLIFICATION = 2.92
-GEMM_DRAM_WRITE_AMPLIFICATION = 1.07
+# residue bytes) comes from the table in profiles/residue_gemm_dram_traffic.md: ncu captures of a
+# smaller launch, one row per kernel variant, scaled here to the full-size launch by the units.
+TRAFFIC_TABLE = os.path.join(os.path.dirname(os.path.abspath(__file__)), "profiles", "residue_gemm_dram_traffic.md")
+
+
+def gemm_dram_amplification(set_name: str, substrate: str):
+    """(read, write) amplification of the variant, or None when the table has no row for it."""
+    try:
+        with open(TRAFFIC_TABLE) as fh:
+            rows = [[c.strip() for c in line.strip().strip("|").split("|")] for line in fh if line.startswith("|")]
+    except OSError:
+        return None
+    for row in rows:
+        if len(row) >= 4 and row[0] == set_name and row[1] == substrate:
+            try:
+                return float(row[2]), float(row[3])
+            except ValueError:
+                return None
+    return None
+
 
 METRIC = "emulated FP64 TFLOPS (2mnk/s)"
 UNIT = "TFLOP/s"
@@ -158,6 +178,57 @@ def run_reference(args, cfg, set_name):
     print(json.dumps(line))
 
 
+def spawn_command(argv, gpus: int, port: int):
+    """Command line that runs this script as `gpus` ranks on this node (one process per GPU)."""
+    return [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={gpus}",
+            "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + list(argv)
+
+
+def free_port() -> int:
+    import socket
+    with socket.socket() as sock:
+        sock.bind(("127.0.0.1", 0))
+        return sock.getsockname()[1]
+
+
+def library_8bit_tflops(torch, seconds: float = 0.25):
+    """A library 8-bit GEMM (8192^3) timed in this run: the practical ceiling of the tensor pipe on this
+    GPU in its present power state.  Returns {"fp8": TFLOP/s or None, "int8": TOP/s or None}."""
+    n = 8192
+    out = {"fp8": None, "int8": None}
+
+    def timed(fn):
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        reps, total = 0, 0.0
+        while total < seconds * 1e3 and reps < 200:
+            e0.record()
+            for _ in range(5):
+                fn()
+            e1.record()
+            torch.cuda.synchronize()
+            total += e0.elapsed_time(e1)
+            reps += 5
+        return 2.0 * n ** 3 * reps / (total * 1e-3) / 1e12
+
+    try:
+        a = torch.randint(-8, 8, (n, n), device="cuda", dtype=torch.int8)
+        b = torch.randint(-8, 8, (n, n), device="cuda", dtype=torch.int8)
+        out["int8"] = timed(lambda: torch._int_mm(a, b))
+    except Exception:
+        pass
+    try:
+        a8 = torch.randn(n, n, device="cuda").to(torch.float8_e4m3fn)
+        b8 = torch.randn(n, n, device="cuda").to(torch.float8_e4m3fn).t()
+        one = torch.ones((), device="cuda")
+        out["fp8"] = timed(lambda: torch._scaled_mm(a8, b8, scale_a=one, scale_b=one, out_dtype=torch.bfloat16))
+    except Exception:
+        pass
+    return out
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -169,9 +240,13 @@ def main():
     ap.add_argument("--substrate", default="fp8", choices=["fp8", "int8", "int8n"],
                     help="int8n = native INT8 residues, one plane per modulus (set A only)")
     ap.add_argument("--shape", default=None, help="m,n,k override (same distribution and seed as --config)")
-    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--e2e-steps", type=int, default=10)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-also", action="store_true", help="skip the other routes and the library 8-bit GEMM")
     args = ap.parse_args()
+    if args.impl != "reference" and args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # run plainly with --gpus N: start the N replica ranks ourselves
+        raise SystemExit(subprocess.call(spawn_command(sys.argv[1:], args.gpus, free_port())))
     if args.warmup < 3 and args.impl != "reference":
         args.warmup = 3
     cfg = syn.CONFIGS[args.config]
@@ -212,7 +287,16 @@ def main():
     hC = torch.from_numpy(np.ascontiguousarray(C0.T)).pin_memory()
     del A, B, C0
     dA, dB, dC = hA.cuda(), hB.cuda(), hC.cuda()
-    core = oz.oz_workspace_bytes(m, n, k, modset, route)
+    # the other routes timed for the `also` key (single GPU, default workload only)
+    also_routes = []
+    if world == 1 and not args.no_also and args.shape is None:
+        for sname, subname in (("E", "fp8"), ("S", "int8"), ("S", "fp8"), ("A", "int8n")):
+            if (sname, subname) != (args.set_name, args.substrate):
+                also_routes.append((sname, subname))
+    sets = {"S": oz.OZ_SET_S, "E": oz.OZ_SET_E, "A": oz.OZ_SET_A}
+    subs = {"fp8": oz.OZ_SUB_FP8, "int8": oz.OZ_SUB_INT8, "int8n": oz.OZ_SUB_INT8_NATIVE}
+    core = max([oz.oz_workspace_bytes(m, n, k, modset, route)] +
+               [oz.oz_workspace_bytes(m, n, k, sets[a], subs[b] | oz.OZ_QUANT_RN | oz.OZ_SCALE_CS) for a, b in also_routes])
     ws_bytes = core + 8 * (m * k + k * n + m * n) + 4096
     ws = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")
     oz.check(oz.oz_set_workspace(ws, ws_bytes), "oz_set_workspace")
@@ -272,6 +356,46 @@ def main():
     oz.check(oz.oz_query_status(stream), "device status after the end-to-end steps")
 
     flops = 2.0 * m * n * k
+
+    # ---- the same workload on the other routes, and with the planes of A and B prepared once
+    def timed_steps(fn, steps=5, warm=2):
+        for _ in range(warm):
+            fn()
+        torch.cuda.synchronize()
+        t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        t0.record(stream)
+        for _ in range(steps):
+            fn()
+        t1.record(stream)
+        torch.cuda.synchronize()
+        return t0.elapsed_time(t1) / steps
+
+    also = []
+    for sname, subname in also_routes:
+        rt2 = subs[subname] | oz.OZ_QUANT_RN | oz.OZ_SCALE_CS
+        r2, _, _ = oz.oz_set_info(sets[sname])
+        passes2 = r2 if subname == "int8n" else 3 * r2
+        ms2 = timed_steps(lambda: oz.check(oz.oz_dgemm_ex(m, n, k, cfg.alpha, dA, m, dB, k, cfg.beta, dC, m,
+                                                          sets[sname], rt2, stream), "oz_dgemm_ex"))
+        oz.check(oz.oz_query_status(stream), "device status (also)")
+        also.append({"modulus_set": sname, "substrate": subname, "value": flops / (ms2 * 1e-3) / 1e12, "unit": UNIT,
+                     "ms_per_step": ms2, "steps": 5,
+                     "roof_frac_of_nominal": flops / (ms2 * 1e-3) / 1e12 / (4500.0 / (passes2 + 1))})
+    if world == 1 and not args.no_also:
+        # planes kept across calls (HPL: the panel's planes serve the whole trailing matrix): operands
+        # prepared once, then products only
+        opA = torch.empty(oz.oz_operand_bytes(0, m, k, modset, route), dtype=torch.uint8, device="cuda")
+        opB = torch.empty(oz.oz_operand_bytes(1, n, k, modset, route), dtype=torch.uint8, device="cuda")
+        oz.check(oz.oz_prepare_operand(0, m, k, dA, m, modset, route, opA, None, stream), "oz_prepare_operand")
+        oz.check(oz.oz_prepare_operand(1, n, k, dB, k, modset, route, opB, None, stream), "oz_prepare_operand")
+        ms3 = timed_steps(lambda: oz.check(oz.oz_dgemm_prepared(m, n, k, cfg.alpha, opA, opB, cfg.beta, dC, m, modset,
+                                                                route, stream), "oz_dgemm_prepared"))
+        oz.check(oz.oz_query_status(stream), "device status (prepared)")
+        also.append({"modulus_set": args.set_name, "substrate": args.substrate, "planes": "prepared once (oz_dgemm_prepared)",
+                     "value": flops / (ms3 * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": ms3, "steps": 5})
+        del opA, opB
+    lib8 = library_8bit_tflops(torch) if (world == 1 and not args.no_also) else {"fp8": None, "int8": None}
+
     if world > 1:
         def rmax(v):
             t = torch.tensor([v], dtype=torch.float64, device="cuda")
@@ -292,13 +416,19 @@ def main():
         value = work / (ms * 1e-3) / 1e12
         lowp_flops = float(passes) * flops                 # p_mma plane products (3r, or r on the native INT8 route)
         gemm_ms = float(stage_ms[2])
-        tensor_peak = 2.0 * peaks["bf16_sustained"]        # 8-bit operands: nominal 2x the bf16 rate
+        # 8-bit operands: nominal 2x the bf16 rate.  The kernel is timed by its own events, a few
+        # milliseconds per launch: the burst figure is its denominator; the other ceilings stand beside it.
+        tensor_peak = 2.0 * peaks["bf16"]
         achieved = lowp_flops / (gemm_ms * 1e-3) / 1e12
         roof_nominal = 4500.0 / (passes + 1)               # P_low/(3r+1), or P_low/(r+1) native INT8, at B200's dense 8-bit rate
         hbm = peaks["hbm_gbs"]
         dec_bytes = 24 * (m * k + k * n) + (p_store_a * m + p_store * n) * k   # two scan passes + convert read; planes written
         rb = oz.oz_residue_elem_bytes(modset)                 # bytes per stored residue
         rec_bytes = (rb * r + 8 + (8 if cfg.beta else 0)) * m * n
+        plane_bytes = float((p_store_a * m + p_store * n) * k)
+        residue_bytes = float(rb) * r * m * n
+        amp = gemm_dram_amplification(args.set_name, args.substrate)
+        lib_peak = lib8["fp8" if args.substrate == "fp8" else "int8"]
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
@@ -313,22 +443,29 @@ def main():
             "roof": {"definition": "P_low/(3r+1)" if passes == 3 * r else "P_low/(r+1)", "nominal_tflops": roof_nominal,
                      "frac_of_nominal": value / world / roof_nominal,
                      "at_measured_peak_tflops": tensor_peak / (passes + 1),
-                     "frac_at_measured_peak": value / world / (tensor_peak / (passes + 1))},
+                     "frac_at_measured_peak": value / world / (tensor_peak / (passes + 1)),
+                     "ms_per_step_x_sm_mhz": ms * clocks["sm_mhz"] if clocks.get("sm_mhz") else None},
             "roofline": {"kernel": "residue_gemm_kernel (tcgen05)", "bound": "tensor", "achieved": achieved,
                          "peak": tensor_peak, "unit": "TFLOP/s", "frac": achieved / tensor_peak,
-                         "peak_source": f"{peaks['source']} bf16 sustained x2 (8-bit operands)",
+                         "peak_source": f"{peaks['source']} bf16 burst x2 (8-bit operands); frac is against this",
                          "frac_of_nominal_4500": achieved / 4500.0,
-                         "traffic": GEMM_DRAM_READ_AMPLIFICATION * (p_store_a * m + p_store * n) * k
-                                    + GEMM_DRAM_WRITE_AMPLIFICATION * float(rb) * r * m * n,
-                         "traffic_unit": "bytes per launch (ncu dram read+write of a smaller launch, scaled by units)",
-                         "algorithmic_dram_bytes": (p_store_a * m + p_store * n) * k + float(rb) * r * m * n,
+                         "frac_of_sustained_x2": achieved / (2.0 * peaks["bf16_sustained"]),
+                         "peak_library_8bit": lib_peak,
+                         "peak_library_8bit_source": "torch 8192^3 8-bit GEMM (torch._scaled_mm e4m3 / torch._int_mm) timed in this run",
+                         "frac_of_library_8bit": achieved / lib_peak if lib_peak else None,
+                         "traffic": amp[0] * plane_bytes + amp[1] * residue_bytes if amp else None,
+                         "traffic_unit": "bytes per launch (ncu dram read+write of a smaller launch of this variant, "
+                                         "scaled by units; profiles/residue_gemm_dram_traffic.md)",
+                         "algorithmic_dram_bytes": plane_bytes + residue_bytes,
                          "ms_per_launch": gemm_ms},
             "stages": {
-                "deconstruct_A_ms": float(stage_ms[0]), "deconstruct_B_ms": float(stage_ms[1]),
+                "deconstruct_A_ms": float(stage_ms[0]), "deconstruct_join_ms": float(stage_ms[1]),
                 "residue_gemm_ms": gemm_ms, "reconstruct_ms": float(stage_ms[3]),
                 "deconstruct_GBps": dec_bytes / ((stage_ms[0] + stage_ms[1]) * 1e-3) / 1e9,
                 "reconstruct_GBps": rec_bytes / (stage_ms[3] * 1e-3) / 1e9,
+                "reconstruct_bytes": rec_bytes,
                 "hbm_peak_GBps": hbm, "hbm_peak_source": peaks["source"]},
+            "also": also,
             "e2e": {"value": work / (e2e_ms * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": e2e_ms,
                     "h2d_bytes_per_step": 8 * (m * k + k * n + (m * n if cfg.beta else 0)),
                     "d2h_bytes_per_step": 8 * m * n, "steps": args.e2e_steps},

@@ -17,7 +17,8 @@
  *   - Matrices are column-major, no transposes: A is m x k (lda >= m), B is k x n
  *     (ldb >= k), C is m x n (ldc >= m).
  *   - Every pointer is a DEVICE pointer owned by the caller unless a comment says
- *     "host".  The library never allocates or frees device memory; scratch comes
+ *     "host", aligned to its element type (8 bytes for matrices, 4 for shifts; OZ_ERR_INVALID_ARG
+ *     otherwise).  The library never allocates or frees device memory; scratch comes
  *     from the workspace registered with oz_set_workspace().
  *   - All work is enqueued on `stream` (a cudaStream_t passed as void*; NULL is the
  *     default stream), or on internal streams that fork from it and join it again inside the
@@ -148,6 +149,31 @@ oz_status_t oz_dgemm_host(int64_t m, int64_t n, int64_t k, double alpha, const d
                           double *C_host, int64_t ldc, oz_modset_t set, uint32_t route,
                           void *stream);
 
+/* Planes kept across calls (storage mode P of Sec. "Storage Modes"; paragraph "O1: convert-once
+ * residue-plane workspace"): an operand that takes part in several products -- the panel of an HPL
+ * trailing update, the operator of an iterative solver -- is deconstructed once into a caller-owned
+ * block and then multiplied any number of times.
+ *
+ * oz_operand_bytes: size of that block for `lines` rows of A (side 0) or columns of B (side 1) and
+ * inner dimension k; 0 for invalid arguments.  The block holds the shifts, the planes in the layout
+ * and pitch that the whole-method calls use internally (not the layout of oz_deconstruct), and the
+ * scan scratch; its content is opaque.
+ * oz_prepare_operand: deconstructs X (same conventions as oz_deconstruct) into `operand` (device
+ * memory, 256-byte aligned, at least oz_operand_bytes()).  Scaling rule, quantiser, substrate and set
+ * come from `route` / `set` and must be the same in every call that uses the block.
+ * oz_dgemm_prepared: C = beta C + alpha A B from two prepared operands (A: m lines, B: n lines, same k,
+ * set and route).  Needs a registered workspace of oz_product_workspace_bytes(m, n, set) bytes (the
+ * residues); launches the residue GEMMs and the reconstruction only.  The result is bit-identical to
+ * oz_dgemm_ex on the same matrices: the shifts of a line depend on that line alone. */
+size_t oz_operand_bytes(int side, int64_t lines, int64_t k, oz_modset_t set, uint32_t route);
+size_t oz_product_workspace_bytes(int64_t m, int64_t n, oz_modset_t set);
+oz_status_t oz_prepare_operand(int side, int64_t lines, int64_t k, const double *X, int64_t ldx,
+                               oz_modset_t set, uint32_t route, void *operand, size_t bytes,
+                               void *stream);
+oz_status_t oz_dgemm_prepared(int64_t m, int64_t n, int64_t k, double alpha, const void *operandA,
+                              const void *operandB, double beta, double *C, int64_t ldc,
+                              oz_modset_t set, uint32_t route, void *stream);
+
 /* Deconstruction of one operand (Algorithm 2; scaling of Eq. 1).
  *   side 0: X is m x k column-major, lines = m rows,    element (i,kk) at X[i + kk*ldx]
  *   side 1: X is k x n column-major, lines = n columns, element (kk,j) at X[kk + j*ldx]
@@ -210,8 +236,9 @@ oz_status_t oz_reconstruct(int64_t m, int64_t n, const void *R, int64_t ldr,
 oz_status_t oz_query_status(void *stream);
 
 /* Optional per-stage timing hook for benchmarks (the paper's Algorithm 1 prices each stage
- * separately).  `events` is a HOST array of 5 cudaEvent_t handles (as void*), or NULL to switch the
- * hook off.  While set, oz_dgemm / oz_dgemm_ex record them on the call's stream: [0] before the
+ * separately), kept per device: it applies to the device that is current when it is set.  `events`
+ * is a HOST array of 5 cudaEvent_t handles (as void*), or NULL to switch the hook off.  While set,
+ * oz_dgemm / oz_dgemm_ex / oz_dgemm_prepared record them on the call's stream: [0] before the
  * first kernel, [1] after the deconstruction of A, [2] once the deconstruction of B -- which runs
  * next to A's on an internal stream that forks from and joins the call's stream -- has finished
  * too, [3] after the residue GEMMs, [4] after the reconstruction.  The handles are copied; the

@@ -26,7 +26,8 @@ OZ_NONFINITE_SHIFT = -(2 ** 31)
 OZ_STATIC_MAX_LINES = 262144
 
 EXPORTS = ["oz_set_info", "oz_plane_count", "oz_plane_count_side", "oz_row_pitch", "oz_residue_elem_bytes", "oz_workspace_bytes", "oz_set_workspace", "oz_dgemm",
-           "oz_dgemm_ex", "oz_dgemm_host", "oz_deconstruct", "oz_deconstruct_static",
+           "oz_dgemm_ex", "oz_dgemm_host", "oz_operand_bytes", "oz_product_workspace_bytes", "oz_prepare_operand",
+           "oz_dgemm_prepared", "oz_deconstruct", "oz_deconstruct_static",
            "oz_residue_gemm", "oz_reconstruct",
            "oz_query_status", "oz_set_stage_events", "oz_launch_count", "oz_status_string"]
 
@@ -68,6 +69,12 @@ def load() -> C.CDLL:
     lib.oz_dgemm.argtypes = [i64, i64, i64, vp, i64, vp, i64, vp, i64, i32, u32, vp]
     lib.oz_dgemm_ex.argtypes = [i64, i64, i64, dbl, vp, i64, vp, i64, dbl, vp, i64, i32, u32, vp]
     lib.oz_dgemm_host.argtypes = lib.oz_dgemm_ex.argtypes
+    lib.oz_operand_bytes.argtypes = [i32, i64, i64, i32, u32]
+    lib.oz_operand_bytes.restype = C.c_size_t
+    lib.oz_product_workspace_bytes.argtypes = [i64, i64, i32]
+    lib.oz_product_workspace_bytes.restype = C.c_size_t
+    lib.oz_prepare_operand.argtypes = [i32, i64, i64, vp, i64, i32, u32, vp, C.c_size_t, vp]
+    lib.oz_dgemm_prepared.argtypes = [i64, i64, i64, dbl, vp, vp, dbl, vp, i64, i32, u32, vp]
     lib.oz_deconstruct.argtypes = [i32, i64, i64, vp, i64, i32, u32, vp, i64, i64, vp, vp, vp]
     lib.oz_deconstruct_static.argtypes = [i32, i64, i64, vp, i64, i32, u32, vp, i64, i64, vp, vp]
     lib.oz_residue_gemm.argtypes = [i64, i64, i64, vp, i64, i64, vp, i64, i64, i32, u32, vp, i64,
@@ -160,6 +167,27 @@ def oz_dgemm_host(m, n, k, alpha, A, lda, B, ldb, beta, Cm, ldc, modset=OZ_SET_S
     """A, B, Cm are HOST tensors (pinned) or raw host addresses."""
     return load().oz_dgemm_host(m, n, k, alpha, _ptr(A), lda, _ptr(B), ldb, beta, _ptr(Cm), ldc,
                                 modset, route, _stream(stream))
+
+
+def oz_operand_bytes(side, lines, k, modset, route=0) -> int:
+    return load().oz_operand_bytes(side, lines, k, modset, route)
+
+
+def oz_product_workspace_bytes(m, n, modset) -> int:
+    return load().oz_product_workspace_bytes(m, n, modset)
+
+
+def oz_prepare_operand(side, lines, k, X, ldx, modset, route, operand, nbytes=None, stream=None) -> int:
+    if nbytes is None:
+        nbytes = operand.numel() * operand.element_size()
+    return load().oz_prepare_operand(side, lines, k, _ptr(X), ldx, modset, route, _ptr(operand), nbytes,
+                                     _stream(stream))
+
+
+def oz_dgemm_prepared(m, n, k, alpha, operandA, operandB, beta, Cm, ldc, modset=OZ_SET_S, route=0,
+                      stream=None) -> int:
+    return load().oz_dgemm_prepared(m, n, k, alpha, _ptr(operandA), _ptr(operandB), beta, _ptr(Cm), ldc,
+                                    modset, route, _stream(stream))
 
 
 def oz_deconstruct(side, lines, k, X, ldx, modset, route, planes, plane_stride, row_pitch, shift,

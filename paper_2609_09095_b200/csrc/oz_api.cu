@@ -27,8 +27,17 @@ cudaEvent_t g_fork[kMaxDevices] = {}, g_join[kMaxDevices] = {};
 void *g_workspace[kMaxDevices] = {};
 size_t g_workspace_bytes[kMaxDevices] = {};
 std::atomic<uint64_t> g_launches{0};
-cudaEvent_t g_stage_events[5] = {};
-bool g_stage_events_on = false;
+// per-stage timing hook: one set of five caller-owned events per device
+cudaEvent_t g_stage_events[kMaxDevices][5] = {};
+bool g_stage_events_on[kMaxDevices] = {};
+
+// the workspace registered for a device (read under the mutex that oz_set_workspace writes it under)
+void registered_workspace(int dev, char **ws, size_t *bytes)
+{
+    std::lock_guard<std::mutex> lock(g_mutex);
+    *ws = static_cast<char *>(g_workspace[dev]);
+    *bytes = g_workspace_bytes[dev];
+}
 
 // Is the integer v exactly representable in E4M3 (the set of Lemma 1)?  If so return its
 // byte code through *code.  OCP E4M3: bias 7, 3 mantissa bits, largest finite value 448.
@@ -239,28 +248,61 @@ struct Carve {
     }
 };
 
+// One deconstructed operand: shifts, scan scratch and planes in one caller-owned block.  Used both
+// for the call-scoped planes inside the workspace and for the planes that a caller keeps across
+// calls (oz_prepare_operand / oz_dgemm_prepared).
+struct OperandLayout {
+    size_t shift, scratch, planes, total;
+    int64_t pitch, stride;
+};
+
+OperandLayout operand_layout(int side, int64_t lines, int64_t k, int set, const Route &rt)
+{
+    OperandLayout o{};
+    Carve c;
+    o.pitch = round_up(k > 0 ? k : 1, 128);   // whole 128-byte lines per TMA box row (k = 5003 -> 5120)
+    o.stride = lines * o.pitch;
+    o.shift = c.take(4 * static_cast<size_t>(lines));
+    o.scratch = c.take(16 * static_cast<size_t>(lines) + 256);
+    o.planes = c.take(static_cast<size_t>(p_store(set, rt.layout(side))) * o.stride);
+    o.total = c.off;
+    return o;
+}
+
+struct OperandView {
+    int32_t *shift;
+    void *scratch;
+    uint8_t *planes;
+    int64_t pitch, stride;
+};
+
+OperandView operand_view(char *base, const OperandLayout &o)
+{
+    return OperandView{reinterpret_cast<int32_t *>(base + o.shift), base + o.scratch,
+                       reinterpret_cast<uint8_t *>(base + o.planes), o.pitch, o.stride};
+}
+
+size_t residue_bytes_total(int64_t m, int64_t n, int set)
+{
+    // the tile-ordered private array of the whole-method calls (whole tiles are stored)
+    return static_cast<size_t>(round_up(static_cast<int64_t>(residue_bytes(set)) * set_r(set) *
+                                        residue_tiling(m, n, set).mod_stride, 256));
+}
+
 struct Layout {
-    size_t shiftA, shiftB, scrA, scrB, PA, PB, R, total;
-    int64_t pitch, strideA, strideB, ldr, mod_stride;
+    OperandLayout A, B;
+    size_t offA, offB, R, total;
 };
 
 Layout make_layout(int64_t m, int64_t n, int64_t k, int set, const Route &rt)
 {
     Layout L{};
-    Carve c;
-    L.pitch = round_up(k > 0 ? k : 1, 128);   // whole 128-byte lines per TMA box row (k = 5003 -> 5120)
-    L.strideA = m * L.pitch;
-    L.strideB = n * L.pitch;
-    L.ldr = round_up(m, 16 / residue_bytes(set));      // residue rows start on 16-byte boundaries
-    L.mod_stride = n * L.ldr;
-    L.shiftA = c.take(4 * static_cast<size_t>(m));
-    L.shiftB = c.take(4 * static_cast<size_t>(n));
-    L.scrA = c.take(16 * static_cast<size_t>(m) + 256);
-    L.scrB = c.take(16 * static_cast<size_t>(n) + 256);
-    L.PA = c.take(static_cast<size_t>(p_store(set, rt.layout(0))) * L.strideA);
-    L.PB = c.take(static_cast<size_t>(p_store(set, rt.layout(1))) * L.strideB);
-    L.R = c.take(static_cast<size_t>(residue_bytes(set)) * set_r(set) * L.mod_stride);
-    L.total = c.off;
+    L.A = operand_layout(0, m, k, set, rt);
+    L.B = operand_layout(1, n, k, set, rt);
+    L.offA = 0;
+    L.offB = L.A.total;
+    L.R = L.offB + L.B.total;
+    L.total = L.R + residue_bytes_total(m, n, set);
     return L;
 }
 
@@ -277,37 +319,75 @@ struct PanelPlan {
     cudaEvent_t *before, *after;
 };
 
+// residue GEMMs + reconstruction from two deconstructed operands (stage events [2]..[4])
+oz_status_t product_impl(int64_t m, int64_t n, int64_t k, double alpha, const OperandView &a,
+                         const OperandView &b, double beta, double *C, int64_t ldc, int set,
+                         const Route &rt, cudaStream_t stream, void *R, int dev, const PanelPlan *plan)
+{
+    const bool ev = g_stage_events_on[dev];
+    if (ev) OZ_CUDA_CHECK(cudaEventRecord(g_stage_events[dev][2], stream));
+    // the residues stay inside this call: tile-ordered, and the two-byte sets skip the canonicalisation
+    oz_status_t st = launch_residue_gemm(m, n, k, a.planes, a.stride, a.pitch, b.planes, b.stride, b.pitch, set,
+                                         rt, R, 0, 0, residue_bytes(set) == 2, true, stream);
+    if (st != OZ_OK) return st;
+    if (ev) OZ_CUDA_CHECK(cudaEventRecord(g_stage_events[dev][3], stream));
+    if (!plan) {
+        st = launch_reconstruct_tiled(m, n, R, a.shift, b.shift, set, alpha, beta, C, ldc, 0, n, stream);
+        if (st != OZ_OK) return st;
+    } else {
+        for (int p = 0; p < plan->np; ++p) {
+            if (plan->wait_before) OZ_CUDA_CHECK(cudaStreamWaitEvent(stream, plan->before[p], 0));
+            st = launch_reconstruct_tiled(m, n, R, a.shift, b.shift, set, alpha, beta, C, ldc, plan->col0[p],
+                                          plan->col0[p + 1], stream);
+            if (st != OZ_OK) return st;
+            OZ_CUDA_CHECK(cudaEventRecord(plan->after[p], stream));
+        }
+    }
+    if (ev) OZ_CUDA_CHECK(cudaEventRecord(g_stage_events[dev][4], stream));
+    return OZ_OK;
+}
+
+// checks shared by the whole-method entry points; *trivial: nothing (more) to do after k == 0 handling
+oz_status_t check_product_args(int64_t m, int64_t n, int64_t k, double alpha, double beta, double *C,
+                               int64_t ldc, int set, uint32_t route, cudaStream_t stream, Route *rt,
+                               bool *trivial)
+{
+    *trivial = true;
+    if (!valid_set(set) || !decode_route_for_set(set, route, rt)) return OZ_ERR_INVALID_ARG;
+    if (m < 0 || n < 0 || k < 0) return OZ_ERR_INVALID_ARG;
+    if (!(alpha == 1.0 || alpha == -1.0) || !(beta == 0.0 || beta == 1.0)) return OZ_ERR_UNSUPPORTED;
+    if (k > OZ_K_MAX) return OZ_ERR_UNSUPPORTED;
+    if (resolve_schedule(set, k, n, true, rt) != OZ_OK) return OZ_ERR_UNSUPPORTED;
+    if (m == 0 || n == 0) return OZ_OK;
+    if (!C || ldc < m || (reinterpret_cast<uintptr_t>(C) & 7u)) return OZ_ERR_INVALID_ARG;
+    if (k == 0) {
+        if (beta == 0.0)
+            OZ_CUDA_CHECK(cudaMemset2DAsync(C, sizeof(double) * ldc, 0, sizeof(double) * m, n, stream));
+        return OZ_OK;
+    }
+    *trivial = false;
+    return OZ_OK;
+}
+
 oz_status_t dgemm_impl(int64_t m, int64_t n, int64_t k, double alpha, const double *A, int64_t lda,
                        const double *B, int64_t ldb, double beta, double *C, int64_t ldc, int set,
                        uint32_t route, cudaStream_t stream, char *ws, size_t ws_bytes,
                        const PanelPlan *plan = nullptr)
 {
     Route rt;
-    if (!valid_set(set) || !decode_route_for_set(set, route, &rt)) return OZ_ERR_INVALID_ARG;
-    if (m < 0 || n < 0 || k < 0) return OZ_ERR_INVALID_ARG;
-    if (!(alpha == 1.0 || alpha == -1.0) || !(beta == 0.0 || beta == 1.0)) return OZ_ERR_UNSUPPORTED;
-    if (k > OZ_K_MAX) return OZ_ERR_UNSUPPORTED;
-    if (resolve_schedule(set, k, n, true, &rt) != OZ_OK) return OZ_ERR_UNSUPPORTED;
-    if (m == 0 || n == 0) return OZ_OK;
-    if (!C || ldc < m) return OZ_ERR_INVALID_ARG;
-    if (k == 0) {
-        if (beta == 0.0)
-            OZ_CUDA_CHECK(cudaMemset2DAsync(C, sizeof(double) * ldc, 0, sizeof(double) * m, n, stream));
-        return OZ_OK;
-    }
-    if (!A || !B || lda < m || ldb < k) return OZ_ERR_INVALID_ARG;
+    bool trivial = true;
+    oz_status_t st = check_product_args(m, n, k, alpha, beta, C, ldc, set, route, stream, &rt, &trivial);
+    if (st != OZ_OK || trivial) return st;
+    if (!A || !B || lda < m || ldb < k || (reinterpret_cast<uintptr_t>(A) & 7u) ||
+        (reinterpret_cast<uintptr_t>(B) & 7u))
+        return OZ_ERR_INVALID_ARG;
     Layout L = make_layout(m, n, k, set, rt);
     if (!ws || ws_bytes < L.total) return OZ_ERR_WORKSPACE;
-    oz_status_t st = ensure_device_ready();
+    st = ensure_device_ready();
     if (st != OZ_OK) return st;
+    const OperandView a = operand_view(ws + L.offA, L.A), b = operand_view(ws + L.offB, L.B);
 
-    int32_t *shiftA = reinterpret_cast<int32_t *>(ws + L.shiftA);
-    int32_t *shiftB = reinterpret_cast<int32_t *>(ws + L.shiftB);
-    uint8_t *PA = reinterpret_cast<uint8_t *>(ws + L.PA);
-    uint8_t *PB = reinterpret_cast<uint8_t *>(ws + L.PB);
-    void *R = ws + L.R;
-
-    // The two operands are deconstructed side by side: B's chain of five short kernels runs on an
+    // The two operands are deconstructed side by side: B's chain of short kernels runs on an
     // internal stream that forks from and joins the caller's (their scratch, planes and shifts are
     // disjoint).  Stage event [1] marks the end of A's chain, [2] the join.
     int dev = 0;
@@ -315,40 +395,18 @@ oz_status_t dgemm_impl(int64_t m, int64_t n, int64_t k, double alpha, const doub
     st = ensure_side_stream(dev);
     if (st != OZ_OK) return st;
     cudaStream_t side = g_side_stream[dev];
-    const bool ev = g_stage_events_on;
-    if (ev) OZ_CUDA_CHECK(cudaEventRecord(g_stage_events[0], stream));
+    const bool ev = g_stage_events_on[dev];
+    if (ev) OZ_CUDA_CHECK(cudaEventRecord(g_stage_events[dev][0], stream));
     OZ_CUDA_CHECK(cudaEventRecord(g_fork[dev], stream));
     OZ_CUDA_CHECK(cudaStreamWaitEvent(side, g_fork[dev], 0));
-    st = launch_deconstruct(1, n, k, B, ldb, set, rt, PB, L.strideB, L.pitch, shiftB, ws + L.scrB, side);
+    st = launch_deconstruct(1, n, k, B, ldb, set, rt, b.planes, b.stride, b.pitch, b.shift, b.scratch, side);
     if (st != OZ_OK) return st;
     OZ_CUDA_CHECK(cudaEventRecord(g_join[dev], side));
-    st = launch_deconstruct(0, m, k, A, lda, set, rt, PA, L.strideA, L.pitch, shiftA, ws + L.scrA, stream);
+    st = launch_deconstruct(0, m, k, A, lda, set, rt, a.planes, a.stride, a.pitch, a.shift, a.scratch, stream);
     if (st != OZ_OK) return st;
-    if (ev) OZ_CUDA_CHECK(cudaEventRecord(g_stage_events[1], stream));
+    if (ev) OZ_CUDA_CHECK(cudaEventRecord(g_stage_events[dev][1], stream));
     OZ_CUDA_CHECK(cudaStreamWaitEvent(stream, g_join[dev], 0));
-    if (ev) OZ_CUDA_CHECK(cudaEventRecord(g_stage_events[2], stream));
-    // the residues stay inside this call: the two-byte sets skip the canonicalisation
-    st = launch_residue_gemm(m, n, k, PA, L.strideA, L.pitch, PB, L.strideB, L.pitch, set, rt, R,
-                             L.ldr, L.mod_stride, residue_bytes(set) == 2, stream);
-    if (st != OZ_OK) return st;
-    if (ev) OZ_CUDA_CHECK(cudaEventRecord(g_stage_events[3], stream));
-    if (!plan) {
-        st = launch_reconstruct(m, n, R, L.ldr, L.mod_stride, shiftA, shiftB, set, alpha, beta, C, ldc,
-                                stream);
-        if (st != OZ_OK) return st;
-    } else {
-        for (int p = 0; p < plan->np; ++p) {
-            const int64_t j0 = plan->col0[p], cols = plan->col0[p + 1] - j0;
-            if (plan->wait_before) OZ_CUDA_CHECK(cudaStreamWaitEvent(stream, plan->before[p], 0));
-            st = launch_reconstruct(m, cols, static_cast<char *>(R) + j0 * L.ldr * residue_bytes(set), L.ldr,
-                                    L.mod_stride, shiftA, shiftB + j0, set, alpha, beta, C + j0 * ldc, ldc,
-                                    stream);
-            if (st != OZ_OK) return st;
-            OZ_CUDA_CHECK(cudaEventRecord(plan->after[p], stream));
-        }
-    }
-    if (ev) OZ_CUDA_CHECK(cudaEventRecord(g_stage_events[4], stream));
-    return OZ_OK;
+    return product_impl(m, n, k, alpha, a, b, beta, C, ldc, set, rt, stream, ws + L.R, dev, plan);
 }
 
 // Side streams and events of the host-buffer entry point, created once per device.
@@ -443,9 +501,11 @@ oz_status_t oz_dgemm_ex(int64_t m, int64_t n, int64_t k, double alpha, const dou
     int dev = 0;
     OZ_CUDA_CHECK(cudaGetDevice(&dev));
     if (dev < 0 || dev >= kMaxDevices) return OZ_ERR_CUDA;
+    char *ws = nullptr;
+    size_t ws_bytes = 0;
+    registered_workspace(dev, &ws, &ws_bytes);
     return dgemm_impl(m, n, k, alpha, A, lda, B, ldb, beta, C, ldc, set, route,
-                      static_cast<cudaStream_t>(stream), static_cast<char *>(g_workspace[dev]),
-                      g_workspace_bytes[dev]);
+                      static_cast<cudaStream_t>(stream), ws, ws_bytes);
 }
 
 oz_status_t oz_dgemm(int64_t m, int64_t n, int64_t k, const double *A, int64_t lda, const double *B,
@@ -471,13 +531,15 @@ oz_status_t oz_dgemm_host(int64_t m, int64_t n, int64_t k, double alpha, const d
     if (!C_host || ldc < m || (k > 0 && (!A_host || !B_host || lda < m || ldb < k)))
         return OZ_ERR_INVALID_ARG;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    char *ws = static_cast<char *>(g_workspace[dev]);
+    char *ws = nullptr;
+    size_t ws_have = 0;
+    registered_workspace(dev, &ws, &ws_have);
     int64_t kk = k > 0 ? k : 1;
     size_t core = make_layout(m, n, kk, set, rt).total;
     size_t bytesA = 8 * static_cast<size_t>(m) * kk, bytesB = 8 * static_cast<size_t>(kk) * n;
     size_t bytesC = 8 * static_cast<size_t>(m) * n;
     size_t offA = core, offB = offA + round_up(bytesA, 256), offC = offB + round_up(bytesB, 256);
-    if (!ws || g_workspace_bytes[dev] < offC + bytesC) return OZ_ERR_WORKSPACE;
+    if (!ws || ws_have < offC + bytesC) return OZ_ERR_WORKSPACE;
     double *dA = reinterpret_cast<double *>(ws + offA);
     double *dB = reinterpret_cast<double *>(ws + offB);
     double *dC = reinterpret_cast<double *>(ws + offC);
@@ -536,6 +598,76 @@ oz_status_t oz_dgemm_host(int64_t m, int64_t n, int64_t k, double alpha, const d
     return OZ_OK;
 }
 
+size_t oz_operand_bytes(int side, int64_t lines, int64_t k, oz_modset_t set, uint32_t route)
+{
+    Route rt;
+    if (!valid_set(set) || !decode_route_for_set(set, route, &rt) || (side != 0 && side != 1) || lines < 0 ||
+        k < 0 || k > OZ_K_MAX)
+        return 0;
+    if (resolve_schedule(set, k, 0, true, &rt) != OZ_OK) return 0;
+    return operand_layout(side, lines > 0 ? lines : 1, k > 0 ? k : 1, set, rt).total;
+}
+
+size_t oz_product_workspace_bytes(int64_t m, int64_t n, oz_modset_t set)
+{
+    if (!valid_set(set) || m < 0 || n < 0) return 0;
+    return residue_bytes_total(m > 0 ? m : 1, n > 0 ? n : 1, set);
+}
+
+oz_status_t oz_prepare_operand(int side, int64_t lines, int64_t k, const double *X, int64_t ldx,
+                               oz_modset_t set, uint32_t route, void *operand, size_t bytes,
+                               void *stream)
+{
+    Route rt;
+    if (!valid_set(set) || !decode_route_for_set(set, route, &rt) || (side != 0 && side != 1))
+        return OZ_ERR_INVALID_ARG;
+    if (lines < 0 || k < 0) return OZ_ERR_INVALID_ARG;
+    if (k > OZ_K_MAX) return OZ_ERR_UNSUPPORTED;
+    if (resolve_schedule(set, k, 0, true, &rt) != OZ_OK) return OZ_ERR_UNSUPPORTED;
+    if (lines == 0 || k == 0) return OZ_OK;           // nothing to keep: a product with k = 0 reads no operand
+    if (!X || !operand || (reinterpret_cast<uintptr_t>(operand) & 255u) || (reinterpret_cast<uintptr_t>(X) & 7u) ||
+        ldx < (side == 0 ? lines : k))
+        return OZ_ERR_INVALID_ARG;
+    const OperandLayout o = operand_layout(side, lines, k, set, rt);
+    if (bytes < o.total) return OZ_ERR_WORKSPACE;
+    oz_status_t st = ensure_device_ready();
+    if (st != OZ_OK) return st;
+    const OperandView v = operand_view(static_cast<char *>(operand), o);
+    return launch_deconstruct(side, lines, k, X, ldx, set, rt, v.planes, v.stride, v.pitch, v.shift, v.scratch,
+                              static_cast<cudaStream_t>(stream));
+}
+
+oz_status_t oz_dgemm_prepared(int64_t m, int64_t n, int64_t k, double alpha, const void *operandA,
+                              const void *operandB, double beta, double *C, int64_t ldc,
+                              oz_modset_t set, uint32_t route, void *stream)
+{
+    int dev = 0;
+    OZ_CUDA_CHECK(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return OZ_ERR_CUDA;
+    Route rt;
+    bool trivial = true;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    oz_status_t st = check_product_args(m, n, k, alpha, beta, C, ldc, set, route, s, &rt, &trivial);
+    if (st != OZ_OK || trivial) return st;
+    if (!operandA || !operandB || (reinterpret_cast<uintptr_t>(operandA) & 255u) ||
+        (reinterpret_cast<uintptr_t>(operandB) & 255u))
+        return OZ_ERR_INVALID_ARG;
+    char *ws = nullptr;
+    size_t ws_bytes = 0;
+    registered_workspace(dev, &ws, &ws_bytes);
+    if (!ws || ws_bytes < residue_bytes_total(m, n, set)) return OZ_ERR_WORKSPACE;
+    st = ensure_device_ready();
+    if (st != OZ_OK) return st;
+    const OperandView a = operand_view(static_cast<char *>(const_cast<void *>(operandA)), operand_layout(0, m, k, set, rt));
+    const OperandView b = operand_view(static_cast<char *>(const_cast<void *>(operandB)), operand_layout(1, n, k, set, rt));
+    if (g_stage_events_on[dev]) {
+        // no deconstruction in this call: the first three events coincide
+        OZ_CUDA_CHECK(cudaEventRecord(g_stage_events[dev][0], s));
+        OZ_CUDA_CHECK(cudaEventRecord(g_stage_events[dev][1], s));
+    }
+    return product_impl(m, n, k, alpha, a, b, beta, C, ldc, set, rt, s, ws, dev, nullptr);
+}
+
 oz_status_t oz_deconstruct(int side, int64_t lines, int64_t k, const double *X, int64_t ldx,
                            oz_modset_t set, uint32_t route, uint8_t *planes, int64_t plane_stride,
                            int64_t row_pitch, int32_t *shift, void *scratch, void *stream)
@@ -550,7 +682,8 @@ oz_status_t oz_deconstruct(int side, int64_t lines, int64_t k, const double *X, 
     if (!planes || !shift || !scratch || (k > 0 && !X)) return OZ_ERR_INVALID_ARG;
     if (row_pitch < k || row_pitch < 16 || (row_pitch & 15) || (plane_stride & 15) ||
         plane_stride < lines * row_pitch || (reinterpret_cast<uintptr_t>(planes) & 15u) ||
-        (reinterpret_cast<uintptr_t>(scratch) & 255u))
+        (reinterpret_cast<uintptr_t>(scratch) & 255u) || (reinterpret_cast<uintptr_t>(shift) & 3u) ||
+        (reinterpret_cast<uintptr_t>(X) & 7u))
         return OZ_ERR_INVALID_ARG;
     if (k > 0 && ldx < (side == 0 ? lines : k)) return OZ_ERR_INVALID_ARG;
     oz_status_t st = ensure_device_ready();
@@ -571,6 +704,7 @@ oz_status_t oz_residue_gemm(int64_t m, int64_t n, int64_t k, const uint8_t *PA, 
     if (resolve_schedule(set, k, 0, false, &rt) != OZ_OK) return OZ_ERR_UNSUPPORTED;
     if (m == 0 || n == 0) return OZ_OK;
     if (!PA || !PB || !R || ldr < m || mod_stride < n * ldr) return OZ_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(R) % static_cast<uintptr_t>(residue_bytes(set))) return OZ_ERR_INVALID_ARG;
     if ((pitchA & 15) || (pitchB & 15) || (strideA & 15) || (strideB & 15) || pitchA < k ||
         pitchB < k || pitchA < 16 || pitchB < 16 || strideA < m * pitchA || strideB < n * pitchB ||
         (reinterpret_cast<uintptr_t>(PA) & 15u) || (reinterpret_cast<uintptr_t>(PB) & 15u))
@@ -578,7 +712,7 @@ oz_status_t oz_residue_gemm(int64_t m, int64_t n, int64_t k, const uint8_t *PA, 
     oz_status_t st = ensure_device_ready();
     if (st != OZ_OK) return st;
     return launch_residue_gemm(m, n, k, PA, strideA, pitchA, PB, strideB, pitchB, set, rt, R, ldr,
-                               mod_stride, false, static_cast<cudaStream_t>(stream));
+                               mod_stride, false, false, static_cast<cudaStream_t>(stream));
 }
 
 oz_status_t oz_reconstruct(int64_t m, int64_t n, const void *R, int64_t ldr, int64_t mod_stride,
@@ -589,6 +723,10 @@ oz_status_t oz_reconstruct(int64_t m, int64_t n, const void *R, int64_t ldr, int
     if (!(alpha == 1.0 || alpha == -1.0) || !(beta == 0.0 || beta == 1.0)) return OZ_ERR_UNSUPPORTED;
     if (m == 0 || n == 0) return OZ_OK;
     if (!R || !shiftA || !shiftB || !C || ldr < m || mod_stride < n * ldr || ldc < m)
+        return OZ_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(R) % static_cast<uintptr_t>(residue_bytes(set)) ||
+        (reinterpret_cast<uintptr_t>(shiftA) & 3u) || (reinterpret_cast<uintptr_t>(shiftB) & 3u) ||
+        (reinterpret_cast<uintptr_t>(C) & 7u))
         return OZ_ERR_INVALID_ARG;
     oz_status_t st = ensure_device_ready();
     if (st != OZ_OK) return st;
@@ -614,13 +752,17 @@ oz_status_t oz_query_status(void *stream)
 
 oz_status_t oz_set_stage_events(void *const *events)
 {
+    int dev = 0;
+    OZ_CUDA_CHECK(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return OZ_ERR_CUDA;
     std::lock_guard<std::mutex> lock(g_mutex);
-    g_stage_events_on = events != nullptr;
-    for (int i = 0; i < 5; ++i)
-        g_stage_events[i] = events ? static_cast<cudaEvent_t>(events[i]) : nullptr;
+    g_stage_events_on[dev] = false;
     if (events)
         for (int i = 0; i < 5; ++i)
-            if (!events[i]) { g_stage_events_on = false; return OZ_ERR_INVALID_ARG; }
+            if (!events[i]) return OZ_ERR_INVALID_ARG;
+    for (int i = 0; i < 5; ++i)
+        g_stage_events[dev][i] = events ? static_cast<cudaEvent_t>(events[i]) : nullptr;
+    g_stage_events_on[dev] = events != nullptr;
     return OZ_OK;
 }
 

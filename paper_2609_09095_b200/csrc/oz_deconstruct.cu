@@ -381,8 +381,9 @@ oz_status_t launch_convert(const double *X, int64_t ldx, int64_t lines, int64_t 
     if (lines * nchunks >= 0x7FFFFFFFll) return OZ_ERR_UNSUPPORTED;   // item numbers are 32-bit
     int64_t need = SIDE == 1 ? (lines * nchunks + 7) / 8
                              : ((lines + kTileLines - 1) / kTileLines) * nchunks;
-    int sms = 148;
-    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, 0);
+    int dev = 0, sms = 148;
+    OZ_CUDA_CHECK(cudaGetDevice(&dev));
+    OZ_CUDA_CHECK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
     int64_t cap = static_cast<int64_t>(sms) * (SIDE == 1 ? 6 : 3);
     int grid = static_cast<int>(need < cap ? need : cap);
     convert_kernel<SET, SIDE, LAYOUT><<<grid, kConvThreads, smem, stream>>>(

@@ -61,7 +61,8 @@ extern "C" oz_status_t oz_deconstruct_static(int side, int64_t lines, int64_t k,
     if (lines == 0) return OZ_OK;
     if (!planes || !shift || (k > 0 && !X)) return OZ_ERR_INVALID_ARG;
     if (row_pitch < k || row_pitch < 16 || (row_pitch & 15) || (plane_stride & 15) ||
-        plane_stride < lines * row_pitch || (reinterpret_cast<uintptr_t>(planes) & 15u))
+        plane_stride < lines * row_pitch || (reinterpret_cast<uintptr_t>(planes) & 15u) ||
+        (reinterpret_cast<uintptr_t>(shift) & 3u) || (reinterpret_cast<uintptr_t>(X) & 7u))
         return OZ_ERR_INVALID_ARG;
     if (k > 0 && ldx < (side == 0 ? lines : k)) return OZ_ERR_INVALID_ARG;
     oz_status_t st = oz::ensure_device_ready();

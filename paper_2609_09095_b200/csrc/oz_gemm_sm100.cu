@@ -24,14 +24,14 @@
 // contiguous in the column-major residue array; a warp transposes its 32 x 64 block through a
 // small swizzled shared-memory buffer so that each store instruction writes whole lines.
 //
-// Kernel structure (one persistent CTA per SM, 640 threads, 96 registers each; launched as
+// Kernel structure (one persistent CTA per SM, 576 threads, up to 112 registers each; launched as
 // clusters of two CTAs that share one tcgen05.mma.cta_group::2 unless n pads badly to 256):
 //   warp 0       TMA producer: 128-byte-swizzled K-major tiles of B (128 lines) and A (256 lines,
 //                or this CTA's half of them in a pair) into a shared-memory ring of 192 KiB
 //                (4 stages of 48 KiB, or 6 of 32 KiB in a pair), no multicast
 //   warp 1       MMA issuer: one lane issues tcgen05.mma (M=128 or 256 across the pair, N=256,
 //                K=32); accumulators live in TMEM, two slots of 256 columns used alternately per job
-//   warps 4..19  epilogue (4 per TMEM lane quarter, 64 columns each): tcgen05.ld the finished slot,
+//   warps 2..17  epilogue (4 per TMEM lane quarter, 64 columns each): tcgen05.ld the finished slot,
 //                reduce each accumulator modulo m_i in FP32 (all values are integers below 2^24,
 //                every step exact), fold it with the job's weight into a per-thread running
 //                combination held in registers, release the slot; after the last job reduce once
@@ -52,6 +52,7 @@
 // word, every role leaves its loops, in-flight copies are given a bounded time to land, TMEM is
 // freed and the kernel returns.
 #include <cuda.h>
+#include <atomic>
 #include <cstdlib>
 
 #include "oz_internal.h"
@@ -80,10 +81,15 @@ struct Tile {
     static constexpr int TILE_J = BLOCK_M * CG;                  // columns of C per work item
 };
 constexpr int TMEM_COLS = 512;                     // two accumulator slots of BLOCK_N columns
-constexpr int NUM_THREADS = 640;
-constexpr int FIRST_EPI_WARP = 4;                  // warps 0..3: producer, MMA issuer, two idle
+constexpr int NUM_THREADS = 576;                   // 18 warps: 112 registers each fit the register file
+constexpr int FIRST_EPI_WARP = 2;                  // warp 0: producer, warp 1: MMA issuer
 constexpr int EPI_WARPS = 16;
 constexpr int COLS_PER_WARP = BLOCK_N / 4;         // four warps share a TMEM lane quarter
+#ifndef OZ_DRAIN_W
+#define OZ_DRAIN_W 16
+#endif
+constexpr int DRAIN_W = OZ_DRAIN_W;                // accumulator columns per tcgen05.ld of a drain: 64 running
+                                                   // values + 16 loaded ones stay inside the 96 registers
 constexpr int XPOSE_BYTES = 16 * 128;                // per epilogue warp: 16 lines x 128 bytes
 constexpr size_t SMEM_BYTES = 4 * 49152 + EPI_WARPS * XPOSE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
 static_assert(Tile<1>::STAGES * Tile<1>::STAGE_BYTES == 4 * 49152 && Tile<2>::STAGES * Tile<2>::STAGE_BYTES == 4 * 49152, "ring size");
@@ -296,8 +302,10 @@ __device__ __forceinline__ void umma_commit(uint32_t bar)
     }
 }
 
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32])
+template <int N>
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[N])
 {
+    static_assert(N == 32, "32 columns");
     asm volatile(
         "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
         "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
@@ -307,6 +315,22 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32])
           "=r"(v[14]), "=r"(v[15]), "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]),
           "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]),
           "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+        : "r"(taddr)
+        : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+// 16 columns of the warp's 32 lanes, with the wait
+template <int N>
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&v)[N])
+{
+    static_assert(N == 16, "16 columns");
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]),
+          "=r"(v[7]), "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]),
+          "=r"(v[14]), "=r"(v[15])
         : "r"(taddr)
         : "memory");
     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
@@ -419,6 +443,15 @@ __device__ __forceinline__ void segment_range(const ModInfo &mi, int job, int se
     *kc1 = min(nk, *kc0 + len);
 }
 
+// acc - m * rint(acc / m) for a pair of integer-valued floats below 2^24 (exact): rint through the
+// 1.5 * 2^23 constant, then one fused multiply-add
+__device__ __forceinline__ float2 mod_balanced2(float2 acc, float2 inv_m2, float2 neg_m2)
+{
+    const float2 big = make_float2(12582912.0f, 12582912.0f), neg_big = make_float2(-12582912.0f, -12582912.0f);
+    const float2 quot = __fadd2_rn(__ffma2_rn(acc, inv_m2, big), neg_big);
+    return __ffma2_rn(quot, neg_m2, acc);
+}
+
 // RB: bytes of one stored residue (2: uint16, 1: uint8 for the all-byte modulus set)
 // DIRECT: native INT8 residues -- one accumulator per modulus, loaded straight into the registers
 //         that otherwise hold the running combination of several accumulators
@@ -426,7 +459,13 @@ __device__ __forceinline__ void segment_range(const ModInfo &mi, int job, int se
 //         [0, m_i) (two-byte residues only).  The reconstruction is indifferent to it -- the CRT
 //         weight of m_i is a multiple of M -- and the epilogue saves the canonicalisation; used for
 //         the residues that stay inside the whole-method calls.
-template <int SUB, int CG, int RB, bool DIRECT, bool LOOSE>
+// TILED: the residue array is the private, tile-ordered one of the whole-method calls (see
+//         residue_tiling() below): the 32 columns x 64 rows that an epilogue warp owns form one
+//         contiguous block, [16-byte chunk][lane], so that every store instruction of a warp writes
+//         512 consecutive bytes straight from registers -- no transposition through shared memory,
+//         which the tensor pipe and the TMA writes need for themselves.  The reconstruction reads
+//         the same order.  Without it the public layout R[mod][j][ldr] is written.
+template <int SUB, int CG, int RB, bool DIRECT, bool LOOSE, bool TILED>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 residue_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB,
                     const __grid_constant__ GemmParams p)
@@ -568,7 +607,8 @@ residue_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
     } else {
         // ------------------------------------------------------------ epilogue
         const int q = warp & 3;                              // TMEM lane quarter this warp may read
-        const int part = (warp - FIRST_EPI_WARP) >> 2;       // which 64 of the tile's 256 TMEM columns
+        const int part = (warp - FIRST_EPI_WARP) >> 2;       // which 64 of the tile's 256 TMEM columns (any four
+                                                             // consecutive warps cover the four lane quarters)
         int slot = 0;
         uint32_t slot_phase = 0;   // bit s = phase of slot s
         bool ok = true;
@@ -577,6 +617,7 @@ residue_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
             const ModInfo &mi = p.mod[it.mod];
             const float mm = mi.m, inv_m = mi.inv_m;
             const float loose_offset = mm + 8388608.0f;          // exact: m < 2^11
+            const float2 inv_m2 = make_float2(inv_m, inv_m), neg_m2 = make_float2(-mm, -mm);
             const uint32_t im = mi.mi, imagic = mi.magic, ibias = mi.bias;
             // running combination per element: FP32 (FP8 route) or INT32 (INT8 routes), as raw bits
             uint32_t comb[COLS_PER_WARP];
@@ -584,11 +625,11 @@ residue_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
 #pragma unroll
                 for (int c = 0; c < COLS_PER_WARP; ++c) comb[c] = 0u;
             }
-            // canonical residues in [0, m), packed 4 / RB to a word in row order
-            uint32_t packed[COLS_PER_WARP * RB / 4];
             for (int job = 0; ok && job < mi.njobs; ++job)
             for (int seg = 0, nseg = job_segments(mi, job); ok && seg < nseg; ++seg) {
-                ok = mbar_wait(tfull_bar + 8 * slot, (slot_phase >> slot) & 1u, abort_flag, p.status);
+                // every lane polls for itself; the verdict is made warp-uniform before anything that
+                // contains a warp barrier depends on it
+                ok = __all_sync(0xFFFFFFFFu, mbar_wait(tfull_bar + 8 * slot, (slot_phase >> slot) & 1u, abort_flag, p.status));
                 if (!ok) break;
                 tc_fence_after();
                 const float wj = mi.w[job];
@@ -602,30 +643,40 @@ residue_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
                     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
                 } else
 #pragma unroll
-                for (int c0 = 0; c0 < COLS_PER_WARP; c0 += 32) {
-                    uint32_t v[32];
-                    tmem_ld32(taddr + c0, v);
+                for (int c0 = 0; c0 < COLS_PER_WARP; c0 += DRAIN_W) {
+                    uint32_t v[DRAIN_W];
+                    if constexpr (DRAIN_W == 32) tmem_ld32(taddr + c0, v);
+                    else tmem_ld16(taddr + c0, v);
                     if constexpr (SUB == 0) {
+                        // two values per instruction (packed FP32 pairs): half the issue slots
+                        const float2 wj2 = make_float2(wj, wj);
                         if (reduce_first) {
 #pragma unroll
-                            for (int e = 0; e < 32; ++e) {
-                                float acc = __uint_as_float(v[e]);
-                                float quot = fmaf(acc, inv_m, 12582912.0f) - 12582912.0f;   // rint(acc/m)
-                                float res = fmaf(-quot, mm, acc);                            // exact, |res| <= ~m/2
-                                comb[c0 + e] = __float_as_uint(fmaf(res, wj, __uint_as_float(comb[c0 + e])));
+                            for (int e = 0; e < DRAIN_W; e += 2) {
+                                const float2 acc = make_float2(__uint_as_float(v[e]), __uint_as_float(v[e + 1]));
+                                const float2 res = mod_balanced2(acc, inv_m2, neg_m2);       // exact, |res| <= ~m/2
+                                const float2 cur = make_float2(__uint_as_float(comb[c0 + e]), __uint_as_float(comb[c0 + e + 1]));
+                                const float2 nxt = __ffma2_rn(res, wj2, cur);
+                                comb[c0 + e] = __float_as_uint(nxt.x);
+                                comb[c0 + e + 1] = __float_as_uint(nxt.y);
                             }
                         } else {
                             // the host has checked that w * acc stays below 2^24 for this k
 #pragma unroll
-                            for (int e = 0; e < 32; ++e)
-                                comb[c0 + e] = __float_as_uint(fmaf(__uint_as_float(v[e]), wj, __uint_as_float(comb[c0 + e])));
+                            for (int e = 0; e < DRAIN_W; e += 2) {
+                                const float2 acc = make_float2(__uint_as_float(v[e]), __uint_as_float(v[e + 1]));
+                                const float2 cur = make_float2(__uint_as_float(comb[c0 + e]), __uint_as_float(comb[c0 + e + 1]));
+                                const float2 nxt = __ffma2_rn(acc, wj2, cur);
+                                comb[c0 + e] = __float_as_uint(nxt.x);
+                                comb[c0 + e + 1] = __float_as_uint(nxt.y);
+                            }
                         }
                     } else {
                         // INT32 accumulators: exact integer arithmetic, no conversions
                         const int iwj = mi.iw[job];
                         if (reduce_first) {
 #pragma unroll
-                            for (int e = 0; e < 32; ++e) {
+                            for (int e = 0; e < DRAIN_W; ++e) {
                                 uint32_t u = v[e] + ibias;                       // non-negative, same residue
                                 uint32_t r = u - __umulhi(u, imagic) * im;       // in [0, 2m)
                                 r = min(r, r - im);
@@ -634,7 +685,7 @@ residue_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
                         } else {
                             // the host has checked that the weighted sum stays inside INT32 for this k
 #pragma unroll
-                            for (int e = 0; e < 32; ++e)
+                            for (int e = 0; e < DRAIN_W; ++e)
                                 comb[c0 + e] = static_cast<uint32_t>(static_cast<int>(v[e]) * iwj + static_cast<int>(comb[c0 + e]));
                         }
                     }
@@ -654,36 +705,81 @@ residue_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
             const int64_t j = jw + lane;
             const int64_t i0 = static_cast<int64_t>(it.tm) * BLOCK_N + part * COLS_PER_WARP;
             if (i0 >= p.m || jw >= p.n) continue;                                 // warp-uniform
+            // last reduction of one combination value: the stored residue in the low bits of a word
+            auto final_bits = [&](uint32_t cv) -> uint32_t {
+                if constexpr (SUB == 0) {
+                    float t = __uint_as_float(cv);
+                    float quot = fmaf(t, inv_m, 12582912.0f) - 12582912.0f;
+                    float res = fmaf(-quot, mm, t);                      // |res| <= ~m/2
+                    if constexpr (LOOSE) {
+                        return __float_as_uint(res + loose_offset);      // res + m in (0, 2m), low mantissa bits
+                    } else {
+                        res = res < 0.0f ? res + mm : res;               // canonical [0, m)
+                        return __float_as_uint(res + 8388608.0f);        // integer in the low mantissa bits
+                    }
+                } else if constexpr (DIRECT) {
+                    uint32_t u = cv + mi.bias30;                          // in (0, 2^31 + 256)
+                    return u - (__umulhi(u, mi.magic39) >> 7) * im;      // exact quotient: canonical [0, m)
+                } else {
+                    uint32_t u = cv + ibias;
+                    uint32_t r = u - __umulhi(u, imagic) * im;           // in [0, 2m)
+                    return LOOSE ? r : min(r, r - im);                   // canonical [0, m) unless LOOSE
+                }
+            };
+            // same for two values at once; the loose FP32 form is done with packed pairs
+            auto final_bits2 = [&](uint32_t c0v, uint32_t c1v, uint32_t &b0, uint32_t &b1) {
+                if constexpr (SUB == 0 && LOOSE) {
+                    const float2 res = mod_balanced2(make_float2(__uint_as_float(c0v), __uint_as_float(c1v)), inv_m2, neg_m2);
+                    const float2 out = __fadd2_rn(res, make_float2(loose_offset, loose_offset));
+                    b0 = __float_as_uint(out.x);
+                    b1 = __float_as_uint(out.y);
+                } else {
+                    b0 = final_bits(c0v);
+                    b1 = final_bits(c1v);
+                }
+            };
+            // four consecutive rows starting at combination value c -> one (RB = 1) or two (RB = 2) words
+            auto pack4 = [&](int c, uint32_t &w0, uint32_t &w1) {
+                uint32_t b0, b1, b2, b3;
+                final_bits2(comb[c], comb[c + 1], b0, b1);
+                final_bits2(comb[c + 2], comb[c + 3], b2, b3);
+                if constexpr (RB == 2) {
+                    w0 = __byte_perm(b0, b1, 0x5410);
+                    w1 = __byte_perm(b2, b3, 0x5410);
+                } else {
+                    w0 = __byte_perm(__byte_perm(b0, b1, 0x0040), __byte_perm(b2, b3, 0x0040), 0x5410);
+                    w1 = 0u;
+                }
+            };
+            constexpr int NCH = COLS_PER_WARP * RB / 16;     // 16-byte chunks of a thread's run of rows
+            if constexpr (TILED) {
+                unsigned char *blk = static_cast<unsigned char *>(p.R) +
+                    ((((static_cast<int64_t>(it.mod) * p.tiles_m + it.tm) * p.tiles_n + it.tn) * CG + rank) * EPI_WARPS +
+                     (part * 4 + q)) * static_cast<int64_t>(NCH * 512) + lane * 16;
+#pragma unroll
+                for (int c = 0; c < NCH; ++c) {
+                    uint4 val;
+                    if constexpr (RB == 2) {
+                        pack4(8 * c, val.x, val.y);
+                        pack4(8 * c + 4, val.z, val.w);
+                    } else {
+                        uint32_t unused;
+                        pack4(16 * c, val.x, unused);
+                        pack4(16 * c + 4, val.y, unused);
+                        pack4(16 * c + 8, val.z, unused);
+                        pack4(16 * c + 12, val.w, unused);
+                    }
+                    *reinterpret_cast<uint4 *>(blk + c * 512) = val;
+                }
+            } else {
+            // residues packed 4 / RB to a word in row order
+            uint32_t packed[COLS_PER_WARP * RB / 4];
 #pragma unroll
             for (int c = 0; c < COLS_PER_WARP; c += 4) {
-                uint32_t bits[4];
-#pragma unroll
-                for (int h = 0; h < 4; ++h) {
-                    if (SUB == 0) {
-                        float t = __uint_as_float(comb[c + h]);
-                        float quot = fmaf(t, inv_m, 12582912.0f) - 12582912.0f;
-                        float res = fmaf(-quot, mm, t);                      // |res| <= ~m/2
-                        if constexpr (LOOSE) {
-                            bits[h] = __float_as_uint(res + loose_offset);   // res + m in (0, 2m), low mantissa bits
-                        } else {
-                            res = res < 0.0f ? res + mm : res;               // canonical [0, m)
-                            bits[h] = __float_as_uint(res + 8388608.0f);     // integer in the low mantissa bits
-                        }
-                    } else if constexpr (DIRECT) {
-                        uint32_t u = comb[c + h] + mi.bias30;                 // in (0, 2^31 + 256)
-                        bits[h] = u - (__umulhi(u, mi.magic39) >> 7) * im;   // exact quotient: canonical [0, m)
-                    } else {
-                        uint32_t u = comb[c + h] + ibias;
-                        uint32_t r = u - __umulhi(u, imagic) * im;           // in [0, 2m)
-                        bits[h] = LOOSE ? r : min(r, r - im);                // canonical [0, m) unless LOOSE
-                    }
-                }
-                if constexpr (RB == 2) {
-                    packed[c >> 1] = __byte_perm(bits[0], bits[1], 0x5410);
-                    packed[(c >> 1) + 1] = __byte_perm(bits[2], bits[3], 0x5410);
-                } else {
-                    packed[c >> 2] = __byte_perm(__byte_perm(bits[0], bits[1], 0x0040),
-                                                 __byte_perm(bits[2], bits[3], 0x0040), 0x5410);
+                if constexpr (RB == 2) pack4(c, packed[c >> 1], packed[(c >> 1) + 1]);
+                else {
+                    uint32_t unused;
+                    pack4(c, packed[c >> 2], unused);
                 }
             }
             unsigned char *rbase = static_cast<unsigned char *>(p.R) + it.mod * p.mod_stride * RB;
@@ -716,7 +812,6 @@ residue_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
                     }
                 } else {
                     // 32 lines x 64 bytes in one pass; lane -> line lane/4 + 8t, 16-byte chunk lane%4
-                    constexpr int NCH = COLS_PER_WARP * RB / 16;     // 16-byte chunks per line
 #pragma unroll
                     for (int c = 0; c < NCH; ++c)
                         *reinterpret_cast<uint4 *>(xp + lane * 64 + (((c ^ (lane >> 1)) & 3) << 4)) =
@@ -742,6 +837,7 @@ residue_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
                             dst[c] = static_cast<unsigned char>((packed[c >> 2] >> (8 * (c & 3))) & 0xFFu);
                     }
             }
+            }   // public layout
         }
     }
 
@@ -791,12 +887,12 @@ bool make_plane_map(CUtensorMap *map, const uint8_t *base, int64_t lines, int64_
     return rc == CUDA_SUCCESS;
 }
 
-template <int SUB, int CG, int RB, bool DIRECT = false, bool LOOSE = false>
+template <int SUB, int CG, int RB, bool DIRECT = false, bool LOOSE = false, bool TILED = false>
 oz_status_t launch_variant(const CUtensorMap &mapA, const CUtensorMap &mapB, const GemmParams &p, int sms,
                            cudaStream_t stream)
 {
     static_assert(!LOOSE || RB == 2, "a representative below 2m needs the two-byte element");
-    auto kernel = residue_gemm_kernel<SUB, CG, RB, DIRECT, LOOSE>;
+    auto kernel = residue_gemm_kernel<SUB, CG, RB, DIRECT, LOOSE, TILED>;
     OZ_CUDA_CHECK(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        static_cast<int>(SMEM_BYTES)));
     int64_t groups = sms / CG;                                    // CTAs, or CTA pairs
@@ -823,20 +919,48 @@ oz_status_t launch_variant(const CUtensorMap &mapA, const CUtensorMap &mapB, con
 
 // Which variant runs: CTA pairs (tcgen05 cta_group::2, tiles of 256 columns) unless that would pad
 // the column count noticeably more than 128-column tiles do (n = 128: one half-empty pair tile).
-// OZ_GEMM_CTA_GROUP=1|2 overrides the choice for experiments.
 static int cta_group_choice(int64_t n)
 {
-    const char *env = getenv("OZ_GEMM_CTA_GROUP");
-    if (env && env[0] == '2') return 2;
-    if (env && env[0] == '1') return 1;
     const int64_t pad1 = round_up(n, BLOCK_M), pad2 = round_up(n, 2 * BLOCK_M);
     return (pad2 * 20 <= pad1 * 21) ? 2 : 1;
+}
+
+// Test hook for the bounded waits, read once when the library is loaded: with
+// OZ_TEST_STALL_PRODUCER=once in the environment the first residue-GEMM launch of the process loads
+// no operand, every role's wait runs into its time limit, the kernel sets OZ_ERR_TIMEOUT and
+// returns cleanly; later launches are normal.  ("1": every launch.)
+static std::atomic<int> g_stall_producer{[] {
+    const char *env = getenv("OZ_TEST_STALL_PRODUCER");
+    if (!env) return 0;
+    return env[0] == '1' ? 1 : (env[0] == 'o' ? 2 : 0);
+}()};
+
+static int take_stall_flag()
+{
+    int v = g_stall_producer.load();
+    if (v == 2) {
+        g_stall_producer.store(0);
+        return 1;
+    }
+    return v;
+}
+
+ResidueTiling residue_tiling(int64_t m, int64_t n, int set)
+{
+    ResidueTiling t;
+    t.cg = cta_group_choice(n);
+    t.tile_cols = BLOCK_M * t.cg;
+    t.tiles_m = static_cast<int>((m + BLOCK_N - 1) / BLOCK_N);
+    t.tiles_n = static_cast<int>((n + t.tile_cols - 1) / t.tile_cols);
+    t.mod_stride = static_cast<int64_t>(t.tiles_m) * t.tiles_n * t.tile_cols * BLOCK_N;
+    (void)set;
+    return t;
 }
 
 oz_status_t launch_residue_gemm(int64_t m, int64_t n, int64_t k, const uint8_t *PA, int64_t strideA,
                                 int64_t pitchA, const uint8_t *PB, int64_t strideB, int64_t pitchB,
                                 int set, const Route &rt, void *R, int64_t ldr,
-                                int64_t mod_stride, bool loose, cudaStream_t stream)
+                                int64_t mod_stride, bool loose, bool tiled, cudaStream_t stream)
 {
     const int cg = cta_group_choice(n);
     GemmParams p{};
@@ -851,12 +975,7 @@ oz_status_t launch_residue_gemm(int64_t m, int64_t n, int64_t k, const uint8_t *
     p.total_items = static_cast<int64_t>(p.r) * p.tiles_m * p.tiles_n;
     if (p.total_items >= 0x7FFFFFFFll) return OZ_ERR_UNSUPPORTED;        // item numbers are 32-bit in the kernel
     p.R = R; p.ldr = ldr; p.mod_stride = mod_stride;
-    // Test hook for the bounded waits: with OZ_TEST_STALL_PRODUCER=1 no operand is ever loaded, every
-    // role's wait runs into its time limit, the kernel sets OZ_ERR_TIMEOUT and returns cleanly.
-    {
-        const char *env = getenv("OZ_TEST_STALL_PRODUCER");
-        p.stall_producer = (env && env[0] == '1') ? 1 : 0;
-    }
+    p.stall_producer = take_stall_flag();
     p.status = device_status_word();
     for (int i = 0; i < p.r; ++i) {
         int mi = modulus(set, i), s = square_root(mi);
@@ -939,29 +1058,21 @@ oz_status_t launch_residue_gemm(int64_t m, int64_t n, int64_t k, const uint8_t *
     OZ_CUDA_CHECK(cudaGetDevice(&dev));
     OZ_CUDA_CHECK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
     // substrate 0: FP8 planes; otherwise INT8 planes (two-limb digits or native residues)
+#define OZ_LAUNCH(SUB, RB, DIRECT, LOOSE, TILED)                                                    \
+    (cg == 2 ? launch_variant<SUB, 2, RB, DIRECT, LOOSE, TILED>(mapA, mapB, p, sms, stream)        \
+             : launch_variant<SUB, 1, RB, DIRECT, LOOSE, TILED>(mapA, mapB, p, sms, stream))
+#define OZ_LAUNCH_SUB(RB, LOOSE, TILED)                                                             \
+    (rt.substrate == 0 ? OZ_LAUNCH(0, RB, false, LOOSE, TILED) : OZ_LAUNCH(1, RB, false, LOOSE, TILED))
     // one accumulator per modulus of at most 128 * 128 * k <= 2^30: the direct drain with the exact division
     if (rt.native() && p.mod[0].nseg_all == 1 && k <= 65536)
-        return cg == 2 ? launch_variant<1, 2, 1, true>(mapA, mapB, p, sms, stream)
-                       : launch_variant<1, 1, 1, true>(mapA, mapB, p, sms, stream);
-    if (rb == 1) {
-        if (cg == 2)
-            return rt.substrate == 0 ? launch_variant<0, 2, 1>(mapA, mapB, p, sms, stream)
-                                     : launch_variant<1, 2, 1>(mapA, mapB, p, sms, stream);
-        return rt.substrate == 0 ? launch_variant<0, 1, 1>(mapA, mapB, p, sms, stream)
-                                 : launch_variant<1, 1, 1>(mapA, mapB, p, sms, stream);
-    }
-    if (loose) {
-        if (cg == 2)
-            return rt.substrate == 0 ? launch_variant<0, 2, 2, false, true>(mapA, mapB, p, sms, stream)
-                                     : launch_variant<1, 2, 2, false, true>(mapA, mapB, p, sms, stream);
-        return rt.substrate == 0 ? launch_variant<0, 1, 2, false, true>(mapA, mapB, p, sms, stream)
-                                 : launch_variant<1, 1, 2, false, true>(mapA, mapB, p, sms, stream);
-    }
-    if (cg == 2)
-        return rt.substrate == 0 ? launch_variant<0, 2, 2>(mapA, mapB, p, sms, stream)
-                                 : launch_variant<1, 2, 2>(mapA, mapB, p, sms, stream);
-    return rt.substrate == 0 ? launch_variant<0, 1, 2>(mapA, mapB, p, sms, stream)
-                             : launch_variant<1, 1, 2>(mapA, mapB, p, sms, stream);
+        return tiled ? OZ_LAUNCH(1, 1, true, false, true) : OZ_LAUNCH(1, 1, true, false, false);
+    if (rb == 1) return tiled ? OZ_LAUNCH_SUB(1, false, true) : OZ_LAUNCH_SUB(1, false, false);
+    // the tile-ordered array is private to the whole-method calls, which also take the loose residues
+    if (tiled) return OZ_LAUNCH_SUB(2, true, true);
+    if (loose) return OZ_LAUNCH_SUB(2, true, false);
+    return OZ_LAUNCH_SUB(2, false, false);
+#undef OZ_LAUNCH_SUB
+#undef OZ_LAUNCH
 }
 
 }  // namespace oz

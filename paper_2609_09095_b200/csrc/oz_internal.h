@@ -11,7 +11,7 @@ namespace oz {
 
 constexpr int kMaxR = 15;          // moduli in the largest supported set (A)
 constexpr int kMaxPlanes = 44;     // stored planes of set A with two-limb digits
-constexpr int kLutWords = 8208;    // >= sum of the moduli of either set (S: 8197, E: 6838)
+constexpr int kLutWords = 8208;    // >= sum of the moduli of any set (S: 8069, E: 6736, A: 3478)
 
 // ---- modulus sets (Sec. 2 step (ii) for S; "Candidate E" and "Candidate A" paragraphs) ---
 constexpr int kNumSets = 3;
@@ -127,18 +127,40 @@ oz_status_t launch_deconstruct(int side, int64_t lines, int64_t k, const double 
                                int64_t row_pitch, int32_t *shift, void *scratch,
                                cudaStream_t stream);
 
+// Tile-ordered private residue array of the whole-method calls.  The output is cut into tiles of
+// 256 rows x tile_cols columns (128, or 256 when CTA pairs are used); a tile is 16 blocks (32 with
+// pairs: rank-major) of 32 columns x 64 rows, one per epilogue warp, block w = quarter + 4 * part
+// covering columns 32 * quarter .. +31 (of the rank's 128) and rows 64 * part .. +63; a block is
+// stored as [16-byte chunk c][column], chunk c holding 16 / residue_bytes consecutive rows.
+// Residue of modulus i: R + i * mod_stride elements, tiles in (tile row, tile column) order.
+struct ResidueTiling {
+    int cg;              // 1: tiles of 128 columns, 2: CTA pairs, tiles of 256 columns
+    int tile_cols;
+    int tiles_m, tiles_n;
+    int64_t mod_stride;  // elements per modulus (tiles are stored whole, padding included)
+};
+ResidueTiling residue_tiling(int64_t m, int64_t n, int set);
+
+// loose: residues in [0, 2 m_i) (two-byte sets); tiled: R is the tile-ordered private array
+// (ldr and mod_stride are then ignored)
 oz_status_t launch_residue_gemm(int64_t m, int64_t n, int64_t k, const uint8_t *PA,
                                 int64_t strideA, int64_t pitchA, const uint8_t *PB,
                                 int64_t strideB, int64_t pitchB, int set, const Route &rt,
-                                void *R, int64_t ldr, int64_t mod_stride, bool loose,
-                                cudaStream_t stream);   // loose: residues in [0, 2 m_i), two-byte sets
+                                void *R, int64_t ldr, int64_t mod_stride, bool loose, bool tiled,
+                                cudaStream_t stream);
+
+// reconstruction from the tile-ordered array, columns [col0, col1) of the m x n output
+oz_status_t launch_reconstruct_tiled(int64_t m, int64_t n, const void *R, const int32_t *shiftA,
+                                     const int32_t *shiftB, int set, double alpha, double beta,
+                                     double *C, int64_t ldc, int64_t col0, int64_t col1,
+                                     cudaStream_t stream);
 
 oz_status_t launch_reconstruct(int64_t m, int64_t n, const void *R, int64_t ldr,
                                int64_t mod_stride, const int32_t *shiftA, const int32_t *shiftB,
                                int set, double alpha, double beta, double *C, int64_t ldc,
                                cudaStream_t stream);
 
-// uploads the reconstruction constants of both sets to the current device
+// uploads the reconstruction constants of every set to the current device
 oz_status_t upload_reconstruct_constants();
 
 #define OZ_CUDA_CHECK(expr)                                  \

@@ -5,9 +5,10 @@
 // CRT fixes c' uniquely, so any exact evaluation gives the same integer; this kernel uses the
 // weighted form
 //     c' = sum_i c_i V_i  -  kappa M,     V_i = ((M/m_i)^-1 mod m_i) (M/m_i) mod M,
-// with every V_i and M cut into three 38-bit chunks (40-bit for the all-byte set).  c_i < 2^10.1
-// (2^8), so each of the three chunk sums is an integer below 2^52 and is formed EXACTLY by FP64
-// fused multiply-adds (r MACs per chunk).  kappa = round(S/M) comes from a floating estimate; the
+// with every V_i and M cut into three 38-bit chunks (40-bit for the all-byte set).  A stored
+// residue is below 2 m_i < 2^11.1 (the whole-method calls keep a representative in (0, 2 m_i); 2^8
+// for the byte set), so each of the three chunk sums is an integer below 2^53 -- at most 2^52.8 --
+// and is formed EXACTLY by FP64 fused multiply-adds (r MACs per chunk).  kappa = round(S/M) comes from a floating estimate; the
 // carry-normalised chunks are then summed with error-free additions, which give the correctly
 // rounded FP64 value directly unless c' lies within a hair of a rounding boundary, of a power of
 // two or of +-M/2 -- those rare outputs take an exact path: the 128-bit integer, an exact range
@@ -31,8 +32,8 @@ struct ReconConst {
 
 __constant__ ReconConst c_recon[kNumSets];
 
-// Chunk width: 38 bits for S and E (residues < 2^10.1, 13 terms: sums < 2^52); 40 bits for the
-// 117.8-bit set A (residues < 2^8, 15 terms: sums < 2^52), so that three chunks cover M.
+// Chunk width: 38 bits for S and E (stored residues < 2^11.1, 13 terms: sums < 2^52.8); 40 bits for
+// the 117.8-bit set A (residues < 2^8, 15 terms: sums < 2^52), so that three chunks cover M.
 __host__ __device__ constexpr int chunk_bits(int set) { return set == 2 ? 40 : 38; }
 __host__ __device__ constexpr double pow2d(int e) { double v = 1.0; for (int i = 0; i < e; ++i) v *= 2.0; return v; }
 constexpr double kRint = 6755399441055744.0;          // 1.5 * 2^52: (x + kRint) - kRint = rint(x)
@@ -80,7 +81,7 @@ __device__ __noinline__ double finish_exact(double T0, double T1, double T2, int
     long long hi = (t0 >> 63) + (t1 >> (64 - cw)) + (lo < static_cast<unsigned long long>(t0) ? 1 : 0) +
                    static_cast<long long>(static_cast<unsigned long long>(t2) << (2 * cw - 64));
     const __int128 M = static_cast<__int128>((static_cast<unsigned __int128>(K.M_hi) << 64) | K.M_lo);
-    const __int128 Mh = M >> 1;     // M is even for both sets
+    const __int128 Mh = M >> 1;     // M is even for every set (each holds a power of two)
     __int128 v = static_cast<__int128>((static_cast<unsigned __int128>(static_cast<unsigned long long>(hi)) << 64) | lo);
     if (v >= Mh) v -= M;
     else if (v < -Mh) v += M;
@@ -173,6 +174,30 @@ __device__ __forceinline__ void store_pair(double *out, double p0, double p1, bo
     }
 }
 
+// the ROWS consecutive rows of column j whose residues are packed in w[]: reconstruct, update C
+template <int SET>
+__device__ __forceinline__ void reconstruct_rows(const uint32_t (&w)[kMaxR], int64_t row, int nrows, int sb,
+                                                 const int32_t *__restrict__ shiftA, double alpha, double beta,
+                                                 double *out, bool vecC)
+{
+    constexpr int ROWS = 4 / residue_bytes(SET);
+    int sa[ROWS];
+#pragma unroll
+    for (int h = 0; h < ROWS; ++h) sa[h] = h < nrows ? shiftA[row + h] : 0;
+    {
+        double p0 = row_value<SET, 0>(w, sa[0], sb, alpha);
+        double p1 = nrows > 1 ? row_value<SET, 1>(w, sa[1], sb, alpha) : 0.0;
+        store_pair(out, p0, p1, nrows > 1, vecC, beta);
+    }
+    if constexpr (ROWS == 4) {
+        if (nrows > 2) {
+            double p2 = row_value<SET, 2>(w, sa[2], sb, alpha);
+            double p3 = nrows > 3 ? row_value<SET, 3>(w, sa[3], sb, alpha) : 0.0;
+            store_pair(out + 2, p2, p3, nrows > 3, vecC, beta);
+        }
+    }
+}
+
 // Each thread reconstructs ROWS consecutive rows of one column: the residues of those rows are one
 // 32-bit word per modulus (two uint16 for S and E, four uint8 for the all-byte set A).
 // Six blocks per SM (40 registers) for the two-byte sets: the kernel is bound by instruction issue
@@ -212,23 +237,45 @@ reconstruct_kernel(const void *__restrict__ Rv, int64_t ldr, int64_t mod_stride,
             w[i] = v;
         }
     }
-    const int sb = shiftB[j];
-    int sa[ROWS];
+    reconstruct_rows<SET>(w, row, nrows, shiftB[j], shiftA, alpha, beta, C + row + j * ldc, vecC != 0);
+}
+
+// Same reconstruction from the tile-ordered private array that the whole-method GEMM writes (see
+// ResidueTiling).  A thread takes one 32-bit word of a 32-column x 64-row block, i.e. ROWS consecutive
+// rows of one column.  The words of one column are dealt to consecutive threads, so that a warp
+// reads and writes 512 contiguous bytes of C (one or two whole columns of the block); its residue
+// loads are 16-byte pieces 512 bytes apart, and the warps of a thread block, which take neighbouring
+// columns, ask for whole 128-byte lines between them.
+// grid: x = (piece of the block, block within the tile, CTA rank of the pair), y = tile column, z = tile row
+template <int SET>
+__global__ void __launch_bounds__(256, residue_bytes(SET) == 2 ? 6 : 5)
+reconstruct_tiled_kernel(const void *__restrict__ Rv, int64_t mod_stride, int cg, int tiles_n, int tn0,
+                         int64_t m, int64_t n, int64_t col0, int64_t col1,
+                         const int32_t *__restrict__ shiftA, const int32_t *__restrict__ shiftB,
+                         double alpha, double beta, double *__restrict__ C, int64_t ldc, int vecC)
+{
+    constexpr int RB = residue_bytes(SET), ROWS = 4 / RB, r = set_r(SET);
+    constexpr int kBlockWords = 64 * 32 * RB / 4;          // words of one 32 x 64 block: 1024 or 512
+    constexpr int kColWords = 64 / ROWS;                   // words of one column of the block: 32 or 16
+    constexpr int kCtaCols = 256 / kColWords;              // columns per thread block: 8 or 16
+    constexpr int kPieces = 32 / kCtaCols;                 // thread blocks per residue block: 4 or 2
+    const uint32_t piece = blockIdx.x % kPieces;
+    const uint32_t wi = (blockIdx.x / kPieces) & 15u;
+    const uint32_t rank = blockIdx.x / (kPieces * 16);     // 0, or 0..1 with CTA pairs
+    const uint32_t tn = static_cast<uint32_t>(tn0) + blockIdx.y, tm = blockIdx.z;
+    const uint32_t lane = piece * kCtaCols + threadIdx.x / kColWords;   // column of the block
+    const uint32_t wq = threadIdx.x % kColWords, c = wq >> 2, sub = wq & 3u;
+    const int64_t row = static_cast<int64_t>(tm) * 256 + (wi >> 2) * 64 + c * (16 / RB) + sub * ROWS;
+    const int64_t j = (static_cast<int64_t>(tn) * cg + rank) * 128 + (wi & 3u) * 32 + lane;
+    if (row >= m || j >= n || j < col0 || j >= col1) return;
+    const int nrows = m - row < ROWS ? static_cast<int>(m - row) : ROWS;
+    const int64_t wb = ((static_cast<int64_t>(tm) * tiles_n + tn) * cg + rank) * 16 + wi;
+    const unsigned char *base = static_cast<const unsigned char *>(Rv) +
+                                (wb * kBlockWords + c * 128 + lane * 4 + sub) * 4;
+    uint32_t w[kMaxR];
 #pragma unroll
-    for (int h = 0; h < ROWS; ++h) sa[h] = h < nrows ? shiftA[row + h] : 0;
-    double *out = C + row + j * ldc;
-    {
-        double p0 = row_value<SET, 0>(w, sa[0], sb, alpha);
-        double p1 = nrows > 1 ? row_value<SET, 1>(w, sa[1], sb, alpha) : 0.0;
-        store_pair(out, p0, p1, nrows > 1, vecC != 0, beta);
-    }
-    if constexpr (ROWS == 4) {
-        if (nrows > 2) {
-            double p2 = row_value<SET, 2>(w, sa[2], sb, alpha);
-            double p3 = nrows > 3 ? row_value<SET, 3>(w, sa[3], sb, alpha) : 0.0;
-            store_pair(out + 2, p2, p3, nrows > 3, vecC != 0, beta);
-        }
-    }
+    for (int i = 0; i < r; ++i) w[i] = *reinterpret_cast<const uint32_t *>(base + i * mod_stride * RB);
+    reconstruct_rows<SET>(w, row, nrows, shiftB[j], shiftA, alpha, beta, C + row + j * ldc, vecC != 0);
 }
 
 }  // namespace
@@ -289,6 +336,32 @@ oz_status_t launch_reconstruct(int64_t m, int64_t n, const void *R, int64_t ldr,
     else
         reconstruct_kernel<1><<<grid, 256, 0, stream>>>(R, ldr, mod_stride, m, n, shiftA, shiftB, alpha,
                                                         beta, C, ldc, vecR, vecC);
+    count_launch();
+    OZ_CUDA_CHECK(cudaGetLastError());
+    return OZ_OK;
+}
+
+oz_status_t launch_reconstruct_tiled(int64_t m, int64_t n, const void *R, const int32_t *shiftA,
+                                     const int32_t *shiftB, int set, double alpha, double beta,
+                                     double *C, int64_t ldc, int64_t col0, int64_t col1,
+                                     cudaStream_t stream)
+{
+    if (col1 <= col0) return OZ_OK;
+    const ResidueTiling t = residue_tiling(m, n, set);
+    const int tn0 = static_cast<int>(col0 / t.tile_cols);
+    const int ntn = static_cast<int>((col1 + t.tile_cols - 1) / t.tile_cols) - tn0;
+    const int pieces = 64 * 32 * residue_bytes(set) / 4 / 256;
+    if (t.tiles_m > 65535 || ntn > 65535) return OZ_ERR_UNSUPPORTED;
+    const int vecC = ((ldc & 1) == 0 && (reinterpret_cast<uintptr_t>(C) & 15u) == 0) ? 1 : 0;
+    const dim3 grid(static_cast<unsigned>(pieces * 16 * t.cg), static_cast<unsigned>(ntn),
+                    static_cast<unsigned>(t.tiles_m));
+#define OZ_RECON_TILED(SET_)                                                                              \
+    reconstruct_tiled_kernel<SET_><<<grid, 256, 0, stream>>>(R, t.mod_stride, t.cg, t.tiles_n, tn0, m, n,  \
+                                                             col0, col1, shiftA, shiftB, alpha, beta, C, ldc, vecC)
+    if (set == 2) OZ_RECON_TILED(2);
+    else if (set == 0) OZ_RECON_TILED(0);
+    else OZ_RECON_TILED(1);
+#undef OZ_RECON_TILED
     count_launch();
     OZ_CUDA_CHECK(cudaGetLastError());
     return OZ_OK;

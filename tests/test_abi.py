@@ -65,3 +65,50 @@ def test_header_is_plain_c(tmp_path):
                    '    return p[0] == 0;\n}\n' % (len(oz.EXPORTS), calls))
     inc = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "include")
     subprocess.run([gcc, "-std=c99", "-Wall", "-Werror", "-pedantic", "-fsyntax-only", "-I", inc, str(src)], check=True)
+
+
+def test_misaligned_pointers_are_rejected_on_the_host():
+    """Pointers that are not aligned to their element type are a host-detectable error of the stage
+    entry points: OZ_ERR_INVALID_ARG comes back before any CUDA call (so this runs without a GPU;
+    the addresses are never dereferenced)."""
+    base = 0x7F0000000000                     # any 256-byte aligned number
+    m, n, k, pitch = 8, 8, 16, 16
+    ok_args = dict(PA=base, PB=base + 4096, R=base + 8192)
+    for set_id, elem in ((oz.OZ_SET_S, 2), (oz.OZ_SET_E, 2)):
+        assert oz.oz_residue_gemm(m, n, k, ok_args["PA"], m * pitch, pitch, ok_args["PB"], n * pitch, pitch, set_id,
+                                  0, ok_args["R"] + 1, m, m * n, 0) == oz.OZ_ERR_INVALID_ARG      # odd address, uint16 residues
+        assert oz.oz_reconstruct(m, n, base + 1, m, m * n, base + 4096, base + 8192, set_id, 1.0, 0.0,
+                                 base + 16384, m, 0) == oz.OZ_ERR_INVALID_ARG
+    # shifts are int32, matrices are double
+    assert oz.oz_reconstruct(m, n, base, m, m * n, base + 4098, base + 8192, oz.OZ_SET_S, 1.0, 0.0, base + 16384, m, 0) \
+        == oz.OZ_ERR_INVALID_ARG
+    assert oz.oz_reconstruct(m, n, base, m, m * n, base + 4096, base + 8194, oz.OZ_SET_A, 1.0, 0.0, base + 16384, m, 0) \
+        == oz.OZ_ERR_INVALID_ARG
+    assert oz.oz_reconstruct(m, n, base, m, m * n, base + 4096, base + 8192, oz.OZ_SET_A, 1.0, 0.0, base + 16388, m, 0) \
+        == oz.OZ_ERR_INVALID_ARG
+    assert oz.oz_deconstruct(0, m, k, base + 4, m, oz.OZ_SET_S, 0, base + 4096, m * pitch, pitch, base + 8192,
+                             base + 16384, 0) == oz.OZ_ERR_INVALID_ARG                        # X not 8-byte aligned
+    assert oz.oz_deconstruct(0, m, k, base, m, oz.OZ_SET_S, 0, base + 4096, m * pitch, pitch, base + 8194,
+                             base + 16384, 0) == oz.OZ_ERR_INVALID_ARG                        # shift not 4-byte aligned
+    assert oz.oz_deconstruct_static(1, n, k, base + 2, k, oz.OZ_SET_S, 0, base + 4096, n * pitch, pitch,
+                                    base + 8192, 0) == oz.OZ_ERR_INVALID_ARG
+
+
+def test_prepared_operand_sizes():
+    """Host-only queries of the planes-kept-across-calls interface."""
+    m, n, k = 16384, 16384, 1024
+    a = oz.oz_operand_bytes(0, m, k, oz.OZ_SET_S, 0)
+    b = oz.oz_operand_bytes(1, n, k, oz.OZ_SET_S, 0)
+    assert 30 * m * k <= a < 30 * m * k + 21 * m + 4096 and a == b
+    assert oz.oz_operand_bytes(0, m, k, oz.OZ_SET_A, oz.OZ_SUB_INT8_NATIVE) < 15 * m * k + 21 * m + 4096
+    assert oz.oz_operand_bytes(2, m, k, oz.OZ_SET_S, 0) == 0
+    assert oz.oz_operand_bytes(0, m, oz.OZ_K_MAX + 1, oz.OZ_SET_S, 0) == 0
+    # inner dimension padded to whole 128-byte lines
+    assert oz.oz_operand_bytes(0, 1000, 5003, oz.OZ_SET_S, 0) >= 30 * 1000 * 5120
+    r = oz.oz_product_workspace_bytes(m, n, oz.OZ_SET_S)
+    assert r == 24 * m * n
+    assert oz.oz_product_workspace_bytes(m, n, oz.OZ_SET_A) == 15 * m * n
+    # planes of both operands + residues = the workspace of the whole-method call
+    assert oz.oz_workspace_bytes(m, n, k, oz.OZ_SET_S, 0) == a + b + r
+    # ragged shapes are stored as whole tiles
+    assert oz.oz_product_workspace_bytes(10007, 9973, oz.OZ_SET_S) == 24 * 10240 * 9984

@@ -52,6 +52,26 @@ def test_two_rank_aggregation_gloo(tmp_path):
     assert bench.aggregate_over_ranks(7.0, 3.0, 1, None, None) == (7.0, 3.0)
 
 
+def test_self_spawned_ranks_gloo():
+    """`bench.py --gpus N` run without torchrun starts its own N ranks: the command line it builds
+    (one process per GPU on 127.0.0.1, the original arguments passed on) brings up a working group."""
+    cmd = bench.spawn_command(["--gpus", "2", "--steps", "3"], 2, _free_port())
+    assert cmd[1:4] == ["-m", "torch.distributed.run", "--nnodes=1"] and "--nproc-per-node=2" in cmd
+    assert cmd[cmd.index("--master-addr") + 1] == "127.0.0.1"
+    assert cmd[-5] == os.path.join(ROOT, "bench.py") and cmd[-4:] == ["--gpus", "2", "--steps", "3"]
+    cmd[-5] = os.path.join(ROOT, "tests", "rank_probe.py")          # same launch line, CPU ranks
+    out = subprocess.run(cmd, capture_output=True, text=True, timeout=600)
+    assert out.returncode == 0, out.stderr
+    got = json.loads([l for l in out.stdout.splitlines() if l.startswith("{")][-1])
+    assert got == {"ms": 11.0, "work": 14.0, "world": 2, "argv": ["--gpus", "2", "--steps", "3"]}
+
+
+def test_traffic_table_lookup():
+    amp = bench.gemm_dram_amplification("S", "fp8")
+    assert amp is None or (len(amp) == 2 and amp[0] >= 1.0 and amp[1] >= 0.9)
+    assert bench.gemm_dram_amplification("no such set", "fp8") is None
+
+
 def test_clock_sample_parser():
     s = bench.ClockSampler(0)
     s.proc = type("P", (), {"terminate": lambda self: None, "wait": lambda self, timeout=None: 0})()

@@ -419,6 +419,31 @@ def test_planes_reproduce_residue_products(name, sub):
         assert (R1[i].T.astype(object) == want % mm).all()
 
 
+@pytest.mark.parametrize("name,sub", [("S", ozo.SUB_FP8), ("S", ozo.SUB_INT8), ("E", ozo.SUB_FP8),
+                                      ("A", ozo.SUB_INT8), ("A", ozo.SUB_INT8_NATIVE)])
+def test_plane_writer_equals_per_element_split_and_encode(name, sub):
+    """The plane writer hoists the split and the encoding of each residue value out of its element
+    loop; this holds it to the plain per-element statement of Algorithm 2: split the residue
+    (Lemma 1 carry included), encode each digit, store it at [plane][line][k]."""
+    rng = np.random.default_rng(11)
+    ms = ozo.modset(SETS[name])
+    lines, k = 3, 41
+    D = np.stack([rng.integers(-(mm // 2), (mm - 1) // 2 + 1, size=(lines, k)) for mm in ms]).astype(np.int16)
+    for i, mm in enumerate(ms):                      # both ends of every centred interval
+        D[i, 0, 0], D[i, 0, 1] = -(mm // 2), (mm - 1) // 2
+    P = ozo.planes(D, SETS[name], sub)
+    plane = 0
+    for i, mm in enumerate(ms):
+        digits_of = (lambda d: [d]) if sub == ozo.SUB_INT8_NATIVE else (lambda d, mm=mm: ozo.split(d, mm))
+        for l in range(lines):
+            for kk in range(k):
+                for q, dg in enumerate(digits_of(int(D[i, l, kk]))):
+                    byte = ozo.e4m3_encode(dg) if sub == ozo.SUB_FP8 else dg & 0xFF
+                    assert P[plane + q, l, kk] == byte
+        plane += len(digits_of(0))
+    assert plane == P.shape[0] and (P[:, :, k:] == 0).all()
+
+
 # ----------------------------------------------------------------- P10: reduces to an exact product
 def test_exact_on_small_integers():
     A, B = syn.special_operands("small_integers", 12, 10, 64)
