@@ -65,6 +65,44 @@ def shift_of_line(line, ms, rule, tbits, k):
     return p + 9 - E
 
 
+def bound_digit(x: float, E: int) -> int:
+    """Accurate mode: the smallest E4M3-representable integer that is >= |x| 2^(4-E)."""
+    if x == 0:
+        return 0
+    g = math.ceil(abs(Fraction(x)) * Fraction(2) ** (4 - E))
+    while g not in _E:
+        g += 1
+    return g
+
+
+def shifts_accurate(A, B, ms):
+    """Accurate mode (Sec. 2 "The FP8 variant": the extra magnitude-bound product).  A: m x k nested
+    lists, B: k x n nested lists of finite floats.  Returns (sigma, tau, rowmax, colmax)."""
+    m, k, n = len(A), len(B), len(B[0])
+    rows = [A[i] for i in range(m)]
+    cols = [[B[kk][j] for kk in range(k)] for j in range(n)]
+
+    def line_exponent(line):
+        nz = [abs(Fraction(x)) for x in line if x != 0]
+        return max(floor_log2(x) for x in nz) if nz else None
+
+    EA, EB = [line_exponent(l) for l in rows], [line_exponent(l) for l in cols]
+    GA = [[bound_digit(x, EA[i]) if EA[i] is not None else 0 for x in rows[i]] for i in range(m)]
+    GB = [[bound_digit(x, EB[j]) if EB[j] is not None else 0 for x in cols[j]] for j in range(n)]
+    Cbar = [[sum(GA[i][kk] * GB[j][kk] for kk in range(k)) for j in range(n)] for i in range(m)]
+    rowmax = [max(Cbar[i]) if n else 0 for i in range(m)]
+    colmax = [max(Cbar[i][j] for i in range(m)) if m else 0 for j in range(n)]
+    Hp = ((product(ms) - 1) // 2 // 129) * 128
+    L = Hp.bit_length() - 1
+
+    def ceil_log2(v):
+        return (v - 1).bit_length() if v > 1 else 0
+
+    sigma = [0 if EA[i] is None else (L - ceil_log2(rowmax[i])) // 2 + 4 - EA[i] for i in range(m)]
+    tau = [0 if EB[j] is None else (L - ceil_log2(colmax[j])) // 2 + 4 - EB[j] for j in range(n)]
+    return sigma, tau, rowmax, colmax
+
+
 def quantise(x: float, sigma: int, quant: str) -> int:
     v = Fraction(x) * Fraction(2) ** sigma
     if quant == "TZ":
@@ -136,8 +174,11 @@ def dgemm(A, B, set_name="S", quant="RN", rule="CS"):
     ms = SETS[set_name]
     m, k, n = len(A), len(B), len(B[0])
     tA, tB = budget_maxexp(ms, k)
-    sig = [shift_of_line(A[i], ms, rule, tA, k) for i in range(m)]
-    tau = [shift_of_line([B[kk][j] for kk in range(k)], ms, rule, tB, k) for j in range(n)]
+    if rule == "ACCURATE":
+        sig, tau, _, _ = shifts_accurate(A, B, ms)
+    else:
+        sig = [shift_of_line(A[i], ms, rule, tA, k) for i in range(m)]
+        tau = [shift_of_line([B[kk][j] for kk in range(k)], ms, rule, tB, k) for j in range(n)]
     QA = [[quantise(A[i][kk], sig[i], quant) for kk in range(k)] for i in range(m)]
     QB = [[quantise(B[kk][j], tau[j], quant) for kk in range(k)] for j in range(n)]
     R = [[[sum(centred(QA[i][kk], mm) * centred(QB[j][kk], mm) for kk in range(k)) % mm

@@ -40,7 +40,7 @@ typedef unsigned __int128 u128;
 
 enum { OZO_SET_S = 0, OZO_SET_E = 1, OZO_SET_A = 2 };
 enum { OZO_QUANT_RN = 0, OZO_QUANT_TZ = 1 };
-enum { OZO_SCALE_MAXEXP = 0, OZO_SCALE_CS = 1 };
+enum { OZO_SCALE_MAXEXP = 0, OZO_SCALE_CS = 1, OZO_SCALE_ACCURATE = 2 };
 /* FP8 / INT8: two-limb digit planes (Sec. 2 "FP8 variant").  INT8_NATIVE: one plane per modulus
  * holding the centred residue itself as a signed byte -- possible for byte moduli only (Sec. 2,
  * paragraph "The substrate transition": byte-modulus residues need no digit split on the INT8
@@ -227,6 +227,116 @@ void ozo_shifts(int side, int64_t lines, int64_t k, const double *X, int64_t ldx
         while (pw < 60 && S <= (G2 >> (2 * (pw + 1)))) ++pw;
         shift[l] = pw + 9 - E;
     }
+}
+
+/* ------------------------------------------------------------------ */
+/* Accurate mode (Sec. 2 "The FP8 variant": one additional FP8 GEMM that  */
+/* estimates an input magnitude bound -- the "+1" of alpha = 3r + 1)      */
+/* ------------------------------------------------------------------ */
+/* The paper names the extra product and leaves its use to the cited analysis.  Reading taken:
+ *   1. E_i = largest exponent of line i (as in the MAXEXP rule).
+ *   2. magnitude digit  g(x) = the smallest integer of the E4M3 grid {0..16, 18, 20, .., 32}
+ *      that is >= |x| 2^(4-E_i); so |x| <= g(x) 2^(E_i-4), and every g is exact in FP8.
+ *   3. bound product    Cbar_ij = sum_k g(a_ik) g(b_kj)  (an integer <= 1024 k, exact in an FP32
+ *      accumulator for k <= 16384): 2^(E_i+F_j-8) Cbar_ij >= (|A||B|)_ij.
+ *   4. row_i = max_j Cbar_ij, col_j = max_i Cbar_ij; rho_i = ceil(log2 row_i), likewise for col_j;
+ *      L = floor(log2 H'), H' = floor(((M-1)/2) / 129) * 128  (a 1/129 margin for the
+ *      half-units that rounding to nearest adds to |a'|, |b'|);
+ *      p_i = floor((L - rho_i) / 2), q_j = floor((L - chi_j) / 2), sigma_i = p_i + 4 - E_i,
+ *      tau_j = q_j + 4 - F_j.
+ * Soundness: |a'_ik| <= 2^p_i g(a_ik) (1 + 2^-(p_i+1)) when g >= 1, so
+ * |c'_ij| <= 2^(p_i+q_j) Cbar_ij (1 + 2^-39) and p_i + q_j <= L - (rho_i + chi_j)/2 <= L - log2 Cbar_ij,
+ * hence |c'_ij| <= 2^L (1 + 2^-39) < (M-1)/2.
+ * Lines of zeros get shift 0, lines with Inf/NaN the sentinel (their digits count as zero). */
+int ozo_bound_digit(double x, int E)
+{
+    fp_parts p = decode(x);
+    if (p.kind != 1) return 0;
+    /* |x| 2^(4-E) = sig 2^(ex-52+4-E) = sig / 2^sh */
+    int sh = 48 + E - p.ex;
+    uint64_t g;
+    if (sh >= 64) g = 1;
+    else if (sh <= 0) g = p.sig << (-sh);          /* cannot exceed 32: |x| < 2^(E+1) */
+    else g = (p.sig >> sh) + ((p.sig & ((1ull << sh) - 1)) ? 1 : 0);
+    if (g > 16 && (g & 1)) ++g;                    /* 17..31 odd -> next even: the E4M3 grid above 16 */
+    return (int)g;
+}
+
+/* floor(log2 H') of the accurate rule for a set */
+int ozo_accurate_budget_log2(int set)
+{
+    u128 H = (modset_product(set) - 1) / 2;
+    u128 Hp = (H / 129) * 128;
+    int L = -1;
+    while (Hp) { ++L; Hp >>= 1; }
+    return L;
+}
+
+static int ceil_log2_u64(uint64_t v)
+{
+    int c = 0;
+    while (((uint64_t)1 << c) < v) ++c;
+    return c;
+}
+
+/* digits G[line*k + kk] and exponents E[line] (INT32_MIN: line of zeros) of one operand;
+ * bad[line] = 1 for a line with Inf/NaN (digits all zero) */
+void ozo_bound_planes(int side, int64_t lines, int64_t k, const double *X, int64_t ldx,
+                      uint8_t *G, int32_t *Eout, int32_t *bad)
+{
+#pragma omp parallel for schedule(static)
+    for (int64_t l = 0; l < lines; ++l) {
+        int any = 0, nf = 0, E = 0;
+        for (int64_t kk = 0; kk < k; ++kk) {
+            fp_parts p = decode(*elem(X, ldx, side, l, kk));
+            if (p.kind == 2) nf = 1;
+            if (p.kind == 1) { if (!any || p.e > E) E = p.e; any = 1; }
+        }
+        bad[l] = nf;
+        Eout[l] = (any && !nf) ? E : INT32_MIN;
+        for (int64_t kk = 0; kk < k; ++kk)
+            G[l * k + kk] = (uint8_t)((any && !nf) ? ozo_bound_digit(*elem(X, ldx, side, l, kk), E) : 0);
+    }
+}
+
+/* shifts of both operands by the accurate rule; rowmax / colmax (may be NULL) receive the maxima of
+ * the bound product */
+int ozo_shifts_accurate(int64_t m, int64_t n, int64_t k, const double *A, int64_t lda,
+                        const double *B, int64_t ldb, int set, int32_t *shiftA, int32_t *shiftB,
+                        uint32_t *rowmax_out, uint32_t *colmax_out)
+{
+    uint8_t *GA = malloc((size_t)(m * k > 0 ? m * k : 1)), *GB = malloc((size_t)(n * k > 0 ? n * k : 1));
+    int32_t *EA = malloc(sizeof(int32_t) * (m > 0 ? m : 1)), *EB = malloc(sizeof(int32_t) * (n > 0 ? n : 1));
+    int32_t *badA = malloc(sizeof(int32_t) * (m > 0 ? m : 1)), *badB = malloc(sizeof(int32_t) * (n > 0 ? n : 1));
+    uint32_t *rowmax = calloc((size_t)(m > 0 ? m : 1), sizeof(uint32_t));
+    uint32_t *colmax = calloc((size_t)(n > 0 ? n : 1), sizeof(uint32_t));
+    if (!GA || !GB || !EA || !EB || !badA || !badB || !rowmax || !colmax) return -1;
+    ozo_bound_planes(0, m, k, A, lda, GA, EA, badA);
+    ozo_bound_planes(1, n, k, B, ldb, GB, EB, badB);
+    for (int64_t j = 0; j < n; ++j) {
+        uint32_t cm = 0;
+#pragma omp parallel for schedule(static) reduction(max : cm)
+        for (int64_t i = 0; i < m; ++i) {
+            uint64_t acc = 0;
+            for (int64_t kk = 0; kk < k; ++kk) acc += (uint64_t)GA[i * k + kk] * GB[j * k + kk];
+            if (acc > rowmax[i]) rowmax[i] = (uint32_t)acc;   /* row i is touched by this thread only */
+            if (acc > cm) cm = (uint32_t)acc;
+        }
+        colmax[j] = cm;
+    }
+    const int L = ozo_accurate_budget_log2(set);
+    for (int64_t i = 0; i < m; ++i)
+        shiftA[i] = badA[i] ? OZO_NONFINITE_SHIFT
+                    : EA[i] == INT32_MIN ? 0                      /* a maximum of 0 counts as 1: rho = 0 */
+                    : ((L - ceil_log2_u64(rowmax[i])) >> 1) + 4 - EA[i];
+    for (int64_t j = 0; j < n; ++j)
+        shiftB[j] = badB[j] ? OZO_NONFINITE_SHIFT
+                    : EB[j] == INT32_MIN ? 0
+                    : ((L - ceil_log2_u64(colmax[j])) >> 1) + 4 - EB[j];
+    if (rowmax_out) memcpy(rowmax_out, rowmax, sizeof(uint32_t) * m);
+    if (colmax_out) memcpy(colmax_out, colmax, sizeof(uint32_t) * n);
+    free(GA); free(GB); free(EA); free(EB); free(badA); free(badB); free(rowmax); free(colmax);
+    return 0;
 }
 
 /* ------------------------------------------------------------------ */
@@ -745,8 +855,12 @@ int ozo_dgemm(int64_t m, int64_t n, int64_t k, const double *A, int64_t lda, con
     uint16_t *R = malloc(sizeof(uint16_t) * r * m * n);
     int64_t *CI = malloc(sizeof(int64_t) * 2 * m * n);
     if (!sA || !sB || !QA || !QB || !DA || !DB || !R || !CI) return -1;
-    ozo_shifts(0, m, k, A, lda, set, rule, tA, sA);
-    ozo_shifts(1, n, k, B, ldb, set, rule, tB, sB);
+    if (rule == OZO_SCALE_ACCURATE) {
+        if (ozo_shifts_accurate(m, n, k, A, lda, B, ldb, set, sA, sB, NULL, NULL)) return -1;
+    } else {
+        ozo_shifts(0, m, k, A, lda, set, rule, tA, sA);
+        ozo_shifts(1, n, k, B, ldb, set, rule, tB, sB);
+    }
     ozo_quantise(0, m, k, A, lda, sA, quant, QA);
     ozo_quantise(1, n, k, B, ldb, sB, quant, QB);
     ozo_residues(m, k, QA, set, DA);

@@ -21,7 +21,7 @@ _LIB = os.path.join(_HERE, "liboz_oracle.so")
 
 SET_S, SET_E, SET_A = 0, 1, 2
 QUANT_RN, QUANT_TZ = 0, 1
-SCALE_MAXEXP, SCALE_CS = 0, 1
+SCALE_MAXEXP, SCALE_CS, SCALE_ACCURATE = 0, 1, 2
 SUB_FP8, SUB_INT8, SUB_INT8_NATIVE = 0, 1, 2
 NONFINITE_SHIFT = -(2**31)
 
@@ -165,6 +165,29 @@ def shifts(side: int, X: np.ndarray, s: int, rule: int, tbits: int) -> np.ndarra
     lib().ozo_shifts(side, _i64(lines), _i64(k), _p(X), _i64(max(X.shape[0], 1)), s, rule,
                      tbits, _p(out))
     return out
+
+
+def bound_digit(x: float, E: int) -> int:
+    return lib().ozo_bound_digit(C.c_double(x), int(E))
+
+
+def accurate_budget_log2(s: int) -> int:
+    return lib().ozo_accurate_budget_log2(s)
+
+
+def shifts_accurate(A: np.ndarray, B: np.ndarray, s: int):
+    """Shifts of both operands by the accurate rule (the extra bound product of Sec. 2 "The FP8
+    variant"); returns (shiftA, shiftB, rowmax, colmax)."""
+    _check_cm(A)
+    _check_cm(B)
+    m, k = A.shape
+    n = B.shape[1]
+    sA, sB = np.zeros(m, dtype=np.int32), np.zeros(n, dtype=np.int32)
+    rm, cm = np.zeros(m, dtype=np.uint32), np.zeros(n, dtype=np.uint32)
+    rc = lib().ozo_shifts_accurate(_i64(m), _i64(n), _i64(k), _p(A), _i64(max(m, 1)), _p(B), _i64(max(k, 1)), s,
+                                   _p(sA), _p(sB), _p(rm), _p(cm))
+    assert rc == 0
+    return sA, sB, rm, cm
 
 
 def quantise(side: int, X: np.ndarray, shift: np.ndarray, quant: int) -> np.ndarray:

@@ -372,6 +372,76 @@ def test_shifts_keep_product_in_range(rule, name):
             assert all(max(abs(int(v)) for v in QA[i]) >= 2**(tA - 1) for i in range(m))
 
 
+# ----------------------------------------------------------------- accurate mode: the "+1" bound product
+def test_bound_digit_is_the_least_e4m3_upper_bound():
+    """Sec. 2 "The FP8 variant": the extra product runs on FP8 operands, so its magnitude digits must
+    be E4M3-exact; the digit is the least grid value not below |x| 2^(4-E)."""
+    grid = sorted(v for v in range(0, 33) if ozo.in_e4m3(v))
+    assert grid == list(range(0, 17)) + list(range(18, 33, 2))
+    E = 3
+    for num in range(0, 16 * 64 + 1):                       # |x| 2^(4-E) = num / 32, up to 32
+        x = num / 32.0 * 2.0 ** (E - 4)
+        g = ozo.bound_digit(x, E)
+        exact = Fraction(num, 32)
+        assert g in grid and g >= exact
+        assert all(v < exact for v in grid if v < g)        # no smaller grid value bounds it
+        assert ozo.bound_digit(-x, E) == g == big.bound_digit(x, E)
+    assert ozo.bound_digit(5e-324, 0) == 1 and ozo.bound_digit(0.0, 0) == 0      # tiny but non-zero counts as 1
+    assert ozo.bound_digit(float(np.nextafter(2.0 ** (E + 1), 0.0)), E) == 32
+
+
+@pytest.mark.parametrize("name", ["S", "E", "A"])
+def test_accurate_shifts_are_sound_and_match_the_restatement(name):
+    """The shifts chosen from the bound product keep every |c'_ij| inside the CRT range -- checked by
+    brute force in exact integers on random operands, on an operand pair that attains the bound
+    (all entries at the top of their binade, equal signs) and with both quantisers -- and equal the
+    big-integer restatement."""
+    rng = np.random.default_rng(31)
+    ms = ozo.modset(SETS[name])
+    M = math.prod(ms)
+    m, n, k = 8, 6, 40
+    A = np.asfortranarray((rng.random((m, k)) - 0.5) * np.exp(3 * rng.standard_normal((m, k))))
+    B = np.asfortranarray((rng.random((k, n)) - 0.5) * np.exp(3 * rng.standard_normal((k, n))))
+    top = float(np.nextafter(2.0, 0.0))
+    A[1, :] = top * 2.0 ** 5                                 # every digit 32, products aligned with column 2
+    B[:, 2] = top * 2.0 ** -7
+    A[4, 1:] = 0.0                                           # a single non-zero
+    A[6, :] = 0.0                                            # a zero line
+    B[:, 4] = 0.0
+    sA, sB, rm, cm = ozo.shifts_accurate(A, B, SETS[name])
+    sig, tau, rowmax, colmax = big.shifts_accurate(A.tolist(), B.tolist(), ms)
+    assert sA.tolist() == sig and sB.tolist() == tau
+    assert rm.tolist() == rowmax and cm.tolist() == colmax
+    assert rm[1] == 1024 * k == cm[2] and sA[6] == 0 and sB[4] == 0
+    L = ozo.accurate_budget_log2(SETS[name])
+    assert 2 ** L <= ((M - 1) // 2 // 129) * 128 < 2 ** (L + 1)
+    for quant in (ozo.QUANT_RN, ozo.QUANT_TZ):
+        QA = ozo.quantise(0, A, sA, quant).astype(object)
+        QB = ozo.quantise(1, B, sB, quant).astype(object)
+        absC = np.abs(QA) @ np.abs(QB).T
+        assert max(int(v) for v in absC.ravel()) <= (M - 1) // 2
+    # on the pair that attains the bound the rule gives up less than three bits of the range
+    # (a bit for each ceiling of a logarithm, half a bit for the halved exponent, the 1/129 margin)
+    assert int(absC[1, 2]) * 8 > (M - 1) // 2
+    # the whole method with this rule: C oracle == restatement
+    Cm, s1, s2, R = ozo.dgemm(A, B, SETS[name], ozo.QUANT_RN, ozo.SCALE_ACCURATE, want_stages=True)
+    Cf, sig2, tau2, Rb, _ = big.dgemm(A.tolist(), B.tolist(), name, "RN", "ACCURATE")
+    assert s1.tolist() == sig2 == sig and s2.tolist() == tau2 and R.tolist() == Rb and Cm.tolist() == Cf
+
+
+def test_accurate_rule_on_a_closed_form_case():
+    """A = ones(m, k), B = ones(k, n): every digit is 16 (|x| 2^(4-0)), the bound product is 256 k,
+    so sigma = tau = floor((L - ceil(log2(256 k))) / 2) + 4."""
+    for name in ("S", "A"):
+        L = ozo.accurate_budget_log2(SETS[name])
+        for k in (1, 3, 64, 100):
+            A, B = np.ones((2, k), order="F"), np.ones((k, 3), order="F")
+            sA, sB, rm, cm = ozo.shifts_accurate(A, B, SETS[name])
+            want = (L - math.ceil(math.log2(256 * k))) // 2 + 4
+            assert rm.tolist() == [256 * k] * 2 and cm.tolist() == [256 * k] * 3
+            assert sA.tolist() == [want] * 2 and sB.tolist() == [want] * 3
+
+
 # ----------------------------------------------------------------- P7: brute force / big ints
 @pytest.mark.parametrize("name,quant,rule", [("S", "RN", "CS"), ("S", "TZ", "MAXEXP"),
                                              ("E", "RN", "MAXEXP"), ("E", "TZ", "CS"),
