@@ -52,7 +52,8 @@ extern "C" {
 typedef enum {
     OZ_OK = 0,
     OZ_ERR_INVALID_ARG = 1,     /* null pointer, negative size, bad leading dimension, bad enum */
-    OZ_ERR_UNSUPPORTED = 2,     /* k > OZ_K_MAX, alpha/beta outside {+-1}/{0,1}                 */
+    OZ_ERR_UNSUPPORTED = 2,     /* k > OZ_K_MAX, alpha/beta outside {+-1}/{0,1}, OZ_SCALE_ACCURATE
+                                 * through a per-operand entry point or with k > 16384             */
     OZ_ERR_WORKSPACE = 3,       /* no workspace registered, or it is too small                  */
     OZ_ERR_CUDA = 4,            /* a CUDA runtime / driver call failed                          */
     OZ_ERR_NONFINITE_INPUT = 5, /* device: Inf/NaN met in an operand                            */
@@ -75,6 +76,14 @@ typedef enum { OZ_SET_S = 0, OZ_SET_E = 1, OZ_SET_A = 2 } oz_modset_t;
 #define OZ_QUANT_TZ     0x020u  /* truncate toward zero (variant Ozaki-II-TZ)                  */
 #define OZ_SCALE_MAXEXP 0x100u  /* shift from the largest exponent of the line (Eq. 2 read literally) */
 #define OZ_SCALE_CS     0x200u  /* shift from the 2-norm of the line, Cauchy-Schwarz bound (default) */
+#define OZ_SCALE_ACCURATE 0x400u /* accurate mode (Sec. 2 "The FP8 variant": one additional FP8 GEMM
+                                  * estimates an input magnitude bound, the "+1" of the 3r + 1 passes):
+                                  * every element gives an E4M3-exact magnitude digit >= |x| 2^(4-E) (E the
+                                  * largest exponent of its line), one extra tensor-core product of the two
+                                  * digit planes bounds (|A||B|)_ij, and the shifts come from the row and
+                                  * column maxima of that product, so that every |c'_ij| stays inside the
+                                  * CRT range.  Whole-method calls only (the shifts of one operand depend on
+                                  * the other): oz_dgemm, oz_dgemm_ex, oz_dgemm_host; k <= 16384.            */
 
 /* Accumulator schedule of the residue GEMMs for non-square moduli on the FP8 substrate.
  * MERGED: two accumulators per modulus, d e = -15 [d0 e0 + (-16 d1) e1] + 16 (d0+d1)(e0+e1)

@@ -129,6 +129,7 @@ bool decode_route(uint32_t route, Route *out)
     else return false;
     if (sc == 0 || sc == OZ_SCALE_CS) out->rule = 1;
     else if (sc == OZ_SCALE_MAXEXP) out->rule = 0;
+    else if (sc == OZ_SCALE_ACCURATE) out->rule = 2;
     else return false;
     return true;
 }
@@ -160,6 +161,15 @@ void budget_maxexp(int set, int64_t k, int *tA, int *tB)
     while (v) { ++T; v >>= 1; }
     *tB = T / 2;
     *tA = T - T / 2;
+}
+
+// floor(log2 H') of the accurate rule: H' = floor(((M-1)/2) / 129) * 128
+int accurate_budget_log2(int set)
+{
+    unsigned __int128 v = ((set_product(set) - 1) / 2 / 129) * 128;
+    int L = -1;
+    while (v) { ++L; v >>= 1; }
+    return L;
 }
 
 void cs_bound_squared(int set, int64_t k, uint64_t *lo, uint64_t *hi)
@@ -201,6 +211,14 @@ oz_status_t ensure_device_ready()
     OZ_CUDA_CHECK(cudaGetSymbolAddress(&p, g_status));
     g_status_addr[dev] = static_cast<unsigned int *>(p);
     oz_status_t st = upload_reconstruct_constants();
+    if (st != OZ_OK) return st;
+    unsigned char codes[33];
+    for (int d = 0; d <= 32; ++d) {
+        int code = 0;
+        e4m3_code(d, &code);            // odd digits above 16 are never produced
+        codes[d] = static_cast<unsigned char>(code);
+    }
+    st = upload_bound_codes(codes);
     if (st != OZ_OK) return st;
     g_ready[dev] = true;
     return OZ_OK;
@@ -397,6 +415,29 @@ oz_status_t dgemm_impl(int64_t m, int64_t n, int64_t k, double alpha, const doub
     cudaStream_t side = g_side_stream[dev];
     const bool ev = g_stage_events_on[dev];
     if (ev) OZ_CUDA_CHECK(cudaEventRecord(g_stage_events[dev][0], stream));
+    if (rt.rule == 2) {
+        // Accurate mode: exponent scans, one magnitude plane per operand (kept in the first plane slot
+        // of each operand, which the conversion overwrites afterwards), the bound product on the
+        // tensor cores, the shifts from its row and column maxima, then the conversion as usual.
+        if (k > kBoundKMax) return OZ_ERR_UNSUPPORTED;
+        st = launch_scan(0, m, k, A, lda, set, rt, a.shift, a.scratch, stream);
+        if (st == OZ_OK) st = launch_scan(1, n, k, B, ldb, set, rt, b.shift, b.scratch, stream);
+        if (st == OZ_OK) st = launch_bound_plane(0, m, k, A, lda, a.scratch, a.planes, a.pitch, stream);
+        if (st == OZ_OK) st = launch_bound_plane(1, n, k, B, ldb, b.scratch, b.planes, b.pitch, stream);
+        if (st == OZ_OK)
+            st = launch_bound_gemm(m, n, k, a.planes, a.pitch, b.planes, b.pitch, bound_maxima(a.scratch, m),
+                                   bound_maxima(b.scratch, n), stream);
+        const int budget = accurate_budget_log2(set);
+        if (st == OZ_OK) st = launch_accurate_finalize(m, a.scratch, budget, a.shift, stream);
+        if (st == OZ_OK) st = launch_accurate_finalize(n, b.scratch, budget, b.shift, stream);
+        if (st == OZ_OK)
+            st = launch_convert_planes(0, m, k, A, lda, set, rt, a.planes, a.stride, a.pitch, a.shift, stream);
+        if (ev && st == OZ_OK) OZ_CUDA_CHECK(cudaEventRecord(g_stage_events[dev][1], stream));
+        if (st == OZ_OK)
+            st = launch_convert_planes(1, n, k, B, ldb, set, rt, b.planes, b.stride, b.pitch, b.shift, stream);
+        if (st != OZ_OK) return st;
+        return product_impl(m, n, k, alpha, a, b, beta, C, ldc, set, rt, stream, ws + L.R, dev, plan);
+    }
     OZ_CUDA_CHECK(cudaEventRecord(g_fork[dev], stream));
     OZ_CUDA_CHECK(cudaStreamWaitEvent(side, g_fork[dev], 0));
     st = launch_deconstruct(1, n, k, B, ldb, set, rt, b.planes, b.stride, b.pitch, b.shift, b.scratch, side);
@@ -624,6 +665,7 @@ oz_status_t oz_prepare_operand(int side, int64_t lines, int64_t k, const double 
     if (lines < 0 || k < 0) return OZ_ERR_INVALID_ARG;
     if (k > OZ_K_MAX) return OZ_ERR_UNSUPPORTED;
     if (resolve_schedule(set, k, 0, true, &rt) != OZ_OK) return OZ_ERR_UNSUPPORTED;
+    if (rt.rule == 2) return OZ_ERR_UNSUPPORTED;      // the accurate rule derives the shifts from both operands
     if (lines == 0 || k == 0) return OZ_OK;           // nothing to keep: a product with k = 0 reads no operand
     if (!X || !operand || (reinterpret_cast<uintptr_t>(operand) & 255u) || (reinterpret_cast<uintptr_t>(X) & 7u) ||
         ldx < (side == 0 ? lines : k))
@@ -649,6 +691,7 @@ oz_status_t oz_dgemm_prepared(int64_t m, int64_t n, int64_t k, double alpha, con
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     oz_status_t st = check_product_args(m, n, k, alpha, beta, C, ldc, set, route, s, &rt, &trivial);
     if (st != OZ_OK || trivial) return st;
+    if (rt.rule == 2) return OZ_ERR_UNSUPPORTED;      // prepared operands carry per-operand shifts
     if (!operandA || !operandB || (reinterpret_cast<uintptr_t>(operandA) & 255u) ||
         (reinterpret_cast<uintptr_t>(operandB) & 255u))
         return OZ_ERR_INVALID_ARG;

@@ -197,6 +197,102 @@ __global__ void scan_finalize_kernel(ScanScratch s, int64_t lines, int rule, int
     shift[i] = (top >> 1) + 9 - E;
 }
 
+// ---- accurate mode (Sec. 2 "The FP8 variant": the additional FP8 product that estimates a
+// magnitude bound, the "+1" of the 3r + 1 schedule) ------------------------------------------
+// Magnitude digit of one element: the smallest integer of the E4M3 grid {0..16, 18, 20, .., 32} that
+// is >= |x| 2^(4-E), E the largest exponent of the line; integer arithmetic on the bit pattern.
+__device__ __forceinline__ uint32_t bound_digit(double x, int E)
+{
+    unsigned long long bits = static_cast<unsigned long long>(__double_as_longlong(x));
+    int be = static_cast<int>((bits >> 52) & 0x7FF);
+    unsigned long long frac = bits & 0xFFFFFFFFFFFFFull;
+    if (be == 0x7FF || (be == 0 && frac == 0)) return 0u;
+    unsigned long long sig = be ? (frac | (1ull << 52)) : frac;
+    int ex = be ? be - 1023 : -1022;
+    int sh = 48 + E - ex;                                 // |x| 2^(4-E) = sig / 2^sh
+    unsigned long long g;
+    if (sh >= 64) g = 1ull;
+    else if (sh <= 0) g = sig << (-sh);
+    else g = (sig >> sh) + ((sig & ((1ull << sh) - 1ull)) ? 1ull : 0ull);
+    uint32_t d = static_cast<uint32_t>(g);
+    if (d > 16u && (d & 1u)) ++d;                         // above 16 the grid holds the even integers
+    return d;
+}
+
+__constant__ unsigned char c_bound_code[33];              // E4M3 byte of the digits 0..32
+
+// One byte per element: the E4M3 code of its magnitude digit, K-major like the residue planes
+// (out[line * pitch + kk]; bytes kk in [k, pitch) are zero).  Lines of zeros and lines with
+// Inf/NaN give zeros.  SIDE 0 goes through a 32 x 32 shared-memory tile so that loads run along
+// the lines and stores along k.
+template <int SIDE>
+__global__ void __launch_bounds__(256)
+bound_plane_kernel(const double *__restrict__ X, int64_t ldx, int64_t lines, int64_t k, ScanScratch s,
+                   uint8_t *__restrict__ out, int64_t pitch)
+{
+    __shared__ unsigned char tile[32][36];
+    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;      // 32 x 8
+    const int64_t kchunks = (pitch + 31) / 32;
+    const int64_t ltiles = (lines + 31) / 32;
+    for (int64_t item = blockIdx.x; item < ltiles * kchunks; item += gridDim.x) {
+        const int64_t lt = item % ltiles, kc = item / ltiles;
+        if (SIDE == 0) {
+            // thread (tx, ty): line lt*32 + tx, inner indices kc*32 + ty + 8 u
+            const int64_t line = lt * 32 + tx;
+            const bool live = line < lines;
+            const int E = live ? s.emax[line] : INT32_MIN;
+            const bool dead = !live || E == INT32_MIN || s.nonfinite[line] != 0;
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int64_t kk = kc * 32 + ty + 8 * u;
+                uint32_t d = (!dead && kk < k) ? bound_digit(X[line + kk * ldx], E) : 0u;
+                tile[tx][ty + 8 * u] = c_bound_code[d];
+            }
+            __syncthreads();
+            // thread: line lt*32 + (threadIdx.x / 8), four bytes at kc*32 + 4 (threadIdx.x % 8)
+            const int lr = threadIdx.x >> 3, kq = (threadIdx.x & 7) * 4;
+            const int64_t oline = lt * 32 + lr, okk = kc * 32 + kq;
+            if (oline < lines && okk < pitch)
+                *reinterpret_cast<uint32_t *>(out + oline * pitch + okk) =
+                    *reinterpret_cast<const uint32_t *>(&tile[lr][kq]);
+            __syncthreads();
+        } else {
+            const int lr = threadIdx.x >> 3, kq = (threadIdx.x & 7) * 4;
+            const int64_t line = lt * 32 + lr, kk0 = kc * 32 + kq;
+            if (line >= lines || kk0 >= pitch) continue;
+            const int E = s.emax[line];
+            const bool dead = E == INT32_MIN || s.nonfinite[line] != 0;
+            uint32_t word = 0u;
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                uint32_t d = (!dead && kk0 + e < k) ? bound_digit(X[kk0 + e + line * ldx], E) : 0u;
+                word |= static_cast<uint32_t>(c_bound_code[d]) << (8 * e);
+            }
+            *reinterpret_cast<uint32_t *>(out + line * pitch + kk0) = word;
+        }
+    }
+}
+
+// shift[line] of the accurate rule from the line's maximum of the bound product (the bit pattern of
+// a non-negative integer-valued float, accumulated with atomicMax in the low word of sumsq[line]):
+//   ((L - ceil(log2 max)) >> 1) + 4 - E
+__global__ void accurate_finalize_kernel(ScanScratch s, int64_t lines, int L, int32_t *shift,
+                                         unsigned int *status)
+{
+    int64_t i = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x;
+    if (i >= lines) return;
+    if (s.nonfinite[i]) {
+        shift[i] = OZ_NONFINITE_SHIFT;
+        atomicOr(status, 1u << OZ_ERR_NONFINITE_INPUT);
+        return;
+    }
+    const int E = s.emax[i];
+    if (E == INT32_MIN) { shift[i] = 0; return; }
+    const uint32_t v = static_cast<uint32_t>(__uint_as_float(static_cast<uint32_t>(s.sumsq[i])));
+    const int clog = v <= 1u ? 0 : 32 - __clz(static_cast<int>(v - 1u));
+    shift[i] = ((L - clog) >> 1) + 4 - E;
+}
+
 // Eq. 1 for one element, fast form: multiplying by the power of two 2^sigma is exact in FP64 (a
 // product that underflows is far below 1/2 and rounds to zero either way), and the hardware
 // conversion rounds to nearest-even or toward zero.  Valid while 2^sigma is a normal double.
@@ -395,10 +491,10 @@ oz_status_t launch_convert(const double *X, int64_t ldx, int64_t lines, int64_t 
 
 }  // namespace
 
-oz_status_t launch_deconstruct(int side, int64_t lines, int64_t k, const double *X, int64_t ldx,
-                               int set, const Route &rt, uint8_t *planes, int64_t plane_stride,
-                               int64_t row_pitch, int32_t *shift, void *scratch,
-                               cudaStream_t stream)
+// scan_init + the scan passes of the route's scale rule [+ the shifts, except for the accurate rule,
+// whose shifts come later from the bound product]
+oz_status_t launch_scan(int side, int64_t lines, int64_t k, const double *X, int64_t ldx, int set,
+                        const Route &rt, int32_t *shift, void *scratch, cudaStream_t stream)
 {
     ScanScratch s = carve_scratch(scratch, lines);
     unsigned int *status = device_status_word();
@@ -432,11 +528,63 @@ oz_status_t launch_deconstruct(int side, int64_t lines, int64_t k, const double 
             count_launch();
         }
     }
-    scan_finalize_kernel<<<blocks1d, 256, 0, stream>>>(s, lines, rt.rule, side == 0 ? tA : tB, g2lo,
-                                                       g2hi, shift, status);
+    if (rt.rule != 2) {
+        scan_finalize_kernel<<<blocks1d, 256, 0, stream>>>(s, lines, rt.rule, side == 0 ? tA : tB, g2lo,
+                                                           g2hi, shift, status);
+        count_launch();
+    }
+    OZ_CUDA_CHECK(cudaGetLastError());
+    return OZ_OK;
+}
+
+// accurate rule: the line's magnitude digits as one K-major E4M3 plane (after launch_scan)
+oz_status_t launch_bound_plane(int side, int64_t lines, int64_t k, const double *X, int64_t ldx,
+                               void *scratch, uint8_t *plane, int64_t pitch, cudaStream_t stream)
+{
+    ScanScratch s = carve_scratch(scratch, lines);
+    int dev = 0, sms = 148;
+    OZ_CUDA_CHECK(cudaGetDevice(&dev));
+    OZ_CUDA_CHECK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    const int64_t need = ((lines + 31) / 32) * ((pitch + 31) / 32);
+    const int64_t cap = static_cast<int64_t>(sms) * 8;
+    const int grid = static_cast<int>(need < cap ? need : cap);
+    if (side == 0) bound_plane_kernel<0><<<grid, 256, 0, stream>>>(X, ldx, lines, k, s, plane, pitch);
+    else bound_plane_kernel<1><<<grid, 256, 0, stream>>>(X, ldx, lines, k, s, plane, pitch);
     count_launch();
     OZ_CUDA_CHECK(cudaGetLastError());
+    return OZ_OK;
+}
 
+// accurate rule: where the bound product accumulates the maximum of line `l` (a 32-bit word, zero
+// after launch_scan): word stride 2 from this address
+unsigned int *bound_maxima(void *scratch, int64_t lines)
+{
+    return reinterpret_cast<unsigned int *>(carve_scratch(scratch, lines).sumsq);
+}
+
+// accurate rule: shifts from the maxima of the bound product
+oz_status_t launch_accurate_finalize(int64_t lines, void *scratch, int budget_log2, int32_t *shift,
+                                     cudaStream_t stream)
+{
+    ScanScratch s = carve_scratch(scratch, lines);
+    accurate_finalize_kernel<<<static_cast<int>((lines + 255) / 256), 256, 0, stream>>>(s, lines, budget_log2, shift,
+                                                                                         device_status_word());
+    count_launch();
+    OZ_CUDA_CHECK(cudaGetLastError());
+    return OZ_OK;
+}
+
+oz_status_t upload_bound_codes(const unsigned char *codes33)
+{
+    OZ_CUDA_CHECK(cudaMemcpyToSymbol(c_bound_code, codes33, 33));
+    return OZ_OK;
+}
+
+// quantise, reduce, look up, store: the planes of one operand from its shifts
+oz_status_t launch_convert_planes(int side, int64_t lines, int64_t k, const double *X, int64_t ldx,
+                                  int set, const Route &rt, uint8_t *planes, int64_t plane_stride,
+                                  int64_t row_pitch, const int32_t *shift, cudaStream_t stream)
+{
     const uint32_t *lut = device_lut(set, rt.substrate);
 #define OZ_CONVERT(SET_, SIDE_, LAYOUT_)                                                                 \
     launch_convert<SET_, SIDE_, LAYOUT_>(X, ldx, lines, k, shift, lut, planes, plane_stride, row_pitch, \
@@ -451,6 +599,17 @@ oz_status_t launch_deconstruct(int side, int64_t lines, int64_t k, const double 
     return OZ_CONVERT_SET(2);
 #undef OZ_CONVERT_SET
 #undef OZ_CONVERT
+}
+
+oz_status_t launch_deconstruct(int side, int64_t lines, int64_t k, const double *X, int64_t ldx,
+                               int set, const Route &rt, uint8_t *planes, int64_t plane_stride,
+                               int64_t row_pitch, int32_t *shift, void *scratch,
+                               cudaStream_t stream)
+{
+    if (rt.rule == 2) return OZ_ERR_UNSUPPORTED;      // the accurate rule needs both operands
+    oz_status_t st = launch_scan(side, lines, k, X, ldx, set, rt, shift, scratch, stream);
+    if (st != OZ_OK) return st;
+    return launch_convert_planes(side, lines, k, X, ldx, set, rt, planes, plane_stride, row_pitch, shift, stream);
 }
 
 }  // namespace oz

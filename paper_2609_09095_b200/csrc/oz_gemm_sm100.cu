@@ -126,6 +126,7 @@ struct GemmParams {
     int64_t total_items;
     void *R;                        // residues: uint16 (RB = 2) or uint8 (RB = 1, byte moduli)
     int64_t ldr, mod_stride;
+    unsigned int *rowmax, *colmax;  // bound product only: one word per row / column, word stride 2
     unsigned int *status;
     ModInfo mod[kMaxR];
 };
@@ -465,7 +466,10 @@ __device__ __forceinline__ float2 mod_balanced2(float2 acc, float2 inv_m2, float
 //         512 consecutive bytes straight from registers -- no transposition through shared memory,
 //         which the tensor pipe and the TMA writes need for themselves.  The reconstruction reads
 //         the same order.  Without it the public layout R[mod][j][ldr] is written.
-template <int SUB, int CG, int RB, bool DIRECT, bool LOOSE, bool TILED>
+// BOUND: not a residue product but the magnitude-bound product of the accurate mode (Sec. 2 "The FP8
+//         variant", the "+1" pass): one plane per operand, one accumulator per tile, and instead of
+//         residues the epilogue reduces the row and column maxima of the tile into p.rowmax / p.colmax.
+template <int SUB, int CG, int RB, bool DIRECT, bool LOOSE, bool TILED, bool BOUND = false>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 residue_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB,
                     const __grid_constant__ GemmParams p)
@@ -705,6 +709,21 @@ residue_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
             const int64_t j = jw + lane;
             const int64_t i0 = static_cast<int64_t>(it.tm) * BLOCK_N + part * COLS_PER_WARP;
             if (i0 >= p.m || jw >= p.n) continue;                                 // warp-uniform
+            if constexpr (BOUND) {
+                // The accumulators are non-negative integers held exactly in FP32: their bit patterns
+                // order like their values, so the maxima are taken on the raw words.
+                uint32_t colv = 0u, keep0 = 0u, keep1 = 0u;
+#pragma unroll
+                for (int c = 0; c < COLS_PER_WARP; ++c) {
+                    colv = max(colv, comb[c]);
+                    const uint32_t rowv = __reduce_max_sync(0xFFFFFFFFu, comb[c]);   // over the warp's 32 columns
+                    if ((c & 31) == lane) { if (c < 32) keep0 = rowv; else keep1 = rowv; }
+                }
+                if (j < p.n && colv) atomicMax(p.colmax + 2 * j, colv);
+                if (i0 + lane < p.m && keep0) atomicMax(p.rowmax + 2 * (i0 + lane), keep0);
+                if (i0 + 32 + lane < p.m && keep1) atomicMax(p.rowmax + 2 * (i0 + 32 + lane), keep1);
+            }
+            if constexpr (!BOUND) {
             // last reduction of one combination value: the stored residue in the low bits of a word
             auto final_bits = [&](uint32_t cv) -> uint32_t {
                 if constexpr (SUB == 0) {
@@ -838,6 +857,7 @@ residue_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
                     }
             }
             }   // public layout
+            }   // residues
         }
     }
 
@@ -887,12 +907,12 @@ bool make_plane_map(CUtensorMap *map, const uint8_t *base, int64_t lines, int64_
     return rc == CUDA_SUCCESS;
 }
 
-template <int SUB, int CG, int RB, bool DIRECT = false, bool LOOSE = false, bool TILED = false>
+template <int SUB, int CG, int RB, bool DIRECT = false, bool LOOSE = false, bool TILED = false, bool BOUND = false>
 oz_status_t launch_variant(const CUtensorMap &mapA, const CUtensorMap &mapB, const GemmParams &p, int sms,
                            cudaStream_t stream)
 {
     static_assert(!LOOSE || RB == 2, "a representative below 2m needs the two-byte element");
-    auto kernel = residue_gemm_kernel<SUB, CG, RB, DIRECT, LOOSE, TILED>;
+    auto kernel = residue_gemm_kernel<SUB, CG, RB, DIRECT, LOOSE, TILED, BOUND>;
     OZ_CUDA_CHECK(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        static_cast<int>(SMEM_BYTES)));
     int64_t groups = sms / CG;                                    // CTAs, or CTA pairs
@@ -1073,6 +1093,49 @@ oz_status_t launch_residue_gemm(int64_t m, int64_t n, int64_t k, const uint8_t *
     return OZ_LAUNCH_SUB(2, false, false);
 #undef OZ_LAUNCH_SUB
 #undef OZ_LAUNCH
+}
+
+// The magnitude-bound product of the accurate mode: one E4M3 plane per operand (digits <= 32, terms
+// <= 1024, so one FP32 accumulator is exact for k <= 16384), the same tiles, TMA ring and tcgen05
+// instructions as the residue products, and an epilogue that keeps only the row and column maxima.
+oz_status_t launch_bound_gemm(int64_t m, int64_t n, int64_t k, const uint8_t *GA, int64_t pitchA,
+                              const uint8_t *GB, int64_t pitchB, unsigned int *rowmax,
+                              unsigned int *colmax, cudaStream_t stream)
+{
+    if (k > kBoundKMax) return OZ_ERR_UNSUPPORTED;
+    const int cg = cta_group_choice(n);
+    GemmParams p{};
+    p.m = m; p.n = n; p.k = k;
+    p.tiles_m = static_cast<int>((m + BLOCK_N - 1) / BLOCK_N);
+    p.tiles_n = static_cast<int>((n + BLOCK_M * cg - 1) / (BLOCK_M * cg));
+    p.nk = static_cast<int>((k + BLOCK_K - 1) / BLOCK_K);
+    if (k == 0) p.nk = 1;
+    p.r = 1;
+    p.total_items = static_cast<int64_t>(p.tiles_m) * p.tiles_n;
+    if (p.total_items >= 0x7FFFFFFFll) return OZ_ERR_UNSUPPORTED;
+    p.stall_producer = 0;
+    p.status = device_status_word();
+    p.rowmax = rowmax;
+    p.colmax = colmax;
+    ModInfo &mo = p.mod[0];
+    mo.m = 1.0f; mo.inv_m = 1.0f; mo.mi = 1u;
+    mo.njobs = 1;
+    mo.kind = 2;                       // one plane, one K-loop
+    mo.w[0] = 1.0f;
+    mo.iw[0] = 1;
+    mo.reduce[0] = 0;
+    mo.planeA0 = mo.planeB0 = 0;
+    mo.nseg = mo.nseg_all = 1;
+    mo.seg_len = mo.seg_len_all = p.nk;
+    CUtensorMap mapA, mapB;
+    if (!make_plane_map(&mapA, GA, m, pitchA, m * pitchA, 1, BLOCK_N / cg) ||
+        !make_plane_map(&mapB, GB, n, pitchB, n * pitchB, 1, BLOCK_M))
+        return OZ_ERR_CUDA;
+    int dev = 0, sms = 148;
+    OZ_CUDA_CHECK(cudaGetDevice(&dev));
+    OZ_CUDA_CHECK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    return cg == 2 ? launch_variant<0, 2, 2, true, false, false, true>(mapA, mapB, p, sms, stream)
+                   : launch_variant<0, 1, 2, true, false, false, true>(mapA, mapB, p, sms, stream);
 }
 
 }  // namespace oz

@@ -101,7 +101,7 @@ struct Route {
         return native() ? kLayoutNative : ((merged() && side == 0) ? kLayoutMerged : kLayoutDigits);
     }
     int quant;      // 0 rn, 1 tz
-    int rule;       // 0 maxexp, 1 cs
+    int rule;       // 0 maxexp, 1 cs, 2 accurate (shifts from the extra bound product)
 };
 bool decode_route(uint32_t route, Route *out);
 bool decode_route_for_set(int set, uint32_t route, Route *out);
@@ -143,6 +143,26 @@ ResidueTiling residue_tiling(int64_t m, int64_t n, int set);
 
 // loose: residues in [0, 2 m_i) (two-byte sets); tiled: R is the tile-ordered private array
 // (ldr and mod_stride are then ignored)
+// pieces of launch_deconstruct, and the steps of the accurate rule between them
+oz_status_t launch_scan(int side, int64_t lines, int64_t k, const double *X, int64_t ldx, int set,
+                        const Route &rt, int32_t *shift, void *scratch, cudaStream_t stream);
+oz_status_t launch_convert_planes(int side, int64_t lines, int64_t k, const double *X, int64_t ldx,
+                                  int set, const Route &rt, uint8_t *planes, int64_t plane_stride,
+                                  int64_t row_pitch, const int32_t *shift, cudaStream_t stream);
+oz_status_t launch_bound_plane(int side, int64_t lines, int64_t k, const double *X, int64_t ldx,
+                               void *scratch, uint8_t *plane, int64_t pitch, cudaStream_t stream);
+unsigned int *bound_maxima(void *scratch, int64_t lines);      // one word per line, word stride 2
+oz_status_t launch_accurate_finalize(int64_t lines, void *scratch, int budget_log2, int32_t *shift,
+                                     cudaStream_t stream);
+oz_status_t upload_bound_codes(const unsigned char *codes33);
+// the bound product on the tensor cores: rowmax[2 i] / colmax[2 j] receive (atomicMax) the bit pattern
+// of max_j / max_i of sum_k GA[i][k] GB[j][k], an integer-valued FP32 number; k <= kBoundKMax
+constexpr int64_t kBoundKMax = 16384;
+oz_status_t launch_bound_gemm(int64_t m, int64_t n, int64_t k, const uint8_t *GA, int64_t pitchA,
+                              const uint8_t *GB, int64_t pitchB, unsigned int *rowmax,
+                              unsigned int *colmax, cudaStream_t stream);
+int accurate_budget_log2(int set);
+
 oz_status_t launch_residue_gemm(int64_t m, int64_t n, int64_t k, const uint8_t *PA,
                                 int64_t strideA, int64_t pitchA, const uint8_t *PB,
                                 int64_t strideB, int64_t pitchB, int set, const Route &rt,
