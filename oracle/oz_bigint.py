@@ -65,6 +65,22 @@ def shift_of_line(line, ms, rule, tbits, k):
     return p + 9 - E
 
 
+def esc_flatness(line, k):
+    """Exponent-span check: floor(2^16 (sum abar)^2 / (k sum abar^2)), abar = ceil(|x| 2^(9-E)); None for
+    a line of zeros."""
+    nz = [abs(Fraction(x)) for x in line if x != 0]
+    if not nz:
+        return None
+    E = max(floor_log2(x) for x in nz)
+    ab = [math.ceil(x * Fraction(2) ** (9 - E)) for x in nz]
+    return (sum(ab) ** 2 * 2 ** 16) // (k * sum(a * a for a in ab))
+
+
+def esc_threshold(ms):
+    """floor(2^32 (16/3) 2^104 / H) up to the truncation of H to its top bits, H = (M-1)/2."""
+    return min(2 ** 32 - 1, (2 ** 120 // 3) // (((product(ms) - 1) // 2) >> 20))
+
+
 def bound_digit(x: float, E: int) -> int:
     """Accurate mode: the smallest E4M3-representable integer that is >= |x| 2^(4-E)."""
     if x == 0:

@@ -230,6 +230,71 @@ void ozo_shifts(int side, int64_t lines, int64_t k, const double *X, int64_t ldx
 }
 
 /* ------------------------------------------------------------------ */
+/* Exponent-span check (Algorithm 1, last line: "ESC check"; Algorithm 3, */
+/* "ESC range check") -- a reading: the paper names the check and leaves  */
+/* its criterion to the cited analysis                                    */
+/* ------------------------------------------------------------------ */
+/* With the norm-based scale rule the quantisation step of line i is about ||a_i||_2 / G,
+ * G = sqrt((M-1)/2).  Under the usual model of independent rounding errors the error of c_ij is
+ * about (step_i ||b_j||_2 + step_j ||a_i||_2) / sqrt(12), while the target 2u (|A||B|)_ij is about
+ * 2u ||a_i||_1 ||b_j||_1 / k for magnitudes spread evenly over k.  Their ratio is
+ *     1 / (G phi(a_i) phi(b_j) 2u sqrt(12)),     phi(x) = ||x||_1 / (sqrt(k) ||x||_2)  in (0, 1],
+ * so what decides whether r moduli deliver FP64-grade accuracy is how evenly each line spreads its
+ * magnitude over its exponent span ("flatness" phi; 1 for a constant line, 1/sqrt(k) for a single
+ * spike).  The check flags a call whose predicted typical ratio exceeds 1/8:
+ *     min_i phi(a_i)^2 * min_j phi(b_j)^2  <  (16/3) 2^104 / ((M-1)/2).
+ * It is evaluated in integers on the quantities of the norm scan: abar = ceil(|x| 2^(9-E)),
+ * q(line) = floor(2^16 (sum abar)^2 / (k sum abar^2)); lines of zeros or with Inf/NaN are skipped;
+ * threshold  thr = floor(floor(2^120 / 3) / (((M-1)/2) >> 20))  against  q_A q_B  (q <= 2^16).
+ * The threshold is a heuristic (parity unpinned); the arithmetic of q and thr is pinned. */
+uint32_t ozo_esc_threshold(int set)
+{
+    u128 H = (modset_product(set) - 1) / 2;
+    u128 t = (((u128)1 << 120) / 3) / (H >> 20);
+    return t > 0xFFFFFFFFu ? 0xFFFFFFFFu : (uint32_t)t;
+}
+
+/* smallest q over the lines of one operand (0xFFFFFFFF when no line counts) */
+uint32_t ozo_esc_flatness(int side, int64_t lines, int64_t k, const double *X, int64_t ldx)
+{
+    uint32_t best = 0xFFFFFFFFu;
+    for (int64_t l = 0; l < lines; ++l) {
+        int any = 0, bad = 0, E = 0;
+        for (int64_t kk = 0; kk < k; ++kk) {
+            fp_parts p = decode(*elem(X, ldx, side, l, kk));
+            if (p.kind == 2) bad = 1;
+            if (p.kind == 1) { if (!any || p.e > E) E = p.e; any = 1; }
+        }
+        if (bad || !any) continue;
+        u128 S = 0, L1 = 0;
+        for (int64_t kk = 0; kk < k; ++kk) {
+            fp_parts p = decode(*elem(X, ldx, side, l, kk));
+            if (p.kind != 1) continue;
+            int sh = 43 + E - p.ex;
+            uint64_t abar;
+            if (sh >= 64) abar = 1;
+            else if (sh <= 0) abar = p.sig << (-sh);
+            else abar = (p.sig >> sh) + ((p.sig & ((1ull << sh) - 1)) ? 1 : 0);
+            S += (u128)abar * abar;
+            L1 += abar;
+        }
+        u128 q = ((L1 * L1) << 16) / ((u128)k * S);
+        if (q < best) best = (uint32_t)q;
+    }
+    return best;
+}
+
+/* 1 when the check flags the pair of operands */
+int ozo_esc_check(int64_t m, int64_t n, int64_t k, const double *A, int64_t lda, const double *B,
+                  int64_t ldb, int set)
+{
+    uint32_t qa = ozo_esc_flatness(0, m, k, A, lda), qb = ozo_esc_flatness(1, n, k, B, ldb);
+    if (qa > 65536u) qa = 65536u;
+    if (qb > 65536u) qb = 65536u;
+    return (uint64_t)qa * qb < (uint64_t)ozo_esc_threshold(set);
+}
+
+/* ------------------------------------------------------------------ */
 /* Accurate mode (Sec. 2 "The FP8 variant": one additional FP8 GEMM that  */
 /* estimates an input magnitude bound -- the "+1" of alpha = 3r + 1)      */
 /* ------------------------------------------------------------------ */

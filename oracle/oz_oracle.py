@@ -167,6 +167,30 @@ def shifts(side: int, X: np.ndarray, s: int, rule: int, tbits: int) -> np.ndarra
     return out
 
 
+def esc_threshold(s: int) -> int:
+    f = lib().ozo_esc_threshold
+    f.restype = C.c_uint32
+    return int(f(s))
+
+
+def esc_flatness(side: int, X: np.ndarray) -> int:
+    """Smallest flatness code q = floor(2^16 phi^2) over the lines of one operand (exponent-span check)."""
+    _check_cm(X)
+    lines = X.shape[0] if side == 0 else X.shape[1]
+    k = X.shape[1] if side == 0 else X.shape[0]
+    f = lib().ozo_esc_flatness
+    f.restype = C.c_uint32
+    return int(f(side, _i64(lines), _i64(k), _p(X), _i64(max(X.shape[0], 1))))
+
+
+def esc_check(A: np.ndarray, B: np.ndarray, s: int) -> bool:
+    _check_cm(A)
+    _check_cm(B)
+    m, k = A.shape
+    n = B.shape[1]
+    return bool(lib().ozo_esc_check(_i64(m), _i64(n), _i64(k), _p(A), _i64(max(m, 1)), _p(B), _i64(max(k, 1)), s))
+
+
 def bound_digit(x: float, E: int) -> int:
     return lib().ozo_bound_digit(C.c_double(x), int(E))
 

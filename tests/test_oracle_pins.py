@@ -372,6 +372,56 @@ def test_shifts_keep_product_in_range(rule, name):
             assert all(max(abs(int(v)) for v in QA[i]) >= 2**(tA - 1) for i in range(m))
 
 
+# ----------------------------------------------------------------- exponent-span check
+def test_esc_flatness_closed_forms_and_range():
+    """q = floor(2^16 phi^2), phi^2 = ||x||_1^2 / (k ||x||_2^2) on the scan's integer magnitudes:
+    1 for a constant line, 1/k for a single spike, between the two by Cauchy-Schwarz."""
+    k = 48
+    const = np.asfortranarray(np.full((1, k), -0.75))
+    assert ozo.esc_flatness(0, const) == 65536
+    spike = np.zeros((1, k), order="F")
+    spike[0, 7] = 3.0e10
+    assert ozo.esc_flatness(0, spike) == 65536 // k
+    two = np.asfortranarray(np.array([[1.0] * 8 + [2.0 ** -3] * 40]))        # abar 512 x 8, 64 x 40
+    l1, s2 = 512 * 8 + 64 * 40, 512 ** 2 * 8 + 64 ** 2 * 40
+    assert ozo.esc_flatness(0, two) == (l1 * l1 * 65536) // (k * s2) == big.esc_flatness(two[0].tolist(), k)
+    assert ozo.esc_flatness(1, np.asfortranarray(two.T)) == ozo.esc_flatness(0, two)   # same line as a column
+    rng = np.random.default_rng(5)
+    X = np.asfortranarray((rng.random((9, k)) - 0.5) * np.exp(3 * rng.standard_normal((9, k))))
+    X[4, :] = 0.0                                                             # a line of zeros is skipped
+    per_line = [big.esc_flatness(X[i].tolist(), k) for i in range(9)]
+    assert per_line[4] is None and all(65536 // k <= q <= 65536 for q in per_line if q is not None)
+    assert ozo.esc_flatness(0, X) == min(q for q in per_line if q is not None)
+    X[2, 3] = np.inf                                                          # so is a line with Inf/NaN
+    assert ozo.esc_flatness(0, X) == min(q for i, q in enumerate(per_line) if q is not None and i != 2)
+    assert ozo.esc_flatness(0, np.zeros((3, k), order="F")) == 2 ** 32 - 1
+
+
+@pytest.mark.parametrize("name", ["S", "E", "A"])
+def test_esc_threshold_formula(name):
+    ms = ozo.modset(SETS[name])
+    H = (math.prod(ms) - 1) // 2
+    thr = ozo.esc_threshold(SETS[name])
+    assert thr == big.esc_threshold(ms)
+    exact = Fraction(16, 3) * 2 ** 104 * 2 ** 32 / H                          # 2^32 (16/3) 2^104 / H
+    assert abs(Fraction(thr) - exact) <= exact / 2 ** 20 + 1
+
+
+@pytest.mark.parametrize("cfg_id,m,n,k", [(1, 64, 64, 256), (2, 48, 40, 4096), (3, 64, 48, 1024), (4, 96, 32, 4096),
+                                          (5, 40, 36, 5003)])
+def test_esc_check_separates_the_benchmark_distributions(cfg_id, m, n, k):
+    """The check is a heuristic, so this is a calibration rather than a pin: on the five benchmark
+    distributions it flags exactly the one whose measured error exceeds 2u(|A||B|) (the lognormal
+    with sigma = 2), for every modulus set."""
+    A, B = syn.operands(syn.CONFIGS[cfg_id], m, n, k)
+    hi, lo, ab = ozo.dd_gemm(A, B)
+    for name in ("S", "E", "A"):
+        flagged = ozo.esc_check(A, B, SETS[name])
+        worst = float((np.abs(ozo.dgemm(A, B, SETS[name]) - hi) / (2 * 2.0 ** -53 * ab)).max())
+        assert flagged == (cfg_id == 5)
+        assert (worst > 1.0) == flagged
+
+
 # ----------------------------------------------------------------- accurate mode: the "+1" bound product
 def test_bound_digit_is_the_least_e4m3_upper_bound():
     """Sec. 2 "The FP8 variant": the extra product runs on FP8 operands, so its magnitude digits must
