@@ -57,7 +57,8 @@ typedef enum {
     OZ_ERR_WORKSPACE = 3,       /* no workspace registered, or it is too small                  */
     OZ_ERR_CUDA = 4,            /* a CUDA runtime / driver call failed                          */
     OZ_ERR_NONFINITE_INPUT = 5, /* device: Inf/NaN met in an operand                            */
-    OZ_ERR_RANGE = 6,           /* device: a quantised value left the representable range       */
+    OZ_ERR_RANGE = 6,           /* device: the exponent-span check flags the operands (see below); the
+                                 * results are computed all the same                             */
     OZ_ERR_TIMEOUT = 7          /* device: a bounded barrier wait ran out                       */
 } oz_status_t;
 
@@ -240,8 +241,19 @@ oz_status_t oz_reconstruct(int64_t m, int64_t n, const void *R, int64_t ldr,
                            oz_modset_t set, double alpha, double beta, double *C, int64_t ldc,
                            void *stream);
 
-/* Synchronises `stream`, then returns and clears the device status word of the current device
- * (OZ_OK, OZ_ERR_NONFINITE_INPUT, OZ_ERR_RANGE, OZ_ERR_TIMEOUT or OZ_ERR_CUDA). */
+/* Synchronises `stream`, then returns and clears the device status of the current device: the first
+ * that applies of OZ_ERR_CUDA, OZ_ERR_TIMEOUT, OZ_ERR_NONFINITE_INPUT, OZ_ERR_RANGE, else OZ_OK.
+ *
+ * OZ_ERR_RANGE is the exponent-span check (Algorithm 1, last line: "ESC check"; the paper leaves the
+ * criterion to its sources, this is the library's reading).  With the norm-based scale rule
+ * (OZ_SCALE_CS, the default) the scan also measures how evenly every line spreads its magnitude,
+ *     phi(x) = ||x||_1 / (sqrt(k) ||x||_2)   (1: constant line, 1/sqrt(k): one spike),
+ * and the status reports OZ_ERR_RANGE when, for the operands deconstructed since the last query,
+ *     min_i phi(a_i)^2 * min_j phi(b_j)^2  <  (16/3) 2^104 / ((M-1)/2),
+ * i.e. when the rounding-error model predicts a typical error above an eighth of 2u (|A||B|)_ij: the
+ * modulus set is then too small for FP64-grade accuracy on this data (escalate to a larger set, e.g.
+ * OZ_SET_A, or use native FP64 for it).  Purely informational: every result is still computed and
+ * matches the method's definition.  Not evaluated with OZ_SCALE_MAXEXP or OZ_SCALE_ACCURATE. */
 oz_status_t oz_query_status(void *stream);
 
 /* Optional per-stage timing hook for benchmarks (the paper's Algorithm 1 prices each stage

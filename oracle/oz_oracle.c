@@ -258,6 +258,7 @@ uint32_t ozo_esc_threshold(int set)
 uint32_t ozo_esc_flatness(int side, int64_t lines, int64_t k, const double *X, int64_t ldx)
 {
     uint32_t best = 0xFFFFFFFFu;
+#pragma omp parallel for schedule(static) reduction(min : best)
     for (int64_t l = 0; l < lines; ++l) {
         int any = 0, bad = 0, E = 0;
         for (int64_t kk = 0; kk < k; ++kk) {

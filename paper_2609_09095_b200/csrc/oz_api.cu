@@ -12,7 +12,10 @@ namespace oz {
 // per-device objects: plane lookup tables and the sticky status word
 // ------------------------------------------------------------------------------------------
 __device__ uint32_t g_lut[kNumSets][3][kLutWords];
+// status block: [0] sticky condition bits; [1], [2] smallest flatness code of the lines of A / B seen
+// since the last query (exponent-span check); [3] the threshold of the modulus set last used
 __device__ unsigned int g_status[4];
+const unsigned int kStatusReset[4] = {0u, 0xFFFFFFFFu, 0xFFFFFFFFu, 0u};
 
 namespace {
 
@@ -172,6 +175,16 @@ int accurate_budget_log2(int set)
     return L;
 }
 
+// Exponent-span check: a call is flagged when  qA qB < floor(floor(2^120 / 3) / (((M-1)/2) >> 20)),
+// i.e. phiA^2 phiB^2 < (16/3) 2^104 / ((M-1)/2), with q = floor(2^16 phi^2) the smallest flatness of an
+// operand's lines (see scan_finalize_kernel).
+unsigned int esc_threshold(int set)
+{
+    unsigned __int128 H = (set_product(set) - 1) / 2;
+    unsigned __int128 t = ((static_cast<unsigned __int128>(1) << 120) / 3) / (H >> 20);
+    return t > 0xFFFFFFFFu ? 0xFFFFFFFFu : static_cast<unsigned int>(t);
+}
+
 void cs_bound_squared(int set, int64_t k, uint64_t *lo, uint64_t *hi)
 {
     uint64_t bnd = isqrt_u128((set_product(set) - 1) / 2);
@@ -203,8 +216,7 @@ oz_status_t ensure_device_ready()
             for (; off < kLutWords; ++off) host_lut[set][sub][off] = 0;
         }
     OZ_CUDA_CHECK(cudaMemcpyToSymbol(g_lut, host_lut, sizeof(host_lut)));
-    unsigned int zero[4] = {0, 0, 0, 0};
-    OZ_CUDA_CHECK(cudaMemcpyToSymbol(g_status, zero, sizeof(zero)));
+    OZ_CUDA_CHECK(cudaMemcpyToSymbol(g_status, kStatusReset, sizeof(kStatusReset)));
     void *p = nullptr;
     OZ_CUDA_CHECK(cudaGetSymbolAddress(&p, g_lut));
     g_lut_addr[dev] = static_cast<const uint32_t *>(p);
@@ -782,14 +794,16 @@ oz_status_t oz_query_status(void *stream)
     oz_status_t st = ensure_device_ready();
     if (st != OZ_OK) return st;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    unsigned int word[4] = {0, 0, 0, 0}, zero[4] = {0, 0, 0, 0};
+    unsigned int word[4] = {0, 0, 0, 0};
     OZ_CUDA_CHECK(cudaStreamSynchronize(s));
     OZ_CUDA_CHECK(cudaMemcpyFromSymbol(word, g_status, sizeof(word)));
-    OZ_CUDA_CHECK(cudaMemcpyToSymbol(g_status, zero, sizeof(zero)));
+    OZ_CUDA_CHECK(cudaMemcpyToSymbol(g_status, kStatusReset, sizeof(kStatusReset)));
     if (cudaGetLastError() != cudaSuccess) return OZ_ERR_CUDA;
     if (word[0] & (1u << OZ_ERR_TIMEOUT)) return OZ_ERR_TIMEOUT;
-    if (word[0] & (1u << OZ_ERR_RANGE)) return OZ_ERR_RANGE;
     if (word[0] & (1u << OZ_ERR_NONFINITE_INPUT)) return OZ_ERR_NONFINITE_INPUT;
+    // exponent-span check: an operand that was not scanned since the last query counts as flat
+    const uint64_t qa = word[1] > 65536u ? 65536u : word[1], qb = word[2] > 65536u ? 65536u : word[2];
+    if (word[3] != 0u && qa * qb < static_cast<uint64_t>(word[3])) return OZ_ERR_RANGE;
     return OZ_OK;
 }
 
@@ -820,7 +834,7 @@ const char *oz_status_string(oz_status_t status)
         case OZ_ERR_WORKSPACE: return "workspace missing or too small";
         case OZ_ERR_CUDA: return "CUDA call failed";
         case OZ_ERR_NONFINITE_INPUT: return "Inf/NaN in an operand";
-        case OZ_ERR_RANGE: return "quantised value out of range";
+        case OZ_ERR_RANGE: return "exponent-span check: operands too unevenly scaled for FP64-grade accuracy with this modulus set";
         case OZ_ERR_TIMEOUT: return "bounded device wait ran out";
     }
     return "unknown status";

@@ -32,10 +32,11 @@ constexpr int kTileLines = 32;         // side 0: lines per shared-memory transp
 constexpr int kTilePitch = kChunk + 1; // doubles per tile row (+1: conflict-free column writes)
 
 struct ScanScratch {
-    unsigned long long *sumsq;  // [lines]
-    int *emax;                  // [lines]
-    int *nonfinite;             // [lines]
+    unsigned long long *sumsq;  // [lines]  sum of squared magnitudes (accurate rule: maximum of the bound product)
+    int *emax;                  // [lines]  largest exponent, INT32_MIN for a line of zeros
+    int *nonfinite;             // [lines]  bit 31: the line holds Inf/NaN; bits 0..30: sum of the magnitudes
 };
+constexpr int kNonfiniteBit = INT32_MIN;
 
 __host__ __device__ inline ScanScratch carve_scratch(void *scratch, int64_t lines)
 {
@@ -104,6 +105,7 @@ scan_kernel(const double *__restrict__ X, int64_t ldx, int64_t lines, int64_t k,
     bool live = line < lines;
     int emax = INT32_MIN, bad = 0;
     unsigned long long acc = 0;
+    unsigned int l1 = 0;          // sum of the magnitudes abar <= 2^10 (exponent-span check): below 2^30 for k <= 2^20
     int E = 0;
     if (PASS == 1 && live) E = s.emax[line];
     // 2^(9-E) as a double, when it is a normal number (not for lines of subnormals only)
@@ -134,6 +136,7 @@ scan_kernel(const double *__restrict__ X, int64_t ldx, int64_t lines, int64_t k,
                     if (abar == 0ull && x != 0.0) abar = 1ull;
                     if (!(y < 2048.0)) abar = 0ull;       // Inf/NaN: the line is flagged, value unused
                     acc += abar * abar;
+                    l1 += static_cast<unsigned int>(abar);
                 } else {
                     unsigned long long bits = static_cast<unsigned long long>(__double_as_longlong(x));
                     int be = static_cast<int>((bits >> 52) & 0x7FF);
@@ -147,6 +150,7 @@ scan_kernel(const double *__restrict__ X, int64_t ldx, int64_t lines, int64_t k,
                     else if (sh <= 0) abar = sig << (-sh);
                     else abar = (sig >> sh) + ((sig & ((1ull << sh) - 1)) ? 1ull : 0ull);
                     acc += abar * abar;
+                    l1 += static_cast<unsigned int>(abar);
                 }
             }
         }
@@ -160,6 +164,7 @@ scan_kernel(const double *__restrict__ X, int64_t ldx, int64_t lines, int64_t k,
                 bad |= __shfl_xor_sync(0xFFFFFFFFu, bad, o);
             } else {
                 acc += __shfl_xor_sync(0xFFFFFFFFu, acc, o);
+                l1 += __shfl_xor_sync(0xFFFFFFFFu, l1, o);
             }
         }
         if (lane != 0) live = false;
@@ -167,21 +172,22 @@ scan_kernel(const double *__restrict__ X, int64_t ldx, int64_t lines, int64_t k,
     if (!live) return;
     if (PASS == 0) {
         if (emax != INT32_MIN) atomicMax(&s.emax[line], emax);
-        if (bad) atomicOr(&s.nonfinite[line], 1);
+        if (bad) atomicOr(&s.nonfinite[line], kNonfiniteBit);
     } else if (acc) {
         atomicAdd(&s.sumsq[line], acc);
+        atomicAdd(&s.nonfinite[line], static_cast<int>(l1));     // never reaches bit 31
     }
 }
 
 // shift[line]: MAXEXP  t - 1 - E;  CS  p + 9 - E with p the largest integer such that
 // 4^p * S <= G^2  (G^2 passed as two 64-bit words).
-__global__ void scan_finalize_kernel(ScanScratch s, int64_t lines, int rule, int tbits,
+__global__ void scan_finalize_kernel(ScanScratch s, int64_t lines, int64_t k, int side, int rule, int tbits,
                                      unsigned long long g2lo, unsigned long long g2hi,
-                                     int32_t *shift, unsigned int *status)
+                                     unsigned int esc_threshold, int32_t *shift, unsigned int *status)
 {
     int64_t i = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x;
     if (i >= lines) return;
-    if (s.nonfinite[i]) {
+    if (s.nonfinite[i] < 0) {
         shift[i] = OZ_NONFINITE_SHIFT;
         atomicOr(status, 1u << OZ_ERR_NONFINITE_INPUT);
         return;
@@ -195,6 +201,14 @@ __global__ void scan_finalize_kernel(ScanScratch s, int64_t lines, int rule, int
     unsigned long long qlo = static_cast<unsigned long long>(q);
     int top = qhi ? 127 - __clzll(static_cast<long long>(qhi)) : 63 - __clzll(static_cast<long long>(qlo));
     shift[i] = (top >> 1) + 9 - E;
+    // Exponent-span check (Algorithm 1, "ESC check"): flatness of the line,
+    // floor(2^16 (sum abar)^2 / (k sum abar^2)); the smallest value of each operand is kept in the
+    // device status block and judged against the set's threshold when the status is queried.
+    const unsigned long long l1 = static_cast<unsigned int>(s.nonfinite[i]);
+    const unsigned __int128 flat = ((static_cast<unsigned __int128>(l1 * l1)) << 16) /
+                                   (static_cast<unsigned __int128>(static_cast<unsigned long long>(k)) * s.sumsq[i]);
+    atomicMin(status + 1 + side, static_cast<unsigned int>(flat));
+    status[3] = esc_threshold;
 }
 
 // ---- accurate mode (Sec. 2 "The FP8 variant": the additional FP8 product that estimates a
@@ -241,7 +255,7 @@ bound_plane_kernel(const double *__restrict__ X, int64_t ldx, int64_t lines, int
             const int64_t line = lt * 32 + tx;
             const bool live = line < lines;
             const int E = live ? s.emax[line] : INT32_MIN;
-            const bool dead = !live || E == INT32_MIN || s.nonfinite[line] != 0;
+            const bool dead = !live || E == INT32_MIN || s.nonfinite[line] < 0;
 #pragma unroll
             for (int u = 0; u < 4; ++u) {
                 const int64_t kk = kc * 32 + ty + 8 * u;
@@ -261,7 +275,7 @@ bound_plane_kernel(const double *__restrict__ X, int64_t ldx, int64_t lines, int
             const int64_t line = lt * 32 + lr, kk0 = kc * 32 + kq;
             if (line >= lines || kk0 >= pitch) continue;
             const int E = s.emax[line];
-            const bool dead = E == INT32_MIN || s.nonfinite[line] != 0;
+            const bool dead = E == INT32_MIN || s.nonfinite[line] < 0;
             uint32_t word = 0u;
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
@@ -281,7 +295,7 @@ __global__ void accurate_finalize_kernel(ScanScratch s, int64_t lines, int L, in
 {
     int64_t i = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x;
     if (i >= lines) return;
-    if (s.nonfinite[i]) {
+    if (s.nonfinite[i] < 0) {
         shift[i] = OZ_NONFINITE_SHIFT;
         atomicOr(status, 1u << OZ_ERR_NONFINITE_INPUT);
         return;
@@ -529,8 +543,8 @@ oz_status_t launch_scan(int side, int64_t lines, int64_t k, const double *X, int
         }
     }
     if (rt.rule != 2) {
-        scan_finalize_kernel<<<blocks1d, 256, 0, stream>>>(s, lines, rt.rule, side == 0 ? tA : tB, g2lo,
-                                                           g2hi, shift, status);
+        scan_finalize_kernel<<<blocks1d, 256, 0, stream>>>(s, lines, k, side, rt.rule, side == 0 ? tA : tB, g2lo,
+                                                           g2hi, esc_threshold(set), shift, status);
         count_launch();
     }
     OZ_CUDA_CHECK(cudaGetLastError());

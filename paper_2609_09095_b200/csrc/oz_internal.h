@@ -162,6 +162,8 @@ oz_status_t launch_bound_gemm(int64_t m, int64_t n, int64_t k, const uint8_t *GA
                               const uint8_t *GB, int64_t pitchB, unsigned int *rowmax,
                               unsigned int *colmax, cudaStream_t stream);
 int accurate_budget_log2(int set);
+// exponent-span check: threshold of the set against the product of the two operands' flatness codes
+unsigned int esc_threshold(int set);
 
 oz_status_t launch_residue_gemm(int64_t m, int64_t n, int64_t k, const uint8_t *PA,
                                 int64_t strideA, int64_t pitchA, const uint8_t *PB,

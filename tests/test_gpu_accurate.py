@@ -86,3 +86,51 @@ def test_accurate_mode_limits():
     # the shifts of one operand depend on the other: no per-operand entry point takes the rule
     assert oz.oz_deconstruct(0, 4, 16, t, 4, oz.OZ_SET_S, rt, u, 64, 16, s, u) == oz.OZ_ERR_UNSUPPORTED
     assert oz.oz_prepare_operand(0, 4, 16, t, 4, oz.OZ_SET_S, rt, u) == oz.OZ_ERR_UNSUPPORTED
+
+
+# ------------------------------------------------------------------ exponent-span check
+@pytest.mark.parametrize("set_name", ["S", "E", "A"])
+def test_exponent_span_status_matches_oracle(set_name):
+    """Algorithm 1, "ESC check": the status of a whole-method call is OZ_ERR_RANGE exactly when the
+    oracle's statement of the check flags the operands -- on the five benchmark distributions, on a
+    spike, and for a single operand through the stage entry point -- and the results are untouched."""
+    import paper_2609_09095_b200 as oz
+    import tests.gpu_helpers as gh
+    sub = "int8n" if set_name == "A" else "fp8"
+    cases = [syn.operands(syn.CONFIGS[c], 96, 80, kk) for c, kk in ((1, 256), (2, 1500), (3, 1024), (4, 2000), (5, 3001))]
+    cases.append(syn.special_operands("spike", 40, 30, 500))
+    seen = set()
+    for A, B in cases:
+        got, st = None, None
+        m, k = A.shape
+        n = B.shape[1]
+        gh.ensure_workspace(oz.oz_workspace_bytes(m, n, k, gh.SETS[set_name], gh.route(sub)))
+        dA, dB = gh.to_dev(A), gh.to_dev(B)
+        import torch
+        dC = torch.zeros((n, m), dtype=torch.float64, device="cuda")
+        oz.check(oz.oz_dgemm(m, n, k, dA, m, dB, k, dC, m, gh.SETS[set_name], gh.route(sub)), "oz_dgemm")
+        st = gh.sync_status(esc=True)
+        flagged = ozo.esc_check(A, B, OSET[set_name])
+        assert st == (oz.OZ_ERR_RANGE if flagged else 0)
+        assert (gh.from_dev(dC) == ozo.dgemm(A, B, OSET[set_name])).all()
+        assert gh.sync_status(esc=True) == 0                     # cleared by the query
+        seen.add(flagged)
+        # the other scale rules do not run the check
+        oz.check(oz.oz_dgemm(m, n, k, dA, m, dB, k, dC, m, gh.SETS[set_name], gh.route(sub, "RN", "MAXEXP")), "oz_dgemm")
+        assert gh.sync_status(esc=True) == 0
+    assert seen == {True, False}
+    # one operand through the stage entry point: the other counts as flat
+    A, B = cases[4]
+    thr = ozo.esc_threshold(OSET[set_name])
+    for side, X in ((0, A), (1, B)):
+        lines = X.shape[0] if side == 0 else X.shape[1]
+        k = X.shape[1] if side == 0 else X.shape[0]
+        p = oz.oz_plane_count_side(gh.SETS[set_name], gh.route(sub), side)
+        pitch = oz.oz_row_pitch(k)
+        planes = torch.empty((p, lines, pitch), dtype=torch.uint8, device="cuda")
+        shift = torch.empty((lines,), dtype=torch.int32, device="cuda")
+        scratch = torch.zeros(16 * lines + 256, dtype=torch.uint8, device="cuda")
+        oz.check(oz.oz_deconstruct(side, lines, k, gh.to_dev(X), X.shape[0], gh.SETS[set_name], gh.route(sub), planes,
+                                   lines * pitch, pitch, shift, scratch), "oz_deconstruct")
+        want = oz.OZ_ERR_RANGE if min(ozo.esc_flatness(side, X), 65536) * 65536 < thr else 0
+        assert gh.sync_status(esc=True) == want

@@ -92,7 +92,7 @@ def test_static_entry_allocates_nothing_and_holds_its_maximum():
     call()
     free_after, _ = torch.cuda.mem_get_info()
     assert free_after == free_before
-    assert oz.oz_query_status() == 0
+    assert oz.oz_query_status() == 0          # uniform lines: the exponent-span check has nothing to say
     assert bool((shift == ref_shift).all()) and bool((planes == ref_planes).all())
     # the line sampled against the oracle: first, last and a few in between
     pick = np.array([0, 1, lines // 2, lines - 2, lines - 1])
