@@ -174,7 +174,9 @@ __device__ __forceinline__ void store_pair(double *out, double p0, double p1, bo
     }
 }
 
-// the ROWS consecutive rows of column j whose residues are packed in w[]: reconstruct, update C
+// the ROWS consecutive rows of column j whose residues are packed in w[]: reconstruct, update C.
+// For beta = 1 the old values of C are requested before the arithmetic starts, so that their latency
+// hides behind it.
 template <int SET>
 __device__ __forceinline__ void reconstruct_rows(const uint32_t (&w)[kMaxR], int64_t row, int nrows, int sb,
                                                  const int32_t *__restrict__ shiftA, double alpha, double beta,
@@ -184,16 +186,26 @@ __device__ __forceinline__ void reconstruct_rows(const uint32_t (&w)[kMaxR], int
     int sa[ROWS];
 #pragma unroll
     for (int h = 0; h < ROWS; ++h) sa[h] = h < nrows ? shiftA[row + h] : 0;
+    const bool whole = vecC && nrows == ROWS;
+    double2 old[ROWS / 2];
+#pragma unroll
+    for (int h = 0; h < ROWS / 2; ++h) old[h] = make_double2(0.0, 0.0);
+    if (whole && beta != 0.0) {
+#pragma unroll
+        for (int h = 0; h < ROWS / 2; ++h) old[h] = *reinterpret_cast<const double2 *>(out + 2 * h);
+    }
     {
         double p0 = row_value<SET, 0>(w, sa[0], sb, alpha);
         double p1 = nrows > 1 ? row_value<SET, 1>(w, sa[1], sb, alpha) : 0.0;
-        store_pair(out, p0, p1, nrows > 1, vecC, beta);
+        if (whole) *reinterpret_cast<double2 *>(out) = make_double2(old[0].x + p0, old[0].y + p1);
+        else store_pair(out, p0, p1, nrows > 1, false, beta);
     }
     if constexpr (ROWS == 4) {
         if (nrows > 2) {
             double p2 = row_value<SET, 2>(w, sa[2], sb, alpha);
             double p3 = nrows > 3 ? row_value<SET, 3>(w, sa[3], sb, alpha) : 0.0;
-            store_pair(out + 2, p2, p3, nrows > 3, vecC, beta);
+            if (whole) *reinterpret_cast<double2 *>(out + 2) = make_double2(old[1].x + p2, old[1].y + p3);
+            else store_pair(out + 2, p2, p3, nrows > 3, false, beta);
         }
     }
 }
