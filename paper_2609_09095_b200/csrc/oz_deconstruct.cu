@@ -478,6 +478,254 @@ convert_kernel(const double *__restrict__ X, int64_t ldx, int64_t lines, int64_t
     }
 }
 
+// ---- whole deconstruction of a group of lines in one kernel ------------------------------------
+// When a few whole lines fit in shared memory next to the look-up table, a thread block loads them
+// once and takes everything from there: largest exponent, the norm sums, the shift, and the
+// conversion into planes.  The operand is then read from HBM once (8 bytes per element instead of
+// 24 with the three-pass kernels above) and one launch replaces five.  The arithmetic is the same,
+// function by function, so the outputs are identical; the sums are integers, hence independent of
+// the order in which the warps add them.  Not for the accurate rule, whose shifts need the other
+// operand.
+struct FusedParams {
+    const double *X;
+    int64_t ldx, lines, k;
+    int group;                 // lines per thread block pass
+    int pitch;                 // doubles per line in shared memory (k + 1: conflict-free for both sides)
+    int side, rule, tbits, tz;
+    unsigned long long g2lo, g2hi;
+    unsigned int esc_threshold;
+    const uint32_t *lut_global;
+    uint8_t *planes;
+    int64_t plane_stride, row_pitch;
+    int32_t *shift;
+    unsigned int *status;
+};
+
+struct FusedLine {             // per-line results in shared memory
+    unsigned long long sumsq;
+    int emax, bad, shift;
+    unsigned int l1;
+};
+
+template <int SET, int SIDE, int LAYOUT>
+__global__ void __launch_bounds__(1024, 1)
+deconstruct_fused_kernel(const __grid_constant__ FusedParams p)
+{
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    uint32_t *lut = reinterpret_cast<uint32_t *>(smem_raw);
+    double *buf = reinterpret_cast<double *>(smem_raw + kLutWords * 4);
+    FusedLine *res = reinterpret_cast<FusedLine *>(buf + static_cast<size_t>(p.group) * p.pitch);
+    const int nthreads = blockDim.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = nthreads >> 5;
+    for (int i = tid; i < kLutWords; i += nthreads) lut[i] = p.lut_global[i];
+    const int64_t ngroups = (p.lines + p.group - 1) / p.group;
+    const int k = static_cast<int>(p.k);
+    for (int64_t g = blockIdx.x; g < ngroups; g += gridDim.x) {
+        const int64_t line0 = g * p.group;
+        const int nl = static_cast<int>(p.lines - line0 < p.group ? p.lines - line0 : p.group);
+        __syncthreads();                 // the previous group's conversion has finished with buf / res
+        // ---- load: nl lines x k doubles, coalesced along the operand's leading dimension
+        if (SIDE == 0) {
+            // element (line, kk) at X[line + kk ldx]: consecutive threads take consecutive lines
+            // (the group size is a power of two on this side: shifts instead of divisions)
+            const int gshift = 31 - __clz(p.group), gmask = p.group - 1;
+            const int total = k << gshift;
+            for (int e0 = tid; e0 < total; e0 += 4 * nthreads) {
+                double v[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int e = e0 + u * nthreads, kk = e >> gshift, l = e & gmask;
+                    v[u] = (e < total && l < nl) ? p.X[line0 + l + static_cast<int64_t>(kk) * p.ldx] : 0.0;
+                }
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int e = e0 + u * nthreads, kk = e >> gshift, l = e & gmask;
+                    if (e < total && l < nl) buf[l * p.pitch + kk] = v[u];
+                }
+            }
+        } else {
+            // batches of independent loads: enough bytes in flight to run at memory speed
+            for (int l0 = 0; l0 < nl; l0 += 4)
+                for (int kk = tid; kk < k; kk += nthreads) {
+                    double v[4];
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) v[u] = l0 + u < nl ? p.X[kk + (line0 + l0 + u) * p.ldx] : 0.0;
+#pragma unroll
+                    for (int u = 0; u < 4; ++u)
+                        if (l0 + u < nl) buf[(l0 + u) * p.pitch + kk] = v[u];
+                }
+        }
+        if (tid < nl) {
+            res[tid].sumsq = 0ull;
+            res[tid].emax = INT32_MIN;
+            res[tid].bad = 0;
+            res[tid].l1 = 0u;
+        }
+        __syncthreads();
+        // ---- the scans: a line is cut into `segs` pieces, one warp per piece
+        const int segs = nwarps >= nl ? nwarps / nl : 1;
+        const int span = (k + segs - 1) / segs;
+        for (int item = warp; item < nl * segs; item += nwarps) {
+            const int l = item / segs, seg = item - l * segs;
+            const int k0 = seg * span, k1 = min(k, k0 + span);
+            int emax = INT32_MIN, bad = 0;
+            for (int kk = k0 + lane; kk < k1; kk += 32) {
+                int e;
+                const int c = classify(buf[l * p.pitch + kk], &e);
+                if (c == 2) bad = 1;
+                if (c == 1 && e > emax) emax = e;
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+                emax = max(emax, __shfl_xor_sync(0xFFFFFFFFu, emax, o));
+                bad |= __shfl_xor_sync(0xFFFFFFFFu, bad, o);
+            }
+            if (lane == 0) {
+                if (emax != INT32_MIN) atomicMax(&res[l].emax, emax);
+                if (bad) atomicOr(&res[l].bad, 1);
+            }
+        }
+        __syncthreads();
+        if (p.rule == 1) {
+            for (int item = warp; item < nl * segs; item += nwarps) {
+                const int l = item / segs, seg = item - l * segs;
+                const int k0 = seg * span, k1 = min(k, k0 + span);
+                const int E = res[l].emax;
+                if (E == INT32_MIN || res[l].bad) continue;              // warp-uniform
+                const bool fast_scale = 9 - E >= -1000 && 9 - E <= 1000;
+                const double scale9 = __hiloint2double((1023 + (fast_scale ? 9 - E : 0)) << 20, 0);
+                unsigned long long acc = 0ull;
+                unsigned int l1 = 0u;
+                for (int kk = k0 + lane; kk < k1; kk += 32) {
+                    const double x = buf[l * p.pitch + kk];
+                    unsigned long long abar;
+                    if (fast_scale) {
+                        const double y = fabs(x) * scale9;
+                        abar = static_cast<unsigned long long>(__double2ll_ru(y));
+                        if (abar == 0ull && x != 0.0) abar = 1ull;
+                    } else {
+                        unsigned long long bits = static_cast<unsigned long long>(__double_as_longlong(x));
+                        int be = static_cast<int>((bits >> 52) & 0x7FF);
+                        unsigned long long frac = bits & 0xFFFFFFFFFFFFFull;
+                        if (be == 0 && frac == 0) continue;
+                        unsigned long long sig = be ? (frac | (1ull << 52)) : frac;
+                        int ex = be ? be - 1023 : -1022;
+                        int sh = 43 + E - ex;                 // |x| 2^(9-E) = sig / 2^sh
+                        if (sh >= 64) abar = 1;
+                        else if (sh <= 0) abar = sig << (-sh);
+                        else abar = (sig >> sh) + ((sig & ((1ull << sh) - 1)) ? 1ull : 0ull);
+                    }
+                    acc += abar * abar;
+                    l1 += static_cast<unsigned int>(abar);
+                }
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) {
+                    acc += __shfl_xor_sync(0xFFFFFFFFu, acc, o);
+                    l1 += __shfl_xor_sync(0xFFFFFFFFu, l1, o);
+                }
+                if (lane == 0 && acc) {
+                    atomicAdd(&res[l].sumsq, acc);
+                    atomicAdd(&res[l].l1, l1);
+                }
+            }
+            __syncthreads();
+        }
+        // ---- the shift of every line (same arithmetic as scan_finalize_kernel)
+        if (tid < nl) {
+            FusedLine &r = res[tid];
+            int sh = 0;
+            if (r.bad) {
+                sh = OZ_NONFINITE_SHIFT;
+                atomicOr(p.status, 1u << OZ_ERR_NONFINITE_INPUT);
+            } else if (r.emax != INT32_MIN) {
+                if (p.rule == 0) {
+                    sh = p.tbits - 1 - r.emax;
+                } else {
+                    unsigned __int128 G2 = (static_cast<unsigned __int128>(p.g2hi) << 64) | p.g2lo;
+                    unsigned __int128 q = G2 / static_cast<unsigned __int128>(r.sumsq);
+                    unsigned long long qhi = static_cast<unsigned long long>(q >> 64);
+                    unsigned long long qlo = static_cast<unsigned long long>(q);
+                    int top = qhi ? 127 - __clzll(static_cast<long long>(qhi)) : 63 - __clzll(static_cast<long long>(qlo));
+                    sh = (top >> 1) + 9 - r.emax;
+                    const unsigned long long l1 = r.l1;
+                    const unsigned __int128 flat = ((static_cast<unsigned __int128>(l1 * l1)) << 16) /
+                                                   (static_cast<unsigned __int128>(static_cast<unsigned long long>(p.k)) * r.sumsq);
+                    atomicMin(p.status + 1 + p.side, static_cast<unsigned int>(flat));
+                    p.status[3] = p.esc_threshold;
+                }
+            }
+            r.shift = sh;
+            p.shift[line0 + tid] = sh;
+        }
+        __syncthreads();
+        // ---- conversion: a thread takes four consecutive inner indices of one line
+        const int quads = static_cast<int>(p.row_pitch >> 2);          // row_pitch is a multiple of 16
+        for (int it = tid; it < nl * quads; it += nthreads) {
+            const int l = it / quads, kb = (it - l * quads) * 4;
+            const int sigma = res[l].shift;
+            const bool dead = sigma == OZ_NONFINITE_SHIFT;
+            double x[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) x[e] = (!dead && kb + e < k) ? buf[l * p.pitch + kb + e] : 0.0;
+            convert4<SET, LAYOUT>(x, dead ? 0 : sigma, p.tz != 0, lut, p.planes + (line0 + l) * p.row_pitch + kb,
+                                  p.plane_stride);
+        }
+    }
+}
+
+// Lines per thread-block pass of the fused kernel and its launch shape; group = 0: not applicable
+// (the lines are too long for shared memory).
+#ifndef OZ_FUSED_MAX_ELEMS
+#define OZ_FUSED_MAX_ELEMS (1ll << 22)
+#endif
+struct FusedShape { int group, threads, grid; size_t smem; };
+
+FusedShape fused_shape(int side, int64_t lines, int64_t k, int sms)
+{
+    FusedShape f{0, 0, 0, 0};
+    if (k < 1 || k > 32768 || lines < 1) return f;
+    // The one-kernel form wins where the call is bound by launch latency; larger operands keep the
+    // three-pass kernels, whose many small blocks hide the memory latency better.
+    if (lines * k > OZ_FUSED_MAX_ELEMS) return f;
+    const size_t line_bytes = static_cast<size_t>(k + 1) * 8;
+    const size_t fixed = kLutWords * 4 + 64 * sizeof(FusedLine) + 64;
+    // two blocks per SM when lines are short enough for that, else one block with more threads
+    const size_t budget2 = 110 * 1024, budget1 = 224 * 1024;
+    int group = static_cast<int>((budget2 - fixed) / line_bytes);
+    int threads = 512;
+    const int min_group = side == 0 ? 4 : 1;         // side 0 loads `group` consecutive doubles per inner index
+    if (group < (side == 0 ? 8 : 2)) {
+        group = static_cast<int>((budget1 - fixed) / line_bytes);
+        threads = 1024;
+    }
+    if (group < min_group) return f;
+    if (group > 32) group = 32;
+    if (side == 0) {
+        int pow2 = 1;
+        while (pow2 * 2 <= group) pow2 *= 2;
+        group = pow2;
+    } else if (group > lines) {
+        group = static_cast<int>(lines);
+    }
+    f.group = group;
+    f.threads = threads;
+    f.smem = fixed + static_cast<size_t>(group) * line_bytes;
+    const int64_t ngroups = (lines + group - 1) / group;
+    const int64_t cap = static_cast<int64_t>(sms) * (threads == 512 ? 2 : 1);
+    f.grid = static_cast<int>(ngroups < cap ? ngroups : cap);
+    return f;
+}
+
+template <int SET, int SIDE, int LAYOUT>
+oz_status_t launch_fused(const FusedParams &p, const FusedShape &f, cudaStream_t stream)
+{
+    auto kernel = deconstruct_fused_kernel<SET, SIDE, LAYOUT>;
+    OZ_CUDA_CHECK(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(f.smem)));
+    kernel<<<f.grid, f.threads, f.smem, stream>>>(p);
+    count_launch();
+    OZ_CUDA_CHECK(cudaGetLastError());
+    return OZ_OK;
+}
+
 template <int SET, int SIDE, int LAYOUT>
 oz_status_t launch_convert(const double *X, int64_t ldx, int64_t lines, int64_t k,
                            const int32_t *shift, const uint32_t *lut, uint8_t *planes,
@@ -621,6 +869,39 @@ oz_status_t launch_deconstruct(int side, int64_t lines, int64_t k, const double 
                                cudaStream_t stream)
 {
     if (rt.rule == 2) return OZ_ERR_UNSUPPORTED;      // the accurate rule needs both operands
+    int dev = 0, sms = 148;
+    OZ_CUDA_CHECK(cudaGetDevice(&dev));
+    OZ_CUDA_CHECK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    const FusedShape f = fused_shape(side, lines, k, sms);
+    if (f.group > 0) {
+        FusedParams p{};
+        p.X = X; p.ldx = ldx; p.lines = lines; p.k = k;
+        p.group = f.group;
+        p.pitch = static_cast<int>(k + 1);
+        p.side = side; p.rule = rt.rule; p.tz = rt.quant;
+        int tA = 0, tB = 0;
+        budget_maxexp(set, k, &tA, &tB);
+        p.tbits = side == 0 ? tA : tB;
+        uint64_t g2lo = 0, g2hi = 0;
+        cs_bound_squared(set, k, &g2lo, &g2hi);
+        p.g2lo = g2lo; p.g2hi = g2hi;
+        p.esc_threshold = esc_threshold(set);
+        p.lut_global = device_lut(set, rt.substrate);
+        p.planes = planes; p.plane_stride = plane_stride; p.row_pitch = row_pitch;
+        p.shift = shift;
+        p.status = device_status_word();
+        const int layout = rt.layout(side);
+#define OZ_FUSED(SET_, SIDE_, LAYOUT_) launch_fused<SET_, SIDE_, LAYOUT_>(p, f, stream)
+#define OZ_FUSED_SET(SET_)                                                                      \
+    (side == 1 ? OZ_FUSED(SET_, 1, kLayoutDigits)                                               \
+               : (layout == kLayoutMerged ? OZ_FUSED(SET_, 0, kLayoutMerged) : OZ_FUSED(SET_, 0, kLayoutDigits)))
+        if (layout == kLayoutNative) return side == 0 ? OZ_FUSED(2, 0, kLayoutNative) : OZ_FUSED(2, 1, kLayoutNative);
+        if (set == 0) return OZ_FUSED_SET(0);
+        if (set == 1) return OZ_FUSED_SET(1);
+        return OZ_FUSED_SET(2);
+#undef OZ_FUSED_SET
+#undef OZ_FUSED
+    }
     oz_status_t st = launch_scan(side, lines, k, X, ldx, set, rt, shift, scratch, stream);
     if (st != OZ_OK) return st;
     return launch_convert_planes(side, lines, k, X, ldx, set, rt, planes, plane_stride, row_pitch, shift, stream);

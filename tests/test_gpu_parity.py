@@ -34,7 +34,9 @@ def _oracle_deconstruct(side, X, set_name, sub, quant, rule):
 @pytest.mark.parametrize("side", [0, 1])
 @pytest.mark.parametrize("lines,k,dist", [(256, 256, "uniform"), (37, 129, "lognormal:2.0"),
                                           (130, 1000, "normal"), (1, 1, "uniform"), (5, 17, "lognormal:0.5"),
-                                          (67, 4101, "lognormal:2.0"), (300, 16, "uniform")])
+                                          (67, 4101, "lognormal:2.0"), (300, 16, "uniform"),
+                                          # too long or too large for the one-kernel deconstruction: the three-pass kernels
+                                          (40, 7001, "normal"), (9, 30011, "lognormal:0.5"), (2100, 2100, "normal")])
 @pytest.mark.parametrize("set_name,sub,quant,rule", [("S", "fp8", "RN", "CS"), ("S", "int8", "TZ", "MAXEXP"),
                                                      ("E", "fp8", "TZ", "CS"), ("E", "int8", "RN", "MAXEXP"),
                                                      ("A", "int8n", "RN", "CS"), ("A", "fp8", "TZ", "MAXEXP")])
