@@ -19,6 +19,11 @@
  * big-integer restatement -- except the accuracy of the method against the true
  * product on inputs with a very wide exponent spread, for which the paper prints
  * no bound: "parity unpinned" for that one quantity (it is measured, not asserted).
+ * Two passages name a step and leave its content to the paper's sources: the extra
+ * bound product of the accurate mode and the "ESC check".  The readings taken are
+ * stated above ozo_bound_digit and ozo_esc_threshold; their arithmetic is pinned
+ * (soundness by brute force, closed forms, the big-integer restatement), the
+ * threshold of the ESC reading is a heuristic: "parity unpinned" for that value.
  *
  * Storage conventions (column-major BLAS shapes, Sec. 2: C = AB, A m x k, B k x n):
  *   side 0: X is m x k, "line" i is row i,    element (i,kk) at X[i + kk*ldx]
