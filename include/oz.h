@@ -33,6 +33,10 @@
  *   - m, n or k equal to zero is OZ_OK (k = 0 gives C = 0, or C unchanged for beta = 1).
  *   - Non-finite contract: an Inf or NaN anywhere in row i of A (column j of B)
  *     makes every C(i,:) (C(:,j)) NaN and sets OZ_ERR_NONFINITE_INPUT.
+ *   - Range of the result: the product is rounded once to 53 bits and then scaled by a power of
+ *     two.  Where that scaling lands below the normal range (|C_ij| < 2^-1022) the value is rounded a
+ *     second time, to the subnormal grid, and where it lands above the largest finite number it
+ *     becomes infinite; such outputs are outside the single-rounding contract.
  *   - One FP32 accumulator of the FP8 route stays exact to k = 32768 (Lemma 1 and the accumulation
  *     invariant of Algorithm 2), an INT32 one to 131071 (native residues) or 4 million (digits).
  *     A longer k is split inside the residue-GEMM kernel into K segments with an accumulator each,

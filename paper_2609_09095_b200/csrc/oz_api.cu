@@ -210,8 +210,8 @@ oz_status_t ensure_device_ready()
             int off = 0;
             for (int i = 0; i < set_r(set); ++i) {
                 int m = modulus(set, i);
-                for (int u = 0; u < m; ++u) host_lut[set][sub][off + u] = lut_entry(u, m, sub);
-                off += m;
+                for (int u = 0; u < kLutSpan * m; ++u) host_lut[set][sub][off + u] = lut_entry(u % m, m, sub);
+                off += kLutSpan * m;
             }
             for (; off < kLutWords; ++off) host_lut[set][sub][off] = 0;
         }

@@ -349,21 +349,27 @@ __device__ __forceinline__ void convert_modulus(const uint32_t (&l0)[4], const u
     // a' = l0 + l1 2^16 + l2 2^32 + l3 2^48 with the top limb SIGNED; `bias` (a multiple of m not
     // below 2^15 c3) keeps the limb sum non-negative, so no separate sign correction is needed.
     constexpr uint32_t bias = ((32768u * c3 + m - 1) / m) * m;
-    // floor(v / m) = (v * ceil(2^39 / m)) >> 39 exactly for v < 2^28
-    constexpr uint32_t magic = static_cast<uint32_t>(((1ull << 39) + m - 1) / m);
+    static_assert(65535ull * (1ull + c1 + c2) + 32767ull * c3 + bias < (1ull << 28), "limb sum below 2^28");
+    // Everything is carried four times too large, so that the remainder is the BYTE offset of the
+    // table entry: v = 4 (limb sum) < 2^30, and floor(v / 4m) = (v * ceil(2^(32+s) / 4m)) >> (32+s)
+    // exactly for s = ceil(log2 m) (the multiplier stays below 2^31).
+    // Per element: four multiply-adds, one multiply-high, a shift, one multiply-subtract, one look-up.
+    constexpr uint32_t m4 = 4u * m;
+    constexpr int s = ceil_log2(m);
+    constexpr uint32_t magic = static_cast<uint32_t>(((1ull << (32 + s)) + m4 - 1) / m4);
+    static_assert(static_cast<unsigned long long>(m4) << 30 <= (1ull << (32 + s)), "exact quotient for v < 2^30");
     constexpr int off = lut_offset(SET, I);
     constexpr int plane = first_plane(SET, I, LAYOUT);
-    static_assert(65535ull * (1ull + c1 + c2) + 32767ull * c3 + bias < (1ull << 28), "limb sum below 2^28");
+    const unsigned char *table = reinterpret_cast<const unsigned char *>(lut + off);
     uint32_t w[4];
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
-        uint32_t v = l3[e] * c3 + bias;          // l3 holds the signed limb in two's complement
-        v = l2[e] * c2 + v;
-        v = l1[e] * c1 + v;
-        v += l0[e];
-        uint32_t q = __umulhi(v, magic) >> 7;
-        uint32_t r = v - q * m;                  // canonical residue in [0, m)
-        w[e] = lut[off + r];
+        uint32_t v = l3[e] * (4u * c3) + 4u * bias;      // l3 holds the signed limb in two's complement
+        v = l2[e] * (4u * c2) + v;
+        v = l1[e] * (4u * c1) + v;
+        v = l0[e] * 4u + v;
+        const uint32_t r4 = v - (__umulhi(v, magic) >> s) * m4;        // 4 (a' mod m), canonical
+        w[e] = *reinterpret_cast<const uint32_t *>(table + r4);
     }
     uint32_t t01 = __byte_perm(w[0], w[1], 0x5140);
     uint32_t t23 = __byte_perm(w[2], w[3], 0x5140);
@@ -424,7 +430,7 @@ convert_kernel(const double *__restrict__ X, int64_t ldx, int64_t lines, int64_t
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     uint32_t *lut = reinterpret_cast<uint32_t *>(smem_raw);
-    for (int i = threadIdx.x; i < kLutWords; i += kConvThreads) lut[i] = lut_global[i];
+    for (int i = threadIdx.x; i < lut_words(SET); i += kConvThreads) lut[i] = lut_global[i];
     __syncthreads();
 
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -447,7 +453,7 @@ convert_kernel(const double *__restrict__ X, int64_t ldx, int64_t lines, int64_t
             convert4<SET, LAYOUT>(x, dead ? 0 : sigma, tz != 0, lut, planes + line * row_pitch + kb, plane_stride);
         }
     } else {
-        double *tile = reinterpret_cast<double *>(smem_raw + kLutWords * 4);
+        double *tile = reinterpret_cast<double *>(smem_raw + lut_words(SET) * 4);
         const uint32_t ltiles = static_cast<uint32_t>((lines + kTileLines - 1) / kTileLines);
         const uint32_t items = ltiles * nchunks;
         for (uint32_t item = blockIdx.x; item < items; item += gridDim.x) {
@@ -513,10 +519,10 @@ deconstruct_fused_kernel(const __grid_constant__ FusedParams p)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     uint32_t *lut = reinterpret_cast<uint32_t *>(smem_raw);
-    double *buf = reinterpret_cast<double *>(smem_raw + kLutWords * 4);
+    double *buf = reinterpret_cast<double *>(smem_raw + lut_words(SET) * 4);
     FusedLine *res = reinterpret_cast<FusedLine *>(buf + static_cast<size_t>(p.group) * p.pitch);
     const int nthreads = blockDim.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = nthreads >> 5;
-    for (int i = tid; i < kLutWords; i += nthreads) lut[i] = p.lut_global[i];
+    for (int i = tid; i < lut_words(SET); i += nthreads) lut[i] = p.lut_global[i];
     const int64_t ngroups = (p.lines + p.group - 1) / p.group;
     const int k = static_cast<int>(p.k);
     for (int64_t g = blockIdx.x; g < ngroups; g += gridDim.x) {
@@ -679,7 +685,7 @@ deconstruct_fused_kernel(const __grid_constant__ FusedParams p)
 #endif
 struct FusedShape { int group, threads, grid; size_t smem; };
 
-FusedShape fused_shape(int side, int64_t lines, int64_t k, int sms)
+FusedShape fused_shape(int set, int side, int64_t lines, int64_t k, int sms)
 {
     FusedShape f{0, 0, 0, 0};
     if (k < 1 || k > 32768 || lines < 1) return f;
@@ -687,7 +693,7 @@ FusedShape fused_shape(int side, int64_t lines, int64_t k, int sms)
     // three-pass kernels, whose many small blocks hide the memory latency better.
     if (lines * k > OZ_FUSED_MAX_ELEMS) return f;
     const size_t line_bytes = static_cast<size_t>(k + 1) * 8;
-    const size_t fixed = kLutWords * 4 + 64 * sizeof(FusedLine) + 64;
+    const size_t fixed = lut_words(set) * 4 + 64 * sizeof(FusedLine) + 64;
     // two blocks per SM when lines are short enough for that, else one block with more threads
     const size_t budget2 = 110 * 1024, budget1 = 224 * 1024;
     int group = static_cast<int>((budget2 - fixed) / line_bytes);
@@ -731,7 +737,7 @@ oz_status_t launch_convert(const double *X, int64_t ldx, int64_t lines, int64_t 
                            const int32_t *shift, const uint32_t *lut, uint8_t *planes,
                            int64_t plane_stride, int64_t row_pitch, int tz, cudaStream_t stream)
 {
-    size_t smem = kLutWords * 4 + (SIDE == 0 ? sizeof(double) * kTileLines * kTilePitch : 0);
+    size_t smem = lut_words(SET) * 4 + (SIDE == 0 ? sizeof(double) * kTileLines * kTilePitch : 0);
     OZ_CUDA_CHECK(cudaFuncSetAttribute(convert_kernel<SET, SIDE, LAYOUT>,
                                        cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        static_cast<int>(smem)));
@@ -742,7 +748,11 @@ oz_status_t launch_convert(const double *X, int64_t ldx, int64_t lines, int64_t 
     int dev = 0, sms = 148;
     OZ_CUDA_CHECK(cudaGetDevice(&dev));
     OZ_CUDA_CHECK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
-    int64_t cap = static_cast<int64_t>(sms) * (SIDE == 1 ? 6 : 3);
+    // persistent blocks: as many as are resident at once (each copies the table once)
+    int per_sm = 1;
+    OZ_CUDA_CHECK(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, convert_kernel<SET, SIDE, LAYOUT>,
+                                                                kConvThreads, smem));
+    int64_t cap = static_cast<int64_t>(sms) * (per_sm > 0 ? per_sm : 1);
     int grid = static_cast<int>(need < cap ? need : cap);
     convert_kernel<SET, SIDE, LAYOUT><<<grid, kConvThreads, smem, stream>>>(
         X, ldx, lines, k, shift, lut, planes, plane_stride, row_pitch, tz);
@@ -872,7 +882,7 @@ oz_status_t launch_deconstruct(int side, int64_t lines, int64_t k, const double 
     int dev = 0, sms = 148;
     OZ_CUDA_CHECK(cudaGetDevice(&dev));
     OZ_CUDA_CHECK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
-    const FusedShape f = fused_shape(side, lines, k, sms);
+    const FusedShape f = fused_shape(rt.layout(side) == kLayoutNative ? 2 : set, side, lines, k, sms);
     if (f.group > 0) {
         FusedParams p{};
         p.X = X; p.ldx = ldx; p.lines = lines; p.k = k;

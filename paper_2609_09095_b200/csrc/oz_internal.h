@@ -11,6 +11,8 @@ namespace oz {
 
 constexpr int kMaxR = 15;          // moduli in the largest supported set (A)
 constexpr int kMaxPlanes = 44;     // stored planes of set A with two-limb digits
+// The plane look-up table of a set holds, per modulus, the packed plane bytes of the residues 0 .. m-1.
+constexpr int kLutSpan = 1;
 constexpr int kLutWords = 8208;    // >= sum of the moduli of any set (S: 8069, E: 6736, A: 3478)
 
 // ---- modulus sets (Sec. 2 step (ii) for S; "Candidate E" and "Candidate A" paragraphs) ---
@@ -69,9 +71,12 @@ __host__ __device__ constexpr int64_t merged_k_limit(int set) { return set == 0 
 __host__ __device__ constexpr int lut_offset(int set, int i)
 {
     int o = 0;
-    for (int j = 0; j < i; ++j) o += modulus(set, j);
+    for (int j = 0; j < i; ++j) o += kLutSpan * modulus(set, j);
     return o;
 }
+
+// words of a set's table, rounded up to whole 16-byte groups
+__host__ __device__ constexpr int lut_words(int set) { return (lut_offset(set, set_r(set)) + 3) / 4 * 4; }
 
 // 2^e mod m
 __host__ __device__ constexpr uint32_t pow2_mod(int e, uint32_t m)
@@ -79,6 +84,14 @@ __host__ __device__ constexpr uint32_t pow2_mod(int e, uint32_t m)
     uint32_t v = 1 % m;
     for (int j = 0; j < e; ++j) v = (v * 2u) % m;
     return v;
+}
+
+// smallest s with 2^s >= m
+__host__ __device__ constexpr int ceil_log2(uint32_t m)
+{
+    int s = 0;
+    while ((1u << s) < m) ++s;
+    return s;
 }
 
 // floor(2^32 / m)
