@@ -772,9 +772,11 @@ residue_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
             };
             constexpr int NCH = COLS_PER_WARP * RB / 16;     // 16-byte chunks of a thread's run of rows
             if constexpr (TILED) {
+                // block (tile, CTA rank, warp), then modulus: the r residue blocks of one 32 x 64 patch of
+                // the output lie next to one another, which is how the reconstruction reads them
                 unsigned char *blk = static_cast<unsigned char *>(p.R) +
-                    ((((static_cast<int64_t>(it.mod) * p.tiles_m + it.tm) * p.tiles_n + it.tn) * CG + rank) * EPI_WARPS +
-                     (part * 4 + q)) * static_cast<int64_t>(NCH * 512) + lane * 16;
+                    (((((static_cast<int64_t>(it.tm) * p.tiles_n + it.tn) * CG + rank) * EPI_WARPS + (part * 4 + q)) * p.r +
+                      it.mod) * static_cast<int64_t>(NCH * 512)) + lane * 16;
 #pragma unroll
                 for (int c = 0; c < NCH; ++c) {
                     uint4 val;

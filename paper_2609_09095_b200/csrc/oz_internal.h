@@ -145,12 +145,13 @@ oz_status_t launch_deconstruct(int side, int64_t lines, int64_t k, const double 
 // pairs: rank-major) of 32 columns x 64 rows, one per epilogue warp, block w = quarter + 4 * part
 // covering columns 32 * quarter .. +31 (of the rank's 128) and rows 64 * part .. +63; a block is
 // stored as [16-byte chunk c][column], chunk c holding 16 / residue_bytes consecutive rows.
-// Residue of modulus i: R + i * mod_stride elements, tiles in (tile row, tile column) order.
+// Order in memory: tile row, tile column, CTA rank, block, modulus -- the r residue blocks of one
+// 32 x 64 patch of the output are consecutive (4 KiB each, 2 KiB for byte residues).
 struct ResidueTiling {
     int cg;              // 1: tiles of 128 columns, 2: CTA pairs, tiles of 256 columns
     int tile_cols;
     int tiles_m, tiles_n;
-    int64_t mod_stride;  // elements per modulus (tiles are stored whole, padding included)
+    int64_t mod_stride;  // elements per modulus in total (tiles are stored whole, padding included)
 };
 ResidueTiling residue_tiling(int64_t m, int64_t n, int set);
 

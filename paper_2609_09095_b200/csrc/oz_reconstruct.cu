@@ -261,7 +261,7 @@ reconstruct_kernel(const void *__restrict__ Rv, int64_t ldr, int64_t mod_stride,
 // grid: x = (piece of the block, block within the tile, CTA rank of the pair), y = tile column, z = tile row
 template <int SET>
 __global__ void __launch_bounds__(256, residue_bytes(SET) == 2 ? 6 : 5)
-reconstruct_tiled_kernel(const void *__restrict__ Rv, int64_t mod_stride, int cg, int tiles_n, int tn0,
+reconstruct_tiled_kernel(const void *__restrict__ Rv, int cg, int tiles_n, int tn0,
                          int64_t m, int64_t n, int64_t col0, int64_t col1,
                          const int32_t *__restrict__ shiftA, const int32_t *__restrict__ shiftB,
                          double alpha, double beta, double *__restrict__ C, int64_t ldc, int vecC)
@@ -282,11 +282,12 @@ reconstruct_tiled_kernel(const void *__restrict__ Rv, int64_t mod_stride, int cg
     if (row >= m || j >= n || j < col0 || j >= col1) return;
     const int nrows = m - row < ROWS ? static_cast<int>(m - row) : ROWS;
     const int64_t wb = ((static_cast<int64_t>(tm) * tiles_n + tn) * cg + rank) * 16 + wi;
+    // the r blocks of this patch are consecutive: modulus i at a compile-time offset
     const unsigned char *base = static_cast<const unsigned char *>(Rv) +
-                                (wb * kBlockWords + c * 128 + lane * 4 + sub) * 4;
+                                ((wb * r) * kBlockWords + c * 128 + lane * 4 + sub) * 4;
     uint32_t w[kMaxR];
 #pragma unroll
-    for (int i = 0; i < r; ++i) w[i] = *reinterpret_cast<const uint32_t *>(base + i * mod_stride * RB);
+    for (int i = 0; i < r; ++i) w[i] = *reinterpret_cast<const uint32_t *>(base + i * (kBlockWords * 4));
     reconstruct_rows<SET>(w, row, nrows, shiftB[j], shiftA, alpha, beta, C + row + j * ldc, vecC != 0);
 }
 
@@ -368,7 +369,7 @@ oz_status_t launch_reconstruct_tiled(int64_t m, int64_t n, const void *R, const 
     const dim3 grid(static_cast<unsigned>(pieces * 16 * t.cg), static_cast<unsigned>(ntn),
                     static_cast<unsigned>(t.tiles_m));
 #define OZ_RECON_TILED(SET_)                                                                              \
-    reconstruct_tiled_kernel<SET_><<<grid, 256, 0, stream>>>(R, t.mod_stride, t.cg, t.tiles_n, tn0, m, n,  \
+    reconstruct_tiled_kernel<SET_><<<grid, 256, 0, stream>>>(R, t.cg, t.tiles_n, tn0, m, n,  \
                                                              col0, col1, shiftA, shiftB, alpha, beta, C, ldc, vecC)
     if (set == 2) OZ_RECON_TILED(2);
     else if (set == 0) OZ_RECON_TILED(0);
