@@ -104,6 +104,14 @@ typedef enum { OZ_SET_S = 0, OZ_SET_E = 1, OZ_SET_A = 2 } oz_modset_t;
 #define OZ_ACC_MERGED   0x1000u
 #define OZ_ACC_SEPARATE 0x2000u
 
+/* Reconstruction of the whole-method calls with the CRT recombination hosted on the INT8 tensor pipe
+ * (Algorithm 3, the "[INT8-TENSOR + SIMT]" branch: about r multiply-accumulates per output as one
+ * small unsigned 8-bit product, then carry, lift and the single rounding in integer arithmetic).
+ * Same results bit for bit.  The default form evaluates the same weighted sum in exact FP64 chunks;
+ * on B200, whose FP64 pipe is as wide as its integer pipe, that form is about 1.8 times faster, so
+ * this bit is for comparison and for parts with a narrow FP64 pipe.  Ignored by the stage entry points. */
+#define OZ_RECON_TENSOR 0x4000u
+
 #define OZ_K_MAX 1048576
 #define OZ_NONFINITE_SHIFT INT32_MIN  /* value of shift[] for a line that holds Inf/NaN */
 

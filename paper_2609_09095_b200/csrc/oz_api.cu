@@ -118,7 +118,8 @@ uint64_t isqrt_u128(unsigned __int128 v)
 bool decode_route(uint32_t route, Route *out)
 {
     uint32_t sub = route & 0x00Fu, q = route & 0x0F0u, sc = route & 0xF00u, ac = route & 0x3000u;
-    if (route & ~0x3FFFu) return false;
+    if (route & ~0x7FFFu) return false;
+    out->hosted = (route & OZ_RECON_TENSOR) != 0;
     if (ac == 0) out->acc = 0;
     else if (ac == OZ_ACC_MERGED) out->acc = 1;
     else if (ac == OZ_ACC_SEPARATE) out->acc = 2;
@@ -231,6 +232,8 @@ oz_status_t ensure_device_ready()
         codes[d] = static_cast<unsigned char>(code);
     }
     st = upload_bound_codes(codes);
+    if (st != OZ_OK) return st;
+    st = upload_hosted_constants();
     if (st != OZ_OK) return st;
     g_ready[dev] = true;
     return OZ_OK;
@@ -361,14 +364,17 @@ oz_status_t product_impl(int64_t m, int64_t n, int64_t k, double alpha, const Op
                                          rt, R, 0, 0, residue_bytes(set) == 2, true, stream);
     if (st != OZ_OK) return st;
     if (ev) OZ_CUDA_CHECK(cudaEventRecord(g_stage_events[dev][3], stream));
+    // the CRT recombination: exact FP64 chunk sums on the FP64 pipe, or (OZ_RECON_TENSOR) one small
+    // unsigned 8-bit product per 128 outputs on the tensor pipe and an integer tail
+    auto reconstruct = rt.hosted ? launch_reconstruct_hosted : launch_reconstruct_tiled;
     if (!plan) {
-        st = launch_reconstruct_tiled(m, n, R, a.shift, b.shift, set, alpha, beta, C, ldc, 0, n, stream);
+        st = reconstruct(m, n, R, a.shift, b.shift, set, alpha, beta, C, ldc, 0, n, stream);
         if (st != OZ_OK) return st;
     } else {
         for (int p = 0; p < plan->np; ++p) {
             if (plan->wait_before) OZ_CUDA_CHECK(cudaStreamWaitEvent(stream, plan->before[p], 0));
-            st = launch_reconstruct_tiled(m, n, R, a.shift, b.shift, set, alpha, beta, C, ldc, plan->col0[p],
-                                          plan->col0[p + 1], stream);
+            st = reconstruct(m, n, R, a.shift, b.shift, set, alpha, beta, C, ldc, plan->col0[p],
+                             plan->col0[p + 1], stream);
             if (st != OZ_OK) return st;
             OZ_CUDA_CHECK(cudaEventRecord(plan->after[p], stream));
         }

@@ -113,6 +113,7 @@ struct Route {
     {
         return native() ? kLayoutNative : ((merged() && side == 0) ? kLayoutMerged : kLayoutDigits);
     }
+    bool hosted;    // whole-method calls: CRT recombination on the INT8 tensor pipe (OZ_RECON_TENSOR)
     int quant;      // 0 rn, 1 tz
     int rule;       // 0 maxexp, 1 cs, 2 accurate (shifts from the extra bound product)
 };
@@ -198,6 +199,13 @@ oz_status_t launch_reconstruct(int64_t m, int64_t n, const void *R, int64_t ldr,
 
 // uploads the reconstruction constants of every set to the current device
 oz_status_t upload_reconstruct_constants();
+oz_status_t upload_hosted_constants();
+
+// reconstruction from the tile-ordered array with the CRT recombination on the INT8 tensor pipe
+oz_status_t launch_reconstruct_hosted(int64_t m, int64_t n, const void *R, const int32_t *shiftA,
+                                      const int32_t *shiftB, int set, double alpha, double beta,
+                                      double *C, int64_t ldc, int64_t col0, int64_t col1,
+                                      cudaStream_t stream);
 
 #define OZ_CUDA_CHECK(expr)                                  \
     do {                                                     \

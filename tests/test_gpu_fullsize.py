@@ -93,6 +93,14 @@ def test_full_size_sampled(cfg_id, set_name, sub):
     assert (got == Co).all()
     # a whole-matrix property that holds at any size: no entry is left unwritten / non-finite
     assert bool(torch.isfinite(dC).all())
+    if cfg_id in (3, 5):
+        # the reconstruction hosted on the tensor pipe gives the same matrix, entry for entry
+        dC2 = gh.to_dev(C0) if C0 is not None else torch.empty((n, m), dtype=torch.float64, device="cuda")
+        oz.check(oz.oz_dgemm_ex(m, n, k, cfg.alpha, dA, m, dB, k, cfg.beta, dC2, m, gh.SETS[set_name],
+                                rt | oz.OZ_RECON_TENSOR), "oz_dgemm_ex, tensor-hosted reconstruction")
+        assert gh.sync_status() == 0
+        assert bool((dC2 == dC).all())
+        del dC2
     del dA, dB, dC
     oz.oz_set_workspace(None)
     gh._ws = None

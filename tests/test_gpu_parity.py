@@ -468,3 +468,74 @@ def test_bounded_waits_time_out_cleanly(n):
                           f"import tests.test_gpu_parity as t; t._stalled_then_normal({n})"],
                          cwd=root, env=env, capture_output=True, text=True, timeout=600)
     assert out.returncode == 0 and "stalled-then-normal ok" in out.stdout, out.stdout + out.stderr
+
+
+def test_whole_method_rounding_boundaries():
+    """The reconstruction of the whole-method calls (tile-ordered residues) at the boundaries of its one
+    rounding: with k = 1 the integer c' is the product of two chosen integers times a power of two, so
+    operands can be built whose products sit exactly on ties (2^53 + 1 and friends: round to even, both
+    ways), one unit either side of a tie, just below and at powers of two, and far beyond 53 bits.
+    Every output must equal the oracle's (and Python's correctly rounded product), with the FP64 form of
+    the reconstruction and with the one hosted on the INT8 tensor pipe."""
+    import tests.gpu_helpers as gh
+    from fractions import Fraction
+    # factor pairs of integers of 54..60 bits with interesting low bits
+    targets = []
+    for base in (2 ** 53, 2 ** 54, 2 ** 57, 3 * 2 ** 52):
+        for delta in (-3, -2, -1, 0, 1, 2, 3, 5, 7):
+            targets.append(base + delta)
+    targets += [2 ** 53 + 2 ** 20 + 1, (2 ** 53 + 1) * 3, (2 ** 53 + 3) * 5, 2 ** 60 - 1, 2 ** 60 + 2 ** 7]
+    rows, cols = [], []
+    for t in targets:                      # t = p * q with p small and odd if possible, else p = 1
+        p = next((d for d in (3, 5, 7, 9, 11, 13, 107, 321) if t % d == 0), 1)
+        q = t // p
+        if q < 2 ** 53:                    # both factors must be exact doubles
+            rows.append(float(p))
+            cols.append(float(q))
+    A = np.asfortranarray(np.array(rows + [-r for r in rows]).reshape(-1, 1))
+    B = np.asfortranarray(np.array(cols).reshape(1, -1))
+    exact = [[Fraction(a) * Fraction(b) for b in B[0]] for a in A[:, 0]]
+    for set_name, sub, recon in (("S", "fp8", None), ("E", "int8", None), ("A", "int8n", None),
+                                 ("S", "fp8", "tensor"), ("E", "fp8", "tensor"), ("A", "int8n", "tensor")):
+        for quant in ("RN", "TZ"):
+            got, st = gh.dgemm(A, B, set_name, gh.route(sub, quant, "CS", recon=recon))
+            oq = ozo.QUANT_RN if quant == "RN" else ozo.QUANT_TZ
+            want = ozo.dgemm(A, B, OSET[set_name], oq, ozo.SCALE_CS)
+            assert st == 0 and (got == want).all()
+            # integers this small are quantised exactly, so the result is the correctly rounded product
+            assert got.tolist() == [[float(v) for v in row] for row in exact]
+
+
+@pytest.mark.parametrize("set_name,sub,m,n,k,alpha,beta", [
+    ("S", "fp8", 700, 515, 384, 1.0, 0.0),          # several tiles, ragged, CTA-pair tiles
+    ("S", "int8", 257, 129, 1000, -1.0, 1.0),
+    ("E", "fp8", 300, 260, 1024, -1.0, 1.0),        # 13 moduli: all sixteen byte positions in use
+    ("A", "int8n", 520, 300, 260, 1.0, 1.0),        # byte residues: four outputs per thread
+    ("A", "fp8", 64, 1030, 96, 1.0, 0.0),
+    ("S", "fp8", 1, 1, 1, 1.0, 0.0),
+])
+def test_reconstruction_hosted_on_the_tensor_pipe(set_name, sub, m, n, k, alpha, beta):
+    """OZ_RECON_TENSOR (Algorithm 3, the INT8-tensor branch of the reconstruction): the CRT
+    recombination as one unsigned 8-bit tcgen05 product per 128 outputs and an integer tail.  Bit for
+    bit the oracle's result, like the FP64 form, also on lines of zeros, spikes and non-finite input."""
+    import paper_2609_09095_b200 as oz
+    import tests.gpu_helpers as gh
+    rng = np.random.default_rng(m + 3 * n + 7 * k)
+    A, B = syn._draw(rng, m, k, "lognormal:0.5"), syn._draw(rng, k, n, "normal")
+    C0 = np.asfortranarray(rng.standard_normal((m, n)))
+    if m > 8 and n > 8:
+        A[3, :] = 0.0
+        B[:, 5] = 0.0
+        A[1, k // 2] = 7.0e30
+    rt = gh.route(sub, "RN", "CS", recon="tensor")
+    got, st = gh.dgemm(A, B, set_name, rt, alpha, beta, C0 if beta else None)
+    want = ozo.dgemm(A, B, OSET[set_name], ozo.QUANT_RN, ozo.SCALE_CS, alpha, beta, C0 if beta else None)
+    assert st == 0 and (got == want).all()
+    plain, st = gh.dgemm(A, B, set_name, gh.route(sub, "RN", "CS"), alpha, beta, C0 if beta else None)
+    assert st == 0 and (plain == got).all()
+    if m > 8 and n > 8:
+        A[2, 0] = np.nan
+        got, st = gh.dgemm(A, B, set_name, rt, alpha, beta, C0 if beta else None)
+        want = ozo.dgemm(A, B, OSET[set_name], ozo.QUANT_RN, ozo.SCALE_CS, alpha, beta, C0 if beta else None)
+        assert st == oz.OZ_ERR_NONFINITE_INPUT
+        assert (np.isnan(got) == np.isnan(want)).all() and (got[~np.isnan(want)] == want[~np.isnan(want)]).all()
