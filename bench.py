@@ -314,7 +314,7 @@ def main():
     esc_flag = [False]
 
     def check_status(where):
-        """Device status; the exponent-span verdict (OZ_ERR_RANGE) is informational and only recorded."""
+        """Device status; the result of the exponent-span check (OZ_ERR_RANGE) is informational and only recorded."""
         st = oz.oz_query_status(stream)
         if st == oz.OZ_ERR_RANGE:
             esc_flag[0] = True

@@ -631,7 +631,7 @@ residue_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
             }
             for (int job = 0; ok && job < mi.njobs; ++job)
             for (int seg = 0, nseg = job_segments(mi, job); ok && seg < nseg; ++seg) {
-                // every lane polls for itself; the verdict is made warp-uniform before anything that
+                // every lane polls for itself; the outcome is made warp-uniform before anything that
                 // contains a warp barrier depends on it
                 ok = __all_sync(0xFFFFFFFFu, mbar_wait(tfull_bar + 8 * slot, (slot_phase >> slot) & 1u, abort_flag, p.status));
                 if (!ok) break;

@@ -320,7 +320,7 @@ reconstruct_hosted_kernel(const void *__restrict__ Rv, int cg, int tiles_n, int 
                 for (int it = 0; it < 256 && !ok; ++it) ok = bar_try_wait(bar, phase);
             }
         }
-        if (__syncthreads_or(ok ? 0 : 1)) {              // block-uniform verdict
+        if (__syncthreads_or(ok ? 0 : 1)) {              // block-uniform outcome
             if (t == 0) atomicOr(status, 1u << OZ_ERR_TIMEOUT);
             alive = false;
             break;

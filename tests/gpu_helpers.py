@@ -37,7 +37,7 @@ def from_dev(t: torch.Tensor) -> np.ndarray:
 
 
 def sync_status(esc: bool = False) -> int:
-    """Device status after a synchronisation.  The verdict of the exponent-span check
+    """Device status after a synchronisation.  The result of the exponent-span check
     (OZ_ERR_RANGE) is informational -- the results are the same with or without it -- so it is
     reported as 0 unless the caller asks for it (the tests that pin the check do)."""
     st = oz.oz_query_status()

@@ -83,7 +83,7 @@ def test_full_size_sampled(cfg_id, set_name, sub):
     gh.ensure_workspace(oz.oz_workspace_bytes(m, n, k, gh.SETS[set_name], rt))
     dC = gh.to_dev(C0) if C0 is not None else torch.empty((n, m), dtype=torch.float64, device="cuda")
     oz.check(oz.oz_dgemm_ex(m, n, k, cfg.alpha, dA, m, dB, k, cfg.beta, dC, m, gh.SETS[set_name], rt), "oz_dgemm_ex")
-    # exponent-span check at full size: the oracle's verdict on the whole operands (config 5 is flagged)
+    # exponent-span check at full size: the oracle's result on the whole operands (config 5 is flagged)
     flagged = ozo.esc_check(A, B, oset)
     assert flagged == (cfg_id == 5)
     assert gh.sync_status(esc=True) == (oz.OZ_ERR_RANGE if flagged else 0)
