@@ -347,7 +347,9 @@ def main():
     oz.oz_set_stage_events(None)
     check_status("device status after the timed steps")
     local_ms = ev0.elapsed_time(ev1) / args.steps
-    stage_ms = np.array([[evs[i].elapsed_time(evs[i + 1]) for i in range(4)] for evs in stage_events]).mean(axis=0)
+    per_step = np.array([[evs[i].elapsed_time(evs[i + 1]) for i in range(4)] for evs in stage_events])
+    stage_ms = per_step.mean(axis=0)
+    step_totals = per_step.sum(axis=1)          # first to last stage event of every timed call
 
     # ---- end to end through the host-buffer entry point (copies inside the timed region)
     def e2e_step():
@@ -404,6 +406,14 @@ def main():
         also.append({"modulus_set": args.set_name, "substrate": args.substrate, "planes": "prepared once (oz_dgemm_prepared)",
                      "value": flops / (ms3 * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": ms3, "steps": 5})
         del opA, opB
+        if k <= 16384:
+            # accurate mode: the shifts from one extra tensor-core product of magnitude digits (3r + 1 passes)
+            rt4 = route & ~oz.OZ_SCALE_CS | oz.OZ_SCALE_ACCURATE
+            ms4 = timed_steps(lambda: oz.check(oz.oz_dgemm_ex(m, n, k, cfg.alpha, dA, m, dB, k, cfg.beta, dC, m, modset,
+                                                              rt4, stream), "oz_dgemm_ex"))
+            check_status("device status (accurate mode)")
+            also.append({"modulus_set": args.set_name, "substrate": args.substrate, "scale_rule": "ACCURATE",
+                         "value": flops / (ms4 * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": ms4, "steps": 5})
     lib8 = library_8bit_tflops(torch) if (world == 1 and not args.no_also) else {"fp8": None, "int8": None}
 
     if world > 1:
@@ -474,6 +484,7 @@ def main():
                 "deconstruct_GBps": dec_bytes / ((stage_ms[0] + stage_ms[1]) * 1e-3) / 1e9,
                 "reconstruct_GBps": rec_bytes / (stage_ms[3] * 1e-3) / 1e9,
                 "reconstruct_bytes": rec_bytes,
+                "call_ms_median": float(np.median(step_totals)), "call_ms_best": float(step_totals.min()),
                 "hbm_peak_GBps": hbm, "hbm_peak_source": peaks["source"]},
             "also": also,
             "e2e": {"value": work / (e2e_ms * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": e2e_ms,
