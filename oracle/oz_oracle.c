@@ -678,9 +678,16 @@ int ozo_pstore_merged(int set, int side)
     return p;
 }
 
-/* plane order per non-square modulus on side 0: d0, -16*d1, d0+d1; on side 1: d0, d1, d0+d1 */
-int ozo_planes_merged(int side, int64_t lines, int64_t k, const int16_t *D, int set, uint8_t *P,
-                      int64_t plane_stride, int64_t row_pitch)
+/* The same regrouping on the INT8 substrate (B200 keeps an INT8 tensor path; -16*d1 reaches -256 and
+ * does not fit a signed byte, so the factor 16 is shared between the operands):
+ *     d e = 15 [ (-d0) e0 + (4 d1)(4 e1) ] + 16 (d0+d1)(e0+e1)
+ * side 0 stores -d0, 4*d1, d0+d1; side 1 stores e0, 4*e1, e0+e1 (|4 d1| <= 64).  The merged term
+ * reaches 196 + 16*256 = 4292, exact in INT32 far beyond any supported k.
+ *
+ * plane order per non-square modulus, FP8: side 0: d0, -16*d1, d0+d1; side 1: d0, d1, d0+d1
+ *                                    INT8: side 0: -d0, 4*d1, d0+d1; side 1: d0, 4*d1, d0+d1 */
+int ozo_planes_merged_sub(int side, int64_t lines, int64_t k, const int16_t *D, int set, int substrate,
+                          uint8_t *P, int64_t plane_stride, int64_t row_pitch)
 {
     int mod[16], r = ozo_modset(set, mod), plane = 0, bad = 0;
     for (int i = 0; i < r; ++i) {
@@ -690,10 +697,23 @@ int ozo_planes_merged(int side, int64_t lines, int64_t k, const int16_t *D, int 
         for (int d = -(mod[i] / 2); 2 * d < mod[i]; ++d) {
             int dg[4] = {0, 0, 0, 0};
             ozo_split(d, mod[i], dg);
-            if (side == 0 && np == 3) dg[1] = -16 * dg[1];
+            if (np == 3) {
+                if (substrate == OZO_SUB_FP8) {
+                    if (side == 0) dg[1] = -16 * dg[1];
+                } else {
+                    if (side == 0) dg[0] = -dg[0];
+                    dg[1] = 4 * dg[1];
+                }
+            }
             for (int q = 0; q < np; ++q) {
-                int byte = ozo_e4m3_encode(dg[q]);
-                if (byte < 0) { bad = 1; byte = 0x7F; }
+                int byte;
+                if (substrate == OZO_SUB_FP8) {
+                    byte = ozo_e4m3_encode(dg[q]);
+                    if (byte < 0) { bad = 1; byte = 0x7F; }
+                } else {
+                    if (dg[q] < -128 || dg[q] > 127) bad = 1;
+                    byte = dg[q] & 0xFF;
+                }
                 code[d + 1024][q] = (uint8_t)byte;
             }
         }
@@ -708,15 +728,24 @@ int ozo_planes_merged(int side, int64_t lines, int64_t k, const int16_t *D, int 
     return bad ? -1 : plane;
 }
 
+int ozo_planes_merged(int side, int64_t lines, int64_t k, const int16_t *D, int set, uint8_t *P,
+                      int64_t plane_stride, int64_t row_pitch)
+{
+    return ozo_planes_merged_sub(side, lines, k, D, set, OZO_SUB_FP8, P, plane_stride, row_pitch);
+}
+
 /* residues from the merged layout: PA in the side-0 layout (-16*d1 in place of d1), PB plain */
-int64_t ozo_plane_products_merged(int64_t m, int64_t n, int64_t k, const uint8_t *PA,
-                                  int64_t strideA, int64_t pitchA, const uint8_t *PB,
-                                  int64_t strideB, int64_t pitchB, int set, uint16_t *R)
+int64_t ozo_plane_products_merged_sub(int64_t m, int64_t n, int64_t k, const uint8_t *PA,
+                                      int64_t strideA, int64_t pitchA, const uint8_t *PB,
+                                      int64_t strideB, int64_t pitchB, int set, int substrate,
+                                      uint16_t *R)
 {
     int mod[16], r = ozo_modset(set, mod), pa = 0, pb = 0;
     int64_t worst = 0;
     int digit_of[256];
-    for (int c = 0; c < 256; ++c) digit_of[c] = plane_digit((uint8_t)c, OZO_SUB_FP8);
+    /* weight of the merged accumulator: -15 [d0 e0 + (-16 d1) e1] on FP8, +15 [(-d0) e0 + (4 d1)(4 e1)] on INT8 */
+    const int w0 = substrate == OZO_SUB_FP8 ? -15 : 15;
+    for (int c = 0; c < 256; ++c) digit_of[c] = plane_digit((uint8_t)c, substrate);
     for (int i = 0; i < r; ++i) {
         int s = ozo_square_root(mod[i]);
         const int npa = ozo_planes_of_merged(mod[i], 0), npb = ozo_planes_of_merged(mod[i], 1);
@@ -735,14 +764,14 @@ int64_t ozo_plane_products_merged(int64_t m, int64_t n, int64_t k, const uint8_t
                         acc0 += (int64_t)a[0] * b[0];
                         acc1 += (int64_t)a[1] * b[0] + (int64_t)a[0] * b[1];
                     } else {
-                        acc0 += (int64_t)a[0] * b[0] + (int64_t)a[1] * b[1];   /* d0 e0 - 16 d1 e1 */
+                        acc0 += (int64_t)a[0] * b[0] + (int64_t)a[1] * b[1];   /* d0 e0 - 16 d1 e1 (INT8: its negative) */
                         acc1 += (int64_t)a[2] * b[2];                           /* (d0+d1)(e0+e1)   */
                     }
                 }
                 int64_t v0 = acc0 < 0 ? -acc0 : acc0, v1 = acc1 < 0 ? -acc1 : acc1;
                 if (v0 > worst_i) worst_i = v0;
                 if (v1 > worst_i) worst_i = v1;
-                int64_t t = s ? acc0 + (int64_t)s * acc1 : -15 * acc0 + 16 * acc1;
+                int64_t t = s ? acc0 + (int64_t)s * acc1 : w0 * acc0 + 16 * acc1;
                 int64_t c = t % mod[i];
                 if (c < 0) c += mod[i];
                 R[((int64_t)i * n + j) * m + ii] = (uint16_t)c;
@@ -752,6 +781,13 @@ int64_t ozo_plane_products_merged(int64_t m, int64_t n, int64_t k, const uint8_t
         pb += npb;
     }
     return worst;
+}
+
+int64_t ozo_plane_products_merged(int64_t m, int64_t n, int64_t k, const uint8_t *PA,
+                                  int64_t strideA, int64_t pitchA, const uint8_t *PB,
+                                  int64_t strideB, int64_t pitchB, int set, uint16_t *R)
+{
+    return ozo_plane_products_merged_sub(m, n, k, PA, strideA, pitchA, PB, strideB, pitchB, set, OZO_SUB_FP8, R);
 }
 
 /* ------------------------------------------------------------------ */

@@ -246,23 +246,27 @@ def pstore_merged(s: int, side: int) -> int:
     return lib().ozo_pstore_merged(s, side)
 
 
-def planes_merged(side: int, D: np.ndarray, s: int, row_pitch: int | None = None) -> np.ndarray:
-    """FP8 planes of the merged-accumulator layout (side 0 stores -16*d1 in place of d1)."""
+def planes_merged(side: int, D: np.ndarray, s: int, row_pitch: int | None = None,
+                  substrate: int = SUB_FP8) -> np.ndarray:
+    """Planes of the merged-accumulator layout.  FP8: side 0 stores -16*d1 in place of d1.
+    INT8: side 0 stores -d0, 4*d1, d0+d1 and side 1 stores d0, 4*d1, d0+d1."""
     r, lines, k = D.shape
     pitch = row_pitch if row_pitch is not None else (k + 15) // 16 * 16
     P = np.full((pstore_merged(s, side), lines, pitch), 0xAA, dtype=np.uint8)
-    rc = lib().ozo_planes_merged(side, _i64(lines), _i64(k), _p(np.ascontiguousarray(D)), s, _p(P),
-                                 _i64(lines * pitch), _i64(pitch))
-    assert rc == pstore_merged(s, side), "a digit was not representable in E4M3"
+    rc = lib().ozo_planes_merged_sub(side, _i64(lines), _i64(k), _p(np.ascontiguousarray(D)), s, substrate, _p(P),
+                                     _i64(lines * pitch), _i64(pitch))
+    assert rc == pstore_merged(s, side), "a digit was not representable on the substrate"
     return P
 
 
-def plane_products_merged(PA: np.ndarray, PB: np.ndarray, k: int, s: int):
+def plane_products_merged(PA: np.ndarray, PB: np.ndarray, k: int, s: int, substrate: int = SUB_FP8):
     _, m, pa = PA.shape
     _, n, pb = PB.shape
     R = np.zeros((len(modset(s)), n, m), dtype=np.uint16)
-    worst = lib().ozo_plane_products_merged(_i64(m), _i64(n), _i64(k), _p(PA), _i64(m * pa), _i64(pa),
-                                            _p(PB), _i64(n * pb), _i64(pb), s, _p(R))
+    f = lib().ozo_plane_products_merged_sub
+    f.restype = C.c_int64
+    worst = f(_i64(m), _i64(n), _i64(k), _p(PA), _i64(m * pa), _i64(pa), _p(PB), _i64(n * pb), _i64(pb), s,
+              substrate, _p(R))
     return R, int(worst)
 
 

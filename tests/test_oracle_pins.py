@@ -223,6 +223,50 @@ def test_merged_accumulator_layout(name):
     assert (R == ozo.products(DA, DB, SETS[name])).all() and w <= 4095 * k
 
 
+@pytest.mark.parametrize("name", ["S", "E", "A"])
+def test_merged_accumulator_layout_on_int8(name):
+    """The N_acc = 2 regrouping on the INT8 substrate: d e = 15 [(-d0) e0 + (4 d1)(4 e1)] + 16 dS eS.
+    The identity holds for every pair of residues of every non-square modulus, every stored value
+    fits a signed byte, the merged term is at most 196 + 16 * 256, and the planes reproduce the
+    residue products."""
+    ms = ozo.modset(SETS[name])
+    nonsq = [m for m in ms if math.isqrt(m) ** 2 != m]
+    worst = 0
+    for m in nonsq:
+        lo, hi = -(m // 2), (m - 1) // 2
+        sp = {d: ozo.split(d, m) for d in range(lo, hi + 1)}
+        assert all(-128 <= -d0 <= 127 and -128 <= 4 * d1 <= 127 and -128 <= ds <= 127 for (d0, d1, ds) in sp.values())
+        probe = list(sp.items())[:: max(1, len(sp) // 61)] + [(lo, sp[lo]), (hi, sp[hi])]
+        for d, (d0, d1, ds) in sp.items():
+            for e, (e0, e1, es) in probe:
+                merged = (-d0) * e0 + (4 * d1) * (4 * e1)
+                assert (15 * merged + 16 * ds * es - d * e) % m == 0
+                worst = max(worst, abs(merged))
+    assert worst <= 196 + 16 * 256 == 4292
+    rng = np.random.default_rng(33)
+    m_, n_, k = 5, 4, 41
+    QA = rng.integers(-2**50, 2**50, size=(m_, k))
+    QB = rng.integers(-2**50, 2**50, size=(n_, k))
+    DA, DB = ozo.residues(QA, SETS[name]), ozo.residues(QB, SETS[name])
+    PA = ozo.planes_merged(0, DA, SETS[name], substrate=ozo.SUB_INT8)
+    PB = ozo.planes_merged(1, DB, SETS[name], substrate=ozo.SUB_INT8)
+    plainA, plainB, p0 = ozo.planes(DA, SETS[name], ozo.SUB_INT8), ozo.planes(DB, SETS[name], ozo.SUB_INT8), 0
+    for mm in ms:
+        if math.isqrt(mm) ** 2 == mm:
+            assert (PA[p0:p0 + 2] == plainA[p0:p0 + 2]).all() and (PB[p0:p0 + 2] == plainB[p0:p0 + 2]).all()
+            p0 += 2
+            continue
+        d0, d1 = plainA[p0].view(np.int8).astype(int), plainA[p0 + 1].view(np.int8).astype(int)
+        assert (PA[p0].view(np.int8) == -d0).all() and (PA[p0 + 1].view(np.int8) == 4 * d1).all()
+        assert (PA[p0 + 2] == plainA[p0 + 2]).all()
+        e1 = plainB[p0 + 1].view(np.int8).astype(int)
+        assert (PB[p0] == plainB[p0]).all() and (PB[p0 + 1].view(np.int8) == 4 * e1).all()
+        assert (PB[p0 + 2] == plainB[p0 + 2]).all()
+        p0 += 3
+    R, w = ozo.plane_products_merged(PA, PB, k, SETS[name], ozo.SUB_INT8)
+    assert (R == ozo.products(DA, DB, SETS[name])).all() and w <= 4292 * k
+
+
 def test_lemma1_is_sharp_at_513():
     def rule(d):
         d0 = (d + 8) % 16 - 8
