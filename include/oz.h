@@ -90,17 +90,22 @@ typedef enum { OZ_SET_S = 0, OZ_SET_E = 1, OZ_SET_A = 2 } oz_modset_t;
                                   * CRT range.  Whole-method calls only (the shifts of one operand depend on
                                   * the other): oz_dgemm, oz_dgemm_ex, oz_dgemm_host; k <= 16384.            */
 
-/* Accumulator schedule of the residue GEMMs for non-square moduli on the FP8 substrate.
+/* Accumulator schedule of the residue GEMMs for non-square moduli on the two digit substrates.
  * MERGED: two accumulators per modulus, d e = -15 [d0 e0 + (-16 d1) e1] + 16 (d0+d1)(e0+e1)
- * (discussion of Table "tuples", N_acc = 2).  The A operand then stores the pre-scaled -16*d1 in
- * the place of d1 (plane order d0, -16*d1, d0+d1; d1 enters only through d1 e1), B is unchanged,
- * and the plane counts stay those of the table.  One merged accumulator is exact while its term
- * stays below 2^24: k <= 4097 for set S, k <= 15420 for sets E and A.  A longer k is cut into equal
- * K segments no longer than that, each with an accumulator of its own that is reduced modulo m_i
- * before the segments are added (split-K inside the kernel; the residues are the same).
+ * (discussion of Table "tuples", N_acc = 2).  The plane counts stay those of the table.
+ *   FP8:  the A operand stores the pre-scaled -16*d1 in the place of d1 (plane order d0, -16*d1,
+ *         d0+d1; d1 enters only through d1 e1), B is unchanged.  One merged accumulator is exact
+ *         while it stays below 2^24: k <= 4097 for set S, k <= 15420 for sets E and A.
+ *   INT8: -16*d1 does not fit a byte, so the factor is shared: A stores -d0, 4*d1, d0+d1 and B stores
+ *         e0, 4*e1, e0+e1; the accumulator (-d0) e0 + (4 d1)(4 e1) is the negative of the bracket and
+ *         takes the weight +15.  Its term is at most 4292, exact in INT32 for k <= 500 000.
+ * A longer k is cut into equal K segments no longer than that, each with an accumulator of its own
+ * that is reduced modulo m_i before the segments are added (split-K inside the kernel; the residues
+ * are the same).
  * SEPARATE: the three accumulators of Eq. 8.  With neither bit, oz_dgemm / oz_dgemm_ex /
- * oz_dgemm_host pick MERGED on the FP8 substrate (their planes are internal), and the stage entry
- * points use SEPARATE.  Planes of A written with MERGED must be multiplied with MERGED. */
+ * oz_dgemm_host pick MERGED on the digit substrates (their planes are internal), and the stage entry
+ * points use SEPARATE.  Planes written with MERGED must be multiplied with MERGED.  Not defined for
+ * OZ_SUB_INT8_NATIVE (one plane per modulus). */
 #define OZ_ACC_MERGED   0x1000u
 #define OZ_ACC_SEPARATE 0x2000u
 
@@ -124,7 +129,7 @@ oz_status_t oz_set_info(oz_modset_t set, int *r, int *p_store, int *moduli);
 int oz_plane_count(oz_modset_t set, uint32_t route);
 
 /* Same, for the operand on `side` (0: A, 1: B).  The counts of the two sides are equal on every
- * route (with OZ_ACC_MERGED the pre-scaled plane takes the place of d1 on A); the function remains
+ * route (with OZ_ACC_MERGED the re-scaled planes take the places of the plain ones); the function remains
  * for callers that size the two plane arrays separately. */
 int oz_plane_count_side(oz_modset_t set, uint32_t route, int side);
 

@@ -90,9 +90,10 @@ uint32_t lut_entry(int u, int m, int substrate)
         else byte = dig[q] & 0xFF;
         word |= static_cast<uint32_t>(byte) << (8 * q);
     }
-    if (substrate == 0 && !s) {              // byte 3: the pre-scaled plane -16*d1 of the merged schedule
+    if (!s) {                                // byte 3: what the merged schedule swaps in
         int byte = 0;
-        e4m3_code(-16 * dig[1], &byte);
+        if (substrate == 0) e4m3_code(-16 * dig[1], &byte);   // FP8: the pre-scaled plane -16*d1
+        else byte = (-dig[0]) & 0xFF;                          // INT8: -d0 (4*d1 is a shift of byte 1)
         word |= static_cast<uint32_t>(byte) << 24;
     }
     return word;
@@ -142,19 +143,19 @@ bool decode_route(uint32_t route, Route *out)
 bool decode_route_for_set(int set, uint32_t route, Route *out)
 {
     if (!decode_route(route, out)) return false;
-    if (out->merged() && out->substrate != 0) return false;   // -16*d1 reaches -256: FP8 planes only
+    if (out->merged() && out->native()) return false;         // one plane per modulus: nothing to merge
     return !(out->native() && set != OZ_SET_A);
 }
 
 // Fixes the accumulator schedule of a call.  `automatic`: the whole-method entry points, whose
-// planes are internal, take the merged schedule on the FP8 substrate (one accumulator drain fewer per
-// non-square modulus at no extra plane; the GEMM cuts a long k into segments that each stay exact);
+// planes are internal, take the merged schedule on the digit substrates (one accumulator drain fewer
+// per non-square modulus at no extra plane; the GEMM cuts a long k into segments that each stay exact);
 // the stage entry points default to separate accumulators because what their d1 plane holds is part
 // of the interface.
 oz_status_t resolve_schedule(int set, int64_t k, int64_t n, bool automatic, Route *rt)
 {
     if (rt->acc == 0)
-        rt->acc = (automatic && rt->substrate == 0 && k > 0) ? 1 : 2;
+        rt->acc = (automatic && !rt->native() && k > 0) ? 1 : 2;
     return OZ_OK;
 }
 

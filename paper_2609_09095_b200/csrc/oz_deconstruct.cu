@@ -373,18 +373,25 @@ __device__ __forceinline__ void convert_modulus(const uint32_t (&l0)[4], const u
     }
     uint32_t t01 = __byte_perm(w[0], w[1], 0x5140);
     uint32_t t23 = __byte_perm(w[2], w[3], 0x5140);
-    *reinterpret_cast<uint32_t *>(out + plane * plane_stride) = __byte_perm(t01, t23, 0x5410);
-    if (LAYOUT == kLayoutNative) return;      // one plane: the centred residue itself
+    const uint32_t first = __byte_perm(t01, t23, 0x5410), second = __byte_perm(t01, t23, 0x7632);
+    if (LAYOUT == kLayoutNative) {            // one plane: the centred residue itself
+        *reinterpret_cast<uint32_t *>(out + plane * plane_stride) = first;
+        return;
+    }
     if (planes_of(m) == 3) {
-        // bytes 2 and 3 of the table words: d0+d1 and the pre-scaled -16*d1, which takes the
-        // place of d1 in the merged layout
+        // bytes 2 and 3 of the table words: d0+d1 and the byte the merged layouts swap in
+        // (FP8: the pre-scaled -16*d1 for d1; INT8: -d0 for d0, with 4*d1 made by a byte-wise shift)
         uint32_t u01 = __byte_perm(w[0], w[1], 0x7362);
         uint32_t u23 = __byte_perm(w[2], w[3], 0x7362);
+        const uint32_t extra = __byte_perm(u01, u23, 0x7632);
+        constexpr bool kI8 = LAYOUT == kLayoutMergedI8A || LAYOUT == kLayoutMergedI8B;
+        *reinterpret_cast<uint32_t *>(out + plane * plane_stride) = LAYOUT == kLayoutMergedI8A ? extra : first;
         *reinterpret_cast<uint32_t *>(out + (plane + 1) * plane_stride) =
-            LAYOUT == kLayoutMerged ? __byte_perm(u01, u23, 0x7632) : __byte_perm(t01, t23, 0x7632);
+            LAYOUT == kLayoutMerged ? extra : (kI8 ? ((second << 2) & 0xFCFCFCFCu) : second);
         *reinterpret_cast<uint32_t *>(out + (plane + 2) * plane_stride) = __byte_perm(u01, u23, 0x5410);
     } else {
-        *reinterpret_cast<uint32_t *>(out + (plane + 1) * plane_stride) = __byte_perm(t01, t23, 0x7632);
+        *reinterpret_cast<uint32_t *>(out + plane * plane_stride) = first;
+        *reinterpret_cast<uint32_t *>(out + (plane + 1) * plane_stride) = second;
     }
 }
 
@@ -862,8 +869,11 @@ oz_status_t launch_convert_planes(int side, int64_t lines, int64_t k, const doub
     launch_convert<SET_, SIDE_, LAYOUT_>(X, ldx, lines, k, shift, lut, planes, plane_stride, row_pitch, \
                                          rt.quant, stream)
 #define OZ_CONVERT_SET(SET_)                                                                             \
-    (side == 1 ? OZ_CONVERT(SET_, 1, kLayoutDigits)                                                      \
-               : (layout == kLayoutMerged ? OZ_CONVERT(SET_, 0, kLayoutMerged) : OZ_CONVERT(SET_, 0, kLayoutDigits)))
+    (side == 1 ? (layout == kLayoutMergedI8B ? OZ_CONVERT(SET_, 1, kLayoutMergedI8B)                    \
+                                             : OZ_CONVERT(SET_, 1, kLayoutDigits))                      \
+               : (layout == kLayoutMerged      ? OZ_CONVERT(SET_, 0, kLayoutMerged)                     \
+                  : layout == kLayoutMergedI8A ? OZ_CONVERT(SET_, 0, kLayoutMergedI8A)                  \
+                                               : OZ_CONVERT(SET_, 0, kLayoutDigits)))
     const int layout = rt.layout(side);
     if (layout == kLayoutNative) return side == 0 ? OZ_CONVERT(2, 0, kLayoutNative) : OZ_CONVERT(2, 1, kLayoutNative);
     if (set == 0) return OZ_CONVERT_SET(0);
@@ -903,8 +913,11 @@ oz_status_t launch_deconstruct(int side, int64_t lines, int64_t k, const double 
         const int layout = rt.layout(side);
 #define OZ_FUSED(SET_, SIDE_, LAYOUT_) launch_fused<SET_, SIDE_, LAYOUT_>(p, f, stream)
 #define OZ_FUSED_SET(SET_)                                                                      \
-    (side == 1 ? OZ_FUSED(SET_, 1, kLayoutDigits)                                               \
-               : (layout == kLayoutMerged ? OZ_FUSED(SET_, 0, kLayoutMerged) : OZ_FUSED(SET_, 0, kLayoutDigits)))
+    (side == 1 ? (layout == kLayoutMergedI8B ? OZ_FUSED(SET_, 1, kLayoutMergedI8B)             \
+                                             : OZ_FUSED(SET_, 1, kLayoutDigits))               \
+               : (layout == kLayoutMerged      ? OZ_FUSED(SET_, 0, kLayoutMerged)              \
+                  : layout == kLayoutMergedI8A ? OZ_FUSED(SET_, 0, kLayoutMergedI8A)           \
+                                               : OZ_FUSED(SET_, 0, kLayoutDigits)))
         if (layout == kLayoutNative) return side == 0 ? OZ_FUSED(2, 0, kLayoutNative) : OZ_FUSED(2, 1, kLayoutNative);
         if (set == 0) return OZ_FUSED_SET(0);
         if (set == 1) return OZ_FUSED_SET(1);

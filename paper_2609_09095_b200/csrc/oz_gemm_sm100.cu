@@ -1043,14 +1043,17 @@ oz_status_t launch_residue_gemm(int64_t m, int64_t n, int64_t k, const uint8_t *
             mo.reduce[1] = skip_all ? 0 : 1;
             mo.reduce[2] = 1;
         } else if (rt.merged()) {
-            // d e = -15 [d0 e0 - 16 d1 e1] + 16 dS eS; merged term <= 4095 (9-bit tail) or 1088 (bytes)
+            // d e = -15 [d0 e0 - 16 d1 e1] + 16 dS eS; merged term <= 4095 (9-bit tail) or 1088 (bytes).
+            // INT8 planes hold -d0 and 4*d1, so the accumulator is the NEGATIVE of the bracket (weight
+            // +15) and its term is bounded by 4292 for every modulus up to 1089.
             mo.njobs = 2;
             mo.kind = 3;
-            mo.w[0] = -15.0f; mo.w[1] = 16.0f; mo.w[2] = 0.0f;
+            mo.w[0] = integer ? 15.0f : -15.0f; mo.w[1] = 16.0f; mo.w[2] = 0.0f;
             // K longer than the exact range of one merged accumulator is cut into equal segments,
             // each drained and reduced on its own (the residues add modulo m).
-            const int64_t merged_term = mi > 256 ? 4095 : 1088;
-            const int seg_max = static_cast<int>(merged_k_limit(set) / BLOCK_K);
+            const int64_t merged_term = integer ? 4292 : (mi > 256 ? 4095 : 1088);
+            const int seg_max = integer ? static_cast<int>(((1ll << 31) - 1) / merged_term / BLOCK_K)
+                                        : static_cast<int>(merged_k_limit(set) / BLOCK_K);
             mo.nseg = (p.nk + seg_max - 1) / seg_max;
             if (mo.nseg < 1) mo.nseg = 1;
             mo.seg_len = (p.nk + mo.nseg - 1) / mo.nseg;

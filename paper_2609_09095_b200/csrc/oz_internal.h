@@ -45,7 +45,11 @@ __host__ __device__ constexpr int square_root(int m)
 //   kLayoutMerged  the A operand of the merged-accumulator schedule (discussion of Table "tuples",
 //                  N_acc = 2): the d1 plane of every non-square modulus holds the pre-scaled -16*d1
 //                  (d1 enters only through d1*e1); same plane count as kLayoutDigits
-constexpr int kLayoutDigits = 0, kLayoutNative = 1, kLayoutMerged = 2;
+//   kLayoutMergedI8A / kLayoutMergedI8B  the same schedule on INT8 digit planes, where -16*d1 does
+//                  not fit a byte: both operands carry 4*d1 in place of d1 and the A operand -d0
+//                  in place of d0, so that (-d0) e0 + (4 d1)(4 e1) = -(d0 e0 - 16 d1 e1)
+constexpr int kLayoutDigits = 0, kLayoutNative = 1, kLayoutMerged = 2, kLayoutMergedI8A = 3,
+              kLayoutMergedI8B = 4;
 
 __host__ __device__ constexpr int planes_of(int m, int layout = kLayoutDigits)
 {
@@ -111,7 +115,10 @@ struct Route {
     // plane layout of the operand on `side` (0: rows of A, 1: columns of B)
     int layout(int side) const
     {
-        return native() ? kLayoutNative : ((merged() && side == 0) ? kLayoutMerged : kLayoutDigits);
+        if (native()) return kLayoutNative;
+        if (!merged()) return kLayoutDigits;
+        if (substrate == 1) return side == 0 ? kLayoutMergedI8A : kLayoutMergedI8B;
+        return side == 0 ? kLayoutMerged : kLayoutDigits;
     }
     bool hosted;    // whole-method calls: CRT recombination on the INT8 tensor pipe (OZ_RECON_TENSOR)
     int quant;      // 0 rn, 1 tz

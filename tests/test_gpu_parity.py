@@ -51,20 +51,23 @@ def test_deconstruct_bit_exact(side, lines, k, dist, set_name, sub, quant, rule)
     assert P.shape == Po.shape and (P == Po).all()
 
 
+@pytest.mark.parametrize("sub", ["fp8", "int8"])
 @pytest.mark.parametrize("set_name,lines,k", [("S", 130, 1000), ("E", 67, 4101), ("A", 37, 129), ("S", 5, 4097)])
-def test_merged_schedule_stages_bit_exact(set_name, lines, k):
-    """Merged accumulators: the A operand carries the pre-scaled -16*d1 planes, B is unchanged, and
-    the two-accumulator GEMM gives the same residues."""
+def test_merged_schedule_stages_bit_exact(set_name, lines, k, sub):
+    """Merged accumulators.  FP8: the A operand carries the pre-scaled -16*d1 planes and B is unchanged.
+    INT8: A carries -d0 and 4*d1, B carries 4*e1.  The two-accumulator GEMM gives the same residues."""
     import tests.gpu_helpers as gh
     rng = np.random.default_rng(lines + k)
     A = syn._draw(rng, lines, k, "lognormal:0.5")
     B = syn._draw(rng, k, 150, "normal")
-    rt = gh.route("fp8", "RN", "CS", acc="merged")
+    rt = gh.route(sub, "RN", "CS", acc="merged")
+    osub = OSUB[sub]
     PA, shA, st = gh.deconstruct(0, A, set_name, rt)
     PB, shB, st2 = gh.deconstruct(1, B, set_name, rt)
-    _, shAo, DA = _oracle_deconstruct(0, A, set_name, "fp8", "RN", "CS")
-    _, shBo, DB = _oracle_deconstruct(1, B, set_name, "fp8", "RN", "CS")
-    PAo, PBo = ozo.planes_merged(0, DA, OSET[set_name]), ozo.planes_merged(1, DB, OSET[set_name])
+    _, shAo, DA = _oracle_deconstruct(0, A, set_name, sub, "RN", "CS")
+    _, shBo, DB = _oracle_deconstruct(1, B, set_name, sub, "RN", "CS")
+    PAo = ozo.planes_merged(0, DA, OSET[set_name], substrate=osub)
+    PBo = ozo.planes_merged(1, DB, OSET[set_name], substrate=osub)
     assert st == 0 and st2 == 0 and (shA == shAo).all() and (shB == shBo).all()
     assert PA.shape == PAo.shape and (PA == PAo).all() and (PB == PBo).all()
     R, st3 = gh.residue_gemm(PA, PB, k, set_name, rt)
@@ -75,11 +78,44 @@ def test_merged_schedule_limits():
     import torch
     import paper_2609_09095_b200 as oz
     import tests.gpu_helpers as gh
-    # the pre-scaled plane takes the place of d1: counts as in the paper's table
+    # the re-scaled planes take the places of the plain ones: counts as in the paper's table
     assert oz.oz_plane_count_side(oz.OZ_SET_S, oz.OZ_ACC_MERGED, 0) == 30
     assert oz.oz_plane_count_side(oz.OZ_SET_S, oz.OZ_ACC_MERGED, 1) == 30
     assert oz.oz_plane_count_side(oz.OZ_SET_E, oz.OZ_ACC_MERGED, 0) == 33
-    assert oz.oz_plane_count_side(oz.OZ_SET_S, oz.OZ_ACC_MERGED | oz.OZ_SUB_INT8, 0) == 0   # FP8 planes only
+    assert oz.oz_plane_count_side(oz.OZ_SET_S, oz.OZ_ACC_MERGED | oz.OZ_SUB_INT8, 0) == 30
+    assert oz.oz_plane_count_side(oz.OZ_SET_S, oz.OZ_ACC_MERGED | oz.OZ_SUB_INT8, 1) == 30
+    # one plane per modulus leaves nothing to merge
+    assert oz.oz_plane_count_side(oz.OZ_SET_A, oz.OZ_ACC_MERGED | oz.OZ_SUB_INT8_NATIVE, 0) == 0
+
+
+@pytest.mark.parametrize("set_name,k", [("S", 1100), ("S", 29700), ("S", 29900), ("E", 33000)])
+def test_merged_schedule_on_int8_with_extreme_digits(set_name, k):
+    """INT8 merged schedule at the edges of its host-side range checks: the largest residues everywhere
+    (term 4292 on the 1089 modulus), k on either side of 29 774, where 15 * 4292 k + 16 * 484 k leaves
+    INT32 and the accumulators are reduced before they are weighted, and past the FP32 depth."""
+    import tests.gpu_helpers as gh
+    rng = np.random.default_rng(k)
+    m, n = 70, 140
+    _, DA = _random_planes(rng, set_name, "int8", m, k, extreme=True)
+    _, DB = _random_planes(rng, set_name, "int8", n, k, extreme=True)
+    top = 0
+    for i, mod in enumerate(ozo.modset(OSET[set_name])):
+        if len(ozo.split(0, mod)) == 2:      # square modulus: no merged accumulator
+            continue
+        # the residue whose own square gives the largest merged term 16 d1^2 - d0^2
+        term = lambda d: 16 * ozo.split(d, mod)[1] ** 2 - ozo.split(d, mod)[0] ** 2
+        d = max(range(-(mod // 2), (mod - 1) // 2 + 1), key=term)
+        top = max(top, term(d))
+        DA[i, :8, :] = DB[i, :8, :] = d
+        if -(mod // 2) <= -d <= (mod - 1) // 2:
+            DA[i, 8:16, :] = -d
+    assert top > (4000 if set_name == "S" else 900)       # 9-bit tail of S; byte moduli
+    PA = ozo.planes_merged(0, DA, OSET[set_name], substrate=ozo.SUB_INT8)
+    PB = ozo.planes_merged(1, DB, OSET[set_name], substrate=ozo.SUB_INT8)
+    want, worst = ozo.plane_products_merged(PA, PB, k, OSET[set_name], substrate=ozo.SUB_INT8)
+    assert (want == ozo.products(DA, DB, OSET[set_name])).all() and worst >= top * k
+    R, st = gh.residue_gemm(PA, PB, k, set_name, gh.route("int8", acc="merged"))
+    assert st == 0 and (R == want).all()
 
 
 @pytest.mark.parametrize("set_name,k", [("S", 4224), ("S", 8321), ("S", 12289), ("E", 16640), ("A", 16640)])
