@@ -81,6 +81,41 @@ def esc_threshold(ms):
     return min(2 ** 32 - 1, (2 ** 120 // 3) // (((product(ms) - 1) // 2) >> 20))
 
 
+def esc_rows(A, B, ms):
+    """Rows of the product that go to the native FP64 path: q(a_i) against the least flat column of B,
+    both capped at 2^16, below the set's threshold.  A: m x k, B: k x n nested lists."""
+    k, n = len(B), len(B[0])
+    qb = [esc_flatness([B[kk][j] for kk in range(k)], k) for j in range(n)]
+    qb = min([min(q, 2 ** 16) for q in qb if q is not None], default=2 ** 16)
+    out = []
+    for row in A:
+        qa = esc_flatness(row, k)
+        out.append(0 if qa is None else int(min(qa, 2 ** 16) * qb < esc_threshold(ms)))
+    return out
+
+
+def _rn(x: Fraction) -> float:
+    return float(x)          # exact rational -> nearest double, ties to even
+
+
+def native_dot(a, b) -> float:
+    """The compensated inner product of the native path, every floating-point operation written as
+    the correctly rounded value of its exact rational result (finite data, no overflow)."""
+    acc, comp = 0.0, 0.0
+    for x, y in zip(a, b):
+        fx, fy = Fraction(x), Fraction(y)
+        p = _rn(fx * fy)
+        pe = _rn(fx * fy - Fraction(p))
+        s = _rn(Fraction(acc) + Fraction(p))
+        bb = _rn(Fraction(s) - Fraction(acc))
+        t1 = _rn(Fraction(acc) - Fraction(_rn(Fraction(s) - Fraction(bb))))
+        t2 = _rn(Fraction(p) - Fraction(bb))
+        se = _rn(Fraction(t1) + Fraction(t2))
+        comp = _rn(Fraction(comp) + Fraction(_rn(Fraction(pe) + Fraction(se))))
+        acc = s
+    return _rn(Fraction(acc) + Fraction(comp))
+
+
 def bound_digit(x: float, E: int) -> int:
     """Accurate mode: the smallest E4M3-representable integer that is >= |x| 2^(4-E)."""
     if x == 0:

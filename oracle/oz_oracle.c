@@ -19,11 +19,13 @@
  * big-integer restatement -- except the accuracy of the method against the true
  * product on inputs with a very wide exponent spread, for which the paper prints
  * no bound: "parity unpinned" for that one quantity (it is measured, not asserted).
- * Two passages name a step and leave its content to the paper's sources: the extra
- * bound product of the accurate mode and the "ESC check".  The readings taken are
- * stated above ozo_bound_digit and ozo_esc_threshold; their arithmetic is pinned
- * (soundness by brute force, closed forms, the big-integer restatement), the
- * threshold of the ESC reading is a heuristic: "parity unpinned" for that value.
+ * Three passages name a step and leave its content to the paper's sources: the extra
+ * bound product of the accurate mode, the "ESC check" and the native-FP64 path for
+ * out-of-range rows.  The readings taken are stated above ozo_bound_digit,
+ * ozo_esc_threshold and ozo_esc_rows; their arithmetic is pinned (soundness by brute
+ * force, closed forms, the big-integer restatement, the error bound of the compensated
+ * dot product), the threshold of the ESC reading is a heuristic: "parity unpinned" for
+ * that value.
  *
  * Storage conventions (column-major BLAS shapes, Sec. 2: C = AB, A m x k, B k x n):
  *   side 0: X is m x k, "line" i is row i,    element (i,kk) at X[i + kk*ldx]
@@ -259,33 +261,39 @@ uint32_t ozo_esc_threshold(int set)
     return t > 0xFFFFFFFFu ? 0xFFFFFFFFu : (uint32_t)t;
 }
 
+/* q of one line; 0xFFFFFFFF for a line that does not count (zeros only, or Inf/NaN) */
+static uint32_t line_flatness(int side, int64_t l, int64_t k, const double *X, int64_t ldx)
+{
+    int any = 0, bad = 0, E = 0;
+    for (int64_t kk = 0; kk < k; ++kk) {
+        fp_parts p = decode(*elem(X, ldx, side, l, kk));
+        if (p.kind == 2) bad = 1;
+        if (p.kind == 1) { if (!any || p.e > E) E = p.e; any = 1; }
+    }
+    if (bad || !any) return 0xFFFFFFFFu;
+    u128 S = 0, L1 = 0;
+    for (int64_t kk = 0; kk < k; ++kk) {
+        fp_parts p = decode(*elem(X, ldx, side, l, kk));
+        if (p.kind != 1) continue;
+        int sh = 43 + E - p.ex;
+        uint64_t abar;
+        if (sh >= 64) abar = 1;
+        else if (sh <= 0) abar = p.sig << (-sh);
+        else abar = (p.sig >> sh) + ((p.sig & ((1ull << sh) - 1)) ? 1 : 0);
+        S += (u128)abar * abar;
+        L1 += abar;
+    }
+    return (uint32_t)(((L1 * L1) << 16) / ((u128)k * S));
+}
+
 /* smallest q over the lines of one operand (0xFFFFFFFF when no line counts) */
 uint32_t ozo_esc_flatness(int side, int64_t lines, int64_t k, const double *X, int64_t ldx)
 {
     uint32_t best = 0xFFFFFFFFu;
 #pragma omp parallel for schedule(static) reduction(min : best)
     for (int64_t l = 0; l < lines; ++l) {
-        int any = 0, bad = 0, E = 0;
-        for (int64_t kk = 0; kk < k; ++kk) {
-            fp_parts p = decode(*elem(X, ldx, side, l, kk));
-            if (p.kind == 2) bad = 1;
-            if (p.kind == 1) { if (!any || p.e > E) E = p.e; any = 1; }
-        }
-        if (bad || !any) continue;
-        u128 S = 0, L1 = 0;
-        for (int64_t kk = 0; kk < k; ++kk) {
-            fp_parts p = decode(*elem(X, ldx, side, l, kk));
-            if (p.kind != 1) continue;
-            int sh = 43 + E - p.ex;
-            uint64_t abar;
-            if (sh >= 64) abar = 1;
-            else if (sh <= 0) abar = p.sig << (-sh);
-            else abar = (p.sig >> sh) + ((p.sig & ((1ull << sh) - 1)) ? 1 : 0);
-            S += (u128)abar * abar;
-            L1 += abar;
-        }
-        u128 q = ((L1 * L1) << 16) / ((u128)k * S);
-        if (q < best) best = (uint32_t)q;
+        uint32_t q = line_flatness(side, l, k, X, ldx);
+        if (q < best) best = q;
     }
     return best;
 }
@@ -910,6 +918,68 @@ void ozo_output(int64_t m, int64_t n, const int64_t *CI, const int32_t *shiftA,
 }
 
 /* ------------------------------------------------------------------ */
+/* Out-of-range rows on the native FP64 path (Algorithm 1, last line:   */
+/* "native-FP64 fallback for out-of-range rows"; Algorithm 3: "re-issue */
+/* out-of-range rows on the native-FP64 path") -- a reading: the paper  */
+/* names the step and leaves both the criterion and the arithmetic open */
+/* ------------------------------------------------------------------ */
+/* Row i of the product is out of range when the exponent-span check fails for it against the
+ * least flat column of B:  min(q(a_i), 2^16) * min(min_j q(b_j), 2^16) < thr  (same q and thr as
+ * ozo_esc_check; rows of zeros and rows with Inf/NaN are never re-issued).  flag[i] = 1 for such
+ * rows; returns their number. */
+int64_t ozo_esc_rows(int64_t m, int64_t n, int64_t k, const double *A, int64_t lda, const double *B,
+                     int64_t ldb, int set, uint8_t *flag)
+{
+    uint32_t qb = ozo_esc_flatness(1, n, k, B, ldb);
+    if (qb > 65536u) qb = 65536u;
+    const uint64_t thr = ozo_esc_threshold(set);
+    int64_t count = 0;
+    for (int64_t i = 0; i < m; ++i) {
+        uint32_t qa = line_flatness(0, i, k, A, lda);
+        flag[i] = 0;
+        if (qa == 0xFFFFFFFFu) continue;
+        if (qa > 65536u) qa = 65536u;
+        if ((uint64_t)qa * qb < thr) { flag[i] = 1; ++count; }
+    }
+    return count;
+}
+
+/* The native path: FP64 arithmetic only, the inner product taken in the order kk = 0 .. k-1 with the
+ * rounding error of every product (one fused multiply-add) and of every addition (the error-free
+ * sum of two doubles) collected in a second double that is added at the end -- the classical
+ * compensated dot product, whose result is as good as if computed in twice the working precision
+ * and then rounded, so that the re-issued rows meet the same 2u (|A||B|) contract as the others.
+ * Columns of B with Inf/NaN give NaN as everywhere else.  C(i,:) is updated for flagged rows only. */
+void ozo_native_rows(int64_t m, int64_t n, int64_t k, const double *A, int64_t lda, const double *B,
+                     int64_t ldb, const uint8_t *flag, double alpha, double beta, double *C, int64_t ldc)
+{
+#pragma omp parallel for schedule(static)
+    for (int64_t j = 0; j < n; ++j) {
+        int bad = 0;
+        for (int64_t kk = 0; kk < k; ++kk)
+            if (decode(B[kk + j * ldb]).kind == 2) bad = 1;
+        for (int64_t i = 0; i < m; ++i) {
+            if (!flag[i]) continue;
+            double acc = 0.0, comp = 0.0;
+            for (int64_t kk = 0; kk < k; ++kk) {
+                double a = A[i + kk * lda], b = B[kk + j * ldb];
+                double p = a * b;
+                double pe = fma(a, b, -p);                  /* a b = p + pe */
+                double s = acc + p;
+                double bb = s - acc;
+                double se = (acc - (s - bb)) + (p - bb);    /* acc + p = s + se */
+                comp = comp + (pe + se);
+                acc = s;
+            }
+            double v = bad ? NAN : acc + comp;
+            double *c = &C[i + j * ldc];
+            if (beta == 0.0) *c = alpha * v;
+            else *c = beta * (*c) + alpha * v;
+        }
+    }
+}
+
+/* ------------------------------------------------------------------ */
 /* Second reference: double-double GEMM (error-free products and sums)  */
 /* ------------------------------------------------------------------ */
 static void dd_add_prod(double *hi, double *lo, double a, double b)
@@ -980,6 +1050,31 @@ int ozo_dgemm(int64_t m, int64_t n, int64_t k, const double *A, int64_t lda, con
     if (R_out) memcpy(R_out, R, sizeof(uint16_t) * r * m * n);
     free(sA); free(sB); free(QA); free(QB); free(DA); free(DB); free(R); free(CI);
     return 0;
+}
+
+/* The whole method with the out-of-range rows re-issued on the native path: the flagged rows of C
+ * come from ozo_native_rows (applied to the caller's old C), all others from the method.  Norm-based
+ * scale rule only (the check is defined on its scan).  Returns the number of re-issued rows, or -1. */
+int64_t ozo_dgemm_fallback(int64_t m, int64_t n, int64_t k, const double *A, int64_t lda,
+                           const double *B, int64_t ldb, double *C, int64_t ldc, int set, int quant,
+                           double alpha, double beta, uint8_t *flag_out)
+{
+    if (m <= 0 || n <= 0 || k <= 0) return ozo_dgemm(m, n, k, A, lda, B, ldb, C, ldc, set, quant, OZO_SCALE_CS, alpha, beta, NULL, NULL, NULL);
+    uint8_t *flag = malloc((size_t)m);
+    double *old = malloc(sizeof(double) * (size_t)m * (size_t)n);
+    if (!flag || !old) return -1;
+    for (int64_t j = 0; j < n; ++j)
+        for (int64_t i = 0; i < m; ++i) old[i + j * m] = C[i + j * ldc];
+    int64_t count = ozo_esc_rows(m, n, k, A, lda, B, ldb, set, flag);
+    if (ozo_dgemm(m, n, k, A, lda, B, ldb, C, ldc, set, quant, OZO_SCALE_CS, alpha, beta, NULL, NULL, NULL)) return -1;
+    /* the flagged rows start again from the old values */
+    for (int64_t j = 0; j < n; ++j)
+        for (int64_t i = 0; i < m; ++i)
+            if (flag[i]) C[i + j * ldc] = old[i + j * m];
+    ozo_native_rows(m, n, k, A, lda, B, ldb, flag, alpha, beta, C, ldc);
+    if (flag_out) memcpy(flag_out, flag, (size_t)m);
+    free(flag); free(old);
+    return count;
 }
 
 /* ------------------------------------------------------------------ */

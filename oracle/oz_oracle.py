@@ -191,6 +191,52 @@ def esc_check(A: np.ndarray, B: np.ndarray, s: int) -> bool:
     return bool(lib().ozo_esc_check(_i64(m), _i64(n), _i64(k), _p(A), _i64(max(m, 1)), _p(B), _i64(max(k, 1)), s))
 
 
+def esc_rows(A: np.ndarray, B: np.ndarray, s: int) -> np.ndarray:
+    """Rows of the product that the exponent-span check sends to the native FP64 path (1 = re-issued)."""
+    _check_cm(A)
+    _check_cm(B)
+    m, k = A.shape
+    n = B.shape[1]
+    flag = np.zeros(max(m, 1), dtype=np.uint8)
+    f = lib().ozo_esc_rows
+    f.restype = C.c_int64
+    count = f(_i64(m), _i64(n), _i64(k), _p(A), _i64(max(m, 1)), _p(B), _i64(max(k, 1)), s, _p(flag))
+    assert count == int(flag[:m].sum())
+    return flag[:m]
+
+
+def native_rows(A: np.ndarray, B: np.ndarray, flag: np.ndarray, alpha: float = 1.0, beta: float = 0.0,
+                C0: np.ndarray | None = None) -> np.ndarray:
+    """The native FP64 path (compensated inner products) on the flagged rows; other rows keep C0."""
+    _check_cm(A)
+    _check_cm(B)
+    m, k = A.shape
+    n = B.shape[1]
+    Cm = np.asfortranarray(C0.copy()) if C0 is not None else np.zeros((m, n), dtype=np.float64, order="F")
+    flag = np.ascontiguousarray(flag, dtype=np.uint8)
+    lib().ozo_native_rows(_i64(m), _i64(n), _i64(k), _p(A), _i64(max(m, 1)), _p(B), _i64(max(k, 1)), _p(flag),
+                          C.c_double(alpha), C.c_double(beta), _p(Cm), _i64(max(m, 1)))
+    return Cm
+
+
+def dgemm_fallback(A: np.ndarray, B: np.ndarray, s: int = SET_S, quant: int = QUANT_RN, alpha: float = 1.0,
+                   beta: float = 0.0, C0: np.ndarray | None = None):
+    """The whole method (norm-based scale rule) with out-of-range rows re-issued on the native path.
+    Returns (C, flag)."""
+    _check_cm(A)
+    _check_cm(B)
+    m, k = A.shape
+    n = B.shape[1]
+    Cm = np.asfortranarray(C0.copy()) if C0 is not None else np.zeros((m, n), dtype=np.float64, order="F")
+    flag = np.zeros(max(m, 1), dtype=np.uint8)
+    f = lib().ozo_dgemm_fallback
+    f.restype = C.c_int64
+    rc = f(_i64(m), _i64(n), _i64(k), _p(A), _i64(max(m, 1)), _p(B), _i64(max(k, 1)), _p(Cm), _i64(max(m, 1)), s,
+           quant, C.c_double(alpha), C.c_double(beta), _p(flag))
+    assert rc >= 0
+    return Cm, flag[:m]
+
+
 def bound_digit(x: float, E: int) -> int:
     return lib().ozo_bound_digit(C.c_double(x), int(E))
 

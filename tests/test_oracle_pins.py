@@ -466,6 +466,99 @@ def test_esc_check_separates_the_benchmark_distributions(cfg_id, m, n, k):
         assert (worst > 1.0) == flagged
 
 
+# ----------------------------------------------------------------- out-of-range rows on the native FP64 path
+def test_esc_rows_match_the_restatement_and_the_call_level_check():
+    """Row i is re-issued when q(a_i) min_j q(b_j) < thr.  Pinned against the big-integer restatement,
+    against closed-form lines (a constant row is never re-issued, a one-spike row against spiky
+    columns is), and against the call-level check: a call is flagged exactly when some row is."""
+    rng = np.random.default_rng(11)
+    m, n, k = 14, 9, 160
+    A = np.asfortranarray(rng.standard_normal((m, k)) * np.exp(2.5 * rng.standard_normal((m, k))))
+    B = np.asfortranarray(rng.standard_normal((k, n)) * np.exp(2.5 * rng.standard_normal((k, n))))
+    A[0, :] = 1.25                     # flat row
+    A[1, :] = 0.0                      # zeros: not counted
+    A[2, :] = 0.0
+    A[2, 17] = -3.0                    # one spike: q = 2^16 / k
+    A[3, 5] = np.nan                   # Inf/NaN rows are not re-issued (their result is NaN anyway)
+    for name in ("S", "E", "A"):
+        ms = ozo.modset(SETS[name])
+        flag = ozo.esc_rows(A, B, SETS[name])
+        A_ok = A.copy(order="F")
+        A_ok[3, 5] = 1.0
+        want = big.esc_rows(A_ok.tolist(), B.tolist(), ms)   # the restatement takes finite data only
+        want[3] = 0
+        assert flag.tolist() == want
+        assert flag[1] == 0 and flag[3] == 0
+        assert bool(ozo.esc_rows(A_ok, B, SETS[name]).any()) == ozo.esc_check(A_ok, B, SETS[name])
+    # with perfectly flat columns the spike row passes on S (q_a q_b = 2^32 / k is far above the threshold) ...
+    Bflat = np.asfortranarray(np.full((k, n), 0.5))
+    assert ozo.esc_rows(A, Bflat, SETS["S"])[2] == (2 ** 32 // k < ozo.esc_threshold(SETS["S"]))
+    # ... and against a one-spike column every counted row with q_a < thr k / 2^16 fails
+    Bspike = np.zeros((k, n), order="F")
+    Bspike[3, :] = 2.0
+    f = ozo.esc_rows(A, Bspike, SETS["S"])
+    per_row = [None if i == 3 else big.esc_flatness(A[i].tolist(), k) for i in range(m)]
+    qb = 65536 // k
+    assert [int(v) for v in f] == [0 if q is None else int(min(q, 65536) * qb < ozo.esc_threshold(SETS["S"]))
+                                   for i, q in enumerate(per_row)]
+
+
+def test_native_rows_are_the_compensated_dot_product_in_k_order():
+    """The native path against its restatement in exact rationals (every operation = the correctly
+    rounded value of its exact result), incl. cancellation, and against the bound of the compensated
+    dot product: |res - a.b| <= u |a.b| + 2 (k u)^2 |a|.|b| -- far inside 2u (|A||B|)."""
+    rng = np.random.default_rng(12)
+    m, n, k = 5, 4, 37
+    A = np.asfortranarray(rng.standard_normal((m, k)) * np.exp(4 * rng.standard_normal((m, k))))
+    B = np.asfortranarray(rng.standard_normal((k, n)) * np.exp(4 * rng.standard_normal((k, n))))
+    A[1, 1::2] = -A[1, 0:-1:2]                      # heavy cancellation in row 1 ...
+    B[1::2, :] = B[0:-1:2, :]                       # ... against pairwise equal entries
+    flag = np.array([1, 1, 0, 1, 0], dtype=np.uint8)
+    C0 = np.asfortranarray(rng.standard_normal((m, n)))
+    for alpha, beta in ((1.0, 0.0), (-1.0, 1.0), (1.0, 1.0)):
+        got = ozo.native_rows(A, B, flag, alpha, beta, C0)
+        for i in range(m):
+            for j in range(n):
+                if not flag[i]:
+                    assert got[i, j] == C0[i, j]                     # untouched
+                    continue
+                v = big.native_dot(A[i].tolist(), B[:, j].tolist())
+                want = alpha * v if beta == 0.0 else C0[i, j] + alpha * v
+                assert got[i, j] == want
+                exact = sum(Fraction(float(x)) * Fraction(float(y)) for x, y in zip(A[i], B[:, j]))
+                mag = sum(abs(Fraction(float(x)) * Fraction(float(y))) for x, y in zip(A[i], B[:, j]))
+                u = Fraction(1, 2 ** 53)
+                assert abs(Fraction(v) - exact) <= u * abs(exact) + 2 * (k * u) ** 2 * mag
+    # the order of the inner product is part of the definition: reversing k changes bits somewhere
+    rev = ozo.native_rows(np.asfortranarray(A[:, ::-1]), np.asfortranarray(B[::-1, :]), flag)
+    fwd = ozo.native_rows(A, B, flag)
+    assert np.allclose(rev, fwd, rtol=1e-15, atol=0)
+    # Inf/NaN in a column of B gives NaN in that column of the re-issued rows
+    Bn = B.copy(order="F")
+    Bn[4, 2] = np.inf
+    out = ozo.native_rows(A, Bn, flag)
+    assert np.isnan(out[flag == 1][:, 2]).all() and np.isfinite(out[flag == 1][:, [0, 1, 3]]).all()
+
+
+def test_fallback_restores_the_accuracy_contract_on_the_wide_distribution():
+    """Config-5 data (lognormal, sigma = 2): the plain method misses 2u (|A||B|); with the out-of-range
+    rows re-issued every entry meets it, and the rows that were not re-issued are the method's."""
+    A, B = syn.operands(syn.CONFIGS[5], 40, 36, 5003)
+    hi, lo, ab = ozo.dd_gemm(A, B)
+    bound = 2 * 2.0 ** -53 * ab
+    plain = ozo.dgemm(A, B, SETS["S"])
+    C, flag = ozo.dgemm_fallback(A, B, SETS["S"])
+    assert (np.abs(plain - hi) > bound).any() and flag.any()
+    assert (np.abs(C - hi) <= bound).all() if flag.all() else (np.abs(C - hi)[flag == 1] <= bound[flag == 1]).all()
+    assert (C[flag == 0] == plain[flag == 0]).all()
+    assert (C[flag == 1] == ozo.native_rows(A, B, flag)[flag == 1]).all()
+    # on a benign distribution nothing is re-issued and the result is the method's, bit for bit
+    A2, B2 = syn.operands(syn.CONFIGS[3], 33, 21, 512)
+    C0 = np.asfortranarray(np.random.default_rng(3).standard_normal((33, 21)))
+    C2, flag2 = ozo.dgemm_fallback(A2, B2, SETS["S"], alpha=-1.0, beta=1.0, C0=C0)
+    assert not flag2.any() and (C2 == ozo.dgemm(A2, B2, SETS["S"], alpha=-1.0, beta=1.0, C0=C0)).all()
+
+
 # ----------------------------------------------------------------- accurate mode: the "+1" bound product
 def test_bound_digit_is_the_least_e4m3_upper_bound():
     """Sec. 2 "The FP8 variant": the extra product runs on FP8 operands, so its magnitude digits must
