@@ -251,6 +251,8 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=10)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-also", action="store_true", help="skip the other routes and the library 8-bit GEMM")
+    ap.add_argument("--fallback", action="store_true",
+                    help="re-issue the rows that fail the exponent-span check on the native FP64 path (OZ_FALLBACK_FP64)")
     args = ap.parse_args()
     if args.impl != "reference" and args.gpus > 1 and "WORLD_SIZE" not in os.environ:
         # run plainly with --gpus N: start the N replica ranks ourselves
@@ -279,7 +281,8 @@ def main():
     m, n, k = cfg.m, cfg.n, cfg.k
     modset = {"S": oz.OZ_SET_S, "E": oz.OZ_SET_E, "A": oz.OZ_SET_A}[args.set_name]
     sub = {"fp8": oz.OZ_SUB_FP8, "int8": oz.OZ_SUB_INT8, "int8n": oz.OZ_SUB_INT8_NATIVE}[args.substrate]
-    route = sub | oz.OZ_QUANT_RN | oz.OZ_SCALE_CS
+    host_route = sub | oz.OZ_QUANT_RN | oz.OZ_SCALE_CS      # the host-buffer entry point has no native path
+    route = host_route | (oz.OZ_FALLBACK_FP64 if args.fallback else 0)
     r, _, _ = oz.oz_set_info(modset)
     p_store = oz.oz_plane_count(modset, route)
     p_store_a = oz.oz_plane_count_side(modset, route, 0)    # same count on both operands
@@ -354,6 +357,7 @@ def main():
     clocks = sampler.stop()
     oz.oz_set_stage_events(None)
     check_status("device status after the timed steps")
+    fallback_rows = oz.oz_query_fallback_rows(stream) // max(args.steps + args.warmup, 1)
     local_ms = ev0.elapsed_time(ev1) / args.steps
     per_step = np.array([[evs[i].elapsed_time(evs[i + 1]) for i in range(4)] for evs in stage_events])
     stage_ms = per_step.mean(axis=0)
@@ -361,7 +365,7 @@ def main():
 
     # ---- end to end through the host-buffer entry point (copies inside the timed region)
     def e2e_step():
-        oz.check(oz.oz_dgemm_host(m, n, k, cfg.alpha, hA, m, hB, k, cfg.beta, hC, m, modset, route, stream),
+        oz.check(oz.oz_dgemm_host(m, n, k, cfg.alpha, hA, m, hB, k, cfg.beta, hC, m, modset, host_route, stream),
                  "oz_dgemm_host")
 
     e2e_step()
@@ -501,6 +505,8 @@ def main():
             "gpu_launches": int(launches), "clocks": clocks,
             "exponent_span_check": "flagged (OZ_ERR_RANGE): the set is too small for FP64-grade accuracy on this data"
                                    if esc_flag[0] else "passed",
+            "native_fp64_rows_per_step": int(fallback_rows) if args.fallback else None,
+            "native_fp64_ms": float(local_ms - step_totals.mean()) if args.fallback else None,   # after the last stage event
         }
         if not args.no_cpu_baseline:
             v, cores, desc = oracle_sample_tflops(cfg, args.set_name)

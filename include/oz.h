@@ -117,6 +117,24 @@ typedef enum { OZ_SET_S = 0, OZ_SET_E = 1, OZ_SET_A = 2 } oz_modset_t;
  * this bit is for comparison and for parts with a narrow FP64 pipe.  Ignored by the stage entry points. */
 #define OZ_RECON_TENSOR 0x4000u
 
+/* Out-of-range rows on the native FP64 path (Algorithm 1, last line: "ESC check; native-FP64 fallback
+ * for out-of-range rows"; Algorithm 3: "ESC range check; re-issue out-of-range rows on the native-FP64
+ * path").  The paper names the step; criterion and arithmetic are the library's reading.  With this bit
+ * oz_dgemm / oz_dgemm_ex apply the exponent-span check of oz_query_status() row by row: row i of the
+ * product is out of range when  min(q(a_i), 2^16) * min(min_j q(b_j), 2^16) < threshold  (q = floor(2^16
+ * phi^2), same threshold).  Such rows are left out of the reconstruction and computed in FP64 from the
+ * caller's old C: each entry is the compensated inner product of its row of A and column of B taken in
+ * the order kk = 0 .. k-1 (product error by one fused multiply-add, addition error by the error-free
+ * sum of two doubles, both collected in a second double that is added at the end), then
+ * C = alpha P or C + alpha P.  The value depends on the data alone, and it meets 2u (|A||B|)_ij like the
+ * emulated rows.  Cost: about ten FP64 operations per multiply-add on the SIMT FP64 pipe, so a call in
+ * which every row fails runs far below the emulated rate -- as the paper says, the fallback does not
+ * accelerate.  OZ_ERR_RANGE is still reported (informational).  oz_query_fallback_rows() returns how
+ * many rows were re-issued.  Needs OZ_SCALE_CS (the check is defined on its scan); not combined with
+ * OZ_RECON_TENSOR; OZ_ERR_UNSUPPORTED from oz_dgemm_host and oz_dgemm_prepared; ignored by the stage
+ * entry points.  Workspace: oz_workspace_bytes() with the same route (5 m + 768 bytes more). */
+#define OZ_FALLBACK_FP64 0x8000u
+
 #define OZ_K_MAX 1048576
 #define OZ_NONFINITE_SHIFT INT32_MIN  /* value of shift[] for a line that holds Inf/NaN */
 
@@ -272,6 +290,10 @@ oz_status_t oz_reconstruct(int64_t m, int64_t n, const void *R, int64_t ldr,
  * OZ_SET_A, or use native FP64 for it).  Purely informational: every result is still computed and
  * matches the method's definition.  Not evaluated with OZ_SCALE_MAXEXP or OZ_SCALE_ACCURATE. */
 oz_status_t oz_query_status(void *stream);
+
+/* Synchronises `stream`, stores in *rows (host) the number of rows that calls with OZ_FALLBACK_FP64
+ * re-issued on the native FP64 path on the current device since the last such query, and clears it. */
+oz_status_t oz_query_fallback_rows(void *stream, int64_t *rows);
 
 /* Optional per-stage timing hook for benchmarks (the paper's Algorithm 1 prices each stage
  * separately), kept per device: it applies to the device that is current when it is set.  `events`

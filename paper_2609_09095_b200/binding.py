@@ -22,6 +22,7 @@ OZ_QUANT_RN, OZ_QUANT_TZ = 0x010, 0x020
 OZ_SCALE_MAXEXP, OZ_SCALE_CS, OZ_SCALE_ACCURATE = 0x100, 0x200, 0x400
 OZ_ACC_MERGED, OZ_ACC_SEPARATE = 0x1000, 0x2000
 OZ_RECON_TENSOR = 0x4000
+OZ_FALLBACK_FP64 = 0x8000
 OZ_K_MAX = 1048576
 OZ_NONFINITE_SHIFT = -(2 ** 31)
 OZ_STATIC_MAX_LINES = 262144
@@ -30,13 +31,13 @@ EXPORTS = ["oz_set_info", "oz_plane_count", "oz_plane_count_side", "oz_row_pitch
            "oz_dgemm_ex", "oz_dgemm_host", "oz_operand_bytes", "oz_product_workspace_bytes", "oz_prepare_operand",
            "oz_dgemm_prepared", "oz_deconstruct", "oz_deconstruct_static",
            "oz_residue_gemm", "oz_reconstruct",
-           "oz_query_status", "oz_set_stage_events", "oz_launch_count", "oz_status_string"]
+           "oz_query_status", "oz_query_fallback_rows", "oz_set_stage_events", "oz_launch_count", "oz_status_string"]
 
 __all__ = EXPORTS + ["EXPORTS", "OzError", "load", "check", "LIB_PATH", "OZ_OK", "OZ_ERR_INVALID_ARG",
                      "OZ_ERR_UNSUPPORTED", "OZ_ERR_WORKSPACE", "OZ_ERR_CUDA",
                      "OZ_ERR_NONFINITE_INPUT", "OZ_ERR_RANGE", "OZ_ERR_TIMEOUT", "OZ_SET_S",
                      "OZ_SET_E", "OZ_SET_A", "OZ_SUB_FP8", "OZ_SUB_INT8", "OZ_SUB_INT8_NATIVE", "OZ_QUANT_RN", "OZ_QUANT_TZ",
-                     "OZ_SCALE_MAXEXP", "OZ_SCALE_CS", "OZ_SCALE_ACCURATE", "OZ_ACC_MERGED", "OZ_ACC_SEPARATE", "OZ_RECON_TENSOR", "OZ_K_MAX", "OZ_NONFINITE_SHIFT", "OZ_STATIC_MAX_LINES"]
+                     "OZ_SCALE_MAXEXP", "OZ_SCALE_CS", "OZ_SCALE_ACCURATE", "OZ_ACC_MERGED", "OZ_ACC_SEPARATE", "OZ_RECON_TENSOR", "OZ_FALLBACK_FP64", "OZ_K_MAX", "OZ_NONFINITE_SHIFT", "OZ_STATIC_MAX_LINES"]
 
 _lib = None
 
@@ -82,6 +83,7 @@ def load() -> C.CDLL:
                                     i64, vp]
     lib.oz_reconstruct.argtypes = [i64, i64, vp, i64, i64, vp, vp, i32, dbl, dbl, vp, i64, vp]
     lib.oz_query_status.argtypes = [vp]
+    lib.oz_query_fallback_rows.argtypes = [vp, C.POINTER(C.c_int64)]
     lib.oz_set_stage_events.argtypes = [C.POINTER(vp)]
     lib.oz_launch_count.restype = C.c_uint64
     lib.oz_status_string.argtypes = [i32]
@@ -220,6 +222,13 @@ def oz_reconstruct(m, n, R, ldr, mod_stride, shiftA, shiftB, modset, alpha, beta
 
 def oz_query_status(stream=None) -> int:
     return load().oz_query_status(_stream(stream))
+
+
+def oz_query_fallback_rows(stream=None) -> int:
+    """Rows re-issued on the native FP64 path since the last such query (synchronises the stream)."""
+    rows = C.c_int64(0)
+    check(load().oz_query_fallback_rows(_stream(stream), C.byref(rows)), "oz_query_fallback_rows")
+    return int(rows.value)
 
 
 def oz_set_stage_events(events) -> int:

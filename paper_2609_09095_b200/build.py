@@ -14,7 +14,7 @@ ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "liboz_b200.so")
 SOURCES = ["oz_api.cu", "oz_deconstruct.cu", "oz_deconstruct_static.cu", "oz_gemm_sm100.cu",
-           "oz_reconstruct.cu", "oz_reconstruct_hosted.cu"]
+           "oz_reconstruct.cu", "oz_reconstruct_hosted.cu", "oz_fallback.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-std=c++17", "-O3", "-lineinfo",
               "-Xcompiler", "-fPIC", "-I" + os.path.join(ROOT, "include"), "-I" + CSRC]
 

@@ -14,8 +14,8 @@ namespace oz {
 __device__ uint32_t g_lut[kNumSets][3][kLutWords];
 // status block: [0] sticky condition bits; [1], [2] smallest flatness code of the lines of A / B seen
 // since the last query (exponent-span check); [3] the threshold of the modulus set last used
-__device__ unsigned int g_status[4];
-const unsigned int kStatusReset[4] = {0u, 0xFFFFFFFFu, 0xFFFFFFFFu, 0u};
+__device__ unsigned int g_status[5];
+const unsigned int kStatusReset[5] = {0u, 0xFFFFFFFFu, 0xFFFFFFFFu, 0u, 0u};
 
 namespace {
 
@@ -119,8 +119,9 @@ uint64_t isqrt_u128(unsigned __int128 v)
 bool decode_route(uint32_t route, Route *out)
 {
     uint32_t sub = route & 0x00Fu, q = route & 0x0F0u, sc = route & 0xF00u, ac = route & 0x3000u;
-    if (route & ~0x7FFFu) return false;
+    if (route & ~0xFFFFu) return false;
     out->hosted = (route & OZ_RECON_TENSOR) != 0;
+    out->fallback = (route & OZ_FALLBACK_FP64) != 0;
     if (ac == 0) out->acc = 0;
     else if (ac == OZ_ACC_MERGED) out->acc = 1;
     else if (ac == OZ_ACC_SEPARATE) out->acc = 2;
@@ -326,6 +327,7 @@ size_t residue_bytes_total(int64_t m, int64_t n, int set)
 struct Layout {
     OperandLayout A, B;
     size_t offA, offB, R, total;
+    size_t fb_flag, fb_list, fb_count;    // native-path bookkeeping (fallback route only)
 };
 
 Layout make_layout(int64_t m, int64_t n, int64_t k, int set, const Route &rt)
@@ -337,6 +339,12 @@ Layout make_layout(int64_t m, int64_t n, int64_t k, int set, const Route &rt)
     L.offB = L.A.total;
     L.R = L.offB + L.B.total;
     L.total = L.R + residue_bytes_total(m, n, set);
+    if (rt.fallback) {
+        L.fb_flag = L.total;
+        L.fb_list = L.fb_flag + static_cast<size_t>(round_up(m, 256));
+        L.fb_count = L.fb_list + static_cast<size_t>(round_up(4 * m, 256));
+        L.total = L.fb_count + 256;
+    }
     return L;
 }
 
@@ -356,7 +364,8 @@ struct PanelPlan {
 // residue GEMMs + reconstruction from two deconstructed operands (stage events [2]..[4])
 oz_status_t product_impl(int64_t m, int64_t n, int64_t k, double alpha, const OperandView &a,
                          const OperandView &b, double beta, double *C, int64_t ldc, int set,
-                         const Route &rt, cudaStream_t stream, void *R, int dev, const PanelPlan *plan)
+                         const Route &rt, cudaStream_t stream, void *R, int dev, const PanelPlan *plan,
+                         const unsigned char *skip_rows = nullptr)
 {
     const bool ev = g_stage_events_on[dev];
     if (ev) OZ_CUDA_CHECK(cudaEventRecord(g_stage_events[dev][2], stream));
@@ -367,8 +376,16 @@ oz_status_t product_impl(int64_t m, int64_t n, int64_t k, double alpha, const Op
     if (ev) OZ_CUDA_CHECK(cudaEventRecord(g_stage_events[dev][3], stream));
     // the CRT recombination: exact FP64 chunk sums on the FP64 pipe, or (OZ_RECON_TENSOR) one small
     // unsigned 8-bit product per 128 outputs on the tensor pipe and an integer tail
-    auto reconstruct = rt.hosted ? launch_reconstruct_hosted : launch_reconstruct_tiled;
-    if (!plan) {
+    auto reconstruct = [&](int64_t m_, int64_t n_, const void *R_, const int32_t *sa, const int32_t *sb, int set_,
+                           double alpha_, double beta_, double *C_, int64_t ldc_, int64_t c0, int64_t c1,
+                           cudaStream_t s_) {
+        return rt.hosted ? launch_reconstruct_hosted(m_, n_, R_, sa, sb, set_, alpha_, beta_, C_, ldc_, c0, c1, s_)
+                         : launch_reconstruct_tiled(m_, n_, R_, sa, sb, set_, alpha_, beta_, C_, ldc_, c0, c1, s_);
+    };
+    if (skip_rows) {
+        st = launch_reconstruct_tiled(m, n, R, a.shift, b.shift, set, alpha, beta, C, ldc, 0, n, stream, skip_rows);
+        if (st != OZ_OK) return st;
+    } else if (!plan) {
         st = reconstruct(m, n, R, a.shift, b.shift, set, alpha, beta, C, ldc, 0, n, stream);
         if (st != OZ_OK) return st;
     } else {
@@ -418,6 +435,8 @@ oz_status_t dgemm_impl(int64_t m, int64_t n, int64_t k, double alpha, const doub
     if (!A || !B || lda < m || ldb < k || (reinterpret_cast<uintptr_t>(A) & 7u) ||
         (reinterpret_cast<uintptr_t>(B) & 7u))
         return OZ_ERR_INVALID_ARG;
+    // out-of-range rows on the native path: defined on the norm scan, FP64 reconstruction, one panel
+    if (rt.fallback && (rt.rule != 1 || rt.hosted || plan)) return OZ_ERR_UNSUPPORTED;
     Layout L = make_layout(m, n, k, set, rt);
     if (!ws || ws_bytes < L.total) return OZ_ERR_WORKSPACE;
     st = ensure_device_ready();
@@ -466,7 +485,17 @@ oz_status_t dgemm_impl(int64_t m, int64_t n, int64_t k, double alpha, const doub
     if (st != OZ_OK) return st;
     if (ev) OZ_CUDA_CHECK(cudaEventRecord(g_stage_events[dev][1], stream));
     OZ_CUDA_CHECK(cudaStreamWaitEvent(stream, g_join[dev], 0));
-    return product_impl(m, n, k, alpha, a, b, beta, C, ldc, set, rt, stream, ws + L.R, dev, plan);
+    if (!rt.fallback) return product_impl(m, n, k, alpha, a, b, beta, C, ldc, set, rt, stream, ws + L.R, dev, plan);
+    // Algorithm 1, last line / Algorithm 3, "ESC range check": the rows that fail the check are left
+    // out of the reconstruction and re-issued on the native FP64 path from the caller's old C
+    unsigned char *flag = reinterpret_cast<unsigned char *>(ws + L.fb_flag);
+    int *list = reinterpret_cast<int *>(ws + L.fb_list);
+    unsigned int *count = reinterpret_cast<unsigned int *>(ws + L.fb_count);
+    st = launch_esc_rows(a.scratch, m, b.scratch, n, k, set, flag, list, count, stream);
+    if (st != OZ_OK) return st;
+    st = product_impl(m, n, k, alpha, a, b, beta, C, ldc, set, rt, stream, ws + L.R, dev, nullptr, flag);
+    if (st != OZ_OK) return st;
+    return launch_native_rows(m, n, k, A, lda, B, ldb, list, count, b.shift, alpha, beta, C, ldc, stream);
 }
 
 // Side streams and events of the host-buffer entry point, created once per device.
@@ -711,6 +740,7 @@ oz_status_t oz_dgemm_prepared(int64_t m, int64_t n, int64_t k, double alpha, con
     oz_status_t st = check_product_args(m, n, k, alpha, beta, C, ldc, set, route, s, &rt, &trivial);
     if (st != OZ_OK || trivial) return st;
     if (rt.rule == 2) return OZ_ERR_UNSUPPORTED;      // prepared operands carry per-operand shifts
+    if (rt.fallback) return OZ_ERR_UNSUPPORTED;       // the native path needs the FP64 operands
     if (!operandA || !operandB || (reinterpret_cast<uintptr_t>(operandA) & 255u) ||
         (reinterpret_cast<uintptr_t>(operandB) & 255u))
         return OZ_ERR_INVALID_ARG;
@@ -804,13 +834,27 @@ oz_status_t oz_query_status(void *stream)
     unsigned int word[4] = {0, 0, 0, 0};
     OZ_CUDA_CHECK(cudaStreamSynchronize(s));
     OZ_CUDA_CHECK(cudaMemcpyFromSymbol(word, g_status, sizeof(word)));
-    OZ_CUDA_CHECK(cudaMemcpyToSymbol(g_status, kStatusReset, sizeof(kStatusReset)));
+    OZ_CUDA_CHECK(cudaMemcpyToSymbol(g_status, kStatusReset, sizeof(word)));   // word 4 has its own query
     if (cudaGetLastError() != cudaSuccess) return OZ_ERR_CUDA;
     if (word[0] & (1u << OZ_ERR_TIMEOUT)) return OZ_ERR_TIMEOUT;
     if (word[0] & (1u << OZ_ERR_NONFINITE_INPUT)) return OZ_ERR_NONFINITE_INPUT;
     // exponent-span check: an operand that was not scanned since the last query counts as flat
     const uint64_t qa = word[1] > 65536u ? 65536u : word[1], qb = word[2] > 65536u ? 65536u : word[2];
     if (word[3] != 0u && qa * qb < static_cast<uint64_t>(word[3])) return OZ_ERR_RANGE;
+    return OZ_OK;
+}
+
+oz_status_t oz_query_fallback_rows(void *stream, int64_t *rows)
+{
+    if (!rows) return OZ_ERR_INVALID_ARG;
+    oz_status_t st = ensure_device_ready();
+    if (st != OZ_OK) return st;
+    OZ_CUDA_CHECK(cudaStreamSynchronize(static_cast<cudaStream_t>(stream)));
+    unsigned int count = 0;
+    const unsigned int zero = 0;
+    OZ_CUDA_CHECK(cudaMemcpyFromSymbol(&count, g_status, sizeof(count), 4 * sizeof(unsigned int)));
+    OZ_CUDA_CHECK(cudaMemcpyToSymbol(g_status, &zero, sizeof(zero), 4 * sizeof(unsigned int)));
+    *rows = static_cast<int64_t>(count);
     return OZ_OK;
 }
 

@@ -211,6 +211,70 @@ __global__ void scan_finalize_kernel(ScanScratch s, int64_t lines, int64_t k, in
     status[3] = esc_threshold;
 }
 
+// ---- out-of-range rows (Algorithm 1, last line; Algorithm 3, "ESC range check; re-issue out-of-range
+// rows on the native-FP64 path") ------------------------------------------------------------------
+// flatness of one scanned line from its norm sums, capped at 2^16; 0xFFFFFFFF for a line that does
+// not count (zeros only, or Inf/NaN)
+__device__ __forceinline__ unsigned int scanned_flatness(const ScanScratch &s, int64_t i, int64_t k)
+{
+    const int nf = s.nonfinite[i];
+    if (nf < 0 || s.emax[i] == INT32_MIN) return 0xFFFFFFFFu;
+    const unsigned long long l1 = static_cast<unsigned int>(nf);
+    const unsigned __int128 flat = ((static_cast<unsigned __int128>(l1 * l1)) << 16) /
+                                   (static_cast<unsigned __int128>(static_cast<unsigned long long>(k)) * s.sumsq[i]);
+    const unsigned int q = static_cast<unsigned int>(flat);
+    return q > 65536u ? 65536u : q;
+}
+
+// One block.  Row i of the product is re-issued when q(a_i) * min_j q(b_j) < threshold.  Writes the
+// flag of every row, the re-issued rows in ascending order, their number, and adds that number to the
+// device status block (word 4).
+__global__ void __launch_bounds__(1024)
+esc_rows_kernel(ScanScratch sA, int64_t m, ScanScratch sB, int64_t n, int64_t k, unsigned int threshold,
+                unsigned char *flag, int *list, unsigned int *count, unsigned int *status)
+{
+    __shared__ unsigned int red[32];
+    __shared__ unsigned int base;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    unsigned int qb = 0xFFFFFFFFu;
+    for (int64_t j = tid; j < n; j += blockDim.x) qb = min(qb, scanned_flatness(sB, j, k));
+    qb = __reduce_min_sync(0xFFFFFFFFu, qb);
+    if (lane == 0) red[warp] = qb;
+    if (tid == 0) base = 0u;
+    __syncthreads();
+    qb = red[lane];
+    qb = __reduce_min_sync(0xFFFFFFFFu, qb);
+    if (qb > 65536u) qb = 65536u;
+    __syncthreads();
+    for (int64_t i0 = 0; i0 < m; i0 += blockDim.x) {
+        const int64_t i = i0 + tid;
+        bool out = false;
+        if (i < m) {
+            const unsigned int qa = scanned_flatness(sA, i, k);
+            out = qa != 0xFFFFFFFFu && static_cast<unsigned long long>(qa) * qb < threshold;
+            flag[i] = out ? 1 : 0;
+        }
+        // ordered compaction: position = rows re-issued so far + those of lower threads
+        const unsigned int ballot = __ballot_sync(0xFFFFFFFFu, out);
+        if (lane == 0) red[warp] = __popc(ballot);
+        __syncthreads();
+        unsigned int before = base;
+        for (int w = 0; w < warp; ++w) before += red[w];
+        if (out) list[before + __popc(ballot & ((1u << lane) - 1u))] = static_cast<int>(i);
+        __syncthreads();
+        if (tid == 0) {
+            unsigned int total = 0;
+            for (int w = 0; w < 32; ++w) total += red[w];
+            base += total;
+        }
+        __syncthreads();
+    }
+    if (tid == 0) {
+        *count = base;
+        if (base) atomicAdd(status + 4, base);
+    }
+}
+
 // ---- accurate mode (Sec. 2 "The FP8 variant": the additional FP8 product that estimates a
 // magnitude bound, the "+1" of the 3r + 1 schedule) ------------------------------------------
 // Magnitude digit of one element: the smallest integer of the E4M3 grid {0..16, 18, 20, .., 32} that
@@ -893,7 +957,7 @@ oz_status_t launch_deconstruct(int side, int64_t lines, int64_t k, const double 
     OZ_CUDA_CHECK(cudaGetDevice(&dev));
     OZ_CUDA_CHECK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
     const FusedShape f = fused_shape(rt.layout(side) == kLayoutNative ? 2 : set, side, lines, k, sms);
-    if (f.group > 0) {
+    if (f.group > 0 && !rt.fallback) {      // the row check reads the scan results of the three-pass form
         FusedParams p{};
         p.X = X; p.ldx = ldx; p.lines = lines; p.k = k;
         p.group = f.group;
@@ -928,6 +992,18 @@ oz_status_t launch_deconstruct(int side, int64_t lines, int64_t k, const double 
     oz_status_t st = launch_scan(side, lines, k, X, ldx, set, rt, shift, scratch, stream);
     if (st != OZ_OK) return st;
     return launch_convert_planes(side, lines, k, X, ldx, set, rt, planes, plane_stride, row_pitch, shift, stream);
+}
+
+// flags, ordered list and number of the rows that go to the native FP64 path, from the scan results
+// that the three-pass deconstruction of both operands left in their scratch blocks
+oz_status_t launch_esc_rows(void *scratchA, int64_t m, void *scratchB, int64_t n, int64_t k, int set,
+                            unsigned char *flag, int *list, unsigned int *count, cudaStream_t stream)
+{
+    esc_rows_kernel<<<1, 1024, 0, stream>>>(carve_scratch(scratchA, m), m, carve_scratch(scratchB, n), n, k,
+                                            esc_threshold(set), flag, list, count, device_status_word());
+    count_launch();
+    OZ_CUDA_CHECK(cudaGetLastError());
+    return OZ_OK;
 }
 
 }  // namespace oz

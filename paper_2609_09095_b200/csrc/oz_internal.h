@@ -121,6 +121,7 @@ struct Route {
         return side == 0 ? kLayoutMerged : kLayoutDigits;
     }
     bool hosted;    // whole-method calls: CRT recombination on the INT8 tensor pipe (OZ_RECON_TENSOR)
+    bool fallback;  // oz_dgemm / oz_dgemm_ex: out-of-range rows re-issued on the native FP64 path
     int quant;      // 0 rn, 1 tz
     int rule;       // 0 maxexp, 1 cs, 2 accurate (shifts from the extra bound product)
 };
@@ -197,7 +198,7 @@ oz_status_t launch_residue_gemm(int64_t m, int64_t n, int64_t k, const uint8_t *
 oz_status_t launch_reconstruct_tiled(int64_t m, int64_t n, const void *R, const int32_t *shiftA,
                                      const int32_t *shiftB, int set, double alpha, double beta,
                                      double *C, int64_t ldc, int64_t col0, int64_t col1,
-                                     cudaStream_t stream);
+                                     cudaStream_t stream, const unsigned char *skip_rows = nullptr);
 
 oz_status_t launch_reconstruct(int64_t m, int64_t n, const void *R, int64_t ldr,
                                int64_t mod_stride, const int32_t *shiftA, const int32_t *shiftB,
@@ -213,6 +214,16 @@ oz_status_t launch_reconstruct_hosted(int64_t m, int64_t n, const void *R, const
                                       const int32_t *shiftB, int set, double alpha, double beta,
                                       double *C, int64_t ldc, int64_t col0, int64_t col1,
                                       cudaStream_t stream);
+
+// Out-of-range rows (Algorithm 1, last line; Algorithm 3, "ESC range check"): flags, ascending list and
+// number of the rows that go to the native FP64 path, from the scan results that the three-pass
+// deconstruction left in the two scratch blocks; and the native path itself
+oz_status_t launch_esc_rows(void *scratchA, int64_t m, void *scratchB, int64_t n, int64_t k, int set,
+                            unsigned char *flag, int *list, unsigned int *count, cudaStream_t stream);
+oz_status_t launch_native_rows(int64_t m, int64_t n, int64_t k, const double *A, int64_t lda,
+                               const double *B, int64_t ldb, const int *list, const unsigned int *count,
+                               const int32_t *shiftB, double alpha, double beta, double *C, int64_t ldc,
+                               cudaStream_t stream);
 
 #define OZ_CUDA_CHECK(expr)                                  \
     do {                                                     \

@@ -155,38 +155,26 @@ __device__ __forceinline__ double row_value(const uint32_t (&w)[kMaxR], int sa, 
     return p * alpha;
 }
 
-__device__ __forceinline__ void store_pair(double *out, double p0, double p1, bool two, bool vec, double beta)
+// scalar stores of up to two consecutive rows; `first` / `second`: which of them are written
+__device__ __forceinline__ void store_pair(double *out, double p0, double p1, bool first, bool second, double beta)
 {
-    if (vec && two) {
-        double2 o;
-        if (beta != 0.0) {
-            double2 old = *reinterpret_cast<const double2 *>(out);
-            o.x = old.x + p0;
-            o.y = old.y + p1;
-        } else {
-            o.x = p0;
-            o.y = p1;
-        }
-        *reinterpret_cast<double2 *>(out) = o;
-    } else {
-        out[0] = beta != 0.0 ? out[0] + p0 : p0;
-        if (two) out[1] = beta != 0.0 ? out[1] + p1 : p1;
-    }
+    if (first) out[0] = beta != 0.0 ? out[0] + p0 : p0;
+    if (second) out[1] = beta != 0.0 ? out[1] + p1 : p1;
 }
 
 // the ROWS consecutive rows of column j whose residues are packed in w[]: reconstruct, update C.
 // For beta = 1 the old values of C are requested before the arithmetic starts, so that their latency
-// hides behind it.
+// hides behind it.  `keep`: bit h set = row h is written (rows that go to the native FP64 path are not).
 template <int SET>
 __device__ __forceinline__ void reconstruct_rows(const uint32_t (&w)[kMaxR], int64_t row, int nrows, int sb,
                                                  const int32_t *__restrict__ shiftA, double alpha, double beta,
-                                                 double *out, bool vecC)
+                                                 double *out, bool vecC, uint32_t keep = 0xFu)
 {
     constexpr int ROWS = 4 / residue_bytes(SET);
     int sa[ROWS];
 #pragma unroll
     for (int h = 0; h < ROWS; ++h) sa[h] = h < nrows ? shiftA[row + h] : 0;
-    const bool whole = vecC && nrows == ROWS;
+    const bool whole = vecC && nrows == ROWS && (keep & ((1u << ROWS) - 1u)) == ((1u << ROWS) - 1u);
     double2 old[ROWS / 2];
 #pragma unroll
     for (int h = 0; h < ROWS / 2; ++h) old[h] = make_double2(0.0, 0.0);
@@ -198,14 +186,14 @@ __device__ __forceinline__ void reconstruct_rows(const uint32_t (&w)[kMaxR], int
         double p0 = row_value<SET, 0>(w, sa[0], sb, alpha);
         double p1 = nrows > 1 ? row_value<SET, 1>(w, sa[1], sb, alpha) : 0.0;
         if (whole) *reinterpret_cast<double2 *>(out) = make_double2(old[0].x + p0, old[0].y + p1);
-        else store_pair(out, p0, p1, nrows > 1, false, beta);
+        else store_pair(out, p0, p1, (keep & 1u) != 0, nrows > 1 && (keep & 2u) != 0, beta);
     }
     if constexpr (ROWS == 4) {
         if (nrows > 2) {
             double p2 = row_value<SET, 2>(w, sa[2], sb, alpha);
             double p3 = nrows > 3 ? row_value<SET, 3>(w, sa[3], sb, alpha) : 0.0;
             if (whole) *reinterpret_cast<double2 *>(out + 2) = make_double2(old[1].x + p2, old[1].y + p3);
-            else store_pair(out + 2, p2, p3, nrows > 3, false, beta);
+            else store_pair(out + 2, p2, p3, (keep & 4u) != 0, nrows > 3 && (keep & 8u) != 0, beta);
         }
     }
 }
@@ -259,12 +247,14 @@ reconstruct_kernel(const void *__restrict__ Rv, int64_t ldr, int64_t mod_stride,
 // loads are 16-byte pieces 512 bytes apart, and the warps of a thread block, which take neighbouring
 // columns, ask for whole 128-byte lines between them.
 // grid: x = (piece of the block, block within the tile, CTA rank of the pair), y = tile column, z = tile row
-template <int SET>
+// SKIP: rows flagged in `skip` are left untouched (they are re-issued on the native FP64 path).
+template <int SET, bool SKIP>
 __global__ void __launch_bounds__(256, residue_bytes(SET) == 2 ? 6 : 5)
 reconstruct_tiled_kernel(const void *__restrict__ Rv, int cg, int tiles_n, int tn0,
                          int64_t m, int64_t n, int64_t col0, int64_t col1,
                          const int32_t *__restrict__ shiftA, const int32_t *__restrict__ shiftB,
-                         double alpha, double beta, double *__restrict__ C, int64_t ldc, int vecC)
+                         double alpha, double beta, double *__restrict__ C, int64_t ldc, int vecC,
+                         const unsigned char *__restrict__ skip)
 {
     constexpr int RB = residue_bytes(SET), ROWS = 4 / RB, r = set_r(SET);
     constexpr int kBlockWords = 64 * 32 * RB / 4;          // words of one 32 x 64 block: 1024 or 512
@@ -281,6 +271,14 @@ reconstruct_tiled_kernel(const void *__restrict__ Rv, int cg, int tiles_n, int t
     const int64_t j = (static_cast<int64_t>(tn) * cg + rank) * 128 + (wi & 3u) * 32 + lane;
     if (row >= m || j >= n || j < col0 || j >= col1) return;
     const int nrows = m - row < ROWS ? static_cast<int>(m - row) : ROWS;
+    uint32_t keep = 0xFu;
+    if constexpr (SKIP) {
+        keep = 0u;
+#pragma unroll
+        for (int h = 0; h < ROWS; ++h)
+            if (h < nrows && !skip[row + h]) keep |= 1u << h;
+        if (!keep) return;
+    }
     const int64_t wb = ((static_cast<int64_t>(tm) * tiles_n + tn) * cg + rank) * 16 + wi;
     // the r blocks of this patch are consecutive: modulus i at a compile-time offset
     const unsigned char *base = static_cast<const unsigned char *>(Rv) +
@@ -288,7 +286,7 @@ reconstruct_tiled_kernel(const void *__restrict__ Rv, int cg, int tiles_n, int t
     uint32_t w[kMaxR];
 #pragma unroll
     for (int i = 0; i < r; ++i) w[i] = *reinterpret_cast<const uint32_t *>(base + i * (kBlockWords * 4));
-    reconstruct_rows<SET>(w, row, nrows, shiftB[j], shiftA, alpha, beta, C + row + j * ldc, vecC != 0);
+    reconstruct_rows<SET>(w, row, nrows, shiftB[j], shiftA, alpha, beta, C + row + j * ldc, vecC != 0, keep);
 }
 
 }  // namespace
@@ -357,7 +355,7 @@ oz_status_t launch_reconstruct(int64_t m, int64_t n, const void *R, int64_t ldr,
 oz_status_t launch_reconstruct_tiled(int64_t m, int64_t n, const void *R, const int32_t *shiftA,
                                      const int32_t *shiftB, int set, double alpha, double beta,
                                      double *C, int64_t ldc, int64_t col0, int64_t col1,
-                                     cudaStream_t stream)
+                                     cudaStream_t stream, const unsigned char *skip)
 {
     if (col1 <= col0) return OZ_OK;
     const ResidueTiling t = residue_tiling(m, n, set);
@@ -368,9 +366,11 @@ oz_status_t launch_reconstruct_tiled(int64_t m, int64_t n, const void *R, const 
     const int vecC = ((ldc & 1) == 0 && (reinterpret_cast<uintptr_t>(C) & 15u) == 0) ? 1 : 0;
     const dim3 grid(static_cast<unsigned>(pieces * 16 * t.cg), static_cast<unsigned>(ntn),
                     static_cast<unsigned>(t.tiles_m));
-#define OZ_RECON_TILED(SET_)                                                                              \
-    reconstruct_tiled_kernel<SET_><<<grid, 256, 0, stream>>>(R, t.cg, t.tiles_n, tn0, m, n,  \
-                                                             col0, col1, shiftA, shiftB, alpha, beta, C, ldc, vecC)
+#define OZ_RECON_TILED(SET_)                                                                               \
+    (skip ? reconstruct_tiled_kernel<SET_, true><<<grid, 256, 0, stream>>>(                                \
+                R, t.cg, t.tiles_n, tn0, m, n, col0, col1, shiftA, shiftB, alpha, beta, C, ldc, vecC, skip) \
+          : reconstruct_tiled_kernel<SET_, false><<<grid, 256, 0, stream>>>(                               \
+                R, t.cg, t.tiles_n, tn0, m, n, col0, col1, shiftA, shiftB, alpha, beta, C, ldc, vecC, nullptr))
     if (set == 2) OZ_RECON_TILED(2);
     else if (set == 0) OZ_RECON_TILED(0);
     else OZ_RECON_TILED(1);

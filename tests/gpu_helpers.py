@@ -10,7 +10,7 @@ import paper_2609_09095_b200 as oz
 SETS = {"S": oz.OZ_SET_S, "E": oz.OZ_SET_E, "A": oz.OZ_SET_A}
 
 
-def route(sub="fp8", quant="RN", rule="CS", acc=None, recon=None) -> int:
+def route(sub="fp8", quant="RN", rule="CS", acc=None, recon=None, fallback=False) -> int:
     r = {"fp8": oz.OZ_SUB_FP8, "int8": oz.OZ_SUB_INT8, "int8n": oz.OZ_SUB_INT8_NATIVE}[sub]
     r |= oz.OZ_QUANT_RN if quant == "RN" else oz.OZ_QUANT_TZ
     r |= {"CS": oz.OZ_SCALE_CS, "MAXEXP": oz.OZ_SCALE_MAXEXP, "ACCURATE": oz.OZ_SCALE_ACCURATE}[rule]
@@ -18,6 +18,8 @@ def route(sub="fp8", quant="RN", rule="CS", acc=None, recon=None) -> int:
         r |= oz.OZ_ACC_MERGED if acc == "merged" else oz.OZ_ACC_SEPARATE
     if recon == "tensor":
         r |= oz.OZ_RECON_TENSOR
+    if fallback:
+        r |= oz.OZ_FALLBACK_FP64
     return r
 
 

@@ -105,3 +105,44 @@ def test_full_size_sampled(cfg_id, set_name, sub):
     oz.oz_set_workspace(None)
     gh._ws = None
     torch.cuda.empty_cache()
+
+
+@pytest.mark.parametrize("set_name,sub", [("S", "fp8"), ("A", "int8n")])
+def test_full_size_fallback_sampled(set_name, sub):
+    """Config 5 at full size with the out-of-range rows re-issued on the native FP64 path: the rows the
+    oracle's check flags on the whole operands are the
+    compensated inner products, the others the method's; every sampled entry meets 2u (|A||B|)
+    against the double-double product where it was re-issued."""
+    import paper_2609_09095_b200 as oz
+    import tests.gpu_helpers as gh
+    cfg = syn.CONFIGS[5]
+    m, n, k = cfg.m, cfg.n, cfg.k
+    rng = np.random.default_rng(cfg.seed + 23)
+    A, B = syn.operands(cfg)
+    oset = OSET[set_name]
+    flag = ozo.esc_rows(A, B, oset)
+    assert flag.any()          # against the least flat of 9973 columns every row fails, on either set
+    rows, cols = _sample(m, rng, 256), _sample(n, rng, 128)
+    As, Bs = np.asfortranarray(A[rows, :]), np.asfortranarray(B[:, cols])
+    native = ozo.native_rows(As, Bs, np.ones(len(rows), dtype=np.uint8))
+    method = ozo.dgemm(As, Bs, oset)          # rows and columns are independent: an exact sub-problem
+    want = np.where(flag[rows][:, None] == 1, native, method)
+    rt = gh.route(sub, "RN", "CS", fallback=True)
+    gh.ensure_workspace(oz.oz_workspace_bytes(m, n, k, gh.SETS[set_name], rt))
+    dA, dB = gh.to_dev(A), gh.to_dev(B)
+    dC = torch.empty((n, m), dtype=torch.float64, device="cuda")
+    oz.oz_query_fallback_rows()
+    oz.check(oz.oz_dgemm(m, n, k, dA, m, dB, k, dC, m, gh.SETS[set_name], rt), "oz_dgemm, native path")
+    assert gh.sync_status(esc=True) == oz.OZ_ERR_RANGE
+    assert oz.oz_query_fallback_rows() == int(flag.sum())
+    ri, ci = torch.from_numpy(rows).cuda(), torch.from_numpy(cols).cuda()
+    got = dC[ci, :][:, ri].cpu().numpy().T
+    assert (got == want).all()
+    hi, _, ab = ozo.dd_gemm(As, Bs)
+    re = flag[rows] == 1
+    assert (np.abs(got - hi)[re] <= (2 * U * ab)[re]).all()
+    assert bool(torch.isfinite(dC).all())
+    del dA, dB, dC
+    oz.oz_set_workspace(None)
+    gh._ws = None
+    torch.cuda.empty_cache()
