@@ -32,8 +32,8 @@ native_rows_kernel(int64_t m, int64_t n, int64_t k, const double *__restrict__ A
     const int64_t r0 = static_cast<int64_t>(blockIdx.y) * kFbRows;
     if (r0 >= rows) return;
     const int64_t c0 = static_cast<int64_t>(blockIdx.x) * kFbCols;
-    __shared__ double As[kFbK][kFbRows + 1];
-    __shared__ double Bs[kFbK][kFbCols + 1];
+    __shared__ __align__(16) double As[kFbK][kFbRows + 2];     // +2: rows stay 16-byte aligned for the pair loads
+    __shared__ __align__(16) double Bs[kFbK][kFbCols + 2];
     __shared__ int64_t row_of[kFbRows];
     const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
     if (tid < kFbRows) row_of[tid] = r0 + tid < rows ? list[r0 + tid] : -1;
@@ -62,11 +62,11 @@ native_rows_kernel(int64_t m, int64_t n, int64_t k, const double *__restrict__ A
         }
         __syncthreads();
         for (int kk = 0; kk < kn; ++kk) {
-            double a[4], b[4];
-#pragma unroll
-            for (int r = 0; r < 4; ++r) a[r] = As[kk][ty * 4 + r];
-#pragma unroll
-            for (int c = 0; c < 4; ++c) b[c] = Bs[kk][tx * 4 + c];
+            const double2 a01 = *reinterpret_cast<const double2 *>(&As[kk][ty * 4]);
+            const double2 a23 = *reinterpret_cast<const double2 *>(&As[kk][ty * 4 + 2]);
+            const double2 b01 = *reinterpret_cast<const double2 *>(&Bs[kk][tx * 4]);
+            const double2 b23 = *reinterpret_cast<const double2 *>(&Bs[kk][tx * 4 + 2]);
+            const double a[4] = {a01.x, a01.y, a23.x, a23.y}, b[4] = {b01.x, b01.y, b23.x, b23.y};
 #pragma unroll
             for (int r = 0; r < 4; ++r)
 #pragma unroll
