@@ -776,6 +776,18 @@ FusedShape fused_shape(int set, int side, int64_t lines, int64_t k, int sms)
     }
     if (group < min_group) return f;
     if (group > 32) group = 32;
+    // small operands: fewer lines per block, so that the blocks cover the machine (a 256 x 256 operand
+    // with 32 lines per block would run on 8 SMs)
+#ifndef OZ_FUSED_SPREAD_MIN
+#define OZ_FUSED_SPREAD_MIN 8
+#endif
+    {
+        const int64_t blocks_wanted = static_cast<int64_t>(sms) * (threads == 512 ? 2 : 1);
+        int64_t spread = (lines + blocks_wanted - 1) / blocks_wanted;
+        const int floor_group = side == 0 ? OZ_FUSED_SPREAD_MIN : 1;
+        if (spread < floor_group) spread = floor_group;
+        if (spread < group) group = static_cast<int>(spread);
+    }
     if (side == 0) {
         int pow2 = 1;
         while (pow2 * 2 <= group) pow2 *= 2;
