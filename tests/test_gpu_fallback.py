@@ -45,6 +45,28 @@ def test_fallback_bit_identical_to_oracle(set_name, sub, m, n, k, sigma, quant):
         assert oz.oz_query_fallback_rows() == 0         # the count is cleared by the query
 
 
+@pytest.mark.parametrize("seed", range(12))
+def test_fallback_random_shapes(seed):
+    """Seeded random shapes, sets, substrates, quantisers, scalars and exponent spreads on the route with
+    the native path: whatever share of the rows the check sends there, the matrix is the oracle's."""
+    import paper_2609_09095_b200 as oz
+    import tests.gpu_helpers as gh
+    rng = np.random.default_rng(7000 + seed)
+    m, n, k = int(rng.integers(1, 400)), int(rng.integers(1, 400)), int(rng.integers(1, 700))
+    set_name, sub = [("S", "fp8"), ("A", "int8n"), ("E", "int8"), ("A", "fp8")][seed % 4]
+    quant = ("RN", "TZ")[int(rng.integers(2))]
+    alpha, beta = (1.0, -1.0)[int(rng.integers(2))], (0.0, 1.0)[int(rng.integers(2))]
+    sigma = (0.5, 1.5, 2.0, 2.5, 3.0)[int(rng.integers(5))]
+    A, B = _wide(rng, m, k, sigma), _wide(rng, k, n, sigma)
+    C0 = np.asfortranarray(rng.standard_normal((m, n))) if beta else None
+    oz.oz_query_fallback_rows()
+    got, st = gh.dgemm(A, B, set_name, gh.route(sub, quant, "CS", fallback=True), alpha, beta, C0)
+    want, flag = ozo.dgemm_fallback(A, B, OSET[set_name], ozo.QUANT_RN if quant == "RN" else ozo.QUANT_TZ,
+                                    alpha, beta, C0)
+    assert st == 0 and oz.oz_query_fallback_rows() == int(flag.sum())
+    assert (got == want).all()
+
+
 def test_fallback_mixes_and_reports():
     """Set A on the sigma = 2.5 data: the check splits the rows, so both paths write into the same C."""
     import paper_2609_09095_b200 as oz

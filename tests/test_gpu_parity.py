@@ -432,6 +432,7 @@ def test_argument_errors_are_reported_on_the_host():
     (4096, 4224, 96, -1.0, 1.0, "S", "fp8"),        # 138 MB of C: two column panels on side streams
     (4100, 8200, 40, 1.0, 0.0, "A", "int8n"),       # four panels, ragged, no upload of C
     (3000, 11200, 24, 1.0, 1.0, "E", "fp8"),        # four panels of unequal width
+    (260, 300, 520, -1.0, 1.0, "S", "int8"),        # INT8 digit planes: merged schedule on both operands
 ])
 def test_dgemm_host_buffers(m, n, k, alpha, beta, set_name, sub):
     """oz_dgemm_host (pinned host operands, copies inside, C in column panels when it is large) against
