@@ -251,6 +251,8 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=10)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-also", action="store_true", help="skip the other routes and the library 8-bit GEMM")
+    ap.add_argument("--fused", action="store_true",
+                    help="storage mode F: A converted inside the product kernel (OZ_STORAGE_FUSED; n <= 128)")
     ap.add_argument("--fallback", action="store_true",
                     help="re-issue the rows that fail the exponent-span check on the native FP64 path (OZ_FALLBACK_FP64)")
     args = ap.parse_args()
@@ -282,7 +284,7 @@ def main():
     modset = {"S": oz.OZ_SET_S, "E": oz.OZ_SET_E, "A": oz.OZ_SET_A}[args.set_name]
     sub = {"fp8": oz.OZ_SUB_FP8, "int8": oz.OZ_SUB_INT8, "int8n": oz.OZ_SUB_INT8_NATIVE}[args.substrate]
     host_route = sub | oz.OZ_QUANT_RN | oz.OZ_SCALE_CS      # the host-buffer entry point has no native path
-    route = host_route | (oz.OZ_FALLBACK_FP64 if args.fallback else 0)
+    route = host_route | (oz.OZ_FALLBACK_FP64 if args.fallback else 0) | (oz.OZ_STORAGE_FUSED if args.fused else 0)
     r, _, _ = oz.oz_set_info(modset)
     p_store = oz.oz_plane_count(modset, route)
     p_store_a = oz.oz_plane_count_side(modset, route, 0)    # same count on both operands
@@ -468,7 +470,7 @@ def main():
             "data": "synthetic",
             "config": {"workload": cfg.name, "m": m, "n": n, "k": k, "alpha": cfg.alpha, "beta": cfg.beta,
                        "modulus_set": args.set_name, "r": r, "substrate": args.substrate, "quantiser": "RN",
-                       "scale_rule": "CS",
+                       "scale_rule": "CS", "storage_mode": "F (A converted inside the product kernel)" if args.fused else "M (materialised planes)",
                        "l2": "inputs larger than L2 (126 MB): A+B %.0f MB, C %.0f MB, planes %.0f MB, residues %.0f MB"
                              % (8e-6 * (m * k + k * n), 8e-6 * m * n, 1e-6 * p_store * (m + n) * k, 1e-6 * rb * r * m * n),
                        "parallelism": f"replicas x{world}" if world > 1 else "single GPU"},

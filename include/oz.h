@@ -135,6 +135,18 @@ typedef enum { OZ_SET_S = 0, OZ_SET_E = 1, OZ_SET_A = 2 } oz_modset_t;
  * entry points.  Workspace: oz_workspace_bytes() with the same route (5 m + 768 bytes more). */
 #define OZ_FALLBACK_FP64 0x8000u
 
+/* Storage mode F for tall-skinny products (Sec. "Storage Modes", mode F; "O4: pipelining"): the planes
+ * of A are never written to memory.  oz_dgemm / oz_dgemm_ex then run only the scan of A (its shifts),
+ * and the product kernel converts each 64-row tile of A into plane bytes inside the shared-memory ring
+ * that feeds the tensor core, four moduli per pass over the tile (the paper's modulus blocking with
+ * n_blk = 4: A is read and quantised r/4 times).  B is deconstructed as always.  Same residues, same
+ * result, bit for bit.  Applies when n <= 128, the substrate is FP8 or INT8 digits (merged schedule,
+ * which the bit implies), and k is within the exact depth of one accumulator (k <= 4097 on set S,
+ * 15420 on sets E and A for FP8; 262144 for INT8 digits); OZ_ERR_UNSUPPORTED otherwise, and with
+ * OZ_SCALE_ACCURATE, OZ_RECON_TENSOR, OZ_FALLBACK_FP64, oz_dgemm_host and oz_dgemm_prepared.  Ignored by
+ * the stage entry points. */
+#define OZ_STORAGE_FUSED 0x10000u
+
 #define OZ_K_MAX 1048576
 #define OZ_NONFINITE_SHIFT INT32_MIN  /* value of shift[] for a line that holds Inf/NaN */
 

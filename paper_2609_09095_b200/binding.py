@@ -23,6 +23,7 @@ OZ_SCALE_MAXEXP, OZ_SCALE_CS, OZ_SCALE_ACCURATE = 0x100, 0x200, 0x400
 OZ_ACC_MERGED, OZ_ACC_SEPARATE = 0x1000, 0x2000
 OZ_RECON_TENSOR = 0x4000
 OZ_FALLBACK_FP64 = 0x8000
+OZ_STORAGE_FUSED = 0x10000
 OZ_K_MAX = 1048576
 OZ_NONFINITE_SHIFT = -(2 ** 31)
 OZ_STATIC_MAX_LINES = 262144
@@ -37,7 +38,7 @@ __all__ = EXPORTS + ["EXPORTS", "OzError", "load", "check", "LIB_PATH", "OZ_OK",
                      "OZ_ERR_UNSUPPORTED", "OZ_ERR_WORKSPACE", "OZ_ERR_CUDA",
                      "OZ_ERR_NONFINITE_INPUT", "OZ_ERR_RANGE", "OZ_ERR_TIMEOUT", "OZ_SET_S",
                      "OZ_SET_E", "OZ_SET_A", "OZ_SUB_FP8", "OZ_SUB_INT8", "OZ_SUB_INT8_NATIVE", "OZ_QUANT_RN", "OZ_QUANT_TZ",
-                     "OZ_SCALE_MAXEXP", "OZ_SCALE_CS", "OZ_SCALE_ACCURATE", "OZ_ACC_MERGED", "OZ_ACC_SEPARATE", "OZ_RECON_TENSOR", "OZ_FALLBACK_FP64", "OZ_K_MAX", "OZ_NONFINITE_SHIFT", "OZ_STATIC_MAX_LINES"]
+                     "OZ_SCALE_MAXEXP", "OZ_SCALE_CS", "OZ_SCALE_ACCURATE", "OZ_ACC_MERGED", "OZ_ACC_SEPARATE", "OZ_RECON_TENSOR", "OZ_FALLBACK_FP64", "OZ_STORAGE_FUSED", "OZ_K_MAX", "OZ_NONFINITE_SHIFT", "OZ_STATIC_MAX_LINES"]
 
 _lib = None
 

@@ -119,9 +119,10 @@ uint64_t isqrt_u128(unsigned __int128 v)
 bool decode_route(uint32_t route, Route *out)
 {
     uint32_t sub = route & 0x00Fu, q = route & 0x0F0u, sc = route & 0xF00u, ac = route & 0x3000u;
-    if (route & ~0xFFFFu) return false;
+    if (route & ~0x1FFFFu) return false;
     out->hosted = (route & OZ_RECON_TENSOR) != 0;
     out->fallback = (route & OZ_FALLBACK_FP64) != 0;
+    out->fused = (route & OZ_STORAGE_FUSED) != 0;
     if (ac == 0) out->acc = 0;
     else if (ac == OZ_ACC_MERGED) out->acc = 1;
     else if (ac == OZ_ACC_SEPARATE) out->acc = 2;
@@ -291,7 +292,7 @@ struct OperandLayout {
     int64_t pitch, stride;
 };
 
-OperandLayout operand_layout(int side, int64_t lines, int64_t k, int set, const Route &rt)
+OperandLayout operand_layout(int side, int64_t lines, int64_t k, int set, const Route &rt, bool whole_method = false)
 {
     OperandLayout o{};
     Carve c;
@@ -299,7 +300,8 @@ OperandLayout operand_layout(int side, int64_t lines, int64_t k, int set, const 
     o.stride = lines * o.pitch;
     o.shift = c.take(4 * static_cast<size_t>(lines));
     o.scratch = c.take(16 * static_cast<size_t>(lines) + 256);
-    o.planes = c.take(static_cast<size_t>(p_store(set, rt.layout(side))) * o.stride);
+    // storage mode F keeps no planes of A: they exist only inside the product kernel's shared memory
+    o.planes = c.take((whole_method && rt.fused && side == 0) ? 0 : static_cast<size_t>(p_store(set, rt.layout(side))) * o.stride);
     o.total = c.off;
     return o;
 }
@@ -333,8 +335,8 @@ struct Layout {
 Layout make_layout(int64_t m, int64_t n, int64_t k, int set, const Route &rt)
 {
     Layout L{};
-    L.A = operand_layout(0, m, k, set, rt);
-    L.B = operand_layout(1, n, k, set, rt);
+    L.A = operand_layout(0, m, k, set, rt, true);
+    L.B = operand_layout(1, n, k, set, rt, true);
     L.offA = 0;
     L.offB = L.A.total;
     L.R = L.offB + L.B.total;
@@ -437,6 +439,7 @@ oz_status_t dgemm_impl(int64_t m, int64_t n, int64_t k, double alpha, const doub
         return OZ_ERR_INVALID_ARG;
     // out-of-range rows on the native path: defined on the norm scan, FP64 reconstruction, one panel
     if (rt.fallback && (rt.rule != 1 || rt.hosted || plan)) return OZ_ERR_UNSUPPORTED;
+    if (rt.fused && rt.rule == 2) return OZ_ERR_UNSUPPORTED;
     Layout L = make_layout(m, n, k, set, rt);
     if (!ws || ws_bytes < L.total) return OZ_ERR_WORKSPACE;
     st = ensure_device_ready();
@@ -475,6 +478,30 @@ oz_status_t dgemm_impl(int64_t m, int64_t n, int64_t k, double alpha, const doub
             st = launch_convert_planes(1, n, k, B, ldb, set, rt, b.planes, b.stride, b.pitch, b.shift, stream);
         if (st != OZ_OK) return st;
         return product_impl(m, n, k, alpha, a, b, beta, C, ldc, set, rt, stream, ws + L.R, dev, plan);
+    }
+    if (rt.fused) {
+        // Storage mode F: only the scan of A runs ahead of the product kernel, which converts A's tiles
+        // itself; B is deconstructed as always (side stream); residues in the public layout
+        if (rt.fallback || rt.hosted || plan || !fused_gemm_applies(m, n, k, set, rt)) return OZ_ERR_UNSUPPORTED;
+        OZ_CUDA_CHECK(cudaEventRecord(g_fork[dev], stream));
+        OZ_CUDA_CHECK(cudaStreamWaitEvent(side, g_fork[dev], 0));
+        st = launch_deconstruct(1, n, k, B, ldb, set, rt, b.planes, b.stride, b.pitch, b.shift, b.scratch, side);
+        if (st != OZ_OK) return st;
+        OZ_CUDA_CHECK(cudaEventRecord(g_join[dev], side));
+        st = launch_scan(0, m, k, A, lda, set, rt, a.shift, a.scratch, stream);
+        if (st != OZ_OK) return st;
+        if (ev) OZ_CUDA_CHECK(cudaEventRecord(g_stage_events[dev][1], stream));
+        OZ_CUDA_CHECK(cudaStreamWaitEvent(stream, g_join[dev], 0));
+        if (ev) OZ_CUDA_CHECK(cudaEventRecord(g_stage_events[dev][2], stream));
+        const int64_t ldr = round_up(m, 64);
+        st = launch_fused_gemm(m, n, k, A, lda, a.shift, b.planes, b.stride, b.pitch, set, rt, ws + L.R, ldr, n * ldr,
+                               stream);
+        if (st != OZ_OK) return st;
+        if (ev) OZ_CUDA_CHECK(cudaEventRecord(g_stage_events[dev][3], stream));
+        st = launch_reconstruct(m, n, ws + L.R, ldr, n * ldr, a.shift, b.shift, set, alpha, beta, C, ldc, stream);
+        if (st != OZ_OK) return st;
+        if (ev) OZ_CUDA_CHECK(cudaEventRecord(g_stage_events[dev][4], stream));
+        return OZ_OK;
     }
     OZ_CUDA_CHECK(cudaEventRecord(g_fork[dev], stream));
     OZ_CUDA_CHECK(cudaStreamWaitEvent(side, g_fork[dev], 0));
@@ -740,7 +767,7 @@ oz_status_t oz_dgemm_prepared(int64_t m, int64_t n, int64_t k, double alpha, con
     oz_status_t st = check_product_args(m, n, k, alpha, beta, C, ldc, set, route, s, &rt, &trivial);
     if (st != OZ_OK || trivial) return st;
     if (rt.rule == 2) return OZ_ERR_UNSUPPORTED;      // prepared operands carry per-operand shifts
-    if (rt.fallback) return OZ_ERR_UNSUPPORTED;       // the native path needs the FP64 operands
+    if (rt.fallback || rt.fused) return OZ_ERR_UNSUPPORTED;   // both need the FP64 operands
     if (!operandA || !operandB || (reinterpret_cast<uintptr_t>(operandA) & 255u) ||
         (reinterpret_cast<uintptr_t>(operandB) & 255u))
         return OZ_ERR_INVALID_ARG;

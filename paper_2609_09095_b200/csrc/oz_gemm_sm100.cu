@@ -56,6 +56,7 @@
 #include <cstdlib>
 
 #include "oz_internal.h"
+#include "oz_convert.cuh"
 
 namespace oz {
 namespace {
@@ -872,6 +873,8 @@ residue_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
     }
 }
 
+#include "oz_gemm_fused.cuh"
+
 // ---------------------------------------------------------------- host side
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *,
                                   const cuuint64_t *, const cuuint64_t *, const cuuint32_t *,
@@ -907,6 +910,39 @@ bool make_plane_map(CUtensorMap *map, const uint8_t *base, int64_t lines, int64_
                      box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                      CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return rc == CUDA_SUCCESS;
+}
+
+// 3-D map over planes[plane][line][kbyte] for the fused kernel: box = 16 bytes x 128 lines x 1 plane,
+// no swizzle (8 rows x 16 bytes land as one contiguous core matrix), out-of-range elements read as zero.
+bool make_core_matrix_map(CUtensorMap *map, const uint8_t *base, int64_t lines, int64_t pitch,
+                          int64_t plane_stride, int planes)
+{
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    cuuint64_t dims[3] = {static_cast<cuuint64_t>(pitch), static_cast<cuuint64_t>(lines),
+                          static_cast<cuuint64_t>(planes)};
+    cuuint64_t strides[2] = {static_cast<cuuint64_t>(pitch), static_cast<cuuint64_t>(plane_stride)};
+    cuuint32_t box[3] = {16, 128, 1};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult rc = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<uint8_t *>(base), dims, strides,
+                     box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+                     CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return rc == CUDA_SUCCESS;
+}
+
+template <int SUB, int SET>
+oz_status_t launch_fused_variant(const CUtensorMap &mapB, const GemmParams &p, const FusedGemmParams &f, int sms,
+                                 cudaStream_t stream)
+{
+    constexpr int LAYOUT_A = SUB == 0 ? kLayoutMerged : kLayoutMergedI8A;
+    auto kernel = fused_gemm_kernel<SUB, SET, LAYOUT_A>;
+    constexpr size_t smem = fused_gemm_smem(SET);
+    OZ_CUDA_CHECK(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
+    const int grid = f.tiles < sms ? f.tiles : sms;
+    kernel<<<grid, F_THREADS, smem, stream>>>(mapB, p, f);
+    count_launch();
+    OZ_CUDA_CHECK(cudaGetLastError());
+    return OZ_OK;
 }
 
 template <int SUB, int CG, int RB, bool DIRECT = false, bool LOOSE = false, bool TILED = false, bool BOUND = false>
@@ -967,38 +1003,11 @@ static int take_stall_flag()
     return v;
 }
 
-ResidueTiling residue_tiling(int64_t m, int64_t n, int set)
+// Per-modulus constants of the epilogue and the accumulator schedule (jobs, weights, which
+// accumulators are reduced before they are weighted, K segments) for inner dimension k; p.r and p.nk
+// (chunks of BLOCK_K) are set by the caller.
+static void fill_mod_info(GemmParams &p, int set, const Route &rt, int64_t k)
 {
-    ResidueTiling t;
-    t.cg = cta_group_choice(n);
-    t.tile_cols = BLOCK_M * t.cg;
-    t.tiles_m = static_cast<int>((m + BLOCK_N - 1) / BLOCK_N);
-    t.tiles_n = static_cast<int>((n + t.tile_cols - 1) / t.tile_cols);
-    t.mod_stride = static_cast<int64_t>(t.tiles_m) * t.tiles_n * t.tile_cols * BLOCK_N;
-    (void)set;
-    return t;
-}
-
-oz_status_t launch_residue_gemm(int64_t m, int64_t n, int64_t k, const uint8_t *PA, int64_t strideA,
-                                int64_t pitchA, const uint8_t *PB, int64_t strideB, int64_t pitchB,
-                                int set, const Route &rt, void *R, int64_t ldr,
-                                int64_t mod_stride, bool loose, bool tiled, cudaStream_t stream)
-{
-    const int cg = cta_group_choice(n);
-    GemmParams p{};
-    p.m = m; p.n = n; p.k = k;
-    p.tiles_m = static_cast<int>((m + BLOCK_N - 1) / BLOCK_N);             // 256 rows of C per tile
-    p.tiles_n = static_cast<int>((n + BLOCK_M * cg - 1) / (BLOCK_M * cg)); // 128 (256) columns of C per tile
-    const int rb = residue_bytes(set);
-    p.vec_store = ((ldr * rb) % 16 == 0 && (mod_stride * rb) % 16 == 0 && (reinterpret_cast<uintptr_t>(R) & 15u) == 0) ? 1 : 0;
-    p.nk = static_cast<int>((k + BLOCK_K - 1) / BLOCK_K);
-    if (k == 0) p.nk = 1;   // one all-zero chunk (the planes' padding) gives residues 0
-    p.r = set_r(set);
-    p.total_items = static_cast<int64_t>(p.r) * p.tiles_m * p.tiles_n;
-    if (p.total_items >= 0x7FFFFFFFll) return OZ_ERR_UNSUPPORTED;        // item numbers are 32-bit in the kernel
-    p.R = R; p.ldr = ldr; p.mod_stride = mod_stride;
-    p.stall_producer = take_stall_flag();
-    p.status = device_status_word();
     for (int i = 0; i < p.r; ++i) {
         int mi = modulus(set, i), s = square_root(mi);
         p.mod[i].m = static_cast<float>(mi);
@@ -1073,6 +1082,41 @@ oz_status_t launch_residue_gemm(int64_t m, int64_t n, int64_t k, const uint8_t *
         }
         for (int j = 0; j < 3; ++j) mo.iw[j] = static_cast<int>(mo.w[j]);
     }
+}
+
+ResidueTiling residue_tiling(int64_t m, int64_t n, int set)
+{
+    ResidueTiling t;
+    t.cg = cta_group_choice(n);
+    t.tile_cols = BLOCK_M * t.cg;
+    t.tiles_m = static_cast<int>((m + BLOCK_N - 1) / BLOCK_N);
+    t.tiles_n = static_cast<int>((n + t.tile_cols - 1) / t.tile_cols);
+    t.mod_stride = static_cast<int64_t>(t.tiles_m) * t.tiles_n * t.tile_cols * BLOCK_N;
+    (void)set;
+    return t;
+}
+
+oz_status_t launch_residue_gemm(int64_t m, int64_t n, int64_t k, const uint8_t *PA, int64_t strideA,
+                                int64_t pitchA, const uint8_t *PB, int64_t strideB, int64_t pitchB,
+                                int set, const Route &rt, void *R, int64_t ldr,
+                                int64_t mod_stride, bool loose, bool tiled, cudaStream_t stream)
+{
+    const int cg = cta_group_choice(n);
+    GemmParams p{};
+    p.m = m; p.n = n; p.k = k;
+    p.tiles_m = static_cast<int>((m + BLOCK_N - 1) / BLOCK_N);             // 256 rows of C per tile
+    p.tiles_n = static_cast<int>((n + BLOCK_M * cg - 1) / (BLOCK_M * cg)); // 128 (256) columns of C per tile
+    const int rb = residue_bytes(set);
+    p.vec_store = ((ldr * rb) % 16 == 0 && (mod_stride * rb) % 16 == 0 && (reinterpret_cast<uintptr_t>(R) & 15u) == 0) ? 1 : 0;
+    p.nk = static_cast<int>((k + BLOCK_K - 1) / BLOCK_K);
+    if (k == 0) p.nk = 1;   // one all-zero chunk (the planes' padding) gives residues 0
+    p.r = set_r(set);
+    p.total_items = static_cast<int64_t>(p.r) * p.tiles_m * p.tiles_n;
+    if (p.total_items >= 0x7FFFFFFFll) return OZ_ERR_UNSUPPORTED;        // item numbers are 32-bit in the kernel
+    p.R = R; p.ldr = ldr; p.mod_stride = mod_stride;
+    p.stall_producer = take_stall_flag();
+    p.status = device_status_word();
+    fill_mod_info(p, set, rt, k);
 
     CUtensorMap mapA, mapB;
     if (!make_plane_map(&mapA, PA, m, pitchA, strideA, p_store(set, rt.layout(0)), BLOCK_N / cg) ||
@@ -1098,6 +1142,56 @@ oz_status_t launch_residue_gemm(int64_t m, int64_t n, int64_t k, const uint8_t *
     return OZ_LAUNCH_SUB(2, false, false);
 #undef OZ_LAUNCH_SUB
 #undef OZ_LAUNCH
+}
+
+// Whether the fused mode applies: merged schedule on digit planes, all of B in one 128-lane tile, and
+// an inner dimension that every accumulator holds exactly without K segments.
+bool fused_gemm_applies(int64_t m, int64_t n, int64_t k, int set, const Route &rt)
+{
+    if (rt.native() || !rt.merged() || n < 1 || n > BLOCK_M || m < 1 || k < 1) return false;
+    if ((m + F_LINES - 1) / F_LINES >= 0x7FFFFFFFll) return false;
+    // one accumulator per job over all of k: FP32 holds the merged term (4095 on the 9-bit tail of S,
+    // 1088 on byte moduli) exactly to 2^24, INT32 the term 4292 far beyond any k taken here; where the
+    // epilogue reduces an accumulator before weighting it is decided for this k by fill_mod_info
+    const int64_t kmax = rt.substrate == 0 ? merged_k_limit(set) : 262144;
+    return k <= kmax;
+}
+
+// Residue products with A converted on the fly (storage mode F): A in FP64 with the shifts of its rows,
+// B's planes materialised in the layout of side 1 of the route; canonical residues in the public layout
+// R[mod][j][ldr], ldr a multiple of 64 and at least m rounded up to 64 (the last tile stores whole).
+oz_status_t launch_fused_gemm(int64_t m, int64_t n, int64_t k, const double *A, int64_t lda, const int32_t *shiftA,
+                              const uint8_t *PB, int64_t strideB, int64_t pitchB, int set, const Route &rt,
+                              void *R, int64_t ldr, int64_t mod_stride, cudaStream_t stream)
+{
+    if (!fused_gemm_applies(m, n, k, set, rt)) return OZ_ERR_UNSUPPORTED;
+    if (ldr % F_LINES != 0 || ldr < round_up(m, F_LINES) || (reinterpret_cast<uintptr_t>(R) & 15u)) return OZ_ERR_INVALID_ARG;
+    GemmParams p{};
+    p.m = m; p.n = n; p.k = k;
+    p.r = set_r(set);
+    p.nk = static_cast<int>((k + BLOCK_K - 1) / BLOCK_K);
+    p.R = R; p.ldr = ldr; p.mod_stride = mod_stride;
+    p.stall_producer = 0;
+    p.status = device_status_word();
+    fill_mod_info(p, set, rt, k);
+    FusedGemmParams f{};
+    f.A = A; f.lda = lda; f.shiftA = shiftA;
+    f.lut_global = device_lut(set, rt.substrate);
+    f.tz = rt.quant;
+    f.tiles = static_cast<int>((m + F_LINES - 1) / F_LINES);
+    f.passes = (p.r + F_GROUP - 1) / F_GROUP;
+    f.nks = static_cast<int>((k + F_K - 1) / F_K);
+    CUtensorMap mapB;
+    if (!make_core_matrix_map(&mapB, PB, n, pitchB, strideB, p_store(set, rt.layout(1)))) return OZ_ERR_CUDA;
+    int dev = 0, sms = 148;
+    OZ_CUDA_CHECK(cudaGetDevice(&dev));
+    OZ_CUDA_CHECK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+#define OZ_FUSED_GEMM(SET_) \
+    (rt.substrate == 0 ? launch_fused_variant<0, SET_>(mapB, p, f, sms, stream) : launch_fused_variant<1, SET_>(mapB, p, f, sms, stream))
+    if (set == 0) return OZ_FUSED_GEMM(0);
+    if (set == 1) return OZ_FUSED_GEMM(1);
+    return OZ_FUSED_GEMM(2);
+#undef OZ_FUSED_GEMM
 }
 
 // The magnitude-bound product of the accurate mode: one E4M3 plane per operand (digits <= 32, terms

@@ -122,6 +122,7 @@ struct Route {
     }
     bool hosted;    // whole-method calls: CRT recombination on the INT8 tensor pipe (OZ_RECON_TENSOR)
     bool fallback;  // oz_dgemm / oz_dgemm_ex: out-of-range rows re-issued on the native FP64 path
+    bool fused;     // oz_dgemm / oz_dgemm_ex: A converted inside the product kernel (storage mode F)
     int quant;      // 0 rn, 1 tz
     int rule;       // 0 maxexp, 1 cs, 2 accurate (shifts from the extra bound product)
 };
@@ -193,6 +194,13 @@ oz_status_t launch_residue_gemm(int64_t m, int64_t n, int64_t k, const uint8_t *
                                 int64_t strideB, int64_t pitchB, int set, const Route &rt,
                                 void *R, int64_t ldr, int64_t mod_stride, bool loose, bool tiled,
                                 cudaStream_t stream);
+
+// Storage mode F: residue products with A converted on the fly inside the kernel (n <= 128, merged
+// schedule on digit planes, k within the exact depth of one accumulator); public residue layout
+bool fused_gemm_applies(int64_t m, int64_t n, int64_t k, int set, const Route &rt);
+oz_status_t launch_fused_gemm(int64_t m, int64_t n, int64_t k, const double *A, int64_t lda, const int32_t *shiftA,
+                              const uint8_t *PB, int64_t strideB, int64_t pitchB, int set, const Route &rt,
+                              void *R, int64_t ldr, int64_t mod_stride, cudaStream_t stream);
 
 // reconstruction from the tile-ordered array, columns [col0, col1) of the m x n output
 oz_status_t launch_reconstruct_tiled(int64_t m, int64_t n, const void *R, const int32_t *shiftA,
