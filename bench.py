@@ -308,7 +308,7 @@ def main():
                 also_routes.append((sname, subname))
     sets = {"S": oz.OZ_SET_S, "E": oz.OZ_SET_E, "A": oz.OZ_SET_A}
     subs = {"fp8": oz.OZ_SUB_FP8, "int8": oz.OZ_SUB_INT8, "int8n": oz.OZ_SUB_INT8_NATIVE}
-    core = max([oz.oz_workspace_bytes(m, n, k, modset, route)] +
+    core = max([oz.oz_workspace_bytes(m, n, k, modset, route), oz.oz_workspace_bytes(m, n, k, modset, host_route)] +
                [oz.oz_workspace_bytes(m, n, k, sets[a], subs[b] | oz.OZ_QUANT_RN | oz.OZ_SCALE_CS) for a, b in also_routes])
     ws_bytes = core + 8 * (m * k + k * n + m * n) + 4096
     ws = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")
