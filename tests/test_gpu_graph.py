@@ -10,13 +10,19 @@ from oracle import oz_oracle as ozo
 pytestmark = pytest.mark.gpu
 
 
-@pytest.mark.parametrize("m,n,k,set_name,sub", [(256, 256, 256, "S", "fp8"),        # one-kernel deconstruction
-                                                (300, 2200, 2100, "A", "int8n")])   # three-pass deconstruction of B
-def test_dgemm_replayed_from_a_cuda_graph(m, n, k, set_name, sub):
+@pytest.mark.parametrize("m,n,k,set_name,sub,mode", [
+    (256, 256, 256, "S", "fp8", None),            # one-kernel deconstruction
+    (300, 2200, 2100, "A", "int8n", None),        # three-pass deconstruction of B
+    (300, 100, 500, "S", "fp8", "fused"),         # storage mode F: A converted inside the product kernel
+    (200, 150, 300, "A", "fp8", "fallback"),      # native FP64 path: the number of re-issued rows varies per replay
+])
+def test_dgemm_replayed_from_a_cuda_graph(m, n, k, set_name, sub, mode):
     import torch
     import paper_2609_09095_b200 as oz
     import tests.gpu_helpers as gh
-    sid, rt = gh.SETS[set_name], gh.route(sub)
+    sid, rt = gh.SETS[set_name], gh.route(sub, fallback=(mode == "fallback"))
+    if mode == "fused":
+        rt |= oz.OZ_STORAGE_FUSED
     oset = {"S": ozo.SET_S, "A": ozo.SET_A}[set_name]
     rng = np.random.default_rng(k)
     gh.ensure_workspace(oz.oz_workspace_bytes(m, n, k, sid, rt))
@@ -32,7 +38,12 @@ def test_dgemm_replayed_from_a_cuda_graph(m, n, k, set_name, sub):
         with torch.cuda.graph(graph, stream=side):
             oz.check(oz.oz_dgemm(m, n, k, dA, m, dB, k, dC, m, sid, rt, torch.cuda.current_stream()), "oz_dgemm (capture)")
     for rep in range(3):
-        A, B = syn._draw(rng, m, k, "uniform"), syn._draw(rng, k, n, "normal")
+        if mode == "fallback":      # exponent spreads from benign to wide: none, some or all rows re-issued
+            sg = (0.5, 2.5, 3.5)[rep]
+            A = np.asfortranarray(rng.standard_normal((m, k)) * np.exp(sg * rng.standard_normal((m, k))))
+            B = np.asfortranarray(rng.standard_normal((k, n)) * np.exp(sg * rng.standard_normal((k, n))))
+        else:
+            A, B = syn._draw(rng, m, k, "uniform"), syn._draw(rng, k, n, "normal")
         dA.copy_(gh.to_dev(A))
         dB.copy_(gh.to_dev(B))
         dC.fill_(-1.0)
@@ -40,4 +51,9 @@ def test_dgemm_replayed_from_a_cuda_graph(m, n, k, set_name, sub):
         graph.replay()
         torch.cuda.synchronize()
         assert gh.sync_status() == 0
-        assert (gh.from_dev(dC) == ozo.dgemm(A, B, oset)).all()
+        if mode == "fallback":
+            want, flag = ozo.dgemm_fallback(A, B, oset)
+            assert oz.oz_query_fallback_rows() == int(flag.sum())
+        else:
+            want = ozo.dgemm(A, B, oset)
+        assert (gh.from_dev(dC) == want).all()
